@@ -1,0 +1,194 @@
+/*
+ * dppo.h — C ABI of libdppo: the hot path of DPPO's pruned GRPO training step on one B200.
+ *
+ * DPPO ("Unbiased Dynamic Pruning for Efficient Group-Based Policy Optimization") prunes prompts
+ * and completions of a GRPO batch at random, reweights what is retained by importance-sampling
+ * factors so that the gradient stays unbiased, packs the retained sequences densely and trains on
+ * them.  This library does, per batch:  group advantages -> candidate sets, pruning masks and
+ * rescaling factors -> Dense Prompt Packing -> one sweep over the LM-head logits that yields the
+ * loss and dlogits.
+ *
+ * Conventions (all entry points)
+ *  - Return value: 0 (DPPO_OK) or a negative dppo_error.  Nothing throws, aborts or prints.
+ *    dppo_last_error() gives the message of the calling thread's last failure.
+ *  - Unless a parameter says "host", array pointers are DEVICE pointers owned by the caller.  The
+ *    library allocates no memory and keeps no state between calls; scratch comes from a caller
+ *    workspace sized by the matching *_workspace_bytes() (a pure host function).
+ *  - Work is enqueued on `stream` (a cudaStream_t passed as void*); there is no host
+ *    synchronisation inside.  Outputs are valid once the stream reaches that point.
+ *  - Host-visible arguments are validated before anything is launched.  Problems only the device
+ *    can see (a unit longer than a row, a target id outside the vocabulary, a wait that ran out)
+ *    are recorded in the caller's `status` word (device int32, first error wins, caller zeroes it)
+ *    as a positive dppo_status; the kernel then finishes without trapping.
+ *  - Every output is a deterministic function of the inputs (no floating-point atomics).
+ */
+#ifndef DPPO_H_
+#define DPPO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DPPO_OK = 0,
+    DPPO_ERR_INVALID_ARG = -1,          /* NULL where data is required, negative size, bad enum       */
+    DPPO_ERR_BAD_SHAPE = -2,            /* sizes inconsistent with each other or above a stated limit */
+    DPPO_ERR_MISALIGNED = -3,           /* base pointer or row stride not a multiple of 16 bytes      */
+    DPPO_ERR_WORKSPACE_TOO_SMALL = -4,
+    DPPO_ERR_UNSUPPORTED = -5,          /* dtype / option this build does not implement               */
+    DPPO_ERR_CUDA = -6                  /* a CUDA runtime call failed (message has the CUDA error)    */
+} dppo_error;
+
+typedef enum {                          /* values of the device status word */
+    DPPO_STATUS_OK = 0,
+    DPPO_STATUS_BAD_LENGTH = 1,         /* pack: a retained unit has length < 1 or > L_row            */
+    DPPO_STATUS_BAD_TARGET = 2,         /* loss: a target id outside [0, V)                           */
+    DPPO_STATUS_TIMEOUT = 3,            /* a bounded device-side wait ran out                         */
+    DPPO_STATUS_BAD_SEGMENTS = 4        /* loss: cu_seqlens does not cover a token                    */
+} dppo_status;
+
+int dppo_version(void);                 /* major*10000 + minor*100 + patch */
+const char* dppo_last_error(void);      /* host string, valid until the thread's next failing call */
+
+/* ------------------------------------------------------------------------------------------------
+ * Group-relative advantages — Eq. 2 (A_i = (r_i - mean)/std over the G completions of a prompt) and
+ * the per-prompt threshold of Eq. 14 (Abar = mean_i |A_i|).
+ *   rewards       f32 [P*G], row-major by prompt
+ *   std_ddof      0 population std (default reading of "std"), 1 sample std
+ *   std_eps       added to std before dividing (1e-6 by default; 0 allowed)
+ *   adv           f32 [P*G] out;  mean_abs_adv f32 [P] out
+ * A group whose rewards are all bitwise equal gets A = 0.  Arithmetic is binary64, one rounded
+ * operation at a time in ascending i, rounded once to f32 — results are reproducible bit for bit.
+ * Errors: INVALID_ARG (NULL, P<0, G<1, ddof not 0/1, eps<0).  P == 0 is a no-op.
+ */
+int dppo_group_advantages(const float* rewards, int P, int G, int std_ddof, double std_eps,
+                          float* adv, float* mean_abs_adv, int32_t* status, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Candidate sets, dynamic pruning masks, importance rescaling, history update —
+ * Eq. 15 (completion policy), Eq. 17 (prompt policy), Eq. 18 (discrete rescaling), Eq. 16 (history).
+ */
+typedef struct {
+    int32_t P, G;
+    double r_q, r_o;        /* pruning probabilities in [0,1): a candidate is pruned when u < r      */
+    int32_t mode;           /* 0: independent Bernoulli draws (Eq. 15, 17).
+                               1: fixed fraction (Appendix A / Algorithm 1): prune the floor(r*|C|)
+                                  candidates with the smallest u, ties to the lower index           */
+    int32_t reverse;        /* 0: low-|A| completions / low-H prompts are the candidates (the paper's
+                               rule); 1: the opposite sets (the ablation of Table 5)                 */
+    uint64_t seed, step;    /* Philox4x32-10 key / counter words when u_q,u_o are NULL:
+                               key=(seed lo,hi), counter=(index, domain, step lo, step hi),
+                               domain 1 prompts (index k), 2 completions (index k*G+i);
+                               u = ((out0 | out1<<32) >> 11) * 2^-53                                 */
+} dppo_prune_params;
+
+/*   adv, mean_abs_adv   outputs of dppo_group_advantages
+ *   H_prev   f32 [P] history scores H_{t-1}(q_k); NULL in the first epoch: no prompt is a candidate
+ *   u_q      f64 [P],  u_o f64 [P*G]: explicit draws in [0,1) replacing the generator (NULL: generate)
+ *   cand_q   u8 [P]    the floor(P/2) prompts with the lowest H_prev (ties: lower index)
+ *   cand_o   u8 [P*G]  |A_i| <= Abar_k, taken as G*|A_i| <= (sum_j |A_j|)*(1+1e-12) in binary64
+ *   keep_q   u8 [P];  keep_o u8 [P*G] (all 0 for a pruned prompt)
+ *   n_keep_q i32 [1] = |S^q|;  n_keep_o i32 [P] = |S^o(q_k)|
+ *   gamma_q  f32 [P]   (|S^q|/P)/(1-P^q);  gamma_o f32 [P*G] (|S^o_k|/G)/(1-P^o); 0 where pruned
+ *   w_seq    f32 [P*G] weight of a completion in the pruned objective read as the mean over retained
+ *                      prompts of gamma_q x mean over retained completions of gamma_o x term:
+ *                      1/(P*G*(1-P^q)*(1-P^o)); 0 where pruned
+ *   H_next   f32 [P]   Abar_k if the prompt was retained (or H_prev is NULL), else H_prev[k]
+ * In mode 1, P^q and P^o in these formulas are the realised fractions floor(r|C|)/|C| (the true
+ * inclusion probabilities), so the weights stay unbiased.
+ * Errors: INVALID_ARG (NULL outputs, r outside [0,1), bad mode), BAD_SHAPE (P*G >= 2^31).
+ */
+int dppo_prune_and_rescale(const dppo_prune_params* p, const float* adv, const float* mean_abs_adv,
+                           const float* H_prev, const double* u_q, const double* u_o,
+                           uint8_t* cand_q, uint8_t* cand_o, uint8_t* keep_q, uint8_t* keep_o,
+                           int32_t* n_keep_q, int32_t* n_keep_o, float* gamma_q, float* gamma_o,
+                           float* w_seq, float* H_next, int32_t* status, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Dense Prompt Packing — Section 4.3 (window-based greedy selection from a candidate pool W of
+ * size N_win, refilled from the stream, into rows of capacity L_row).
+ */
+typedef struct {
+    int32_t n_max;          /* units offered (retained or not)                                       */
+    int32_t L_row;          /* row capacity in tokens                                                */
+    int32_t N_win;          /* pool size, >= 1                                                       */
+    int32_t policy;         /* 0 first unit in pool order that fits; 1 longest that fits (ties: oldest) */
+} dppo_pack_params;
+
+size_t dppo_pack_workspace_bytes(const dppo_pack_params* p);
+
+/*   len        i32 [n_max] tokens of each unit (prompt + response)
+ *   keep       u8  [n_max] or NULL: units with keep == 0 are not in the stream
+ *   loss_len   i32 [n_max] or NULL: loss (response) tokens of each unit; NULL: = len
+ *   order      i32 [n_max] out: order[p] = unit placed p-th, for p < n_units; -1 beyond
+ *   row_of, off_in_row  i32 [n_max] out, indexed by unit; -1 for units not in the stream
+ *   row_fill   i32 [n_max] out: tokens used in row r, for r < n_rows; 0 beyond
+ *   cu_seqlens i32 [n_max+1] out: exclusive scan of loss_len in placement order; entries past
+ *              n_units repeat the total, so the array is non-decreasing over its whole length
+ *   counts     i32 [4] out: n_units, n_rows, total tokens, total loss tokens
+ * A retained unit with length < 1 or > L_row sets status DPPO_STATUS_BAD_LENGTH and packs nothing
+ * (counts = 0).  Errors: INVALID_ARG, BAD_SHAPE (n_max above the limit the workspace query
+ * reports as 0 bytes), WORKSPACE_TOO_SMALL.
+ */
+int dppo_pack_prompts(const dppo_pack_params* p, const int32_t* len, const uint8_t* keep,
+                      const int32_t* loss_len, int32_t* order, int32_t* row_of, int32_t* off_in_row,
+                      int32_t* row_fill, int32_t* cu_seqlens, int32_t* counts,
+                      void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Fused loss sweep over the logits — Eq. 1 (clipped surrogate minus beta x KL, 1/|o_i| per sequence,
+ * KL estimator rho_hat - log rho_hat - 1) with the sequence weights of dppo_prune_and_rescale, and
+ * its gradient with respect to the logits.
+ *
+ * For token t of sequence s (cu_seqlens[s] <= t < cu_seqlens[s+1]), target y, A = adv[s], W =
+ * w[s]/|o_s|:  z = logits[t,:]/temperature;  lse = log sum_v exp z_v;  logp = z_y - lse;
+ * rho = exp(logp - logp_old);  d = logp_ref - logp;  kl = e^d - d - 1;
+ * surr = min(rho A, clip(rho, 1-eps_lo, 1+eps_hi) A);  loss = -sum_t W (surr - beta kl);
+ * g = dloss/dlogp = -W (A rho [clipped branch not strictly smaller] + beta (e^d - 1));
+ * dlogits[t,v] = g ([v == y] - exp(z_v - lse)) / temperature.
+ */
+typedef enum { DPPO_F32 = 0, DPPO_BF16 = 1 } dppo_dtype;
+
+typedef struct {
+    int64_t T_max;          /* rows of logits / upper bound of loss tokens                           */
+    int32_t V;              /* vocabulary size                                                       */
+    int32_t dtype;          /* dppo_dtype of logits and dlogits                                      */
+    int64_t row_stride;     /* elements between consecutive rows (>= V; bytes a multiple of 16)      */
+    int32_t S_max;          /* cu_seqlens has S_max+1 entries, non-decreasing, last >= true T        */
+    int32_t reserved;       /* 0                                                                     */
+    double eps_lo, eps_hi;  /* clip range 1-eps_lo .. 1+eps_hi (the paper: both 0.2)                 */
+    double beta;            /* KL coefficient                                                        */
+    double temperature;     /* > 0 (the paper: 1)                                                    */
+} dppo_loss_params;
+
+size_t dppo_grpo_loss_workspace_bytes(const dppo_loss_params* p);
+
+/*   logits       [T_max x row_stride] of dtype, read-only unless dlogits aliases it
+ *   target       i32 [T_max] sampled token ids
+ *   logp_old, logp_ref  f32 [T_max] log-probs of the target under the old / reference policy
+ *   cu_seqlens   i32 [S_max+1]
+ *   n_tokens_dev i32 [1] true number of tokens T <= T_max on the device, or NULL (T = T_max);
+ *                rows >= T are neither read nor written
+ *   adv, w       f32: advantage and sequence weight of each sequence, read at index seg_map[s]
+ *                when seg_map (i32 [S_max], e.g. the packer's `order`) is given, else at index s
+ *   dlogits      same dtype/stride as logits; may alias logits (in place); NULL: forward only
+ *   logp_out, lse_out   f32 [T_max] or NULL
+ *   loss_out     f32 [5]: loss, policy-gradient part -sum W surr, sum W kl, clipped fraction, T
+ * Errors: INVALID_ARG, BAD_SHAPE, MISALIGNED (logits/dlogits base or row stride), UNSUPPORTED
+ * (dtype), WORKSPACE_TOO_SMALL.  Device status: BAD_TARGET (that row's dlogits are zeroed and it
+ * adds nothing to the loss), BAD_SEGMENTS.
+ */
+int dppo_grpo_loss_fwd_bwd(const dppo_loss_params* p, const void* logits, const int32_t* target,
+                           const float* logp_old, const float* logp_ref, const int32_t* cu_seqlens,
+                           const int32_t* n_tokens_dev, const float* adv, const float* w,
+                           const int32_t* seg_map, void* dlogits, float* logp_out, float* lse_out,
+                           float* loss_out, void* workspace, size_t workspace_bytes,
+                           int32_t* status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DPPO_H_ */

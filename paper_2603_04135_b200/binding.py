@@ -1,0 +1,129 @@
+"""ctypes binding of libdppo.so: same names as include/dppo.h, argument marshalling only.
+
+Array arguments are torch tensors (their device pointer is passed), raw integer addresses, or None
+for the nullable ones.  Every function raises DppoError on a non-zero return code.  There is no
+fallback: if the library has not been built, importing this module raises.
+"""
+import ctypes
+import os
+
+import torch
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libdppo.so")
+if not os.path.exists(_LIB_PATH):
+    raise ImportError("libdppo.so is not built: run `python -m paper_2603_04135_b200.build` "
+                      "(the CUDA library is the only implementation; there is no CPU path)")
+lib = ctypes.CDLL(_LIB_PATH)
+
+F32, BF16 = 0, 1
+STATUS_OK, STATUS_BAD_LENGTH, STATUS_BAD_TARGET, STATUS_TIMEOUT, STATUS_BAD_SEGMENTS = 0, 1, 2, 3, 4
+ERR_INVALID_ARG, ERR_BAD_SHAPE, ERR_MISALIGNED, ERR_WORKSPACE_TOO_SMALL, ERR_UNSUPPORTED, ERR_CUDA = \
+    -1, -2, -3, -4, -5, -6
+
+
+class DppoError(RuntimeError):
+    def __init__(self, code, message):
+        super().__init__("libdppo error %d: %s" % (code, message))
+        self.code = code
+
+
+class PruneParams(ctypes.Structure):
+    _fields_ = [("P", ctypes.c_int32), ("G", ctypes.c_int32), ("r_q", ctypes.c_double), ("r_o", ctypes.c_double),
+                ("mode", ctypes.c_int32), ("reverse", ctypes.c_int32), ("seed", ctypes.c_uint64),
+                ("step", ctypes.c_uint64)]
+
+
+class PackParams(ctypes.Structure):
+    _fields_ = [("n_max", ctypes.c_int32), ("L_row", ctypes.c_int32), ("N_win", ctypes.c_int32),
+                ("policy", ctypes.c_int32)]
+
+
+class LossParams(ctypes.Structure):
+    _fields_ = [("T_max", ctypes.c_int64), ("V", ctypes.c_int32), ("dtype", ctypes.c_int32),
+                ("row_stride", ctypes.c_int64), ("S_max", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("eps_lo", ctypes.c_double), ("eps_hi", ctypes.c_double), ("beta", ctypes.c_double),
+                ("temperature", ctypes.c_double)]
+
+
+_vp = ctypes.c_void_p
+lib.dppo_version.restype = ctypes.c_int
+lib.dppo_last_error.restype = ctypes.c_char_p
+lib.dppo_group_advantages.restype = ctypes.c_int
+lib.dppo_group_advantages.argtypes = [_vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_double, _vp, _vp, _vp, _vp]
+lib.dppo_prune_and_rescale.restype = ctypes.c_int
+lib.dppo_prune_and_rescale.argtypes = [ctypes.POINTER(PruneParams)] + [_vp] * 17
+lib.dppo_pack_workspace_bytes.restype = ctypes.c_size_t
+lib.dppo_pack_workspace_bytes.argtypes = [ctypes.POINTER(PackParams)]
+lib.dppo_pack_prompts.restype = ctypes.c_int
+lib.dppo_pack_prompts.argtypes = [ctypes.POINTER(PackParams)] + [_vp] * 10 + [ctypes.c_size_t, _vp, _vp]
+lib.dppo_grpo_loss_workspace_bytes.restype = ctypes.c_size_t
+lib.dppo_grpo_loss_workspace_bytes.argtypes = [ctypes.POINTER(LossParams)]
+lib.dppo_grpo_loss_fwd_bwd.restype = ctypes.c_int
+lib.dppo_grpo_loss_fwd_bwd.argtypes = [ctypes.POINTER(LossParams)] + [_vp] * 14 + [ctypes.c_size_t, _vp, _vp]
+
+
+def _ptr(x):
+    if x is None:
+        return None
+    if isinstance(x, torch.Tensor):
+        return x.data_ptr()
+    return int(x)
+
+
+def _stream(stream):
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream if torch.cuda.is_available() else None
+    if isinstance(stream, torch.cuda.Stream):
+        return stream.cuda_stream
+    return int(stream)
+
+
+def _check(rc):
+    if rc != 0:
+        raise DppoError(rc, lib.dppo_last_error().decode("utf-8", "replace"))
+
+
+def version():
+    return lib.dppo_version()
+
+
+def last_error():
+    return lib.dppo_last_error().decode("utf-8", "replace")
+
+
+def group_advantages(rewards, P, G, adv, mean_abs_adv, std_ddof=0, std_eps=1e-6, status=None, stream=None):
+    _check(lib.dppo_group_advantages(_ptr(rewards), P, G, std_ddof, std_eps, _ptr(adv), _ptr(mean_abs_adv),
+                                     _ptr(status), _stream(stream)))
+
+
+def prune_and_rescale(params, adv, mean_abs_adv, H_prev, u_q, u_o, cand_q, cand_o, keep_q, keep_o,
+                      n_keep_q, n_keep_o, gamma_q, gamma_o, w_seq, H_next, status=None, stream=None):
+    _check(lib.dppo_prune_and_rescale(ctypes.byref(params), _ptr(adv), _ptr(mean_abs_adv), _ptr(H_prev),
+                                      _ptr(u_q), _ptr(u_o), _ptr(cand_q), _ptr(cand_o), _ptr(keep_q),
+                                      _ptr(keep_o), _ptr(n_keep_q), _ptr(n_keep_o), _ptr(gamma_q),
+                                      _ptr(gamma_o), _ptr(w_seq), _ptr(H_next), _ptr(status), _stream(stream)))
+
+
+def pack_workspace_bytes(params):
+    return lib.dppo_pack_workspace_bytes(ctypes.byref(params))
+
+
+def pack_prompts(params, len_, keep, loss_len, order, row_of, off_in_row, row_fill, cu_seqlens, counts,
+                 workspace, workspace_bytes, status=None, stream=None):
+    _check(lib.dppo_pack_prompts(ctypes.byref(params), _ptr(len_), _ptr(keep), _ptr(loss_len), _ptr(order),
+                                 _ptr(row_of), _ptr(off_in_row), _ptr(row_fill), _ptr(cu_seqlens),
+                                 _ptr(counts), _ptr(workspace), workspace_bytes, _ptr(status), _stream(stream)))
+
+
+def grpo_loss_workspace_bytes(params):
+    return lib.dppo_grpo_loss_workspace_bytes(ctypes.byref(params))
+
+
+def grpo_loss_fwd_bwd(params, logits, target, logp_old, logp_ref, cu_seqlens, n_tokens_dev, adv, w, seg_map,
+                      dlogits, logp_out, lse_out, loss_out, workspace, workspace_bytes, status=None,
+                      stream=None):
+    _check(lib.dppo_grpo_loss_fwd_bwd(ctypes.byref(params), _ptr(logits), _ptr(target), _ptr(logp_old),
+                                      _ptr(logp_ref), _ptr(cu_seqlens), _ptr(n_tokens_dev), _ptr(adv), _ptr(w),
+                                      _ptr(seg_map), _ptr(dlogits), _ptr(logp_out), _ptr(lse_out),
+                                      _ptr(loss_out), _ptr(workspace), workspace_bytes, _ptr(status),
+                                      _stream(stream)))

@@ -1,0 +1,168 @@
+// Dense Prompt Packing (Section 4.3): window-based greedy packing of the retained units into rows.
+//
+// The packer is sequential by nature — every pick depends on the space the previous pick left — so it
+// runs as ONE warp.  The pool W never has to be materialised: units enter it in stream order and
+// leave it without reordering, so at any time W = { unplaced stream positions j < min(n, N_win +
+// #placed) } and "pool order" is position order.  The warp therefore keeps a placed-bitmask in
+// shared memory and finds the pick with a ballot over 32 positions at a time, starting at the lowest
+// unplaced position.  Stream compaction (keep mask -> stream) and the cu_seqlens scan ride along.
+#include "common.cuh"
+
+namespace dppo {
+
+constexpr int kPackMaxUnits = 65536;           // bitmask of 2048 words in shared memory
+constexpr int kPackSmemLens = 8192;            // stream lengths cached in shared memory up to this n_max
+
+struct PackWorkspace {                         // carved from the caller's workspace, all i32 [n_max]
+    int32_t* stream;                           // unit index of stream position j
+    int32_t* slen;                             // its length
+};
+
+template <bool kLensInSmem>
+__global__ void __launch_bounds__(32)
+pack_prompts_kernel(dppo_pack_params prm, const int32_t* __restrict__ len,
+                    const uint8_t* __restrict__ keep, const int32_t* __restrict__ loss_len,
+                    int32_t* __restrict__ order, int32_t* __restrict__ row_of,
+                    int32_t* __restrict__ off_in_row, int32_t* __restrict__ row_fill,
+                    int32_t* __restrict__ cu_seqlens, int32_t* __restrict__ counts,
+                    PackWorkspace ws, int32_t* status) {
+    __shared__ uint32_t placed[kPackMaxUnits / 32];
+    __shared__ int32_t lens_smem[kLensInSmem ? kPackSmemLens : 1];
+    const int lane = threadIdx.x;
+    const int n_max = prm.n_max, L = prm.L_row;
+
+    // ---- stream compaction, validation, output defaults
+    int n = 0;
+    long long total_tokens = 0;
+    bool bad = false;
+    for (int base = 0; base < n_max; base += 32) {
+        const int u = base + lane;
+        const bool in = u < n_max && (keep == nullptr || keep[u] != 0);
+        const int l = in ? len[u] : 0;
+        if (u < n_max) { order[u] = -1; row_of[u] = -1; off_in_row[u] = -1; row_fill[u] = 0; }
+        const unsigned m = __ballot_sync(0xffffffffu, in);
+        if (in) {
+            const int pos = n + __popc(m & ((1u << lane) - 1u));
+            ws.stream[pos] = u;
+            if (kLensInSmem) lens_smem[pos] = l; else ws.slen[pos] = l;
+            bad = bad || l < 1 || l > L;
+        }
+        n += __popc(m);
+        long long t = l;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+        total_tokens += t;
+    }
+    for (int w = lane; w < (n + 31) / 32; w += 32) placed[w] = 0u;
+    bad = __any_sync(0xffffffffu, bad);
+    __syncwarp();
+    if (bad) {
+        if (lane == 0) { set_status(status, DPPO_STATUS_BAD_LENGTH); counts[0] = counts[1] = counts[2] = counts[3] = 0; }
+        for (int p = lane; p <= n_max; p += 32) cu_seqlens[p] = 0;
+        return;
+    }
+    const int32_t* slen = kLensInSmem ? lens_smem : ws.slen;
+
+    // ---- greedy placement
+    int n_placed = 0, lo = 0, row = 0, remaining = L, loss_cum = 0;
+    while (n_placed < n) {
+        const int fetched = min(n, prm.N_win + n_placed);       // stream positions that have entered W
+        int pick = -1;
+        if (prm.policy == 0) {                                   // first unit in pool order that fits
+            for (int base = lo & ~31; base < fetched; base += 32) {
+                const int j = base + lane;
+                const bool ok = j >= lo && j < fetched && !((placed[j >> 5] >> (j & 31)) & 1u) && slen[j] <= remaining;
+                const unsigned m = __ballot_sync(0xffffffffu, ok);
+                if (m) { pick = base + __ffs(m) - 1; break; }
+            }
+        } else {                                                 // longest unit that fits, ties to the oldest
+            long long best = -1;                                 // (len << 32) | (0x7fffffff - j)
+            for (int base = lo & ~31; base < fetched; base += 32) {
+                const int j = base + lane;
+                const bool ok = j >= lo && j < fetched && !((placed[j >> 5] >> (j & 31)) & 1u) && slen[j] <= remaining;
+                long long key = ok ? (((long long)slen[j] << 32) | (long long)(0x7fffffff - j)) : -1;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) key = max(key, __shfl_xor_sync(0xffffffffu, key, o));
+                best = max(best, key);
+            }
+            if (best >= 0) pick = 0x7fffffff - (int)(best & 0xffffffffLL);
+        }
+        if (pick < 0) {                                          // nothing in W fits: close the row
+            if (lane == 0) row_fill[row] = L - remaining;
+            ++row;
+            remaining = L;
+            continue;
+        }
+        const int l = slen[pick];
+        if (lane == 0) {
+            const int u = ws.stream[pick];
+            order[n_placed] = u;
+            row_of[u] = row;
+            off_in_row[u] = L - remaining;
+            cu_seqlens[n_placed] = loss_cum;
+            placed[pick >> 5] |= 1u << (pick & 31);
+            loss_cum += loss_len ? loss_len[u] : l;
+        }
+        loss_cum = __shfl_sync(0xffffffffu, loss_cum, 0);
+        __syncwarp();
+        remaining -= l;
+        ++n_placed;
+        if (pick == lo) {                                        // advance to the next unplaced position
+            ++lo;
+            while (lo < n) {
+                const uint32_t w = ~placed[lo >> 5] & (0xffffffffu << (lo & 31));
+                if (w) { lo = (lo & ~31) + __ffs(w) - 1; break; }
+                lo = (lo & ~31) + 32;
+            }
+            lo = min(lo, n);
+        }
+    }
+    const int n_rows = n > 0 ? row + 1 : 0;
+    if (lane == 0) {
+        if (n > 0) row_fill[row] = L - remaining;
+        counts[0] = n; counts[1] = n_rows; counts[2] = (int32_t)total_tokens; counts[3] = loss_cum;
+    }
+    for (int p = n + lane; p <= n_max; p += 32) cu_seqlens[p] = loss_cum;
+}
+
+static size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
+
+}  // namespace dppo
+
+extern "C" size_t dppo_pack_workspace_bytes(const dppo_pack_params* p) {
+    if (!p || p->n_max < 0 || p->n_max > dppo::kPackMaxUnits) return 0;
+    return 2 * dppo::align_up((size_t)(p->n_max > 0 ? p->n_max : 1) * sizeof(int32_t));
+}
+
+extern "C" int dppo_pack_prompts(const dppo_pack_params* p, const int32_t* len, const uint8_t* keep,
+                                 const int32_t* loss_len, int32_t* order, int32_t* row_of,
+                                 int32_t* off_in_row, int32_t* row_fill, int32_t* cu_seqlens,
+                                 int32_t* counts, void* workspace, size_t workspace_bytes,
+                                 int32_t* status, void* stream) {
+    using namespace dppo;
+    if (!p) return fail(DPPO_ERR_INVALID_ARG, "pack_prompts: NULL params");
+    if (p->n_max < 0 || p->L_row < 1 || p->N_win < 1 || (p->policy != 0 && p->policy != 1))
+        return fail(DPPO_ERR_INVALID_ARG, "pack_prompts: n_max=%d L_row=%d N_win=%d policy=%d", p->n_max,
+                    p->L_row, p->N_win, p->policy);
+    if (p->n_max > kPackMaxUnits)
+        return fail(DPPO_ERR_BAD_SHAPE, "pack_prompts: n_max=%d above the limit %d", p->n_max, kPackMaxUnits);
+    if (!cu_seqlens || !counts) return fail(DPPO_ERR_INVALID_ARG, "pack_prompts: NULL cu_seqlens/counts");
+    if (p->n_max > 0 && (!len || !order || !row_of || !off_in_row || !row_fill))
+        return fail(DPPO_ERR_INVALID_ARG, "pack_prompts: NULL array");
+    const size_t need = dppo_pack_workspace_bytes(p);
+    if (!workspace || workspace_bytes < need)
+        return fail(DPPO_ERR_WORKSPACE_TOO_SMALL, "pack_prompts: workspace %zu < %zu bytes", workspace_bytes, need);
+    if (((uintptr_t)workspace & 15) != 0) return fail(DPPO_ERR_MISALIGNED, "pack_prompts: workspace not 16-byte aligned");
+    PackWorkspace ws;
+    ws.stream = (int32_t*)workspace;
+    ws.slen = (int32_t*)((char*)workspace + need / 2);
+    cudaStream_t s = (cudaStream_t)stream;
+    if (p->n_max <= kPackSmemLens)
+        pack_prompts_kernel<true><<<1, 32, 0, s>>>(*p, len, keep, loss_len, order, row_of, off_in_row, row_fill,
+                                                   cu_seqlens, counts, ws, status);
+    else
+        pack_prompts_kernel<false><<<1, 32, 0, s>>>(*p, len, keep, loss_len, order, row_of, off_in_row, row_fill,
+                                                    cu_seqlens, counts, ws, status);
+    DPPO_CHECK_LAUNCH("pack_prompts launch");
+    return DPPO_OK;
+}

@@ -1,0 +1,117 @@
+"""One pruned-GRPO batch step on the device: buffers + the four library calls in order.
+
+This is plumbing around :mod:`.binding`: it allocates device memory with torch, copies the small
+per-batch inputs in, issues the library calls on the current CUDA stream and copies results back.
+All arithmetic happens inside libdppo.
+"""
+import torch
+
+from . import binding as B
+
+
+class DppoStep:
+    """Buffers for a batch of P prompts x G completions and a loss sweep over at most T_max tokens.
+
+    prune_pack():  rewards -> advantages -> candidate sets, masks, gamma, w_seq, H_next -> packing of the
+                   retained completions (unit = prompt + response tokens) into rows of L_row, with
+                   cu_seqlens over the response tokens in packed order.
+    loss():        fused sweep over logits [T, V] of the retained response tokens in packed order.
+    """
+
+    def __init__(self, P, G, L_row, N_win, r_q, r_o, V, dtype, T_max, eps_lo=0.2, eps_hi=0.2, beta=0.04,
+                 temperature=1.0, mode=0, reverse=0, policy=0, std_ddof=0, std_eps=1e-6, device="cuda"):
+        if not torch.cuda.is_available():
+            raise RuntimeError("DppoStep needs a CUDA device: libdppo has no CPU path")
+        self.P, self.G, self.n = P, G, P * G
+        self.V, self.T_max = V, T_max
+        self.dtype = dtype
+        self.std_ddof, self.std_eps = std_ddof, std_eps
+        dev = torch.device(device)
+        self.device = dev
+        n = self.n
+        f32 = dict(dtype=torch.float32, device=dev)
+        i32 = dict(dtype=torch.int32, device=dev)
+        u8 = dict(dtype=torch.uint8, device=dev)
+        self.rewards = torch.zeros(n, **f32)
+        self.H_prev = torch.zeros(P, **f32)
+        self.has_history = False
+        self.unit_len = torch.zeros(n, **i32)
+        self.loss_len = torch.zeros(n, **i32)
+        self.adv = torch.zeros(n, **f32)
+        self.mean_abs_adv = torch.zeros(P, **f32)
+        self.cand_q = torch.zeros(P, **u8); self.cand_o = torch.zeros(n, **u8)
+        self.keep_q = torch.zeros(P, **u8); self.keep_o = torch.zeros(n, **u8)
+        self.n_keep_q = torch.zeros(1, **i32); self.n_keep_o = torch.zeros(P, **i32)
+        self.gamma_q = torch.zeros(P, **f32); self.gamma_o = torch.zeros(n, **f32)
+        self.w_seq = torch.zeros(n, **f32); self.H_next = torch.zeros(P, **f32)
+        self.order = torch.zeros(n, **i32); self.row_of = torch.zeros(n, **i32)
+        self.off_in_row = torch.zeros(n, **i32); self.row_fill = torch.zeros(n, **i32)
+        self.cu_seqlens = torch.zeros(n + 1, **i32); self.counts = torch.zeros(4, **i32)
+        self.status = torch.zeros(1, **i32)
+        self.loss_out = torch.zeros(5, **f32)
+        self.logp_out = torch.zeros(max(T_max, 1), **f32); self.lse_out = torch.zeros(max(T_max, 1), **f32)
+
+        self.prune_params = B.PruneParams(P, G, r_q, r_o, mode, reverse, 0, 0)
+        self.pack_params = B.PackParams(n, L_row, N_win, policy)
+        self.loss_params = B.LossParams(T_max, V, B.BF16 if dtype == "bf16" else B.F32, V, n, 0,
+                                        eps_lo, eps_hi, beta, temperature)
+        self.pack_ws_bytes = B.pack_workspace_bytes(self.pack_params)
+        self.pack_ws = torch.zeros(max(self.pack_ws_bytes, 16), dtype=torch.uint8, device=dev)
+        self.loss_ws_bytes = B.grpo_loss_workspace_bytes(self.loss_params)
+        self.loss_ws = torch.zeros(max(self.loss_ws_bytes, 16), dtype=torch.uint8, device=dev)
+
+    # -- inputs ------------------------------------------------------------------------------------
+    def set_batch(self, rewards, unit_len, loss_len, H_prev=None):
+        """Copy the per-batch host inputs (numpy / torch) to the device."""
+        self.rewards.copy_(torch.as_tensor(rewards, dtype=torch.float32).reshape(-1), non_blocking=True)
+        self.unit_len.copy_(torch.as_tensor(unit_len, dtype=torch.int32).reshape(-1), non_blocking=True)
+        self.loss_len.copy_(torch.as_tensor(loss_len, dtype=torch.int32).reshape(-1), non_blocking=True)
+        self.has_history = H_prev is not None
+        if self.has_history:
+            self.H_prev.copy_(torch.as_tensor(H_prev, dtype=torch.float32).reshape(-1), non_blocking=True)
+
+    # -- library calls -----------------------------------------------------------------------------
+    def advantages(self, rewards=None, adv=None, mean_abs_adv=None):
+        B.group_advantages(self.rewards if rewards is None else rewards, self.P, self.G,
+                           self.adv if adv is None else adv,
+                           self.mean_abs_adv if mean_abs_adv is None else mean_abs_adv,
+                           self.std_ddof, self.std_eps, self.status)
+
+    def prune(self, seed, step, u_q=None, u_o=None):
+        self.prune_params.seed, self.prune_params.step = seed, step
+        B.prune_and_rescale(self.prune_params, self.adv, self.mean_abs_adv,
+                            self.H_prev if self.has_history else None, u_q, u_o,
+                            self.cand_q, self.cand_o, self.keep_q, self.keep_o, self.n_keep_q, self.n_keep_o,
+                            self.gamma_q, self.gamma_o, self.w_seq, self.H_next, self.status)
+
+    def pack(self):
+        B.pack_prompts(self.pack_params, self.unit_len, self.keep_o, self.loss_len, self.order, self.row_of,
+                       self.off_in_row, self.row_fill, self.cu_seqlens, self.counts, self.pack_ws,
+                       self.pack_ws_bytes, self.status)
+
+    def prune_pack(self, seed=0, step=0, u_q=None, u_o=None):
+        self.advantages()
+        self.prune(seed, step, u_q, u_o)
+        self.pack()
+
+    def loss(self, logits, target, logp_old, logp_ref, dlogits=None, row_stride=None):
+        """Loss sweep over the retained tokens; the true token count is read on the device from the
+        packer's counts.  dlogits may be `logits` itself (in place) or None (forward only)."""
+        self.loss_params.row_stride = self.V if row_stride is None else row_stride
+        B.grpo_loss_fwd_bwd(self.loss_params, logits, target, logp_old, logp_ref, self.cu_seqlens,
+                            self.counts[3:4], self.adv, self.w_seq, self.order, dlogits, self.logp_out,
+                            self.lse_out, self.loss_out, self.loss_ws, self.loss_ws_bytes, self.status)
+
+    # -- results -----------------------------------------------------------------------------------
+    def n_tokens(self):
+        """Retained loss tokens T of the last prune_pack (synchronises)."""
+        return int(self.counts[3].item())
+
+    def prune_results(self):
+        names = ["adv", "mean_abs_adv", "cand_q", "cand_o", "keep_q", "keep_o", "n_keep_q", "n_keep_o",
+                 "gamma_q", "gamma_o", "w_seq", "H_next"]
+        return {k: getattr(self, k).cpu().numpy() for k in names}
+
+    def pack_results(self):
+        names = ["order", "row_of", "off_in_row", "row_fill", "cu_seqlens", "counts", "status"]
+        return {k: getattr(self, k).cpu().numpy() for k in names}

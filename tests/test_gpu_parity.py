@@ -1,0 +1,370 @@
+"""GPU-vs-oracle parity through the C ABI (run with -m gpu on a B200).
+
+Integer / byte / index outputs (candidate sets, masks, counts, packing layout, cu_seqlens) and the
+float outputs of the small steps (advantages, gamma, w_seq, H_next) must match bit for bit; the loss
+within 1e-4 relative; dlogits element-wise (see parity_util.assert_dlogits_close).
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2603_04135_b200 import synth
+from parity_util import (oracle_prune_pack, assert_prune_equal, assert_pack_equal, rows_to_f64, pick_rows,
+                         assert_dlogits_close, clip_decision_is_stable, oracle_forward_all_rows)
+
+pytestmark = pytest.mark.gpu
+
+
+def _step(w, T_max, **kw):
+    from paper_2603_04135_b200.step import DppoStep
+    args = dict(P=w.P, G=w.G, L_row=w.L_row, N_win=w.N_win, r_q=w.r_q, r_o=w.r_o, V=max(w.V, 1), dtype=w.dtype,
+                T_max=T_max, eps_lo=w.eps, eps_hi=w.eps, beta=w.beta)
+    args.update(kw)
+    return DppoStep(**args)
+
+
+# ------------------------------------------------------------------------------------------- steps 1-4
+@pytest.mark.parametrize("G", [1, 2, 3, 4, 5, 8, 16])
+@pytest.mark.parametrize("ddof", [0, 1])
+def test_advantages_bit_exact(G, ddof):
+    from paper_2603_04135_b200 import binding as B
+    rng = np.random.default_rng(G * 10 + ddof)
+    P = 257
+    r = (rng.random((P, G)) < rng.random((P, 1))).astype(np.float32)
+    r[5:40] = rng.normal(size=(35, G)).astype(np.float32)          # continuous rewards
+    r[40:50] = np.float32(0.7)                                     # all equal
+    for eps in (1e-6, 0.0):
+        want_adv, want_mabs = oracle.group_advantages(r, ddof=ddof, std_eps=eps)
+        d_r = torch.from_numpy(r).cuda()
+        adv = torch.full((P * G,), -1.0, device="cuda"); mabs = torch.full((P,), -1.0, device="cuda")
+        B.group_advantages(d_r, P, G, adv, mabs, ddof, eps)
+        assert np.array_equal(adv.cpu().numpy().view(np.uint32), want_adv.reshape(-1).view(np.uint32))
+        assert np.array_equal(mabs.cpu().numpy().view(np.uint32), want_mabs.view(np.uint32))
+
+
+@pytest.mark.parametrize("name", ["config0", "config1", "config2"])
+@pytest.mark.parametrize("history", [True, False])
+def test_prune_pack_bit_exact_on_configs(name, history):
+    w = synth.WORKLOADS[name]
+    for seed in range(6):
+        batch = synth.make_batch(w, seed)
+        ref = oracle_prune_pack(batch, w, seed, step=seed + 3, use_history=history)
+        st = _step(w, 1)
+        st.set_batch(batch.rewards, batch.unit_len, batch.loss_len, ref["H_prev"])
+        st.prune_pack(seed=seed, step=seed + 3)
+        assert_prune_equal(st.prune_results(), ref)
+        assert_pack_equal(st.pack_results(), ref["pack"], w.P * w.G)
+        assert st.pack_results()["status"][0] == 0
+
+
+def test_config2_sweep_bit_exact_and_density():
+    w = synth.WORKLOADS["config2"]
+    batch = synth.make_batch(w, 2)
+    naive_rows = None
+    for r_q in (0.0, 0.25, 0.5):
+        for r_o in (0.0, 0.25, 0.5):
+            for N_win in (4, 16, 64):
+                ref = oracle_prune_pack(batch, w, 2, step=11, r_q=r_q, r_o=r_o, N_win=N_win)
+                st = _step(w, 1, r_q=r_q, r_o=r_o, N_win=N_win)
+                st.set_batch(batch.rewards, batch.unit_len, batch.loss_len, ref["H_prev"])
+                st.prune_pack(seed=2, step=11)
+                assert_prune_equal(st.prune_results(), ref)
+                res = st.pack_results()
+                assert_pack_equal(res, ref["pack"], w.P * w.G)
+                n_units, n_rows, tokens, _ = (int(x) for x in res["counts"])
+                if n_units:
+                    density = tokens / (n_rows * w.L_row)
+                    kept = batch.unit_len[ref["prune"]["keep_o"].reshape(-1) == 1]
+                    padded = tokens / (n_units * kept.max())
+                    assert 0 < density <= 1 and 0 < padded <= 1
+
+
+def test_prune_explicit_draws_and_modes():
+    w = synth.WORKLOADS["config2"]
+    batch = synth.make_batch(w, 7)
+    rng = np.random.default_rng(3)
+    u_q = rng.random(w.P); u_o = rng.random((w.P, w.G))
+    u_q[:4] = [0.0, 0.25, 0.24999999999999997, 0.9999999999999999]      # exact boundary of u < r
+    for reverse in (False, True):
+        ref = oracle_prune_pack(batch, w, 0, 0, u_q=u_q, u_o=u_o, reverse=reverse)
+        st = _step(w, 1, reverse=int(reverse))
+        st.set_batch(batch.rewards, batch.unit_len, batch.loss_len, ref["H_prev"])
+        st.prune_pack(u_q=torch.from_numpy(u_q).cuda(), u_o=torch.from_numpy(u_o.reshape(-1)).cuda())
+        assert_prune_equal(st.prune_results(), ref)
+        assert_pack_equal(st.pack_results(), ref["pack"], w.P * w.G)
+
+
+def test_prune_many_seeds_matches_generator_stream():
+    # masks across many (seed, step) pairs: any difference in the counter-based generator shows up here
+    w = synth.scaled(synth.WORKLOADS["config2"], P=64, G=16, r_q=0.5, r_o=0.5)
+    batch = synth.make_batch(w, 1)
+    st = _step(w, 1)
+    for seed, step in [(0, 0), (1, 0), (0, 1), (2**40 + 5, 2**33 + 1), (2**64 - 1, 2**64 - 1), (123456789, 42)]:
+        ref = oracle_prune_pack(batch, w, seed, step)
+        st.set_batch(batch.rewards, batch.unit_len, batch.loss_len, ref["H_prev"])
+        st.prune_pack(seed=seed, step=step)
+        assert_prune_equal(st.prune_results(), ref)
+
+
+# ------------------------------------------------------------------------------------------- step 5
+@pytest.mark.parametrize("policy", [0, 1])
+def test_pack_random_streams(policy):
+    from paper_2603_04135_b200 import binding as B
+    rng = np.random.default_rng(policy)
+    for trial in range(40):
+        n = int(rng.integers(0, 300))
+        L = int(rng.integers(20, 400))
+        lens = rng.integers(1, L + 1, size=n).astype(np.int32)
+        if trial % 3 == 0 and n:
+            lens = np.minimum(lens, max(1, L // 8)).astype(np.int32)       # many units per row
+        keep = (rng.random(n) < 0.7).astype(np.uint8) if trial % 2 else None
+        loss_len = rng.integers(0, 50, size=n).astype(np.int32) if trial % 4 else None
+        N_win = int(rng.choice([1, 2, 4, 16, 31, 32, 33, 64, 1000]))
+        ref = oracle.pack_prompts(lens, L, N_win, keep=keep, loss_len=loss_len, best_fit=bool(policy))
+        got = _run_pack(B, lens, keep, loss_len, L, N_win, policy)
+        assert got["status"][0] == 0
+        assert_pack_equal(got, ref, n)
+
+
+def _run_pack(B, lens, keep, loss_len, L, N_win, policy):
+    n = len(lens)
+    i32 = dict(dtype=torch.int32, device="cuda")
+    d_len = torch.from_numpy(np.asarray(lens, dtype=np.int32)).cuda() if n else torch.zeros(1, **i32)
+    d_keep = torch.from_numpy(keep).cuda() if keep is not None else None
+    d_loss = torch.from_numpy(loss_len).cuda() if loss_len is not None else None
+    outs = {k: torch.full((max(n, 1),), 77, **i32) for k in ("order", "row_of", "off_in_row", "row_fill")}
+    cu = torch.full((n + 1,), 77, **i32); counts = torch.full((4,), 77, **i32); status = torch.zeros(1, **i32)
+    prm = B.PackParams(n, L, N_win, policy)
+    nbytes = B.pack_workspace_bytes(prm)
+    ws = torch.zeros(max(nbytes, 16), dtype=torch.uint8, device="cuda")
+    B.pack_prompts(prm, d_len, d_keep, d_loss, outs["order"], outs["row_of"], outs["off_in_row"], outs["row_fill"],
+                   cu, counts, ws, nbytes, status)
+    res = {k: v.cpu().numpy()[:n] for k, v in outs.items()}
+    res.update(cu_seqlens=cu.cpu().numpy(), counts=counts.cpu().numpy(), status=status.cpu().numpy())
+    return res
+
+
+def test_pack_dataset_scale_and_bad_length():
+    from paper_2603_04135_b200 import binding as B
+    rng = np.random.default_rng(5)
+    # a dataset-sized stream of prompt lengths (the paper packs its 7.5k-8.5k prompts at initialisation),
+    # L_max = the longest sample; larger than the shared-memory length cache
+    n = 8500
+    lens = np.clip(np.rint(np.exp(rng.normal(math.log(150), 0.6, size=n))), 16, 1024).astype(np.int32)
+    L = int(lens.max())
+    for N_win in (8, 64):
+        ref = oracle.pack_prompts(lens, L, N_win)
+        got = _run_pack(B, lens, None, None, L, N_win, 0)
+        assert_pack_equal(got, ref, n)
+    lens2 = np.array([5, 9, 30, 2], dtype=np.int32)
+    got = _run_pack(B, lens2, None, None, 20, 4, 0)
+    assert got["status"][0] == B.STATUS_BAD_LENGTH and (got["counts"] == 0).all()
+    got = _run_pack(B, lens2, np.array([1, 1, 0, 1], dtype=np.uint8), None, 20, 4, 0)
+    assert got["status"][0] == 0 and got["counts"][0] == 3
+
+
+# ------------------------------------------------------------------------------------------- steps 6-8
+def _loss_case(V, dtype, T, S, seed, sigma_noise=0.05, logit_sigma=2.0, tau=1.0, pad=0, in_place=False,
+               forward_only=False, n_tokens=None, beta=0.04, eps=(0.2, 0.2)):
+    """Runs dppo_grpo_loss_fwd_bwd on a random case and compares everything with the oracle."""
+    from paper_2603_04135_b200 import binding as B
+    w = synth.scaled(synth.WORKLOADS["config0"], V=V, dtype=dtype, logit_sigma=logit_sigma)
+    tok = synth.make_token_inputs(w, T, seed, device="cuda", sigma_old=sigma_noise, sigma_ref=2 * sigma_noise)
+    rng = np.random.default_rng(seed)
+    T_true = T if n_tokens is None else n_tokens
+    cuts = np.sort(rng.choice(np.arange(1, T_true), size=min(S - 1, T_true - 1), replace=False)) if T_true > 1 else []
+    cu = np.concatenate([[0], cuts, [T_true]]).astype(np.int32)
+    S_real = len(cu) - 1
+    S_max = S_real + 3                                               # padded tail repeats the total
+    cu_pad = np.concatenate([cu, np.full(S_max - S_real, T_true)]).astype(np.int32)
+    adv = rng.normal(size=S_max).astype(np.float32); adv[0] = 0.0
+    wseq = (rng.random(S_max) * 0.1).astype(np.float32)
+    seg_map = rng.permutation(S_max).astype(np.int32)
+    per16 = 4 if dtype == "f32" else 8                                # row stride must be a multiple of 16 bytes
+    stride = -(-(V + pad) // per16) * per16
+    pad = stride - V
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    buf = torch.zeros((T, stride), dtype=tdt, device="cuda")
+    buf[:, :V] = tok.logits
+    logits_before = buf.clone()
+    dl = buf if in_place else (None if forward_only else torch.full((T, stride), 7.0, dtype=tdt, device="cuda"))
+    prm = B.LossParams(T, V, B.BF16 if dtype == "bf16" else B.F32, stride, S_max, 0, eps[0], eps[1], beta, tau)
+    nbytes = B.grpo_loss_workspace_bytes(prm)
+    ws = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+    loss_out = torch.zeros(5, device="cuda"); logp_out = torch.zeros(T, device="cuda"); lse_out = torch.zeros(T, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ntd = torch.tensor([T_true], dtype=torch.int32, device="cuda") if n_tokens is not None else None
+    B.grpo_loss_fwd_bwd(prm, buf, tok.target, tok.logp_old, tok.logp_ref, torch.from_numpy(cu_pad).cuda(), ntd,
+                        torch.from_numpy(adv).cuda(), torch.from_numpy(wseq).cuda(), torch.from_numpy(seg_map).cuda(),
+                        dl, logp_out, lse_out, loss_out, ws, nbytes, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+
+    z = logits_before[:T_true, :V].to(torch.float64).cpu().numpy()
+    ref = oracle.grpo_loss(z, tok.target.cpu().numpy(), tok.logp_old.cpu().numpy(), tok.logp_ref.cpu().numpy(), cu,
+                           adv[seg_map][:S_real], wseq[seg_map][:S_real], eps[0], eps[1], beta, tau,
+                           want_dlogits=not forward_only)
+    lo = loss_out.cpu().numpy().astype(np.float64)
+    stable = clip_decision_is_stable(ref["rho"], eps[0], eps[1])
+    assert stable.all(), "test case sits on a clip boundary; change the seed"
+    assert abs(lo[0] - ref["loss"]) <= 1e-4 * abs(ref["loss"]) + 1e-7 * ref["abs_sum"]
+    assert abs(lo[0] - ref["loss"]) <= 1e-4 * ref["abs_sum"]
+    assert abs(lo[1] - ref["pg"]) <= 1e-4 * ref["abs_sum"] and abs(lo[2] - ref["kl"]) <= 1e-4 * max(ref["kl"], 1e-12) + 1e-9
+    assert abs(lo[3] - ref["clip_frac"]) < 1e-6 and lo[4] == T_true
+    tol = 1e-5 if dtype == "bf16" else 2e-6
+    assert np.abs(logp_out.cpu().numpy()[:T_true] - ref["logp"]).max() <= tol
+    assert np.abs(lse_out.cpu().numpy()[:T_true] - ref["lse"]).max() <= tol
+    if not forward_only:
+        got = dl[:T_true, :V].to(torch.float64).cpu().numpy()
+        assert_dlogits_close(got, ref["dlogits"], ref["g"], dtype)
+        if not in_place:
+            assert torch.equal(buf, logits_before)                   # inputs untouched
+            assert (dl[T_true:] == 7.0).all()                        # rows past T untouched
+            if pad:
+                assert (dl[:, V:] == 7.0).all()                      # padding columns untouched
+    return ref
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("V", [1, 3, 5, 8, 1000, 1024, 4099, 32768])
+def test_loss_small_vocab_shapes(dtype, V):
+    _loss_case(V, dtype, T=67, S=5, seed=V)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_loss_options(dtype):
+    V = 2056
+    _loss_case(V, dtype, T=50, S=4, seed=1, pad=8)                           # strided rows
+    _loss_case(V, dtype, T=50, S=4, seed=2, in_place=True)                   # dlogits aliases logits
+    _loss_case(V, dtype, T=50, S=4, seed=3, forward_only=True)
+    _loss_case(V, dtype, T=50, S=4, seed=4, n_tokens=37)                     # true T below T_max
+    _loss_case(V, dtype, T=50, S=4, seed=5, tau=1.7)
+    _loss_case(V, dtype, T=50, S=4, seed=6, beta=0.0, eps=(0.2, 0.5))        # decoupled clip range
+    _loss_case(V, dtype, T=1, S=1, seed=7)
+    _loss_case(V, dtype, T=300, S=300, seed=8)                               # one token per sequence
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_loss_all_clip_branches(dtype):
+    # log-ratio noise 0.3: clipped and unclipped tokens of both advantage signs, and A = 0
+    ref = _loss_case(1024, dtype, T=400, S=12, seed=21, sigma_noise=0.3, logit_sigma=1.0)
+    A, rho, cl = ref["A"], ref["rho"], ref["clipped"]
+    assert (cl & (A > 0) & (rho > 1.2)).any() and (cl & (A < 0) & (rho < 0.8)).any()
+    assert (~cl & (A > 0)).any() and (~cl & (A < 0)).any() and (A == 0).any()
+
+
+def test_loss_full_vocab_bf16_rows():
+    # Qwen3 vocabulary: rows of 151,936 bf16 (several tiles, 16-byte multiple), plus a ragged variant
+    _loss_case(151936, "bf16", T=24, S=3, seed=31)
+    _loss_case(151936 - 5, "bf16", T=9, S=2, seed=32, pad=5)
+    _loss_case(151936, "f32", T=6, S=2, seed=33)
+
+
+def test_loss_bad_target_and_empty():
+    from paper_2603_04135_b200 import binding as B
+    V, T = 512, 8
+    w = synth.scaled(synth.WORKLOADS["config0"], V=V)
+    tok = synth.make_token_inputs(w, T, 0, device="cuda")
+    tok.target[3] = V                                                 # outside the vocabulary
+    cu = torch.tensor([0, T], dtype=torch.int32, device="cuda")
+    adv = torch.ones(1, device="cuda"); ws_ = torch.ones(1, device="cuda")
+    prm = B.LossParams(T, V, B.F32, V, 1, 0, 0.2, 0.2, 0.04, 1.0)
+    nbytes = B.grpo_loss_workspace_bytes(prm)
+    ws = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+    dl = torch.full((T, V), 7.0, device="cuda"); loss_out = torch.zeros(5, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B.grpo_loss_fwd_bwd(prm, tok.logits, tok.target, tok.logp_old, tok.logp_ref, cu, None, adv, ws_, None, dl, None,
+                        None, loss_out, ws, nbytes, status)
+    assert status.item() == B.STATUS_BAD_TARGET
+    assert (dl[3] == 0).all() and (dl[2] != 7.0).all() and torch.isfinite(loss_out).all()
+    # T_max = 0: only the reduction runs
+    prm0 = B.LossParams(0, V, B.F32, V, 0, 0, 0.2, 0.2, 0.04, 1.0)
+    B.grpo_loss_fwd_bwd(prm0, None, None, None, None, None, None, None, None, None, None, None, None, loss_out, ws,
+                        nbytes, None)
+    assert (loss_out.cpu().numpy() == 0).all()
+    # host-side validation
+    for bad, code in [(B.LossParams(T, V, 7, V, 1, 0, 0.2, 0.2, 0.04, 1.0), B.ERR_UNSUPPORTED),
+                      (B.LossParams(T, V, B.F32, V - 1, 1, 0, 0.2, 0.2, 0.04, 1.0), B.ERR_BAD_SHAPE),
+                      (B.LossParams(T, V, B.F32, V + 1, 1, 0, 0.2, 0.2, 0.04, 1.0), B.ERR_MISALIGNED),
+                      (B.LossParams(T, V, B.F32, V, 1, 0, 0.2, 0.2, 0.04, 0.0), B.ERR_INVALID_ARG)]:
+        with pytest.raises(B.DppoError) as e:
+            B.grpo_loss_fwd_bwd(bad, tok.logits, tok.target, tok.logp_old, tok.logp_ref, cu, None, adv, ws_, None, dl,
+                                None, None, loss_out, ws, nbytes, status)
+        assert e.value.code == code
+    with pytest.raises(B.DppoError) as e:
+        B.grpo_loss_fwd_bwd(prm, tok.logits, tok.target, tok.logp_old, tok.logp_ref, cu, None, adv, ws_, None, dl, None,
+                            None, loss_out, ws, 16, status)
+    assert e.value.code == B.ERR_WORKSPACE_TOO_SMALL
+
+
+# ------------------------------------------------------------------------------------------- whole path
+def _run_config(w, seed, n_sample_rows, all_rows, use_history=True, in_place=False):
+    batch = synth.make_batch(w, seed)
+    ref = oracle_prune_pack(batch, w, seed, step=1, use_history=use_history)
+    pk = ref["pack"]
+    T = pk["counts"][3]
+    st = _step(w, T)
+    st.set_batch(batch.rewards, batch.unit_len, batch.loss_len, ref["H_prev"])
+    st.prune_pack(seed=seed, step=1)
+    assert_prune_equal(st.prune_results(), ref)
+    assert_pack_equal(st.pack_results(), pk, w.P * w.G)
+    assert st.n_tokens() == T
+    tok = synth.make_token_inputs(w, T, seed, device="cuda")
+    dl = tok.logits.clone() if in_place else torch.empty_like(tok.logits)
+    st.loss(dl if in_place else tok.logits, tok.target, tok.logp_old, tok.logp_ref, dl)
+    torch.cuda.synchronize()
+    assert st.status.item() == 0
+
+    order = np.asarray(pk["order"], dtype=np.int64)
+    adv_seg = ref["adv"].reshape(-1)[order]; w_seg = ref["prune"]["w_seq"].reshape(-1)[order]
+    cu = np.asarray(pk["cu_seqlens"])
+    target = tok.target.cpu().numpy(); lo = tok.logp_old.cpu().numpy(); lr = tok.logp_ref.cpu().numpy()
+    rows = pick_rows(cu, T, n_sample_rows, seed)
+    sub = oracle.grpo_loss(rows_to_f64(tok.logits, rows), target, lo, lr, cu, adv_seg, w_seg, w.eps, w.eps, w.beta,
+                           rows=rows, chunk=64)
+    stable = clip_decision_is_stable(sub["rho"], w.eps, w.eps)
+    assert stable.mean() > 0.99
+    got = rows_to_f64(dl, rows)
+    assert_dlogits_close(got, sub["dlogits"], sub["g"], w.dtype, clip_margin_ok=stable)
+    tol = 1e-5 if w.dtype == "bf16" else 2e-6
+    assert np.abs(st.logp_out.cpu().numpy()[rows] - sub["logp"]).max() <= tol
+    assert np.abs(st.lse_out.cpu().numpy()[rows] - sub["lse"]).max() <= tol
+    out = st.loss_out.cpu().numpy().astype(np.float64)
+    assert out[4] == T
+    if all_rows:
+        full = oracle_forward_all_rows(tok.logits, target, lo, lr, cu, adv_seg, w_seg, w.eps, w.eps, w.beta,
+                                       processes=0 if all_rows == "inline" else None)
+        assert np.abs(st.logp_out.cpu().numpy()[:T] - full["logp"]).max() <= tol
+        assert abs(out[0] - full["loss"]) <= 1e-4 * abs(full["loss"]), (out[0], full["loss"], full["abs_sum"])
+        assert abs(out[0] - full["loss"]) <= 1e-4 * full["abs_sum"]
+        assert abs(out[1] - full["pg"]) <= 1e-4 * full["abs_sum"]
+        assert abs(out[2] - full["kl"]) <= 1e-4 * full["kl"] + 1e-9
+        assert abs(out[3] - full["clip_frac"]) <= 2.0 / max(T, 1)
+    return T
+
+
+@pytest.mark.parametrize("history", [True, False])
+def test_config0_whole_path(history):
+    for seed in (0, 1, 2):
+        _run_config(synth.WORKLOADS["config0"], seed, 64, all_rows="inline", use_history=history)
+
+
+def test_config0_in_place():
+    _run_config(synth.WORKLOADS["config0"], 0, 64, all_rows="inline", in_place=True)
+
+
+def test_config1_whole_path():
+    T = _run_config(synth.WORKLOADS["config1"], 1, 192, all_rows="pool")
+    assert T > 10000
+
+
+def test_config3_full_size_sampled_rows():
+    # the benchmark's launch configuration: in place, full vocabulary, every retained token
+    free, _ = torch.cuda.mem_get_info()
+    if free < 90e9:
+        pytest.skip("needs ~70 GB of free device memory")
+    T = _run_config(synth.WORKLOADS["config3"], 3, 384, all_rows=False, in_place=True)
+    assert T > 60000
