@@ -320,7 +320,7 @@ def token_terms(logp, logp_old, logp_ref, A, eps_lo, eps_hi, beta):
     surr = np.where(clipped, s2, s1)
     j = surr - beta * kl
     dj = np.where(clipped, 0.0, A * rho) + beta * (rho_hat - 1.0)
-    return dict(rho=rho, kl=kl, surr=surr, j=j, dj=dj, clipped=clipped)
+    return dict(rho=rho, rho_hat=rho_hat, kl=kl, surr=surr, j=j, dj=dj, clipped=clipped)
 
 
 def grpo_loss(logits, target, logp_old, logp_ref, cu_seqlens, adv_seg, w_seg,
@@ -361,7 +361,7 @@ def grpo_loss(logits, target, logp_old, logp_ref, cu_seqlens, adv_seg, w_seg,
         loss=-math.fsum(W * tt["j"]), pg=-math.fsum(W * tt["surr"]), kl=math.fsum(W * tt["kl"]),
         abs_sum=math.fsum(np.abs(W * tt["j"])),
         clip_frac=(float(tt["clipped"].sum()) / n) if n else 0.0, T=T,
-        logp=logp, lse=lse, g=g, rho=tt["rho"], clipped=tt["clipped"], W=W, A=A, seg=seg)
+        logp=logp, lse=lse, g=g, rho=tt["rho"], rho_hat=tt["rho_hat"], clipped=tt["clipped"], W=W, A=A, seg=seg)
     if want_dlogits:
         dl = np.empty((n, logits.shape[1]), dtype=np.float64)
         for a in range(0, n, chunk):

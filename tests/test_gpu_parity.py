@@ -13,7 +13,7 @@ import torch
 import oracle
 from paper_2603_04135_b200 import synth
 from parity_util import (oracle_prune_pack, assert_prune_equal, assert_pack_equal, rows_to_f64, pick_rows,
-                         assert_dlogits_close, clip_decision_is_stable, oracle_forward_all_rows)
+                         assert_dlogits_close, clip_decision_is_stable, oracle_forward_all_rows, LOGP_TOL)
 
 pytestmark = pytest.mark.gpu
 
@@ -214,12 +214,12 @@ def _loss_case(V, dtype, T, S, seed, sigma_noise=0.05, logit_sigma=2.0, tau=1.0,
     assert abs(lo[0] - ref["loss"]) <= 1e-4 * ref["abs_sum"]
     assert abs(lo[1] - ref["pg"]) <= 1e-4 * ref["abs_sum"] and abs(lo[2] - ref["kl"]) <= 1e-4 * max(ref["kl"], 1e-12) + 1e-9
     assert abs(lo[3] - ref["clip_frac"]) < 1e-6 and lo[4] == T_true
-    tol = 1e-5 if dtype == "bf16" else 2e-6
+    tol = LOGP_TOL[dtype]
     assert np.abs(logp_out.cpu().numpy()[:T_true] - ref["logp"]).max() <= tol
     assert np.abs(lse_out.cpu().numpy()[:T_true] - ref["lse"]).max() <= tol
     if not forward_only:
         got = dl[:T_true, :V].to(torch.float64).cpu().numpy()
-        assert_dlogits_close(got, ref["dlogits"], ref["g"], dtype)
+        assert_dlogits_close(got, ref, dtype, beta)
         if not in_place:
             assert torch.equal(buf, logits_before)                   # inputs untouched
             assert (dl[T_true:] == 7.0).all()                        # rows past T untouched
@@ -328,8 +328,8 @@ def _run_config(w, seed, n_sample_rows, all_rows, use_history=True, in_place=Fal
     stable = clip_decision_is_stable(sub["rho"], w.eps, w.eps)
     assert stable.mean() > 0.99
     got = rows_to_f64(dl, rows)
-    assert_dlogits_close(got, sub["dlogits"], sub["g"], w.dtype, clip_margin_ok=stable)
-    tol = 1e-5 if w.dtype == "bf16" else 2e-6
+    assert_dlogits_close(got, sub, w.dtype, w.beta, rows_ok=stable)
+    tol = LOGP_TOL[w.dtype]
     assert np.abs(st.logp_out.cpu().numpy()[rows] - sub["logp"]).max() <= tol
     assert np.abs(st.lse_out.cpu().numpy()[rows] - sub["lse"]).max() <= tol
     out = st.loss_out.cpu().numpy().astype(np.float64)
