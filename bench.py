@@ -1,0 +1,325 @@
+#!/usr/bin/env python
+"""Benchmark of the pruned-GRPO hot path: valid tokens/s and fraction of the HBM roofline.
+
+One step = one pass of the whole path over one synthetic batch: group advantages -> candidate sets,
+pruning masks, rescaling -> Dense Prompt Packing -> fused loss sweep (forward + dlogits).  The
+workload is the large fused-loss configuration (32 prompts x 8 completions, 64-1024 response tokens,
+bf16 logits over a 151,936-token vocabulary, pruning probabilities 0.25 / 0.25).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+N > 1 is launched with torch.distributed.run, one rank per GPU; every rank works on its own batch
+(no data-path collective) and rank 0 reports the whole-job throughput with the max time over ranks.
+`--impl reference` times the float64 CPU oracle on the host cores instead (rank 0 only).
+"""
+import argparse
+import json
+import multiprocessing as mp
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2603_04135_b200 import synth
+
+METRIC = "valid tokens/sec of pruned GRPO loss fwd+bwd"
+UNIT = "tokens/s"
+WORKLOAD = "config3"
+WORKLOAD_TEXT = WORKLOAD + ": P=32 G=8, response 64-1024 tokens, V=151936 bf16 logits, r_q=r_o=0.25, L_row=8192, N_win=16"
+
+
+def measured_peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+# --------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index = gpu_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            time.sleep(0.3)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, smax, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1])); smax.append(float(parts[2])); power.append(float(parts[3]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------------------- oracle legs
+def oracle_prune_pack(w, batch, seed, step):
+    import oracle
+    adv, mabs = oracle.group_advantages(batch.rewards)
+    H_prev = oracle.group_advantages(batch.rewards_prev)[1]
+    pr = oracle.prune_and_rescale(adv, mabs, H_prev, w.r_q, w.r_o, seed=seed, step=step)
+    pk = oracle.pack_prompts(batch.unit_len, w.L_row, w.N_win, keep=pr["keep_o"].reshape(-1), loss_len=batch.loss_len)
+    order = np.asarray(pk["order"], dtype=np.int64)
+    return pk, adv.reshape(-1)[order], pr["w_seq"].reshape(-1)[order]
+
+
+def oracle_sample_tasks(w, tok_cpu, rows, pk, adv_seg, w_seg, rows_per_task):
+    is_bf16 = tok_cpu.logits.dtype == torch.bfloat16
+    T = pk["counts"][3]
+    target = np.zeros(T, dtype=np.int64); lo = np.zeros(T); lr = np.zeros(T)
+    target[rows] = tok_cpu.target.numpy(); lo[rows] = tok_cpu.logp_old.numpy(); lr[rows] = tok_cpu.logp_ref.numpy()
+    cu = np.asarray(pk["cu_seqlens"])
+    tasks = []
+    for a in range(0, len(rows), rows_per_task):
+        b = min(len(rows), a + rows_per_task)
+        blk = tok_cpu.logits[a:b]
+        chunk = blk.view(torch.int16).numpy().view(np.uint16) if is_bf16 else blk.numpy()
+        tasks.append((chunk, is_bf16, rows[a:b], target, lo, lr, cu, adv_seg, w_seg, w.eps, w.eps, w.beta, 1.0))
+    return tasks
+
+
+def time_oracle(w, seed, n_rows, steps, warmup, pool, cores):
+    """Times the oracle as it stands: steps 1-5 on the full batch, then loss forward + backward on a
+    bounded sample of n_rows token rows spread over `cores` worker processes."""
+    from oracle import rows_worker
+    batch = synth.make_batch(w, seed)
+    pk, adv_seg, w_seg = oracle_prune_pack(w, batch, seed, 1)
+    T = pk["counts"][3]
+    rng = np.random.default_rng(seed)
+    rows = np.sort(rng.choice(T, size=min(n_rows, T), replace=False))
+    tok = synth.make_token_inputs(w, len(rows), seed, device="cpu", rows_per_chunk=64)
+    tasks = oracle_sample_tasks(w, tok, rows, pk, adv_seg, w_seg, max(1, len(rows) // (cores * 2)))
+    times = []
+    for it in range(warmup + steps):
+        t0 = time.perf_counter()
+        oracle_prune_pack(w, batch, seed, 1)
+        done = sum(r[2] for r in pool.map(rows_worker.fwd_bwd_rows, tasks))
+        dt = time.perf_counter() - t0
+        assert done == len(rows)
+        if it >= warmup:
+            times.append(dt)
+    return len(rows), T, times
+
+
+def run_reference(args):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return 0
+    w = synth.WORKLOADS[WORKLOAD]
+    cores = min(os.cpu_count() or 1, 64)
+    with mp.get_context("spawn").Pool(cores) as pool:
+        n_rows, T, times = time_oracle(w, 3, args.ref_rows, args.steps, args.warmup, pool, cores)
+    ms = 1e3 * sum(times) / len(times)
+    value = n_rows / (ms / 1e3)
+    sample = "%d of the batch's %d retained token rows per step (fwd+bwd, V=%d) plus steps 1-5 on the full batch" % (
+        n_rows, T, w.V)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD_TEXT + "; CPU oracle on a row sample", "rows_per_step": n_rows},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+# --------------------------------------------------------------------------------------- ours
+def run_ours(args):
+    from paper_2603_04135_b200.step import DppoStep      # raises if libdppo.so is missing: no fallback
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (the library has no CPU path)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+
+    # CPU-baseline pool first (spawned workers; never forked after CUDA is up)
+    pool, cores = None, 0
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cores = min(os.cpu_count() or 1, 64)
+        pool = mp.get_context("spawn").Pool(cores)
+
+    w = synth.WORKLOADS[WORKLOAD]
+    seed = 3 + rank                                       # every rank has its own batch (data parallel)
+    batch = synth.make_batch(w, seed)
+
+    T_cap = int(batch.loss_len.sum())                     # unpruned upper bound of loss tokens
+    st = DppoStep(w.P, w.G, w.L_row, w.N_win, w.r_q, w.r_o, w.V, w.dtype, T_cap, w.eps, w.eps, w.beta, device=dev)
+    # history scores: the previous epoch's mean |A| per prompt (Eq. 16), produced by the library itself
+    prev = torch.from_numpy(batch.rewards_prev.reshape(-1).copy()).to(dev)
+    H_prev = torch.zeros(w.P, device=dev); scratch = torch.zeros(w.P * w.G, device=dev)
+    st.advantages(rewards=prev, adv=scratch, mean_abs_adv=H_prev)
+    st.set_batch(batch.rewards, batch.unit_len, batch.loss_len, H_prev)
+    st.prune_pack(seed=seed, step=1)
+    T = st.n_tokens()
+    assert st.status.item() == 0 and 0 < T <= T_cap
+    free, _ = torch.cuda.mem_get_info()
+    need = 2 * T * w.V * 2 + (4 << 30)
+    if need > free:
+        raise RuntimeError("not enough device memory for %s: need %.1f GB, free %.1f GB" % (WORKLOAD, need / 1e9, free / 1e9))
+    tok = synth.make_token_inputs(w, T, seed, device=dev)
+    dlogits = torch.empty_like(tok.logits)
+
+    def one_step(ev0=None, ev1=None):
+        st.prune_pack(seed=seed, step=1)
+        if ev0 is not None:
+            ev0.record()
+        st.loss(tok.logits, tok.target, tok.logp_old, tok.logp_ref, dlogits)
+        if ev1 is not None:
+            ev1.record()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        one_step()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    k_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for i in range(args.steps):
+        one_step(*k_ev[i])
+    e1.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = e0.elapsed_time(e1)
+    loss_ms = sum(a.elapsed_time(b) for a, b in k_ev) / args.steps
+    assert st.status.item() == 0
+    loss_value = float(st.loss_out[0].item())
+
+    # ---- end to end: host buffers in, loss scalars out, through DppoStep.step_from_host
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    host_tok = {k: torch.empty(getattr(tok, k).shape, dtype=getattr(tok, k).dtype, pin_memory=True)
+                for k in ("logits", "target", "logp_old", "logp_ref")}
+    for k in host_tok:
+        host_tok[k].copy_(getattr(tok, k))
+    dev_tok = {k: getattr(tok, k) for k in host_tok}
+    host_batch = {"rewards": torch.from_numpy(batch.rewards.reshape(-1).copy()).pin_memory(),
+                  "unit_len": torch.from_numpy(batch.unit_len.copy()).pin_memory(),
+                  "loss_len": torch.from_numpy(batch.loss_len.copy()).pin_memory(),
+                  "H_prev": H_prev.cpu().pin_memory()}
+    st.step_from_host(host_batch, host_tok, dev_tok, seed, 1, dlogits)          # warm-up
+    barrier()
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(e2e_steps):
+        out_host, h2d, d2h = st.step_from_host(host_batch, host_tok, dev_tok, seed, 1, dlogits)
+    t1.record()
+    barrier()
+    e2e_ms = t0.elapsed_time(t1) / e2e_steps
+    del host_tok
+
+    # ---- max over ranks, totals over ranks
+    stats = torch.tensor([total_ms, loss_ms, e2e_ms], dtype=torch.float64, device=dev)
+    tokens = torch.tensor([float(T)], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(stats, op=dist.ReduceOp.MAX)
+        dist.all_reduce(tokens, op=dist.ReduceOp.SUM)
+    total_ms, loss_ms, e2e_ms = (float(x) for x in stats.tolist())
+    T_all = float(tokens.item())
+
+    if rank == 0:
+        ms_per_step = total_ms / args.steps
+        peak, peak_kind = measured_peaks()
+        bytes_per_token = w.V * 2 + w.V * 2               # read the bf16 logits once, write bf16 dlogits once
+        achieved = T * bytes_per_token / (loss_ms / 1e3) / 1e9
+        line = {
+            "metric": METRIC, "value": T_all / (ms_per_step / 1e3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD_TEXT, "valid_tokens_per_gpu": T,
+                       "sequences_retained": int(st.counts[0].item()),
+                       "arithmetic": "bf16 logits and dlogits, f32 row sums, f64 per-token scalar stage and loss sum",
+                       "l2": "inputs (%.1f GB) far larger than L2; no flush" % (T * w.V * 2 / 1e9),
+                       "parallelism": "dp%d, independent batches" % world},
+            "clocks": clocks,
+            "e2e": {"value": T_all / (e2e_ms / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+            "gpu_launches": 5 * args.steps,
+            "roofline": {"bound": "hbm", "kernel": "grpo loss sweep (rows kernel + its 1-block reduction)",
+                         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "peak_source": peak_kind + " STREAM-style copy", "kernel_ms": loss_ms,
+                         "algorithmic_bytes_per_token": bytes_per_token, "traffic": None},
+            "loss": loss_value,
+        }
+        if pool is not None:
+            n_rows, _, times = time_oracle(w, seed, args.ref_rows, 1, 0, pool, cores)
+            pool.close(); pool.join()
+            line["cpu_baseline"] = {"value": n_rows / times[0], "unit": UNIT, "cores": cores, "kind": "oracle",
+                                    "sample": "%d of %d retained token rows, fwd+bwd, plus steps 1-5 on the full batch"
+                                              % (n_rows, T)}
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--ref-rows", type=int, default=2048, help="token rows in the oracle's timed sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "ours" and args.warmup < 3:
+        args.warmup = 3
+    sys.exit(run_reference(args) if args.impl == "reference" else run_ours(args))
+
+
+if __name__ == "__main__":
+    main()

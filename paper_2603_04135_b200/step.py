@@ -102,6 +102,31 @@ class DppoStep:
                             self.counts[3:4], self.adv, self.w_seq, self.order, dlogits, self.logp_out,
                             self.lse_out, self.loss_out, self.loss_ws, self.loss_ws_bytes, self.status)
 
+    def step_from_host(self, batch_host, token_host, dev_tokens, seed=0, step=0, dlogits=None):
+        """The whole path from HOST buffers: copies the batch inputs and the token inputs (logits, targets,
+        old / reference log-probs; pinned host tensors) to the device, runs advantages -> prune -> pack ->
+        loss sweep, and returns the five loss scalars on the host (this synchronises).
+
+        batch_host: dict with pinned tensors rewards, unit_len, loss_len and optionally H_prev.
+        token_host / dev_tokens: dicts with logits, target, logp_old, logp_ref (host source, device
+        destination).  Returns (loss_out as a host tensor, bytes copied host->device, bytes device->host).
+        """
+        h2d = 0
+        for name in ("rewards", "unit_len", "loss_len"):
+            getattr(self, name).copy_(batch_host[name], non_blocking=True)
+            h2d += batch_host[name].numel() * batch_host[name].element_size()
+        self.has_history = batch_host.get("H_prev") is not None
+        if self.has_history:
+            self.H_prev.copy_(batch_host["H_prev"], non_blocking=True)
+            h2d += batch_host["H_prev"].numel() * 4
+        for name in ("logits", "target", "logp_old", "logp_ref"):
+            dev_tokens[name].copy_(token_host[name], non_blocking=True)
+            h2d += token_host[name].numel() * token_host[name].element_size()
+        self.prune_pack(seed, step)
+        self.loss(dev_tokens["logits"], dev_tokens["target"], dev_tokens["logp_old"], dev_tokens["logp_ref"], dlogits)
+        out = self.loss_out.cpu()                         # device -> host read of the result; synchronises
+        return out, h2d, out.numel() * 4
+
     # -- results -----------------------------------------------------------------------------------
     def n_tokens(self):
         """Retained loss tokens T of the last prune_pack (synchronises)."""
