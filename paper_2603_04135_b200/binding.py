@@ -40,7 +40,7 @@ class PackParams(ctypes.Structure):
 
 class LossParams(ctypes.Structure):
     _fields_ = [("T_max", ctypes.c_int64), ("V", ctypes.c_int32), ("dtype", ctypes.c_int32),
-                ("row_stride", ctypes.c_int64), ("S_max", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("row_stride", ctypes.c_int64), ("S_max", ctypes.c_int32), ("variant", ctypes.c_int32),
                 ("eps_lo", ctypes.c_double), ("eps_hi", ctypes.c_double), ("beta", ctypes.c_double),
                 ("temperature", ctypes.c_double)]
 

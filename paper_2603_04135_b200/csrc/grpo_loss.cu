@@ -12,101 +12,11 @@
 
 namespace dppo {
 
-// ---- 16-byte vectors ------------------------------------------------------------------------------
-template <bool kBf16> struct Elems;
-template <> struct Elems<true> {
-    static constexpr int kPerVec = 8;
-    static __device__ __forceinline__ void unpack(const uint4& q, float (&f)[8]) {
-        f[0] = __uint_as_float(q.x << 16); f[1] = __uint_as_float(q.x & 0xffff0000u);
-        f[2] = __uint_as_float(q.y << 16); f[3] = __uint_as_float(q.y & 0xffff0000u);
-        f[4] = __uint_as_float(q.z << 16); f[5] = __uint_as_float(q.z & 0xffff0000u);
-        f[6] = __uint_as_float(q.w << 16); f[7] = __uint_as_float(q.w & 0xffff0000u);
-    }
-    static __device__ __forceinline__ uint4 pack(const float (&f)[8]) {
-        uint4 q;
-        __nv_bfloat162 a = __floats2bfloat162_rn(f[0], f[1]), b = __floats2bfloat162_rn(f[2], f[3]);
-        __nv_bfloat162 c = __floats2bfloat162_rn(f[4], f[5]), d = __floats2bfloat162_rn(f[6], f[7]);
-        q.x = *reinterpret_cast<uint32_t*>(&a); q.y = *reinterpret_cast<uint32_t*>(&b);
-        q.z = *reinterpret_cast<uint32_t*>(&c); q.w = *reinterpret_cast<uint32_t*>(&d);
-        return q;
-    }
-    static __device__ __forceinline__ float load1(const void* row, int v) {
-        return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(row)[v]);
-    }
-    static __device__ __forceinline__ void store1(void* row, int v, float x) {
-        reinterpret_cast<__nv_bfloat16*>(row)[v] = __float2bfloat16_rn(x);
-    }
-};
-template <> struct Elems<false> {
-    static constexpr int kPerVec = 4;
-    static __device__ __forceinline__ void unpack(const uint4& q, float (&f)[4]) {
-        f[0] = __uint_as_float(q.x); f[1] = __uint_as_float(q.y);
-        f[2] = __uint_as_float(q.z); f[3] = __uint_as_float(q.w);
-    }
-    static __device__ __forceinline__ uint4 pack(const float (&f)[4]) {
-        return make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]), __float_as_uint(f[3]));
-    }
-    static __device__ __forceinline__ float load1(const void* row, int v) {
-        return reinterpret_cast<const float*>(row)[v];
-    }
-    static __device__ __forceinline__ void store1(void* row, int v, float x) {
-        reinterpret_cast<float*>(row)[v] = x;
-    }
-};
-
-// ---- scalar stage (one thread per row) -----------------------------------------------------------
-// ref2/sum2: the row's sum of 2^(z c) is sum2 * 2^ref2 with c = log2(e)/temperature as used in pass 1.
-__device__ RowScalars row_scalar_stage(const LossArgs& a, long long t, float ref2, float sum2) {
-    RowScalars out;
-    const double lse2 = (double)ref2 + log2((double)sum2);           // base-2 log-sum-exp of z c
-    const double lse = lse2 * 0.6931471805599453;                    // natural log-sum-exp of z / temperature
-    out.lse2_hi = (float)lse2;
-    out.lse2_lo = (float)(lse2 - (double)out.lse2_hi);
-    out.g_over_tau = 0.0f;
-    out.valid = false;
-    const int y = a.target[t];
-    RowTerms terms = {0.0, 0.0, 0.0, 0.0};
-    float logp_f = 0.0f;
-    // sequence of this token: the last s with cu_seqlens[s] <= t
-    int lo = 0, hi = a.S_max;                                        // invariant: cu[lo] <= t (checked below)
-    while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if ((long long)a.cu_seqlens[mid] <= t) lo = mid; else hi = mid;
-    }
-    const long long seg_lo = a.cu_seqlens[lo], seg_hi = a.cu_seqlens[lo + 1];
-    if (a.S_max < 1 || t < seg_lo || t >= seg_hi) {
-        set_status(a.status, DPPO_STATUS_BAD_SEGMENTS);
-    } else if (y < 0 || y >= a.V) {
-        set_status(a.status, DPPO_STATUS_BAD_TARGET);
-    } else {
-        const int idx = a.seg_map ? a.seg_map[lo] : lo;
-        const double A = (double)a.adv[idx];
-        const double W = (double)a.w[idx] / (double)(seg_hi - seg_lo);
-        const double zy = (double)(a.bf16 ? Elems<true>::load1(a.logits + t * a.row_bytes, y)
-                                          : Elems<false>::load1(a.logits + t * a.row_bytes, y)) / a.temperature;
-        const double logp = zy - lse;
-        const double rho = exp(logp - (double)a.logp_old[t]);
-        const double d = (double)a.logp_ref[t] - logp;
-        const double rho_hat = exp(d);
-        const double kl = rho_hat - d - 1.0;
-        const double s1 = rho * A;
-        const double s2 = fmin(fmax(rho, 1.0 - a.eps_lo), 1.0 + a.eps_hi) * A;
-        const bool clipped = s2 < s1;
-        const double surr = clipped ? s2 : s1;
-        const double dj = (clipped ? 0.0 : A * rho) + a.beta * (rho_hat - 1.0);
-        terms.loss = -W * (surr - a.beta * kl);
-        terms.pg = -W * surr;
-        terms.kl = W * kl;
-        terms.clipped = clipped ? 1.0 : 0.0;
-        out.g_over_tau = (float)(-W * dj / a.temperature);
-        out.valid = true;
-        logp_f = (float)logp;
-    }
-    a.terms[t] = terms;
-    if (a.logp_out) a.logp_out[t] = logp_f;
-    if (a.lse_out) a.lse_out[t] = (float)lse;
-    return out;
-}
+// ---- kernel choice for variant 0 (from measurements on B200 at V = 151,936) --------------------------
+constexpr int kClusterMinV = 16384;                 // shorter rows: the general kernel's second pass hits L1/L2
+constexpr int kClusterAuto = 4;                     // smallest cluster tried first
+constexpr int kClusterThreads = 256;
+constexpr size_t kClusterMaxSlice = 76 * 1024;      // slice bytes per CTA: keeps three CTAs resident per SM
 
 // ---- general kernel --------------------------------------------------------------------------------
 constexpr int kRowThreads = 512;
@@ -267,6 +177,7 @@ extern "C" int dppo_grpo_loss_fwd_bwd(const dppo_loss_params* p, const void* log
     if (p->row_stride < p->V) return fail(DPPO_ERR_BAD_SHAPE, "grpo_loss: row_stride %lld < V %d", (long long)p->row_stride, p->V);
     if (!(p->temperature > 0.0) || !(p->eps_lo >= 0.0) || !(p->eps_hi >= 0.0) || !(p->beta == p->beta))
         return fail(DPPO_ERR_INVALID_ARG, "grpo_loss: temperature must be > 0, eps >= 0, beta a number");
+    if (p->variant < 0) return fail(DPPO_ERR_INVALID_ARG, "grpo_loss: variant %d", p->variant);
     if (p->T_max >= ((int64_t)1 << 31)) return fail(DPPO_ERR_BAD_SHAPE, "grpo_loss: T_max must be below 2^31");
     if (!loss_out) return fail(DPPO_ERR_INVALID_ARG, "grpo_loss: NULL loss_out");
     const size_t esize = p->dtype == DPPO_BF16 ? 2 : 4;
@@ -293,7 +204,22 @@ extern "C" int dppo_grpo_loss_fwd_bwd(const dppo_loss_params* p, const void* log
     a.scale2 = (float)(1.4426950408889634 / p->temperature);
     cudaStream_t s = (cudaStream_t)stream;
     if (p->T_max > 0) {
-        const int rc = launch_rows_general(a, s);
+        // variant: 0 picks the kernel from the shape; 1 forces the general kernel; C*10000 + threads
+        // forces the cluster kernel with C CTAs per row (a tuning aid; unsupported shapes are an error)
+        int rc;
+        if (p->variant == 1) {
+            rc = launch_rows_general(a, s);
+        } else if (p->variant >= 10000) {
+            rc = launch_rows_cluster(a, p->variant / 10000, p->variant % 10000, s);
+        } else {
+            rc = DPPO_ERR_UNSUPPORTED;
+            if (a.bf16 && p->V >= kClusterMinV) {
+                const int nvec = p->V >> 3;
+                for (int C = kClusterAuto; C <= 8 && rc == DPPO_ERR_UNSUPPORTED; C *= 2)
+                    if ((size_t)((nvec + C - 1) / C) * 16 <= kClusterMaxSlice) rc = launch_rows_cluster(a, C, kClusterThreads, s);
+            }
+            if (rc == DPPO_ERR_UNSUPPORTED) rc = launch_rows_general(a, s);
+        }
         if (rc != DPPO_OK) return rc;
     }
     return launch_loss_reduce(a, loss_out, s);

@@ -39,9 +39,154 @@ struct LossArgs {
     float scale2;            // log2(e) / temperature as the f32 both passes multiply by
 };
 
-__device__ RowScalars row_scalar_stage(const LossArgs& a, long long t, float ref2, float sum2);
+// ---- 16-byte vectors ------------------------------------------------------------------------------
+template <bool kBf16> struct Elems;
+template <> struct Elems<true> {
+    static constexpr int kPerVec = 8;
+    static __device__ __forceinline__ void unpack(const uint4& q, float (&f)[8]) {
+        f[0] = __uint_as_float(q.x << 16); f[1] = __uint_as_float(q.x & 0xffff0000u);
+        f[2] = __uint_as_float(q.y << 16); f[3] = __uint_as_float(q.y & 0xffff0000u);
+        f[4] = __uint_as_float(q.z << 16); f[5] = __uint_as_float(q.z & 0xffff0000u);
+        f[6] = __uint_as_float(q.w << 16); f[7] = __uint_as_float(q.w & 0xffff0000u);
+    }
+    static __device__ __forceinline__ uint4 pack(const float (&f)[8]) {
+        uint4 q;
+        __nv_bfloat162 a = __floats2bfloat162_rn(f[0], f[1]), b = __floats2bfloat162_rn(f[2], f[3]);
+        __nv_bfloat162 c = __floats2bfloat162_rn(f[4], f[5]), d = __floats2bfloat162_rn(f[6], f[7]);
+        q.x = *reinterpret_cast<uint32_t*>(&a); q.y = *reinterpret_cast<uint32_t*>(&b);
+        q.z = *reinterpret_cast<uint32_t*>(&c); q.w = *reinterpret_cast<uint32_t*>(&d);
+        return q;
+    }
+    static __device__ __forceinline__ float load1(const void* row, int v) {
+        return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(row)[v]);
+    }
+    static __device__ __forceinline__ void store1(void* row, int v, float x) {
+        reinterpret_cast<__nv_bfloat16*>(row)[v] = __float2bfloat16_rn(x);
+    }
+};
+template <> struct Elems<false> {
+    static constexpr int kPerVec = 4;
+    static __device__ __forceinline__ void unpack(const uint4& q, float (&f)[4]) {
+        f[0] = __uint_as_float(q.x); f[1] = __uint_as_float(q.y);
+        f[2] = __uint_as_float(q.z); f[3] = __uint_as_float(q.w);
+    }
+    static __device__ __forceinline__ uint4 pack(const float (&f)[4]) {
+        return make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]), __float_as_uint(f[3]));
+    }
+    static __device__ __forceinline__ float load1(const void* row, int v) {
+        return reinterpret_cast<const float*>(row)[v];
+    }
+    static __device__ __forceinline__ void store1(void* row, int v, float x) {
+        reinterpret_cast<float*>(row)[v] = x;
+    }
+};
+
+// ---- scalar stage -------------------------------------------------------------------------------------
+// What one token row needs besides its logits; gathered once per row (one thread, or one warp ahead of
+// time while the row is still in flight).
+struct RowInputs {
+    double A;                // advantage of the token's sequence
+    double W;                // w[seq] / |o_seq|
+    double zy;               // z[y] / temperature
+    double logp_old, logp_ref;
+    int y;
+    int state;               // 0 ok, else the dppo_status to report (row adds nothing, dlogits zero)
+};
+
+__device__ __forceinline__ void row_inputs_from_segment(const LossArgs& a, long long t, int seg, RowInputs& in) {
+    in.A = in.W = in.zy = in.logp_old = in.logp_ref = 0.0;
+    in.y = a.target[t];
+    in.state = 0;
+    const long long seg_lo = a.cu_seqlens[seg], seg_hi = a.cu_seqlens[seg + 1];
+    if (a.S_max < 1 || t < seg_lo || t >= seg_hi) { in.state = DPPO_STATUS_BAD_SEGMENTS; return; }
+    if (in.y < 0 || in.y >= a.V) { in.state = DPPO_STATUS_BAD_TARGET; return; }
+    const int idx = a.seg_map ? a.seg_map[seg] : seg;
+    in.A = (double)a.adv[idx];
+    in.W = (double)a.w[idx] / (double)(seg_hi - seg_lo);
+    in.zy = (double)(a.bf16 ? Elems<true>::load1(a.logits + t * a.row_bytes, in.y)
+                            : Elems<false>::load1(a.logits + t * a.row_bytes, in.y)) / a.temperature;
+    in.logp_old = (double)a.logp_old[t];
+    in.logp_ref = (double)a.logp_ref[t];
+}
+
+// One thread: binary search for the last s with cu_seqlens[s] <= t, then the gather.
+__device__ __forceinline__ void row_gather(const LossArgs& a, long long t, RowInputs& in) {
+    int lo = 0, hi = a.S_max;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if ((long long)a.cu_seqlens[mid] <= t) lo = mid; else hi = mid;
+    }
+    row_inputs_from_segment(a, t, lo, in);
+}
+
+// One warp: the same search 32 probes at a time (one memory round trip per factor of 32); lane 0
+// gathers.  `in` is written by lane 0 only.
+__device__ __forceinline__ void row_gather_warp(const LossArgs& a, long long t, int lane, RowInputs& in) {
+    int lo = 0, hi = a.S_max;
+    while (hi - lo > 1) {
+        const int step = (hi - lo + 31) >> 5;                        // probes at lo + step, lo + 2 step, ...
+        const long long idx = (long long)lo + (long long)(lane + 1) * step;
+        const bool le = idx < hi && (long long)a.cu_seqlens[idx] <= t;
+        const int n = __popc(__ballot_sync(0xffffffffu, le));        // cu_seqlens is non-decreasing: a prefix of lanes
+        lo += n * step;
+        hi = min(hi, lo + step);
+    }
+    if (lane == 0) row_inputs_from_segment(a, t, lo, in);
+}
+
+// ref2/sum2: the row's sum of 2^(z c) is sum2 * 2^ref2 with c = log2(e)/temperature as used in pass 1.
+// write: only one CTA of a cluster that shares a row stores the row's outputs.
+__device__ __forceinline__ RowScalars row_finish(const LossArgs& a, long long t, const RowInputs& in, float ref2,
+                                                 float sum2, bool write = true) {
+    RowScalars out;
+    const double lse2 = (double)ref2 + log2((double)sum2);           // base-2 log-sum-exp of z c
+    const double lse = lse2 * 0.6931471805599453;                    // natural log-sum-exp of z / temperature
+    out.lse2_hi = (float)lse2;
+    out.lse2_lo = (float)(lse2 - (double)out.lse2_hi);
+    out.g_over_tau = 0.0f;
+    out.valid = false;
+    RowTerms terms = {0.0, 0.0, 0.0, 0.0};
+    float logp_f = 0.0f;
+    if (in.state != 0) {
+        if (write) set_status(a.status, in.state);
+    } else {
+        const double A = in.A, W = in.W;
+        const double logp = in.zy - lse;
+        const double rho = exp(logp - in.logp_old);
+        const double d = in.logp_ref - logp;
+        const double rho_hat = exp(d);
+        const double kl = rho_hat - d - 1.0;
+        const double s1 = rho * A;
+        const double s2 = fmin(fmax(rho, 1.0 - a.eps_lo), 1.0 + a.eps_hi) * A;
+        const bool clipped = s2 < s1;
+        const double surr = clipped ? s2 : s1;
+        const double dj = (clipped ? 0.0 : A * rho) + a.beta * (rho_hat - 1.0);
+        terms.loss = -W * (surr - a.beta * kl);
+        terms.pg = -W * surr;
+        terms.kl = W * kl;
+        terms.clipped = clipped ? 1.0 : 0.0;
+        out.g_over_tau = (float)(-W * dj / a.temperature);
+        out.valid = true;
+        logp_f = (float)logp;
+    }
+    if (write) {
+        a.terms[t] = terms;
+        if (a.logp_out) a.logp_out[t] = logp_f;
+        if (a.lse_out) a.lse_out[t] = (float)lse;
+    }
+    return out;
+}
+
+__device__ __forceinline__ RowScalars row_scalar_stage(const LossArgs& a, long long t, float ref2, float sum2) {
+    RowInputs in;
+    row_gather(a, t, in);
+    return row_finish(a, t, in, ref2, sum2, true);
+}
 
 int launch_rows_general(const LossArgs& a, cudaStream_t s);
+// Cluster kernel: the row is split over `cluster` CTAs that keep their slice in shared memory.
+// Returns DPPO_ERR_UNSUPPORTED (nothing launched) when the shape or the device cannot take it.
+int launch_rows_cluster(const LossArgs& a, int cluster, int threads, cudaStream_t s);
 int launch_loss_reduce(const LossArgs& a, float* loss_out, cudaStream_t s);
 
 }  // namespace dppo

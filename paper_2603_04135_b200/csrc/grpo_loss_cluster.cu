@@ -1,0 +1,297 @@
+// Loss sweep for long bf16 rows: the row never comes back from HBM.
+//
+// A logit row of the full vocabulary (151,936 bf16 = 297 KB) does not fit one SM's shared memory, and
+// dlogits cannot be written before the row's log-sum-exp is known.  Instead of reading the row twice,
+// a thread-block cluster of C CTAs splits it: each CTA pulls its slice into shared memory with bulk
+// async copies (no multicast), reduces (max, sum 2^x) over the slice, the C partial pairs are
+// exchanged through distributed shared memory, every CTA repeats the cheap scalar stage, and the
+// second pass runs out of shared memory straight into streaming global stores.  HBM traffic is the
+// algorithmic minimum: one read and one write per element.  Several CTAs per SM sit in different
+// phases (copy in flight / reducing / storing), which is what overlaps the memory system with the
+// exp work.
+#include <cooperative_groups.h>
+
+#include "common.cuh"
+#include "grpo_loss.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace dppo {
+
+constexpr int kMaxCluster = 8;
+constexpr int kChunks = 4;                    // bulk copies (and mbarriers) per slice
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // give up on a copy after 2 s
+
+struct ClusterStatic {
+    unsigned long long bar[kChunks];          // one mbarrier per bulk copy of the slice
+    unsigned long long xbar;                  // completes when every CTA's (reference, sum) pair has landed in x[]
+    unsigned long long x[kMaxCluster];        // pair of CTA k: low word = reference, high word = sum (f32 bits)
+    float red_a[32], red_b[32];
+    RowInputs in;
+    RowScalars row;
+    int failed;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait on phase `parity` of an mbarrier; false when the limit ran out.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    const unsigned long long t0 = global_ns();
+    for (;;) {
+        uint32_t done;
+        asm volatile("{\n\t.reg .pred p;\n\t"
+                     "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                     "selp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (done) return true;
+        if (global_ns() - t0 > kWaitLimitNs) return false;
+    }
+}
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// The cluster barrier is used once, as a start-up handshake ("my mbarriers exist"): no data rides on it.
+__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.aligned;" ::: "memory"); }
+
+// 8-byte store into CTA `rank`'s shared memory that also signals that CTA's mbarrier (8 bytes of tx).
+__device__ __forceinline__ void remote_store_signal(uint32_t local_slot, uint32_t local_bar, int rank, unsigned long long v) {
+    uint32_t rslot, rbar;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rslot) : "r"(local_slot), "r"(rank));
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rbar) : "r"(local_bar), "r"(rank));
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b64 [%0], %1, [%2];"
+                 :: "r"(rslot), "l"(v), "r"(rbar) : "memory");
+}
+
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS)
+grpo_loss_cluster_kernel(const LossArgs a, const int C, const int vec_per_cta) {
+    extern __shared__ __align__(128) unsigned char slice_raw[];
+    __shared__ ClusterStatic st;
+    uint4* slice = reinterpret_cast<uint4*>(slice_raw);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int rank = blockIdx.x % C;                        // cluster dims are (C,1,1): consecutive blocks
+    const long long t = blockIdx.x / C;
+    const long long T = a.n_tokens_dev ? min((long long)*a.n_tokens_dev, a.T_max) : a.T_max;
+    if (t >= T) return;                                     // uniform over the cluster: nobody reaches a barrier
+
+    const int nvec = a.V >> 3;                              // whole 16-byte vectors of the row
+    const int v0 = rank * vec_per_cta;
+    const int nv = max(0, min(vec_per_cta, nvec - v0));     // vectors of this CTA's slice
+    const int chunk_vec = (nv + kChunks - 1) / kChunks;
+    const char* row = a.logits + t * a.row_bytes;
+    const float c = a.scale2;
+
+    // ---- issue the slice's bulk copies
+    if (tid == 0) {
+        st.failed = 0;
+#pragma unroll
+        for (int k = 0; k < kChunks; ++k)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(&st.bar[k])));
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(&st.xbar)));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        // the exchange expects one 8-byte pair from each CTA of the cluster (its own included)
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(smem_u32(&st.xbar)), "r"(8u * C) : "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+#pragma unroll
+        for (int k = 0; k < kChunks; ++k) {
+            const int b = k * chunk_vec, e = min(nv, b + chunk_vec);
+            if (e > b) {
+                const uint32_t bytes = (uint32_t)(e - b) * 16u;
+                const uint32_t bar = smem_u32(&st.bar[k]);
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
+                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                             :: "r"(smem_u32(slice + b)), "l"(row + (size_t)(v0 + b) * 16), "r"(bytes), "r"(bar)
+                             : "memory");
+            }
+        }
+    }
+    __syncthreads();                                        // barriers initialised before anyone polls them
+    cluster_arrive_relaxed();                               // handshake: this CTA's mbarriers exist (waited on before the exchange)
+
+    // ---- while the slice is in flight: one warp finds the token's sequence and gathers the side inputs
+    if (warp == (THREADS > 32 ? 1 : 0)) row_gather_warp(a, t, lane, st.in);
+
+    // ---- pass 1a: slice maximum (packed bf16 max), chunk by chunk as the copies land
+    __nv_bfloat162 mx2 = __float2bfloat162_rn(-INFINITY);
+    bool ok = true;
+#pragma unroll
+    for (int k = 0; k < kChunks; ++k) {
+        const int b = k * chunk_vec, e = min(nv, b + chunk_vec);
+        if (e > b) {
+            ok = mbar_wait(smem_u32(&st.bar[k]), 0) && ok;
+            for (int i = b + tid; i < e; i += THREADS) {
+                const uint4 q = slice[i];
+                mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&q.x));
+                mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&q.y));
+                mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&q.z));
+                mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&q.w));
+            }
+        }
+    }
+    if (!ok) st.failed = 1;                                 // benign race: every writer stores 1
+    float m = fmaxf(__low2float(mx2), __high2float(mx2));
+    // the row's ragged tail (V % 8 elements) belongs to the last CTA and is read from global memory
+    const int tail0 = nvec << 3;
+    float ztail = -INFINITY;
+    if (rank == C - 1 && tail0 + tid < a.V) {
+        ztail = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(row)[tail0 + tid]);
+        m = fmaxf(m, ztail);
+    }
+    m = warp_max(m);
+    if (lane == 0) st.red_a[warp] = m;
+    __syncthreads();
+    m = st.red_a[lane < THREADS / 32 ? lane : 0];
+    m = warp_max(m);                                        // every warp ends with the CTA maximum
+    const float r = m * c;                                  // -inf for an empty slice
+
+    // ---- pass 1b: sum of 2^(z c - r) over the slice
+    float s = 0.0f;
+    if (nv > 0 || ztail > -INFINITY) {
+        float s0 = 0.0f, s1 = 0.0f;
+        for (int i = tid; i < nv; i += THREADS) {
+            const uint4 q = slice[i];
+            s0 += ex2(fmaf(__uint_as_float(q.x << 16), c, -r)) + ex2(fmaf(__uint_as_float(q.y << 16), c, -r));
+            s1 += ex2(fmaf(__uint_as_float(q.x & 0xffff0000u), c, -r)) + ex2(fmaf(__uint_as_float(q.y & 0xffff0000u), c, -r));
+            s0 += ex2(fmaf(__uint_as_float(q.z << 16), c, -r)) + ex2(fmaf(__uint_as_float(q.w << 16), c, -r));
+            s1 += ex2(fmaf(__uint_as_float(q.z & 0xffff0000u), c, -r)) + ex2(fmaf(__uint_as_float(q.w & 0xffff0000u), c, -r));
+        }
+        s = s0 + s1;
+        if (ztail > -INFINITY) s += ex2(fmaf(ztail, c, -r));
+    }
+    s = warp_sum(s);
+    if (lane == 0) st.red_b[warp] = s;
+    __syncthreads();
+
+    // ---- exchange (r, s) with the other CTAs of the cluster: one remote store + signal per peer, then
+    //      thread 0 waits for all C pairs on its own mbarrier and runs the scalar stage (every CTA
+    //      repeats it; rank 0 writes the row's outputs)
+    cluster_wait();                                         // every CTA of the cluster has initialised its mbarriers
+    if (warp == 0) {
+        float ss = lane < THREADS / 32 ? st.red_b[lane] : 0.0f;
+        ss = warp_sum(ss);
+        if (lane < C) {
+            const float rr = st.failed ? __int_as_float(0x7fc00000) : r;   // a NaN reference marks a copy that timed out
+            const unsigned long long v = (unsigned long long)__float_as_uint(rr) | ((unsigned long long)__float_as_uint(ss) << 32);
+            remote_store_signal(smem_u32(&st.x[rank]), smem_u32(&st.xbar), lane, v);
+        }
+        if (lane == 0) {
+            const bool arrived = mbar_wait(smem_u32(&st.xbar), 0);
+            float R = -INFINITY;
+            bool failed = !arrived;
+            for (int k = 0; k < C && arrived; ++k) {
+                const float xr = __uint_as_float((uint32_t)st.x[k]);
+                failed = failed || (xr != xr);
+                R = fmaxf(R, xr);
+            }
+            float S = 0.0f;
+            for (int k = 0; k < C && !failed; ++k) {
+                const float xr = __uint_as_float((uint32_t)st.x[k]), xs = __uint_as_float((uint32_t)(st.x[k] >> 32));
+                S += (xr == -INFINITY) ? 0.0f : xs * exp2f(xr - R);
+            }
+            if (failed) {
+                if (rank == 0) {
+                    set_status(a.status, DPPO_STATUS_TIMEOUT);
+                    const RowTerms zero = {0.0, 0.0, 0.0, 0.0};
+                    a.terms[t] = zero;
+                    if (a.logp_out) a.logp_out[t] = 0.0f;
+                    if (a.lse_out) a.lse_out[t] = 0.0f;
+                }
+                RowScalars bad; bad.lse2_hi = 0.0f; bad.lse2_lo = 0.0f; bad.g_over_tau = 0.0f; bad.valid = false;
+                st.row = bad;
+            } else {
+                st.row = row_finish(a, t, st.in, R, S, rank == 0);
+            }
+        }
+    }
+    __syncthreads();
+    const RowScalars rs = st.row;
+
+    // ---- pass 2: dlogits = g/tau (onehot - 2^(z c - lse2)), shared memory -> streaming global stores
+    if (a.dlogits) {
+        char* drow = a.dlogits + t * a.row_bytes;
+        uint4* dst = reinterpret_cast<uint4*>(drow) + v0;
+        const float ng = rs.valid ? -rs.g_over_tau : 0.0f;
+        const float lse2 = rs.lse2_hi;                       // bf16 output: the low word of the split is below its rounding
+        const int y = rs.valid ? a.target[t] : -1;
+        const int yvec = (y >= 0 ? (y >> 3) : -1) - v0;     // vector of the target relative to this slice
+        const bool live = !st.failed;                        // after a timeout the slice is not read: zeros go out
+        for (int i = tid; i < nv; i += THREADS) {
+            uint4 q = live ? slice[i] : make_uint4(0, 0, 0, 0);
+            float f[8];
+            f[0] = ng * ex2(fmaf(__uint_as_float(q.x << 16), c, -lse2));
+            f[1] = ng * ex2(fmaf(__uint_as_float(q.x & 0xffff0000u), c, -lse2));
+            f[2] = ng * ex2(fmaf(__uint_as_float(q.y << 16), c, -lse2));
+            f[3] = ng * ex2(fmaf(__uint_as_float(q.y & 0xffff0000u), c, -lse2));
+            f[4] = ng * ex2(fmaf(__uint_as_float(q.z << 16), c, -lse2));
+            f[5] = ng * ex2(fmaf(__uint_as_float(q.z & 0xffff0000u), c, -lse2));
+            f[6] = ng * ex2(fmaf(__uint_as_float(q.w << 16), c, -lse2));
+            f[7] = ng * ex2(fmaf(__uint_as_float(q.w & 0xffff0000u), c, -lse2));
+            if (i == yvec) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) if (e == (y & 7)) f[e] -= ng;
+            }
+            __stcs(dst + i, Elems<true>::pack(f));
+        }
+        if (rank == C - 1 && tail0 + tid < a.V) {
+            const int v = tail0 + tid;
+            const float p = ex2(fmaf(ztail, c, -lse2));
+            reinterpret_cast<__nv_bfloat16*>(drow)[v] = __float2bfloat16_rn(ng * p - (v == y ? ng : 0.0f));
+        }
+    }
+}
+
+// ---- host side ---------------------------------------------------------------------------------------
+template <int THREADS>
+static int launch_cluster_t(const LossArgs& a, int C, int vec_per_cta, size_t dyn_bytes, cudaStream_t s) {
+    auto kernel = grpo_loss_cluster_kernel<THREADS>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_bytes);
+    if (e != cudaSuccess) { cudaGetLastError(); return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: %zu bytes of shared memory refused", dyn_bytes); }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(a.T_max * C), 1, 1);
+    cfg.blockDim = dim3(THREADS, 1, 1);
+    cfg.dynamicSmemBytes = dyn_bytes;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)C; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    int max_clusters = 0;
+    e = cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &cfg);
+    if (e != cudaSuccess || max_clusters < 1) { cudaGetLastError(); return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: cluster of %d CTAs does not fit this device", C); }
+    e = cudaLaunchKernelEx(&cfg, kernel, a, C, vec_per_cta);
+    if (e != cudaSuccess) return cuda_fail(e, "grpo_loss cluster launch");
+    return DPPO_OK;
+}
+
+int launch_rows_cluster(const LossArgs& a, int C, int threads, cudaStream_t s) {
+    if (!a.bf16) return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: bf16 rows only");
+    if (C != 2 && C != 4 && C != 8) return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: cluster size %d", C);
+    if ((a.V & 7) >= threads) return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: tail");
+    if (a.T_max * C >= (1ll << 31)) return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: grid too large");
+    const int nvec = a.V >> 3;
+    const int vec_per_cta = (nvec + C - 1) / C;
+    const size_t dyn_bytes = (size_t)(vec_per_cta > 0 ? vec_per_cta : 1) * 16;
+    if (dyn_bytes > 220 * 1024) return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: slice of %zu bytes exceeds shared memory", dyn_bytes);
+    if (dyn_bytes / kChunks + 16 >= (1u << 20)) return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: chunk too large");
+    switch (threads) {
+        case 128: return launch_cluster_t<128>(a, C, vec_per_cta, dyn_bytes, s);
+        case 256: return launch_cluster_t<256>(a, C, vec_per_cta, dyn_bytes, s);
+        case 512: return launch_cluster_t<512>(a, C, vec_per_cta, dyn_bytes, s);
+        case 1024: return launch_cluster_t<1024>(a, C, vec_per_cta, dyn_bytes, s);
+    }
+    return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: %d threads", threads);
+}
+
+}  // namespace dppo

@@ -23,6 +23,7 @@ def main():
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"])
     ap.add_argument("--in-place", action="store_true")
     ap.add_argument("--seqs", type=int, default=16)
+    ap.add_argument("--variant", type=int, default=0, help="kernel variant (see dppo_loss_params.variant)")
     args = ap.parse_args()
     w = synth.scaled(synth.WORKLOADS["config3"], V=args.vocab, dtype=args.dtype)
     T, S = args.rows, args.seqs
@@ -32,7 +33,7 @@ def main():
     adv = torch.from_numpy(rng.normal(size=S).astype(np.float32)).cuda()
     wseq = torch.full((S,), 1.0 / S, device="cuda")
     dl = tok.logits if args.in_place else torch.empty_like(tok.logits)
-    prm = B.LossParams(T, w.V, B.BF16 if args.dtype == "bf16" else B.F32, w.V, S, 0, w.eps, w.eps, w.beta, 1.0)
+    prm = B.LossParams(T, w.V, B.BF16 if args.dtype == "bf16" else B.F32, w.V, S, args.variant, w.eps, w.eps, w.beta, 1.0)
     nbytes = B.grpo_loss_workspace_bytes(prm)
     ws = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
     loss_out = torch.zeros(5, device="cuda")

@@ -168,7 +168,7 @@ def test_pack_dataset_scale_and_bad_length():
 
 # ------------------------------------------------------------------------------------------- steps 6-8
 def _loss_case(V, dtype, T, S, seed, sigma_noise=0.05, logit_sigma=2.0, tau=1.0, pad=0, in_place=False,
-               forward_only=False, n_tokens=None, beta=0.04, eps=(0.2, 0.2)):
+               forward_only=False, n_tokens=None, beta=0.04, eps=(0.2, 0.2), variant=0):
     """Runs dppo_grpo_loss_fwd_bwd on a random case and compares everything with the oracle."""
     from paper_2603_04135_b200 import binding as B
     w = synth.scaled(synth.WORKLOADS["config0"], V=V, dtype=dtype, logit_sigma=logit_sigma)
@@ -191,7 +191,7 @@ def _loss_case(V, dtype, T, S, seed, sigma_noise=0.05, logit_sigma=2.0, tau=1.0,
     buf[:, :V] = tok.logits
     logits_before = buf.clone()
     dl = buf if in_place else (None if forward_only else torch.full((T, stride), 7.0, dtype=tdt, device="cuda"))
-    prm = B.LossParams(T, V, B.BF16 if dtype == "bf16" else B.F32, stride, S_max, 0, eps[0], eps[1], beta, tau)
+    prm = B.LossParams(T, V, B.BF16 if dtype == "bf16" else B.F32, stride, S_max, variant, eps[0], eps[1], beta, tau)
     nbytes = B.grpo_loss_workspace_bytes(prm)
     ws = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
     loss_out = torch.zeros(5, device="cuda"); logp_out = torch.zeros(T, device="cuda"); lse_out = torch.zeros(T, device="cuda")
@@ -261,6 +261,30 @@ def test_loss_full_vocab_bf16_rows():
     _loss_case(151936, "bf16", T=24, S=3, seed=31)
     _loss_case(151936 - 5, "bf16", T=9, S=2, seed=32, pad=5)
     _loss_case(151936, "f32", T=6, S=2, seed=33)
+
+
+@pytest.mark.parametrize("C", [2, 4, 8])
+def test_loss_cluster_kernel_variants(C):
+    # the shared-memory cluster kernel, forced: full vocabulary, ragged tails, slices that are empty
+    for threads in (128, 256, 512):
+        v = C * 10000 + threads
+        _loss_case(151936, "bf16", T=13, S=3, seed=40 + C, variant=v)
+    v = C * 10000 + 256
+    _loss_case(151936 - 5, "bf16", T=7, S=2, seed=50 + C, variant=v)              # tail of 3 elements, padded stride
+    _loss_case(151936, "bf16", T=9, S=2, seed=51 + C, variant=v, in_place=True)
+    _loss_case(151936, "bf16", T=9, S=2, seed=52 + C, variant=v, forward_only=True)
+    _loss_case(151936, "bf16", T=9, S=2, seed=53 + C, variant=v, n_tokens=5, tau=1.3)
+    _loss_case(4099, "bf16", T=33, S=4, seed=54 + C, variant=v)
+    _loss_case(24, "bf16", T=33, S=4, seed=55 + C, variant=v)                    # 3 vectors: most slices are empty
+    _loss_case(5, "bf16", T=20, S=2, seed=56 + C, variant=v)                     # tail only
+    _loss_case(65536, "bf16", T=300, S=7, seed=57 + C, variant=v, sigma_noise=0.3)
+
+
+def test_loss_auto_dispatch_matches_forced_kernels():
+    # variant 0 on a long bf16 row takes the cluster kernel; outputs agree with the general kernel's
+    a = _loss_case(151936, "bf16", T=11, S=2, seed=60, variant=0)
+    b = _loss_case(151936, "bf16", T=11, S=2, seed=60, variant=1)
+    assert a["loss"] == b["loss"]                                                # same oracle case both times
 
 
 def test_loss_bad_target_and_empty():
