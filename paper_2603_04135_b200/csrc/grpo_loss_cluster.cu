@@ -6,15 +6,15 @@
 // async copies (no multicast), reduces (max, sum 2^x) over the slice, the C partial pairs are
 // exchanged through distributed shared memory, every CTA repeats the cheap scalar stage, and the
 // second pass runs out of shared memory straight into streaming global stores.  HBM traffic is the
-// algorithmic minimum: one read and one write per element.  Several CTAs per SM sit in different
-// phases (copy in flight / reducing / storing), which is what overlaps the memory system with the
-// exp work.
-#include <cooperative_groups.h>
+// algorithmic minimum: one read and one write per element.  The exponentials of the first pass are
+// written back over the logits as fp16 (they lie in (0,1], relative to the slice maximum), so the
+// second pass is a scale-and-convert with no exp: one MUFU op per element in total.  Several CTAs
+// per SM sit in different phases (copy in flight / reducing / storing), which is what overlaps the
+// memory system with the exp work.
+#include <cuda_fp16.h>
 
 #include "common.cuh"
 #include "grpo_loss.cuh"
-
-namespace cg = cooperative_groups;
 
 namespace dppo {
 
@@ -52,6 +52,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
         if (done) return true;
         if (global_ns() - t0 > kWaitLimitNs) return false;
     }
+}
+
+__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
+    const __half2 h = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&h);
+}
+// Two fp16 exponentials -> two bf16 gradient entries: e * sc - sub (sub is g/tau at the target, else 0).
+__device__ __forceinline__ uint32_t scale_pair(uint32_t h2, float sc, float sub_lo, float sub_hi) {
+    const float2 e = __half22float2(*reinterpret_cast<const __half2*>(&h2));
+    const __nv_bfloat162 b = __floats2bfloat162_rn(fmaf(e.x, sc, -sub_lo), fmaf(e.y, sc, -sub_hi));
+    return *reinterpret_cast<const uint32_t*>(&b);
 }
 
 __device__ __forceinline__ float ex2(float x) {
@@ -157,18 +168,24 @@ grpo_loss_cluster_kernel(const LossArgs a, const int C, const int vec_per_cta) {
     const float r = m * c;                                  // -inf for an empty slice
 
     // ---- pass 1b: sum of 2^(z c - r) over the slice
-    float s = 0.0f;
+    float s = 0.0f, etail = 0.0f;
     if (nv > 0 || ztail > -INFINITY) {
         float s0 = 0.0f, s1 = 0.0f;
         for (int i = tid; i < nv; i += THREADS) {
             const uint4 q = slice[i];
-            s0 += ex2(fmaf(__uint_as_float(q.x << 16), c, -r)) + ex2(fmaf(__uint_as_float(q.y << 16), c, -r));
-            s1 += ex2(fmaf(__uint_as_float(q.x & 0xffff0000u), c, -r)) + ex2(fmaf(__uint_as_float(q.y & 0xffff0000u), c, -r));
-            s0 += ex2(fmaf(__uint_as_float(q.z << 16), c, -r)) + ex2(fmaf(__uint_as_float(q.w << 16), c, -r));
-            s1 += ex2(fmaf(__uint_as_float(q.z & 0xffff0000u), c, -r)) + ex2(fmaf(__uint_as_float(q.w & 0xffff0000u), c, -r));
+            const float e0 = ex2(fmaf(__uint_as_float(q.x << 16), c, -r)), e1 = ex2(fmaf(__uint_as_float(q.x & 0xffff0000u), c, -r));
+            const float e2 = ex2(fmaf(__uint_as_float(q.y << 16), c, -r)), e3 = ex2(fmaf(__uint_as_float(q.y & 0xffff0000u), c, -r));
+            const float e4 = ex2(fmaf(__uint_as_float(q.z << 16), c, -r)), e5 = ex2(fmaf(__uint_as_float(q.z & 0xffff0000u), c, -r));
+            const float e6 = ex2(fmaf(__uint_as_float(q.w << 16), c, -r)), e7 = ex2(fmaf(__uint_as_float(q.w & 0xffff0000u), c, -r));
+            s0 += (e0 + e2) + (e4 + e6);
+            s1 += (e1 + e3) + (e5 + e7);
+            // the exponentials replace the logits in place, as fp16 pairs: the second pass needs no exp
+            uint4 h;
+            h.x = pack_half2(e0, e1); h.y = pack_half2(e2, e3); h.z = pack_half2(e4, e5); h.w = pack_half2(e6, e7);
+            slice[i] = h;
         }
         s = s0 + s1;
-        if (ztail > -INFINITY) s += ex2(fmaf(ztail, c, -r));
+        if (ztail > -INFINITY) { etail = ex2(fmaf(ztail, c, -r)); s += etail; }
     }
     s = warp_sum(s);
     if (lane == 0) st.red_b[warp] = s;
@@ -223,31 +240,23 @@ grpo_loss_cluster_kernel(const LossArgs a, const int C, const int vec_per_cta) {
         char* drow = a.dlogits + t * a.row_bytes;
         uint4* dst = reinterpret_cast<uint4*>(drow) + v0;
         const float ng = rs.valid ? -rs.g_over_tau : 0.0f;
-        const float lse2 = rs.lse2_hi;                       // bf16 output: the low word of the split is below its rounding
+        // softmax = e * 2^(r - lse2) with e relative to this CTA's reference r
+        const float sc = ng * ex2((r - rs.lse2_hi) - rs.lse2_lo);
         const int y = rs.valid ? a.target[t] : -1;
         const int yvec = (y >= 0 ? (y >> 3) : -1) - v0;     // vector of the target relative to this slice
-        const bool live = !st.failed;                        // after a timeout the slice is not read: zeros go out
         for (int i = tid; i < nv; i += THREADS) {
-            uint4 q = live ? slice[i] : make_uint4(0, 0, 0, 0);
-            float f[8];
-            f[0] = ng * ex2(fmaf(__uint_as_float(q.x << 16), c, -lse2));
-            f[1] = ng * ex2(fmaf(__uint_as_float(q.x & 0xffff0000u), c, -lse2));
-            f[2] = ng * ex2(fmaf(__uint_as_float(q.y << 16), c, -lse2));
-            f[3] = ng * ex2(fmaf(__uint_as_float(q.y & 0xffff0000u), c, -lse2));
-            f[4] = ng * ex2(fmaf(__uint_as_float(q.z << 16), c, -lse2));
-            f[5] = ng * ex2(fmaf(__uint_as_float(q.z & 0xffff0000u), c, -lse2));
-            f[6] = ng * ex2(fmaf(__uint_as_float(q.w << 16), c, -lse2));
-            f[7] = ng * ex2(fmaf(__uint_as_float(q.w & 0xffff0000u), c, -lse2));
-            if (i == yvec) {
-#pragma unroll
-                for (int e = 0; e < 8; ++e) if (e == (y & 7)) f[e] -= ng;
-            }
-            __stcs(dst + i, Elems<true>::pack(f));
+            const uint4 q = slice[i];
+            const int ysel = (i == yvec) ? (y & 7) : -1;        // position of the target inside this vector, if any
+            uint4 o;
+            o.x = scale_pair(q.x, sc, ysel == 0 ? ng : 0.0f, ysel == 1 ? ng : 0.0f);
+            o.y = scale_pair(q.y, sc, ysel == 2 ? ng : 0.0f, ysel == 3 ? ng : 0.0f);
+            o.z = scale_pair(q.z, sc, ysel == 4 ? ng : 0.0f, ysel == 5 ? ng : 0.0f);
+            o.w = scale_pair(q.w, sc, ysel == 6 ? ng : 0.0f, ysel == 7 ? ng : 0.0f);
+            __stcs(dst + i, o);
         }
         if (rank == C - 1 && tail0 + tid < a.V) {
             const int v = tail0 + tid;
-            const float p = ex2(fmaf(ztail, c, -lse2));
-            reinterpret_cast<__nv_bfloat16*>(drow)[v] = __float2bfloat16_rn(ng * p - (v == y ? ng : 0.0f));
+            reinterpret_cast<__nv_bfloat16*>(drow)[v] = __float2bfloat16_rn(sc * etail - (v == y ? ng : 0.0f));
         }
     }
 }
