@@ -139,6 +139,34 @@ int dppo_pack_prompts(const dppo_pack_params* p, const int32_t* len, const uint8
                       void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
 
 /* ------------------------------------------------------------------------------------------------
+ * Packing without a caller workspace.  (The paper has no counterpart: this entry point exists for the
+ * sake of callers, not of the method.)
+ *
+ * Same operation, same arguments and same results as dppo_pack_prompts, minus `workspace`: the
+ * scratch is a fixed 64 KB array inside the library's device image.  It is meant for callers that
+ * have no way to hand over device scratch at the point of the call: host code that is given only
+ * its input and output buffers by a framework and owns no allocator, or a training loop whose
+ * device memory is entirely reserved by a pool, where a cudaMalloc would fail or would stall every
+ * stream while it runs.  The call itself allocates nothing (no cudaMalloc / cudaFree, no library
+ * allocation).
+ *
+ *  - Limit: n_max <= dppo_pack_static_max_units() (8192 units); larger requests return
+ *    DPPO_ERR_BAD_SHAPE and launch nothing.  Every GPU that loads the library holds the 64 KB until
+ *    the process ends, used or not.
+ *  - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ *    that device current) and caches it; make that first call before starting any stream capture.
+ *  - All calls on a device share the one array.  It keeps whatever the previous call left there;
+ *    the kernel never reads a slot before writing it, so nothing needs clearing.  Two calls whose
+ *    kernels can overlap on the GPU (different streams, no ordering between them) race on it:
+ *    keep calls on one stream or order them yourself.
+ */
+int dppo_pack_static_max_units(void);
+int dppo_pack_prompts_static(const dppo_pack_params* p, const int32_t* len, const uint8_t* keep,
+                             const int32_t* loss_len, int32_t* order, int32_t* row_of,
+                             int32_t* off_in_row, int32_t* row_fill, int32_t* cu_seqlens,
+                             int32_t* counts, int32_t* status, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
  * Fused loss sweep over the logits — Eq. 1 (clipped surrogate minus beta x KL, 1/|o_i| per sequence,
  * KL estimator rho_hat - log rho_hat - 1) with the sequence weights of dppo_prune_and_rescale, and
  * its gradient with respect to the logits.

@@ -56,6 +56,9 @@ lib.dppo_pack_workspace_bytes.restype = ctypes.c_size_t
 lib.dppo_pack_workspace_bytes.argtypes = [ctypes.POINTER(PackParams)]
 lib.dppo_pack_prompts.restype = ctypes.c_int
 lib.dppo_pack_prompts.argtypes = [ctypes.POINTER(PackParams)] + [_vp] * 10 + [ctypes.c_size_t, _vp, _vp]
+lib.dppo_pack_static_max_units.restype = ctypes.c_int
+lib.dppo_pack_prompts_static.restype = ctypes.c_int
+lib.dppo_pack_prompts_static.argtypes = [ctypes.POINTER(PackParams)] + [_vp] * 11
 lib.dppo_grpo_loss_workspace_bytes.restype = ctypes.c_size_t
 lib.dppo_grpo_loss_workspace_bytes.argtypes = [ctypes.POINTER(LossParams)]
 lib.dppo_grpo_loss_fwd_bwd.restype = ctypes.c_int
@@ -113,6 +116,19 @@ def pack_prompts(params, len_, keep, loss_len, order, row_of, off_in_row, row_fi
     _check(lib.dppo_pack_prompts(ctypes.byref(params), _ptr(len_), _ptr(keep), _ptr(loss_len), _ptr(order),
                                  _ptr(row_of), _ptr(off_in_row), _ptr(row_fill), _ptr(cu_seqlens),
                                  _ptr(counts), _ptr(workspace), workspace_bytes, _ptr(status), _stream(stream)))
+
+
+def pack_static_max_units():
+    return lib.dppo_pack_static_max_units()
+
+
+def pack_prompts_static(params, len_, keep, loss_len, order, row_of, off_in_row, row_fill, cu_seqlens, counts,
+                        status=None, stream=None):
+    """dppo_pack_prompts without a workspace argument: scratch is a fixed array inside the library
+    (at most pack_static_max_units() units); nothing is allocated by the call."""
+    _check(lib.dppo_pack_prompts_static(ctypes.byref(params), _ptr(len_), _ptr(keep), _ptr(loss_len), _ptr(order),
+                                        _ptr(row_of), _ptr(off_in_row), _ptr(row_fill), _ptr(cu_seqlens),
+                                        _ptr(counts), _ptr(status), _stream(stream)))
 
 
 def grpo_loss_workspace_bytes(params):

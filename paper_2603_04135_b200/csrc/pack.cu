@@ -127,6 +127,35 @@ pack_prompts_kernel(dppo_pack_params prm, const int32_t* __restrict__ len,
 
 static size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
 
+// ---- scratch for dppo_pack_prompts_static ------------------------------------------------------
+// Lives in the library's device image: every GPU that loads the library holds these 64 KB until the
+// process exits.  Layout: stream positions [0, kPackStaticMaxUnits), their lengths after that.
+constexpr int kPackStaticMaxUnits = 8192;
+static __device__ __align__(256) int32_t g_pack_static_scratch[2 * kPackStaticMaxUnits];
+
+constexpr int kMaxDevices = 64;
+static int32_t* g_pack_static_ptr[kMaxDevices];          // device address of the array, per device ordinal
+
+// Device address of the scratch array on the current device.  In host code the array's name is only a
+// handle for the runtime; the address a kernel can use comes from cudaGetSymbolAddress, asked once per
+// device with that device current.
+static int pack_static_scratch(int32_t** out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "pack_prompts_static: cudaGetDevice");
+    if (dev < 0 || dev >= kMaxDevices) return fail(DPPO_ERR_UNSUPPORTED, "pack_prompts_static: device ordinal %d", dev);
+    int32_t* p = __atomic_load_n(&g_pack_static_ptr[dev], __ATOMIC_ACQUIRE);
+    if (p == nullptr) {
+        void* sym = nullptr;
+        e = cudaGetSymbolAddress(&sym, g_pack_static_scratch);
+        if (e != cudaSuccess || sym == nullptr) return cuda_fail(e, "pack_prompts_static: cudaGetSymbolAddress");
+        p = static_cast<int32_t*>(sym);
+        __atomic_store_n(&g_pack_static_ptr[dev], p, __ATOMIC_RELEASE);   // racing threads store the same value
+    }
+    *out = p;
+    return DPPO_OK;
+}
+
 }  // namespace dppo
 
 extern "C" size_t dppo_pack_workspace_bytes(const dppo_pack_params* p) {
@@ -164,5 +193,35 @@ extern "C" int dppo_pack_prompts(const dppo_pack_params* p, const int32_t* len, 
         pack_prompts_kernel<false><<<1, 32, 0, s>>>(*p, len, keep, loss_len, order, row_of, off_in_row, row_fill,
                                                     cu_seqlens, counts, ws, status);
     DPPO_CHECK_LAUNCH("pack_prompts launch");
+    return DPPO_OK;
+}
+
+extern "C" int dppo_pack_static_max_units(void) { return dppo::kPackStaticMaxUnits; }
+
+extern "C" int dppo_pack_prompts_static(const dppo_pack_params* p, const int32_t* len, const uint8_t* keep,
+                                        const int32_t* loss_len, int32_t* order, int32_t* row_of,
+                                        int32_t* off_in_row, int32_t* row_fill, int32_t* cu_seqlens,
+                                        int32_t* counts, int32_t* status, void* stream) {
+    using namespace dppo;
+    if (!p) return fail(DPPO_ERR_INVALID_ARG, "pack_prompts_static: NULL params");
+    if (p->n_max < 0 || p->L_row < 1 || p->N_win < 1 || (p->policy != 0 && p->policy != 1))
+        return fail(DPPO_ERR_INVALID_ARG, "pack_prompts_static: n_max=%d L_row=%d N_win=%d policy=%d", p->n_max,
+                    p->L_row, p->N_win, p->policy);
+    if (p->n_max > kPackStaticMaxUnits)
+        return fail(DPPO_ERR_BAD_SHAPE, "pack_prompts_static: n_max=%d exceeds the built-in scratch (%d units); "
+                    "use dppo_pack_prompts with a caller workspace", p->n_max, kPackStaticMaxUnits);
+    if (!cu_seqlens || !counts) return fail(DPPO_ERR_INVALID_ARG, "pack_prompts_static: NULL cu_seqlens/counts");
+    if (p->n_max > 0 && (!len || !order || !row_of || !off_in_row || !row_fill))
+        return fail(DPPO_ERR_INVALID_ARG, "pack_prompts_static: NULL array");
+    int32_t* scratch = nullptr;
+    const int rc = pack_static_scratch(&scratch);
+    if (rc != DPPO_OK) return rc;
+    PackWorkspace ws;
+    ws.stream = scratch;
+    ws.slen = scratch + kPackStaticMaxUnits;
+    // Nothing in the scratch has to start at zero: the kernel writes every stream slot it later reads.
+    pack_prompts_kernel<true><<<1, 32, 0, (cudaStream_t)stream>>>(*p, len, keep, loss_len, order, row_of, off_in_row,
+                                                                  row_fill, cu_seqlens, counts, ws, status);
+    DPPO_CHECK_LAUNCH("pack_prompts_static launch");
     return DPPO_OK;
 }
