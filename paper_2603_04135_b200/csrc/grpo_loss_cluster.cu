@@ -58,10 +58,10 @@ __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
     const __half2 h = __floats2half2_rn(lo, hi);
     return *reinterpret_cast<const uint32_t*>(&h);
 }
-// Two fp16 exponentials -> two bf16 gradient entries: e * sc - sub (sub is g/tau at the target, else 0).
-__device__ __forceinline__ uint32_t scale_pair(uint32_t h2, float sc, float sub_lo, float sub_hi) {
+// Two fp16 exponentials -> two bf16 gradient entries e * sc.
+__device__ __forceinline__ uint32_t scale_pair(uint32_t h2, float sc) {
     const float2 e = __half22float2(*reinterpret_cast<const __half2*>(&h2));
-    const __nv_bfloat162 b = __floats2bfloat162_rn(fmaf(e.x, sc, -sub_lo), fmaf(e.y, sc, -sub_hi));
+    const __nv_bfloat162 b = __floats2bfloat162_rn(e.x * sc, e.y * sc);
     return *reinterpret_cast<const uint32_t*>(&b);
 }
 
@@ -142,6 +142,7 @@ grpo_loss_cluster_kernel(const LossArgs a, const int C, const int vec_per_cta) {
         const int b = k * chunk_vec, e = min(nv, b + chunk_vec);
         if (e > b) {
             ok = mbar_wait(smem_u32(&st.bar[k]), 0) && ok;
+#pragma unroll 4
             for (int i = b + tid; i < e; i += THREADS) {
                 const uint4 q = slice[i];
                 mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&q.x));
@@ -171,6 +172,7 @@ grpo_loss_cluster_kernel(const LossArgs a, const int C, const int vec_per_cta) {
     float s = 0.0f, etail = 0.0f;
     if (nv > 0 || ztail > -INFINITY) {
         float s0 = 0.0f, s1 = 0.0f;
+#pragma unroll 2
         for (int i = tid; i < nv; i += THREADS) {
             const uint4 q = slice[i];
             const float e0 = ex2(fmaf(__uint_as_float(q.x << 16), c, -r)), e1 = ex2(fmaf(__uint_as_float(q.x & 0xffff0000u), c, -r));
@@ -244,15 +246,20 @@ grpo_loss_cluster_kernel(const LossArgs a, const int C, const int vec_per_cta) {
         const float sc = ng * ex2((r - rs.lse2_hi) - rs.lse2_lo);
         const int y = rs.valid ? a.target[t] : -1;
         const int yvec = (y >= 0 ? (y >> 3) : -1) - v0;     // vector of the target relative to this slice
+#pragma unroll 4
         for (int i = tid; i < nv; i += THREADS) {
             const uint4 q = slice[i];
-            const int ysel = (i == yvec) ? (y & 7) : -1;        // position of the target inside this vector, if any
             uint4 o;
-            o.x = scale_pair(q.x, sc, ysel == 0 ? ng : 0.0f, ysel == 1 ? ng : 0.0f);
-            o.y = scale_pair(q.y, sc, ysel == 2 ? ng : 0.0f, ysel == 3 ? ng : 0.0f);
-            o.z = scale_pair(q.z, sc, ysel == 4 ? ng : 0.0f, ysel == 5 ? ng : 0.0f);
-            o.w = scale_pair(q.w, sc, ysel == 6 ? ng : 0.0f, ysel == 7 ? ng : 0.0f);
+            o.x = scale_pair(q.x, sc); o.y = scale_pair(q.y, sc);
+            o.z = scale_pair(q.z, sc); o.w = scale_pair(q.w, sc);
             __stcs(dst + i, o);
+        }
+        // the one element that also carries the onehot term: the thread that stored its vector redoes it
+        if (yvec >= 0 && yvec < nv && (yvec % THREADS) == tid) {
+            const uint32_t word = reinterpret_cast<const uint32_t*>(slice + yvec)[(y & 7) >> 1];
+            const float2 e = __half22float2(*reinterpret_cast<const __half2*>(&word));
+            const float ey = (y & 1) ? e.y : e.x;
+            reinterpret_cast<__nv_bfloat16*>(drow)[y] = __float2bfloat16_rn(fmaf(ey, sc, -ng));
         }
         if (rank == C - 1 && tail0 + tid < a.V) {
             const int v = tail0 + tid;
