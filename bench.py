@@ -36,6 +36,26 @@ WORKLOAD = "config3"
 WORKLOAD_TEXT = WORKLOAD + ": P=32 G=8, response 64-1024 tokens, V=151936 bf16 logits, r_q=r_o=0.25, L_row=8192, N_win=16"
 
 
+# DRAM traffic of the dominant kernel from its last ncu capture (profiles/loss_sweep_cluster_kernel.md):
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch over 8192 rows of this vocabulary.  Traffic
+# grows in proportion to the rows, so a launch over T rows moves T times the per-row figure.  The record
+# is tied to the kernel sources it was taken from: once they change, `traffic` is reported as null.
+TRAFFIC_CAPTURE = {"rows": 8192, "dram_bytes": 2489454000 + 2431901000,
+                   "source_sha256": "ccce8c8ef8b758288946abbb8ff96c386f98c44113cb5bb88e3e4c004c6459eb"}
+
+
+def captured_traffic_per_row():
+    import hashlib
+    base = os.path.join(ROOT, "paper_2603_04135_b200", "csrc")
+    try:
+        src = b"".join(open(os.path.join(base, f), "rb").read() for f in ("grpo_loss_cluster.cu", "grpo_loss.cuh"))
+    except OSError:
+        return None
+    if hashlib.sha256(src).hexdigest() != TRAFFIC_CAPTURE["source_sha256"]:
+        return None
+    return TRAFFIC_CAPTURE["dram_bytes"] / TRAFFIC_CAPTURE["rows"]
+
+
 def measured_peaks():
     try:
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
@@ -58,7 +78,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.FIELDS,
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "200"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             time.sleep(0.3)
         except Exception:
@@ -204,6 +224,7 @@ def run_ours(args):
         raise RuntimeError("not enough device memory for %s: need %.1f GB, free %.1f GB" % (WORKLOAD, need / 1e9, free / 1e9))
     tok = synth.make_token_inputs(w, T, seed, device=dev)
     dlogits = torch.empty_like(tok.logits)
+    st.loss_params.T_max = T          # the logits hold exactly the retained tokens (the same pruning every step)
 
     def one_step(ev0=None, ev1=None):
         st.prune_pack(seed=seed, step=1)
@@ -222,7 +243,7 @@ def run_ours(args):
         one_step()
     barrier()
     sampler = ClockSampler(local_rank)
-    if rank == 0:
+    if rank == 0 and not args.no_clock_sampling:
         sampler.start()
     k_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -290,7 +311,9 @@ def run_ours(args):
             "roofline": {"bound": "hbm", "kernel": "grpo loss sweep (rows kernel + its 1-block reduction)",
                          "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_source": peak_kind + " STREAM-style copy", "kernel_ms": loss_ms,
-                         "algorithmic_bytes_per_token": bytes_per_token, "traffic": None},
+                         "algorithmic_bytes_per_token": bytes_per_token,
+                         "traffic": (captured_traffic_per_row() * T) if captured_traffic_per_row() else None,
+                         "traffic_note": "ncu dram bytes of an 8192-row capture of the same kernel, scaled by rows"},
             "loss": loss_value,
         }
         if pool is not None:
@@ -315,6 +338,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--ref-rows", type=int, default=2048, help="token rows in the oracle's timed sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-clock-sampling", action="store_true", help="do not poll nvidia-smi during the timed region")
     args = ap.parse_args()
     if args.impl == "ours" and args.warmup < 3:
         args.warmup = 3

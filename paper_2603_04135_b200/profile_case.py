@@ -23,6 +23,9 @@ def main():
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"])
     ap.add_argument("--in-place", action="store_true")
     ap.add_argument("--seqs", type=int, default=16)
+    ap.add_argument("--full-call", action="store_true",
+                    help="pass everything the training step passes: device token count, seg_map, logp/lse outputs")
+    ap.add_argument("--back-to-back", action="store_true", help="enqueue all iterations before synchronising")
     ap.add_argument("--variant", type=int, default=0, help="kernel variant (see dppo_loss_params.variant)")
     args = ap.parse_args()
     w = synth.scaled(synth.WORKLOADS["config3"], V=args.vocab, dtype=args.dtype)
@@ -39,13 +42,23 @@ def main():
     loss_out = torch.zeros(5, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     esize = 2 if args.dtype == "bf16" else 4
+    ntd = seg_map = logp_out = lse_out = None
+    if args.full_call:
+        ntd = torch.tensor([T], dtype=torch.int32, device="cuda")
+        seg_map = torch.arange(S, dtype=torch.int32, device="cuda")
+        logp_out = torch.zeros(T, device="cuda"); lse_out = torch.zeros(T, device="cuda")
+    events = []
     for it in range(args.iters):
         e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
         e0.record()
-        B.grpo_loss_fwd_bwd(prm, tok.logits, tok.target, tok.logp_old, tok.logp_ref, cu, None, adv, wseq, None, dl,
-                            None, None, loss_out, ws, nbytes, status)
+        B.grpo_loss_fwd_bwd(prm, tok.logits, tok.target, tok.logp_old, tok.logp_ref, cu, ntd, adv, wseq, seg_map, dl,
+                            logp_out, lse_out, loss_out, ws, nbytes, status)
         e1.record()
-        torch.cuda.synchronize()
+        events.append((e0, e1))
+        if not args.back_to_back:
+            torch.cuda.synchronize()
+    torch.cuda.synchronize()
+    for it, (e0, e1) in enumerate(events):
         ms = e0.elapsed_time(e1)
         print("iter %d: %.3f ms  %.1f GB/s algorithmic  loss %.6g  status %d" % (
             it, ms, 2 * T * w.V * esize / ms / 1e6, loss_out[0].item(), status.item()))
