@@ -117,24 +117,41 @@ def draw_uniforms(seed, step, P, G):
     return u_q, u_o
 
 
-def prune_masks(cand_q, cand_o, u_q, u_o, r_q, r_o):
-    """Independent pruning with probability r of each candidate (Eq. 15, 17).
+def prune_masks(cand_q, cand_o, u_q, u_o, r_q, r_o, mode=0):
+    """Pruning of the candidates (Eq. 15, 17).
 
-    A prompt is pruned iff cand_q and u_q < r_q; a completion is pruned iff
-    cand_o and u_o < r_o; every completion of a pruned prompt goes with it.
-    Returns keep_q u8[P], keep_o u8[P,G], n_keep_q = |S^q|, n_keep_o[k] = |S^o(q_k)|
-    (0 for a pruned prompt).
+    mode 0 — independent draws: a prompt is pruned iff cand_q and u_q < r_q; a
+    completion iff cand_o and u_o < r_o.
+    mode 1 — fixed fraction (Appendix A, Algorithm 1): of the prompt candidates
+    B the floor(r_q*|B|) with the smallest (u, index) are pruned; of each
+    prompt's completion candidates C the floor(r_o*|C|) with the smallest
+    (u, index).
+    Every completion of a pruned prompt goes with it.  Returns keep_q u8[P],
+    keep_o u8[P,G], n_keep_q = |S^q|, n_keep_o[k] = |S^o(q_k)| (0 for a pruned
+    prompt).
     """
     cand_q = np.asarray(cand_q); cand_o = np.asarray(cand_o)
     P, G = cand_o.shape
     keep_q = np.ones(P, dtype=np.uint8)
     keep_o = np.ones((P, G), dtype=np.uint8)
-    for k in range(P):
-        if cand_q[k] and float(u_q[k]) < r_q:
+    if mode == 0:
+        for k in range(P):
+            if cand_q[k] and float(u_q[k]) < r_q:
+                keep_q[k] = 0
+            for i in range(G):
+                if cand_o[k, i] and float(u_o[k, i]) < r_o:
+                    keep_o[k, i] = 0
+    else:
+        B = [k for k in range(P) if cand_q[k]]
+        for k in sorted(B, key=lambda k: (float(u_q[k]), k))[: int(math.floor(r_q * len(B)))]:
             keep_q[k] = 0
-        for i in range(G):
-            if (not keep_q[k]) or (cand_o[k, i] and float(u_o[k, i]) < r_o):
+        for k in range(P):
+            C = [i for i in range(G) if cand_o[k, i]]
+            for i in sorted(C, key=lambda i: (float(u_o[k, i]), i))[: int(math.floor(r_o * len(C)))]:
                 keep_o[k, i] = 0
+    for k in range(P):
+        if not keep_q[k]:
+            keep_o[k, :] = 0
     n_keep_q = int(keep_q.sum())
     n_keep_o = keep_o.sum(axis=1).astype(np.int32)
     return keep_q, keep_o, n_keep_q, n_keep_o
@@ -143,11 +160,13 @@ def prune_masks(cand_q, cand_o, u_q, u_o, r_q, r_o):
 # --------------------------------------------------------------------------
 # Step 4 — discrete importance rescaling (Eq. 18) and the history update (Eq. 16)
 # --------------------------------------------------------------------------
-def rescale(cand_q, cand_o, keep_q, keep_o, r_q, r_o, mean_abs_adv, H_prev):
+def rescale(cand_q, cand_o, keep_q, keep_o, r_q, r_o, mean_abs_adv, H_prev, mode=0):
     """gamma_q[k] = (|S^q|/|Q|) / (1 - P^q(q_k)),
     gamma_o[k,i] = (|S^o(q_k)|/|O|) / (1 - P^o(o_i))                      (Eq. 18)
     for retained items (0 for pruned ones), with P^q = r_q on prompt candidates
-    and 0 elsewhere, P^o likewise (Eq. 15, 17).
+    and 0 elsewhere, P^o likewise (Eq. 15, 17).  In fixed-fraction mode the
+    probability that a candidate is pruned is the realised fraction
+    floor(r|C|)/|C| of its candidate set, and that is what P stands for.
 
     w_seq[k,i] is the weight of completion (k,i) in the pruned objective read as
     the mean over RETAINED prompts of gamma_q times the mean over RETAINED
@@ -167,14 +186,24 @@ def rescale(cand_q, cand_o, keep_q, keep_o, r_q, r_o, mean_abs_adv, H_prev):
     gamma_o = np.zeros((P, G), dtype=np.float32)
     w_seq = np.zeros((P, G), dtype=np.float32)
     H_next = np.zeros(P, dtype=np.float32)
+    n_B = int(cand_q.sum())
+    if mode == 0:
+        Pq_cand = r_q
+    else:
+        Pq_cand = (float(int(math.floor(r_q * n_B))) / n_B) if n_B > 0 else 0.0
     for k in range(P):
-        Pq = r_q if cand_q[k] else 0.0
+        Pq = Pq_cand if cand_q[k] else 0.0
         n_o = int(keep_o[k].sum())
+        n_C = int(cand_o[k].sum())
+        if mode == 0:
+            Po_cand = r_o
+        else:
+            Po_cand = (float(int(math.floor(r_o * n_C))) / n_C) if n_C > 0 else 0.0
         if keep_q[k]:
             gamma_q[k] = np.float32((n_q / P) / (1.0 - Pq))
         for i in range(G):
             if keep_o[k, i]:
-                Po = r_o if cand_o[k, i] else 0.0
+                Po = Po_cand if cand_o[k, i] else 0.0
                 gamma_o[k, i] = np.float32((n_o / G) / (1.0 - Po))
                 w_seq[k, i] = np.float32(1.0 / ((float(P * G) * (1.0 - Pq)) * (1.0 - Po)))
         if keep_q[k] or H_prev is None:
@@ -185,7 +214,7 @@ def rescale(cand_q, cand_o, keep_q, keep_o, r_q, r_o, mean_abs_adv, H_prev):
 
 
 def prune_and_rescale(adv, mean_abs_adv, H_prev, r_q, r_o, seed=0, step=0,
-                      u_q=None, u_o=None, reverse=False):
+                      u_q=None, u_o=None, reverse=False, mode=0):
     """Steps 2-4 in one call; u_q/u_o override the generator when given."""
     adv = np.asarray(adv, dtype=np.float32)
     P, G = adv.shape
@@ -195,9 +224,9 @@ def prune_and_rescale(adv, mean_abs_adv, H_prev, r_q, r_o, seed=0, step=0,
         dq, do = draw_uniforms(seed, step, P, G)
         u_q = dq if u_q is None else u_q
         u_o = do if u_o is None else u_o
-    keep_q, keep_o, n_keep_q, n_keep_o = prune_masks(cand_q, cand_o, u_q, u_o, r_q, r_o)
+    keep_q, keep_o, n_keep_q, n_keep_o = prune_masks(cand_q, cand_o, u_q, u_o, r_q, r_o, mode=mode)
     gamma_q, gamma_o, w_seq, H_next = rescale(cand_q, cand_o, keep_q, keep_o, r_q, r_o,
-                                              mean_abs_adv, H_prev)
+                                              mean_abs_adv, H_prev, mode=mode)
     return dict(cand_q=cand_q, cand_o=cand_o, keep_q=keep_q, keep_o=keep_o,
                 n_keep_q=n_keep_q, n_keep_o=n_keep_o, gamma_q=gamma_q, gamma_o=gamma_o,
                 w_seq=w_seq, H_next=H_next)

@@ -12,13 +12,13 @@ from paper_2603_04135_b200 import synth
 
 
 def oracle_prune_pack(batch, w, seed, step, use_history=True, reverse=False, best_fit=False,
-                      r_q=None, r_o=None, N_win=None, L_row=None, u_q=None, u_o=None):
+                      r_q=None, r_o=None, N_win=None, L_row=None, u_q=None, u_o=None, mode=0):
     """Steps 1-5 on the CPU.  The history score is mean |A| of the earlier-epoch rewards (Eq. 16)."""
     adv, mabs = oracle.group_advantages(batch.rewards)
     H_prev = oracle.group_advantages(batch.rewards_prev)[1] if use_history else None
     pr = oracle.prune_and_rescale(adv, mabs, H_prev, w.r_q if r_q is None else r_q,
                                   w.r_o if r_o is None else r_o, seed=seed, step=step, reverse=reverse,
-                                  u_q=u_q, u_o=u_o)
+                                  u_q=u_q, u_o=u_o, mode=mode)
     pk = oracle.pack_prompts(batch.unit_len, w.L_row if L_row is None else L_row,
                              w.N_win if N_win is None else N_win, keep=pr["keep_o"].reshape(-1),
                              loss_len=batch.loss_len, best_fit=best_fit)

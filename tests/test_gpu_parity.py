@@ -88,13 +88,16 @@ def test_prune_explicit_draws_and_modes():
     rng = np.random.default_rng(3)
     u_q = rng.random(w.P); u_o = rng.random((w.P, w.G))
     u_q[:4] = [0.0, 0.25, 0.24999999999999997, 0.9999999999999999]      # exact boundary of u < r
+    u_o[3, :4] = u_o[3, 4]                                              # ties between draws (fixed-fraction order)
     for reverse in (False, True):
-        ref = oracle_prune_pack(batch, w, 0, 0, u_q=u_q, u_o=u_o, reverse=reverse)
-        st = _step(w, 1, reverse=int(reverse))
-        st.set_batch(batch.rewards, batch.unit_len, batch.loss_len, ref["H_prev"])
-        st.prune_pack(u_q=torch.from_numpy(u_q).cuda(), u_o=torch.from_numpy(u_o.reshape(-1)).cuda())
-        assert_prune_equal(st.prune_results(), ref)
-        assert_pack_equal(st.pack_results(), ref["pack"], w.P * w.G)
+        for mode in (0, 1):
+            for r in (0.25, 0.6):
+                ref = oracle_prune_pack(batch, w, 0, 0, u_q=u_q, u_o=u_o, reverse=reverse, mode=mode, r_q=r, r_o=r)
+                st = _step(w, 1, reverse=int(reverse), mode=mode, r_q=r, r_o=r)
+                st.set_batch(batch.rewards, batch.unit_len, batch.loss_len, ref["H_prev"])
+                st.prune_pack(u_q=torch.from_numpy(u_q).cuda(), u_o=torch.from_numpy(u_o.reshape(-1)).cuda())
+                assert_prune_equal(st.prune_results(), ref)
+                assert_pack_equal(st.pack_results(), ref["pack"], w.P * w.G)
 
 
 def test_prune_many_seeds_matches_generator_stream():
@@ -107,6 +110,12 @@ def test_prune_many_seeds_matches_generator_stream():
         st.set_batch(batch.rewards, batch.unit_len, batch.loss_len, ref["H_prev"])
         st.prune_pack(seed=seed, step=step)
         assert_prune_equal(st.prune_results(), ref)
+    st1 = _step(w, 1, mode=1)                                            # fixed fraction through the generator
+    for seed, step in [(5, 6), (2**63, 3)]:
+        ref = oracle_prune_pack(batch, w, seed, step, mode=1)
+        st1.set_batch(batch.rewards, batch.unit_len, batch.loss_len, ref["H_prev"])
+        st1.prune_pack(seed=seed, step=step)
+        assert_prune_equal(st1.prune_results(), ref)
 
 
 # ------------------------------------------------------------------------------------------- step 5

@@ -341,3 +341,69 @@ def test_variance_factor_matches_printed_values():
             assert factor <= printed and printed - factor < 0.02
         else:
             assert math.isclose(factor, printed, rel_tol=1e-3)
+
+
+# ---------------------------------------------------------------- fixed-fraction mode (Appendix A, Algorithm 1)
+def test_fixed_fraction_counts_and_choice():
+    adv, mabs, H = _fixed_case(P=6, G=4, seed=21)
+    P, G = adv.shape
+    rng = np.random.default_rng(1)
+    u_q = rng.random(P); u_o = rng.random((P, G))
+    for r_q, r_o in [(0.5, 0.5), (0.4, 0.7), (0.0, 0.99), (0.99, 0.0)]:
+        out = oracle.prune_and_rescale(adv, mabs, H, r_q, r_o, u_q=u_q, u_o=u_o, mode=1)
+        B = [k for k in range(P) if out["cand_q"][k]]
+        m_q = math.floor(r_q * len(B))
+        pruned_q = [k for k in B if not out["keep_q"][k]]
+        assert len(pruned_q) == m_q                                  # floor(r_q |B|) prompts go
+        assert sorted(pruned_q) == sorted(sorted(B, key=lambda k: (u_q[k], k))[:m_q])   # the smallest draws
+        assert all(out["keep_q"][k] for k in range(P) if k not in B)
+        for k in range(P):
+            C = [i for i in range(G) if out["cand_o"][k, i]]
+            m_o = math.floor(r_o * len(C))
+            if out["keep_q"][k]:
+                pruned_o = [i for i in C if not out["keep_o"][k, i]]
+                assert len(pruned_o) == m_o
+                assert sorted(pruned_o) == sorted(sorted(C, key=lambda i: (u_o[k, i], i))[:m_o])
+                # weights use the realised fraction as the pruning probability
+                for i in range(G):
+                    if out["keep_o"][k, i]:
+                        Pq = (m_q / len(B)) if k in B else 0.0
+                        Po = (m_o / len(C)) if i in C else 0.0
+                        assert math.isclose(out["w_seq"][k, i], 1 / (P * G * (1 - Pq) * (1 - Po)), rel_tol=1e-6)
+            else:
+                assert out["keep_o"][k].sum() == 0
+
+
+def test_fixed_fraction_is_unbiased_with_realised_fraction_only():
+    # enumerate every equally likely choice of the pruned subsets
+    P, G, r_q, r_o = 4, 4, 0.5, 0.5
+    r = np.array([[1, 0, 0, 0], [1, 1, 0, 1], [0, 1, 0, 0], [1, 0, 1, 0]], dtype=np.float32)   # |C| = 3, 3, 3, 4
+    adv, mabs = oracle.group_advantages(r)
+    H = np.array([0.1, 0.9, 0.2, 0.8], dtype=np.float32)
+    ell = np.random.default_rng(3).normal(size=(P, G))
+    cand_o = oracle.completion_candidates(adv); cand_q = oracle.prompt_candidates(H, P)
+    B = [k for k in range(P) if cand_q[k]]
+    Cs = [[i for i in range(G) if cand_o[k, i]] for k in range(P)]
+    m_q = math.floor(r_q * len(B)); m_os = [math.floor(r_o * len(C)) for C in Cs]
+    assert any(r_o * len(C) != m for C, m in zip(Cs, m_os))          # a case where floor() bites
+    choices = [list(itertools.combinations(B, m_q))] + [list(itertools.combinations(C, m)) for C, m in zip(Cs, m_os)]
+    total, total_eq18, n = 0.0, 0.0, 0
+    for pick in itertools.product(*choices):
+        u_q = np.full(P, 0.9); u_o = np.full((P, G), 0.9)
+        for k in pick[0]:
+            u_q[k] = 0.1
+        for k in range(P):
+            for i in pick[1 + k]:
+                u_o[k, i] = 0.1
+        out = oracle.prune_and_rescale(adv, mabs, H, r_q, r_o, u_q=u_q, u_o=u_o, mode=1)
+        total += float((out["w_seq"].astype(np.float64) * ell).sum())
+        # Eq. 18 taken literally (P = r) on the same masks
+        lit = 0.0
+        for k in range(P):
+            for i in range(G):
+                if out["keep_o"][k, i]:
+                    lit += ell[k, i] / (P * G * (1 - (r_q if cand_q[k] else 0)) * (1 - (r_o if cand_o[k, i] else 0)))
+        total_eq18 += lit
+        n += 1
+    assert math.isclose(total / n, ell.mean(), abs_tol=2e-7)
+    assert abs(total_eq18 / n - ell.mean()) > 1e-3                   # the printed factors are biased here
