@@ -184,6 +184,7 @@ def run_reference(args):
 # --------------------------------------------------------------------------------------- ours
 def run_ours(args):
     from paper_2603_04135_b200.step import DppoStep      # raises if libdppo.so is missing: no fallback
+    from paper_2603_04135_b200 import dp
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -205,7 +206,7 @@ def run_ours(args):
         pool = mp.get_context("spawn").Pool(cores)
 
     w = synth.WORKLOADS[WORKLOAD]
-    seed = 3 + rank                                       # every rank has its own batch (data parallel)
+    seed = dp.rank_seed(3, rank)                          # every rank has its own batch (data parallel)
     batch = synth.make_batch(w, seed)
 
     T_cap = int(batch.loss_len.sum())                     # unpruned upper bound of loss tokens
@@ -282,13 +283,7 @@ def run_ours(args):
     del host_tok
 
     # ---- max over ranks, totals over ranks
-    stats = torch.tensor([total_ms, loss_ms, e2e_ms], dtype=torch.float64, device=dev)
-    tokens = torch.tensor([float(T)], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(stats, op=dist.ReduceOp.MAX)
-        dist.all_reduce(tokens, op=dist.ReduceOp.SUM)
-    total_ms, loss_ms, e2e_ms = (float(x) for x in stats.tolist())
-    T_all = float(tokens.item())
+    (total_ms, loss_ms, e2e_ms), T_all = dp.combine_over_ranks([total_ms, loss_ms, e2e_ms], T, device=dev)
 
     if rank == 0:
         ms_per_step = total_ms / args.steps
@@ -296,7 +291,7 @@ def run_ours(args):
         bytes_per_token = w.V * 2 + w.V * 2               # read the bf16 logits once, write bf16 dlogits once
         achieved = T * bytes_per_token / (loss_ms / 1e3) / 1e9
         line = {
-            "metric": METRIC, "value": T_all / (ms_per_step / 1e3), "unit": UNIT, "n_gpus": world,
+            "metric": METRIC, "value": dp.throughput(T_all, ms_per_step), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": WORKLOAD_TEXT, "valid_tokens_per_gpu": T,
@@ -305,7 +300,7 @@ def run_ours(args):
                        "l2": "inputs (%.1f GB) far larger than L2; no flush" % (T * w.V * 2 / 1e9),
                        "parallelism": "dp%d, independent batches" % world},
             "clocks": clocks,
-            "e2e": {"value": T_all / (e2e_ms / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "e2e": {"value": dp.throughput(T_all, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "steps": e2e_steps},
             "gpu_launches": 5 * args.steps,
             "roofline": {"bound": "hbm", "kernel": "grpo loss sweep (rows kernel + its 1-block reduction)",
