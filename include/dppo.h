@@ -217,6 +217,36 @@ int dppo_grpo_loss_fwd_bwd(const dppo_loss_params* p, const void* logits, const 
                            float* loss_out, void* workspace, size_t workspace_bytes,
                            int32_t* status, void* stream);
 
+/* ------------------------------------------------------------------------------------------------
+ * Fused LM-head + loss: the same loss as dppo_grpo_loss_fwd_bwd with the logits z = hidden W^T
+ * produced on the fly by the tensor cores and never written to memory (Eq. 1's pi_theta is the
+ * log-softmax of exactly these logits).
+ *
+ *   loss     the loss parameters; dtype must be DPPO_BF16; row_stride and variant are ignored
+ *   H        hidden width, a multiple of 64
+ *   hidden   bf16 [T_max x H] row-major, one row per loss token in packed order
+ *   W        bf16 [V x H] row-major LM-head weight
+ *   dhidden  bf16 [T_max x H] out, dW [V x H] out: the backward; not built yet — pass NULL for both
+ *            (forward only: loss_out, logp_out, lse_out), anything else returns DPPO_ERR_UNSUPPORTED
+ *   other arguments as in dppo_grpo_loss_fwd_bwd; the workspace holds the same per-row terms.
+ * Errors: INVALID_ARG, BAD_SHAPE (H not a multiple of 64), MISALIGNED, UNSUPPORTED, WORKSPACE_TOO_SMALL,
+ * CUDA (tensor-map creation).  Device status: BAD_TARGET, BAD_SEGMENTS, TIMEOUT.
+ */
+typedef struct {
+    dppo_loss_params loss;
+    int32_t H;
+    int32_t reserved;       /* 0 */
+} dppo_lmhead_params;
+
+size_t dppo_lmhead_workspace_bytes(const dppo_lmhead_params* p);
+
+int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hidden, const void* W,
+                          const int32_t* target, const float* logp_old, const float* logp_ref,
+                          const int32_t* cu_seqlens, const int32_t* n_tokens_dev, const float* adv,
+                          const float* w, const int32_t* seg_map, void* dhidden, void* dW,
+                          float* logp_out, float* lse_out, float* loss_out, void* workspace,
+                          size_t workspace_bytes, int32_t* status, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

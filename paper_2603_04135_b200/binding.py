@@ -45,6 +45,10 @@ class LossParams(ctypes.Structure):
                 ("temperature", ctypes.c_double)]
 
 
+class LmheadParams(ctypes.Structure):
+    _fields_ = [("loss", LossParams), ("H", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
 _vp = ctypes.c_void_p
 lib.dppo_version.restype = ctypes.c_int
 lib.dppo_last_error.restype = ctypes.c_char_p
@@ -63,6 +67,12 @@ lib.dppo_grpo_loss_workspace_bytes.restype = ctypes.c_size_t
 lib.dppo_grpo_loss_workspace_bytes.argtypes = [ctypes.POINTER(LossParams)]
 lib.dppo_grpo_loss_fwd_bwd.restype = ctypes.c_int
 lib.dppo_grpo_loss_fwd_bwd.argtypes = [ctypes.POINTER(LossParams)] + [_vp] * 14 + [ctypes.c_size_t, _vp, _vp]
+
+
+lib.dppo_lmhead_workspace_bytes.restype = ctypes.c_size_t
+lib.dppo_lmhead_workspace_bytes.argtypes = [ctypes.POINTER(LmheadParams)]
+lib.dppo_lmhead_grpo_loss.restype = ctypes.c_int
+lib.dppo_lmhead_grpo_loss.argtypes = [ctypes.POINTER(LmheadParams)] + [_vp] * 16 + [ctypes.c_size_t, _vp, _vp]
 
 
 def _ptr(x):
@@ -143,3 +153,15 @@ def grpo_loss_fwd_bwd(params, logits, target, logp_old, logp_ref, cu_seqlens, n_
                                       _ptr(seg_map), _ptr(dlogits), _ptr(logp_out), _ptr(lse_out),
                                       _ptr(loss_out), _ptr(workspace), workspace_bytes, _ptr(status),
                                       _stream(stream)))
+
+
+def lmhead_workspace_bytes(params):
+    return lib.dppo_lmhead_workspace_bytes(ctypes.byref(params))
+
+
+def lmhead_grpo_loss(params, hidden, W, target, logp_old, logp_ref, cu_seqlens, n_tokens_dev, adv, w, seg_map,
+                     dhidden, dW, logp_out, lse_out, loss_out, workspace, workspace_bytes, status=None, stream=None):
+    _check(lib.dppo_lmhead_grpo_loss(ctypes.byref(params), _ptr(hidden), _ptr(W), _ptr(target), _ptr(logp_old),
+                                     _ptr(logp_ref), _ptr(cu_seqlens), _ptr(n_tokens_dev), _ptr(adv), _ptr(w),
+                                     _ptr(seg_map), _ptr(dhidden), _ptr(dW), _ptr(logp_out), _ptr(lse_out),
+                                     _ptr(loss_out), _ptr(workspace), workspace_bytes, _ptr(status), _stream(stream)))

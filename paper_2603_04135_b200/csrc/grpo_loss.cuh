@@ -93,7 +93,9 @@ struct RowInputs {
     int state;               // 0 ok, else the dppo_status to report (row adds nothing, dlogits zero)
 };
 
-__device__ __forceinline__ void row_inputs_from_segment(const LossArgs& a, long long t, int seg, RowInputs& in) {
+// load_zy = false: the caller supplies z[y] itself (the fused LM-head has no logits in memory).
+__device__ __forceinline__ void row_inputs_from_segment(const LossArgs& a, long long t, int seg, RowInputs& in,
+                                                        bool load_zy = true) {
     in.A = in.W = in.zy = in.logp_old = in.logp_ref = 0.0;
     in.y = a.target[t];
     in.state = 0;
@@ -103,20 +105,21 @@ __device__ __forceinline__ void row_inputs_from_segment(const LossArgs& a, long 
     const int idx = a.seg_map ? a.seg_map[seg] : seg;
     in.A = (double)a.adv[idx];
     in.W = (double)a.w[idx] / (double)(seg_hi - seg_lo);
-    in.zy = (double)(a.bf16 ? Elems<true>::load1(a.logits + t * a.row_bytes, in.y)
-                            : Elems<false>::load1(a.logits + t * a.row_bytes, in.y)) / a.temperature;
+    if (load_zy)
+        in.zy = (double)(a.bf16 ? Elems<true>::load1(a.logits + t * a.row_bytes, in.y)
+                                : Elems<false>::load1(a.logits + t * a.row_bytes, in.y)) / a.temperature;
     in.logp_old = (double)a.logp_old[t];
     in.logp_ref = (double)a.logp_ref[t];
 }
 
 // One thread: binary search for the last s with cu_seqlens[s] <= t, then the gather.
-__device__ __forceinline__ void row_gather(const LossArgs& a, long long t, RowInputs& in) {
+__device__ __forceinline__ void row_gather(const LossArgs& a, long long t, RowInputs& in, bool load_zy = true) {
     int lo = 0, hi = a.S_max;
     while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;
         if ((long long)a.cu_seqlens[mid] <= t) lo = mid; else hi = mid;
     }
-    row_inputs_from_segment(a, t, lo, in);
+    row_inputs_from_segment(a, t, lo, in, load_zy);
 }
 
 // One warp: the same search 32 probes at a time (one memory round trip per factor of 32); lane 0

@@ -174,8 +174,8 @@ def make_token_inputs(w: Workload, T: int, seed: int, device="cpu", sigma_old=No
 
 
 def make_lmhead_inputs(w: Workload, T: int, seed: int, device="cpu"):
-    """hidden bf16 [T, H] ~ N(0,1), LM-head weight bf16 [V, H] ~ N(0, 1/H), uniform targets and
-    perturbed old / reference log-probs centred on z[y]-E[lse] with z ~ N(0,1)."""
+    """hidden bf16 [T, H] ~ N(0,1), LM-head weight bf16 [V, H] ~ N(0, 1/H) (so logits ~ N(0,1)), uniform
+    targets and old / reference log-probs = z[y] - E[lse] + N(0, sigma)."""
     dev = torch.device(device)
     gen = torch.Generator(device=dev)
     gen.manual_seed((int(seed) * 1000003 + 0x1EAD) & 0x7FFFFFFFFFFF)
@@ -187,7 +187,10 @@ def make_lmhead_inputs(w: Workload, T: int, seed: int, device="cpu"):
         W[a:b] = (torch.randn((b - a, w.H), generator=gen, device=dev, dtype=torch.float32)
                   / math.sqrt(w.H)).to(torch.bfloat16)
     target = torch.randint(0, w.V, (T,), generator=gen, device=dev).to(torch.int32)
-    centre = -expected_lse(w) * torch.ones((T,), device=dev, dtype=torch.float32)
+    # the sampled token's logit (one dot product per token) minus the closed-form mean log-sum-exp of
+    # N(0,1) logits centres the old / reference log-probs near the current policy's
+    zy = (hidden.float() * W[target.long()].float()).sum(dim=1)
+    centre = zy - expected_lse(w)
     logp_old = centre + w.sigma_old * torch.randn((T,), generator=gen, device=dev, dtype=torch.float32)
     logp_ref = centre + w.sigma_ref * torch.randn((T,), generator=gen, device=dev, dtype=torch.float32)
     return hidden, W, target, logp_old, logp_ref
