@@ -226,16 +226,21 @@ int dppo_grpo_loss_fwd_bwd(const dppo_loss_params* p, const void* logits, const 
  *   H        hidden width, a multiple of 64
  *   hidden   bf16 [T_max x H] row-major, one row per loss token in packed order
  *   W        bf16 [V x H] row-major LM-head weight
- *   dhidden  bf16 [T_max x H] out, dW [V x H] out: the backward; not built yet — pass NULL for both
- *            (forward only: loss_out, logp_out, lse_out), anything else returns DPPO_ERR_UNSUPPORTED
- *   other arguments as in dppo_grpo_loss_fwd_bwd; the workspace holds the same per-row terms.
+ *   backward 0: forward only (loss_out, logp_out, lse_out; dhidden and dW must be NULL).
+ *            1: also the gradients, dhidden = D W and dW = D^T hidden with D = dlogits recomputed from the
+ *            same GEMM for 8192 tokens at a time into workspace scratch (bf16; never the full [T x V]);
+ *            the workspace then also holds K-major copies of W and hidden
+ *   dhidden  bf16 [T_max x H] out (rows at or past the true token count are zero)
+ *   dW       f32 [V x H] out (overwritten, not accumulated into)
+ *   other arguments as in dppo_grpo_loss_fwd_bwd.  The workspace (dppo_lmhead_workspace_bytes, which
+ *   depends on `backward`) must be 1024-byte aligned.
  * Errors: INVALID_ARG, BAD_SHAPE (H not a multiple of 64), MISALIGNED, UNSUPPORTED, WORKSPACE_TOO_SMALL,
  * CUDA (tensor-map creation).  Device status: BAD_TARGET, BAD_SEGMENTS, TIMEOUT.
  */
 typedef struct {
     dppo_loss_params loss;
     int32_t H;
-    int32_t reserved;       /* 0 */
+    int32_t backward;
 } dppo_lmhead_params;
 
 size_t dppo_lmhead_workspace_bytes(const dppo_lmhead_params* p);

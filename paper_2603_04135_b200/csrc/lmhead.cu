@@ -1,17 +1,22 @@
-// Fused LM-head + GRPO loss: the logits z = hidden W^T are produced tile by tile by the 5th-generation
-// tensor cores (tcgen05.mma, accumulators in tensor memory) and consumed on the spot — the row-wise
-// log-sum-exp and the sampled token's logit are folded in as each 128 x 256 tile leaves TMEM, so the
-// [T x V] logits never exist in HBM (Eq. 1's pi_theta(o_t | ...) is a log-softmax of exactly these).
+// Fused LM-head + GRPO loss on the 5th-generation tensor cores.
 //
-// One persistent CTA per SM owns 128 tokens at a time and sweeps the whole vocabulary:
-//   warp 0      TMA producer: 64-wide K slabs of hidden (128 rows) and of W (256 rows), 128B-swizzled,
-//               into a 4-stage shared-memory ring (no multicast)
-//   warp 1      one elected thread issues tcgen05.mma (M=128, N=256, K=16 x 4 per slab) into one of two
+// Forward: the logits z = hidden W^T are produced tile by tile (tcgen05.mma, accumulators in tensor
+// memory) and consumed on the spot — the row-wise log-sum-exp and the sampled token's logit are folded
+// in as each 128 x 256 tile leaves TMEM, so the [T x V] logits never exist in HBM (Eq. 1's
+// pi_theta(o_t | ...) is a log-softmax of exactly these).
+//
+// Backward: dlogits D = g (onehot - softmax)/tau is recomputed from the same GEMM, one chunk of tokens at
+// a time, into a bounded bf16 scratch (never the full [T x V]); dhidden = D W and dW = D^T hidden are
+// two more runs of the same GEMM core over that chunk.
+//
+// One GEMM core serves all four uses; operands are always K-major (transposed copies of W and hidden
+// are made once per call), only the epilogue differs.  One persistent CTA per SM:
+//   warp 0      TMA producer: 64-wide K slabs of A (128 rows) and of B (256 rows), 128B-swizzled, into
+//               a 4-stage shared-memory ring (no multicast)
+//   warp 1      one thread issues tcgen05.mma (M=128, N=256, K=16 x 4 per slab) into one of two
 //               256-column TMEM accumulators; tcgen05.commit releases smem stages / publishes the tile
-//   warps 2-5   epilogue: each thread owns one token row; tcgen05.ld 32 columns at a time, online
-//               (max, sum 2^x) in the base-2 domain, picks up z[y]; after the last vocabulary tile the
-//               binary64 scalar stage of the loss sweep (same code) writes the row's terms
-// While the epilogue drains accumulator b, the MMA warp already fills accumulator 1-b.
+//   warps 2-5   epilogue: each thread owns one row of the tile and reads it 32 columns at a time with
+//               tcgen05.ld; while it drains accumulator b the MMA warp already fills accumulator 1-b
 // Every wait is bounded; on a timeout the CTA records DPPO_STATUS_TIMEOUT, leaves its loops, frees its
 // tensor memory and returns.
 #include <cuda.h>
@@ -21,8 +26,8 @@
 
 namespace dppo {
 
-constexpr int kBM = 128;                 // tokens per tile (TMEM lanes)
-constexpr int kBN = 256;                 // vocabulary entries per tile (TMEM columns of one accumulator)
+constexpr int kBM = 128;                 // rows per tile (TMEM lanes)
+constexpr int kBN = 256;                 // columns per tile (TMEM columns of one accumulator)
 constexpr int kBK = 64;                  // K slab: 64 bf16 = one 128-byte swizzle row
 constexpr int kStages = 4;
 constexpr int kStageBytesA = kBM * kBK * 2;                  // 16 KB
@@ -31,6 +36,7 @@ constexpr int kStageBytes = kStageBytesA + kStageBytesB;
 constexpr int kLmThreads = 192;
 constexpr int kTmemCols = 512;
 constexpr unsigned long long kLmWaitLimitNs = 2000000000ull;
+constexpr int kChunkTokens = 8192;       // tokens whose dlogits are held in scratch at a time
 
 struct LmShared {
     unsigned long long full[kStages];    // TMA bytes have landed in stage s
@@ -49,16 +55,20 @@ __device__ __forceinline__ unsigned long long lm_global_ns() {
     return t;
 }
 
+__device__ __forceinline__ bool lm_try(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done != 0;
+}
+
 // Bounded wait; also leaves when another role has raised the abort flag.
 __device__ __forceinline__ bool lm_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     const unsigned long long t0 = lm_global_ns();
     for (;;) {
-        uint32_t done;
-        asm volatile("{\n\t.reg .pred p;\n\t"
-                     "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-                     "selp.u32 %0, 1, 0, p;\n\t}"
-                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-        if (done) return true;
+        if (lm_try(bar, parity)) return true;
         if (*abort_flag) return false;
         if (lm_global_ns() - t0 > kLmWaitLimitNs) { *abort_flag = 1; return false; }
     }
@@ -68,12 +78,7 @@ __device__ __forceinline__ bool lm_wait(uint32_t bar, uint32_t parity, volatile 
 __device__ __forceinline__ bool lm_wait_plain(uint32_t bar, uint32_t parity, unsigned long long limit_ns) {
     const unsigned long long t0 = lm_global_ns();
     for (;;) {
-        uint32_t done;
-        asm volatile("{\n\t.reg .pred p;\n\t"
-                     "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-                     "selp.u32 %0, 1, 0, p;\n\t}"
-                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-        if (done) return true;
+        if (lm_try(bar, parity)) return true;
         if (lm_global_ns() - t0 > limit_ns) return false;
     }
 }
@@ -99,22 +104,43 @@ __device__ __forceinline__ uint64_t lm_smem_desc(uint32_t smem_addr) {
 // Instruction descriptor of kind::f16: D = f32, A = B = bf16, both K-major, N = 256, M = 128.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
 
-struct LmArgs {
-    LossArgs loss;          // side inputs, outputs, scalars (logits / dlogits unused)
-    int H;
+// What a launch of the GEMM core covers.  Tile j of a CTA is
+//   row sweep : m = blockIdx.x + (j / n_ntiles) * gridDim.x, n = j % n_ntiles   (a row block keeps its CTA)
+//   flat      : id = blockIdx.x + j * gridDim.x; m_fast ? (m = id % n_mtiles, n = id / n_mtiles)
+//                                                        : (m = id / n_ntiles, n = id % n_ntiles)
+struct GemmShape {
     int n_mtiles, n_ntiles, n_ksteps;
+    int a_row0;                          // row offset added to A's TMA coordinate
+    int m_fast;
 };
 
+template <bool kRowSweep>
+__device__ __forceinline__ bool tile_of(const GemmShape& gs, uint32_t j, int& m, int& n) {
+    if (kRowSweep) {
+        m = blockIdx.x + (int)(j / (uint32_t)gs.n_ntiles) * gridDim.x;
+        n = (int)(j % (uint32_t)gs.n_ntiles);
+        return m < gs.n_mtiles;
+    }
+    const long long id = (long long)blockIdx.x + (long long)j * gridDim.x;
+    if (id >= (long long)gs.n_mtiles * gs.n_ntiles) return false;
+    if (gs.m_fast) { m = (int)(id % gs.n_mtiles); n = (int)(id / gs.n_mtiles); }
+    else           { m = (int)(id / gs.n_ntiles); n = (int)(id % gs.n_ntiles); }
+    return true;
+}
+
+// ---- the GEMM core --------------------------------------------------------------------------------
+// Epi (one copy per epilogue thread = per tile row):
+//   void row_begin(int m, int row)                       row sweep: at n == 0; flat: every tile
+//   void chunk(int m, int n, int row, int ch, uint32_t (&v)[32])   32 accumulator columns (f32 bits)
+//   void row_end(int m, int row)                         row sweep: after the last n; flat: every tile
+template <class Epi, bool kRowSweep>
 __global__ void __launch_bounds__(kLmThreads, 1)
-lmhead_fwd_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_constant__ CUtensorMap map_w,
-                  const LmArgs g) {
+lm_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const GemmShape gs, Epi epi, int32_t* status) {
     extern __shared__ unsigned char lm_raw[];
     __shared__ LmShared sh;
     const uint32_t tiles = (lm_smem_u32(lm_raw) + 1023u) & ~1023u;      // 1024-byte aligned ring (swizzle atoms)
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const LossArgs& a = g.loss;
-    const long long T = a.n_tokens_dev ? min((long long)*a.n_tokens_dev, a.T_max) : a.T_max;
-    const int n_mtiles = (int)min((long long)g.n_mtiles, (T + kBM - 1) / kBM);
     volatile int* abort_flag = &sh.abort;
 
     if (tid == 0) {
@@ -143,28 +169,27 @@ lmhead_fwd_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_c
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            uint32_t it = 0;                                             // slab counter over the whole CTA lifetime
-            for (int m = blockIdx.x; m < n_mtiles && !*abort_flag; m += gridDim.x) {
-                for (int n = 0; n < g.n_ntiles && !*abort_flag; ++n) {
-                    for (int k = 0; k < g.n_ksteps; ++k, ++it) {
-                        const uint32_t s = it % kStages, use = it / kStages;
-                        if (use > 0 && !lm_wait(lm_smem_u32(&sh.empty[s]), (use - 1) & 1, abort_flag)) break;
-                        const uint32_t bar = lm_smem_u32(&sh.full[s]);
-                        const uint32_t dst_a = tiles + s * kStageBytes, dst_b = dst_a + kStageBytesA;
-                        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"((uint32_t)kStageBytes) : "memory");
-                        asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-                                     :: "r"(dst_a), "l"(&map_hidden), "r"(bar), "r"(k * kBK), "r"(m * kBM) : "memory");
-                        asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-                                     :: "r"(dst_b), "l"(&map_w), "r"(bar), "r"(k * kBK), "r"(n * kBN) : "memory");
-                    }
+            uint32_t it = 0;                                             // slab counter over the CTA's lifetime
+            int m, n;
+            for (uint32_t j = 0; tile_of<kRowSweep>(gs, j, m, n) && !*abort_flag; ++j) {
+                for (int k = 0; k < gs.n_ksteps; ++k, ++it) {
+                    const uint32_t s = it % kStages, use = it / kStages;
+                    if (use > 0 && !lm_wait(lm_smem_u32(&sh.empty[s]), (use - 1) & 1, abort_flag)) break;
+                    const uint32_t bar = lm_smem_u32(&sh.full[s]);
+                    const uint32_t dst_a = tiles + s * kStageBytes, dst_b = dst_a + kStageBytesA;
+                    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"((uint32_t)kStageBytes) : "memory");
+                    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                                 :: "r"(dst_a), "l"(&map_a), "r"(bar), "r"(k * kBK), "r"(gs.a_row0 + m * kBM) : "memory");
+                    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                                 :: "r"(dst_b), "l"(&map_b), "r"(bar), "r"(k * kBK), "r"(n * kBN) : "memory");
                 }
             }
             if (*abort_flag) {
                 // leaving early: give this thread's own copies in flight a bounded chance to land before
                 // the CTA (and its shared memory) goes away
                 const uint32_t pending = it < (uint32_t)kStages ? it : (uint32_t)kStages;
-                for (uint32_t j = 0; j < pending; ++j) {
-                    const uint32_t i2 = it - 1 - j;
+                for (uint32_t i = 0; i < pending; ++i) {
+                    const uint32_t i2 = it - 1 - i;
                     lm_wait_plain(lm_smem_u32(&sh.full[i2 % kStages]), (i2 / kStages) & 1, 200000000ull);
                 }
             }
@@ -172,111 +197,282 @@ lmhead_fwd_kernel(const __grid_constant__ CUtensorMap map_hidden, const __grid_c
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            uint32_t it = 0, tile = 0;
-            for (int m = blockIdx.x; m < n_mtiles && !*abort_flag; m += gridDim.x) {
-                for (int n = 0; n < g.n_ntiles && !*abort_flag; ++n, ++tile) {
-                    const uint32_t b = tile & 1, use_b = tile >> 1;
-                    if (use_b > 0 && !lm_wait(lm_smem_u32(&sh.acc_empty[b]), (use_b - 1) & 1, abort_flag)) break;
+            uint32_t it = 0;
+            int m, n;
+            for (uint32_t j = 0; tile_of<kRowSweep>(gs, j, m, n) && !*abort_flag; ++j) {
+                const uint32_t b = j & 1, use_b = j >> 1;
+                if (use_b > 0 && !lm_wait(lm_smem_u32(&sh.acc_empty[b]), (use_b - 1) & 1, abort_flag)) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t d_tmem = tmem_base + b * kBN;
+                bool ok = true;
+                for (int k = 0; k < gs.n_ksteps; ++k, ++it) {
+                    const uint32_t s = it % kStages, use = it / kStages;
+                    if (!lm_wait(lm_smem_u32(&sh.full[s]), use & 1, abort_flag)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const uint32_t d_tmem = tmem_base + b * kBN;
-                    bool ok = true;
-                    for (int k = 0; k < g.n_ksteps; ++k, ++it) {
-                        const uint32_t s = it % kStages, use = it / kStages;
-                        if (!lm_wait(lm_smem_u32(&sh.full[s]), use & 1, abort_flag)) { ok = false; break; }
-                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                        const uint32_t sa = tiles + s * kStageBytes, sb = sa + kStageBytesA;
-                        const uint64_t da = lm_smem_desc(sa), db = lm_smem_desc(sb);
+                    const uint32_t sa = tiles + s * kStageBytes, sb = sa + kStageBytesA;
+                    const uint64_t da = lm_smem_desc(sa), db = lm_smem_desc(sb);
 #pragma unroll
-                        for (int kk = 0; kk < kBK / 16; ++kk) {          // 16 K elements = 32 bytes inside the swizzle row
-                            const uint32_t accumulate = (k > 0 || kk > 0) ? 1u : 0u;
-                            asm volatile("{\n\t.reg .pred p;\n\t"
-                                         "setp.ne.b32 p, %4, 0;\n\t"
-                                         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                                         :: "r"(d_tmem), "l"(da + (uint64_t)(kk * 2)), "l"(db + (uint64_t)(kk * 2)),
-                                            "r"(kIdesc), "r"(accumulate) : "memory");
-                        }
-                        // frees this smem stage once the MMAs issued so far have read it
-                        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
-                                     :: "r"(lm_smem_u32(&sh.empty[s])) : "memory");
+                    for (int kk = 0; kk < kBK / 16; ++kk) {              // 16 K elements = 32 bytes inside the swizzle row
+                        const uint32_t accumulate = (k > 0 || kk > 0) ? 1u : 0u;
+                        asm volatile("{\n\t.reg .pred p;\n\t"
+                                     "setp.ne.b32 p, %4, 0;\n\t"
+                                     "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                                     :: "r"(d_tmem), "l"(da + (uint64_t)(kk * 2)), "l"(db + (uint64_t)(kk * 2)),
+                                        "r"(kIdesc), "r"(accumulate) : "memory");
                     }
-                    if (!ok) break;
+                    // frees this smem stage once the MMAs issued so far have read it
                     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
-                                 :: "r"(lm_smem_u32(&sh.acc_full[b])) : "memory");
+                                 :: "r"(lm_smem_u32(&sh.empty[s])) : "memory");
                 }
+                if (!ok) break;
+                asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                             :: "r"(lm_smem_u32(&sh.acc_full[b])) : "memory");
             }
         }
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..5)
         const int q = warp & 3;                                          // TMEM lane quarter this warp may read
         const int row = q * 32 + lane;
-        const float c = a.scale2;
-        uint32_t tile = 0;
-        for (int m = blockIdx.x; m < n_mtiles; m += gridDim.x) {
-            const long long t = (long long)m * kBM + row;
-            const bool live = t < T;
-            RowInputs in;
-            in.state = 0; in.y = -1;
-            if (live) row_gather(a, t, in, false);
-            const int y = (live && in.state == 0) ? in.y : -1;
-            float m2 = -INFINITY, s = 0.0f, zy = 0.0f;
-            bool ok = true;
-            for (int n = 0; n < g.n_ntiles; ++n, ++tile) {
-                const uint32_t b = tile & 1, use_b = tile >> 1;
-                // warp-uniform outcome: the tcgen05.ld below must be executed by all 32 lanes together
-                if (!__all_sync(0xffffffffu, lm_wait(lm_smem_u32(&sh.acc_full[b]), use_b & 1, abort_flag))) { ok = false; break; }
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + b * kBN;
+        int m, n;
+        for (uint32_t j = 0; tile_of<kRowSweep>(gs, j, m, n); ++j) {
+            const uint32_t b = j & 1, use_b = j >> 1;
+            if (!kRowSweep || n == 0) epi.row_begin(m, row);
+            // warp-uniform outcome: the tcgen05.ld below must be executed by all 32 lanes together
+            if (!__all_sync(0xffffffffu, lm_wait(lm_smem_u32(&sh.acc_full[b]), use_b & 1, abort_flag))) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + b * kBN;
 #pragma unroll 1
-                for (int ch = 0; ch < kBN / 32; ++ch) {
-                    uint32_t v[32];
-                    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-                                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-                                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-                                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-                                   "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-                                   "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-                                   "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-                                 : "r"(taddr + (uint32_t)(ch * 32)) : "memory");
-                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                    const int col0 = n * kBN + ch * 32;
-                    const int valid = a.V - col0;                        // columns of this chunk inside the vocabulary
-                    float cm = -INFINITY;
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        float x = __uint_as_float(v[j]);
-                        if (j == y - col0) zy = x;
-                        x = (j < valid) ? x * c : -INFINITY;
-                        v[j] = __float_as_uint(x);
-                        cm = fmaxf(cm, x);
-                    }
-                    if (cm > m2) { s *= lm_ex2(m2 - cm); m2 = cm; }
-                    float acc0 = 0.0f, acc1 = 0.0f;
-#pragma unroll
-                    for (int j = 0; j < 32; j += 2) {
-                        acc0 += lm_ex2(__uint_as_float(v[j]) - m2);
-                        acc1 += lm_ex2(__uint_as_float(v[j + 1]) - m2);
-                    }
-                    s += acc0 + acc1;
-                }
-                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-                __syncwarp();
-                if (lane == 0) lm_arrive(lm_smem_u32(&sh.acc_empty[b]));
+            for (int ch = 0; ch < kBN / 32; ++ch) {
+                uint32_t v[32];
+                asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                             "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                             "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                             : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                               "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+                               "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+                               "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                             : "r"(taddr + (uint32_t)(ch * 32)) : "memory");
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                epi.chunk(m, n, row, ch, v);
             }
-            if (!ok) break;
-            if (live) {
-                in.zy = (double)zy / a.temperature;
-                row_finish(a, t, in, m2, s, true);
-            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) lm_arrive(lm_smem_u32(&sh.acc_empty[b]));
+            if (!kRowSweep || n == gs.n_ntiles - 1) epi.row_end(m, row);
         }
     }
 
     // ---- common exit: nobody touches tensor memory any more, then the allocating warp frees it
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    if (tid == 0 && sh.abort) set_status(a.status, DPPO_STATUS_TIMEOUT);
+    if (tid == 0 && sh.abort) set_status(status, DPPO_STATUS_TIMEOUT);
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
+    }
+}
+
+// ---- epilogues ------------------------------------------------------------------------------------
+struct RowInfo {             // what the backward needs from the forward, per token
+    float lse2_hi, lse2_lo;  // base-2 log-sum-exp of z * scale2
+    float g_over_tau;        // dloss/dlogp / temperature (0 for rows that add nothing)
+    int y;                   // target, -1 if the row is invalid
+};
+
+// Forward: online (max, sum 2^x) over the vocabulary, z[y], then the loss's scalar stage.
+struct EpiLse {
+    LossArgs a;
+    RowInfo* info;           // nullable
+    // per-thread state
+    RowInputs in;
+    long long T;
+    float m2, s, zy;
+    int y;
+    bool live;
+    __device__ __forceinline__ void row_begin(int m, int row) {
+        T = a.n_tokens_dev ? min((long long)*a.n_tokens_dev, a.T_max) : a.T_max;
+        const long long t = (long long)m * kBM + row;
+        live = t < T;
+        in.state = 0; in.y = -1;
+        if (live) row_gather(a, t, in, false);
+        y = (live && in.state == 0) ? in.y : -1;
+        m2 = -INFINITY; s = 0.0f; zy = 0.0f;
+    }
+    __device__ __forceinline__ void chunk(int, int n, int, int ch, uint32_t (&v)[32]) {
+        const int col0 = n * kBN + ch * 32;
+        const int valid = a.V - col0;                                // columns of this chunk inside the vocabulary
+        const float c = a.scale2;
+        if (y >= col0 && y < col0 + 32) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) if (j == y - col0) zy = __uint_as_float(v[j]);
+        }
+        float cm = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            const float x = (j < valid) ? __uint_as_float(v[j]) * c : -INFINITY;
+            v[j] = __float_as_uint(x);
+            cm = fmaxf(cm, x);
+        }
+        if (cm > m2) { s *= lm_ex2(m2 - cm); m2 = cm; }
+        float acc0 = 0.0f, acc1 = 0.0f;
+#pragma unroll
+        for (int j = 0; j < 32; j += 2) {
+            acc0 += lm_ex2(__uint_as_float(v[j]) - m2);
+            acc1 += lm_ex2(__uint_as_float(v[j + 1]) - m2);
+        }
+        s += acc0 + acc1;
+    }
+    __device__ __forceinline__ void row_end(int m, int row) {
+        const long long t = (long long)m * kBM + row;
+        if (!live) {
+            if (info && t < a.T_max) { RowInfo z; z.lse2_hi = 0.0f; z.lse2_lo = 0.0f; z.g_over_tau = 0.0f; z.y = -1; info[t] = z; }
+            return;
+        }
+        in.zy = (double)zy / a.temperature;
+        const RowScalars rs = row_finish(a, t, in, m2, s, true);
+        if (info) {
+            RowInfo ri;
+            ri.lse2_hi = rs.lse2_hi; ri.lse2_lo = rs.lse2_lo;
+            ri.g_over_tau = rs.valid ? rs.g_over_tau : 0.0f;
+            ri.y = rs.valid ? in.y : -1;
+            info[t] = ri;
+        }
+    }
+};
+
+// Backward, step 1: dlogits of a chunk of tokens, written as bf16 both ways round:
+//   D  [chunk tokens x ldd]  (row = token)       feeds dhidden = D W
+//   Dt [V x ldt]             (row = vocabulary)  feeds dW = D^T hidden
+// Rows past the true token count get g = 0 from the forward, i.e. zeros.
+struct EpiDlogits {
+    const RowInfo* info;
+    __nv_bfloat16* D;
+    __nv_bfloat16* Dt;
+    long long t0, tc;        // first token of the chunk, tokens in the chunk
+    long long ldd, ldt;
+    int V;
+    float c;
+    RowInfo ri;
+    bool live;
+    __device__ __forceinline__ void row_begin(int m, int row) {
+        const long long r = (long long)m * kBM + row;
+        live = r < tc;
+        if (live) ri = info[t0 + r];
+        else { ri.lse2_hi = 0.0f; ri.lse2_lo = 0.0f; ri.g_over_tau = 0.0f; ri.y = -1; }
+    }
+    __device__ __forceinline__ void chunk(int m, int n, int row, int ch, uint32_t (&v)[32]) {
+        const int col0 = n * kBN + ch * 32;
+        if (col0 >= V || !live) return;
+        const long long r = (long long)m * kBM + row;                // token index inside the chunk
+        const float g = ri.g_over_tau;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            const float p = lm_ex2(fmaf(__uint_as_float(v[j]), c, -ri.lse2_hi) - ri.lse2_lo);
+            float d = -g * p;
+            if (col0 + j == ri.y) d += g;
+            v[j] = __float_as_uint(d);
+        }
+        if (col0 + 32 <= V) {                                        // ldd is a multiple of 8: 16-byte stores
+            uint32_t pk[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+                pk[j] = *reinterpret_cast<const uint32_t*>(&b2);
+            }
+            uint4* dst = reinterpret_cast<uint4*>(D + r * ldd + col0);
+            dst[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            dst[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+            dst[2] = make_uint4(pk[8], pk[9], pk[10], pk[11]);
+            dst[3] = make_uint4(pk[12], pk[13], pk[14], pk[15]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (col0 + j < V) D[r * ldd + col0 + j] = __float2bfloat16_rn(__uint_as_float(v[j]));
+        }
+        // transposed copy: for a fixed column the 32 lanes of a warp write 32 consecutive tokens (64 bytes)
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+            if (col0 + j < V) Dt[(long long)(col0 + j) * ldt + r] = __float2bfloat16_rn(__uint_as_float(v[j]));
+    }
+    __device__ __forceinline__ void row_end(int, int) {}
+};
+
+// C[rows x ldc] = acc as bf16 (dhidden).
+struct EpiStoreBf16 {
+    __nv_bfloat16* C;
+    long long ldc, row0, rows;   // output row of tile row 0; rows that exist in C
+    int cols;
+    __device__ __forceinline__ void row_begin(int, int) {}
+    __device__ __forceinline__ void chunk(int m, int n, int row, int ch, uint32_t (&v)[32]) {
+        const long long r = row0 + (long long)m * kBM + row;
+        const int col0 = n * kBN + ch * 32;
+        if (r >= rows || col0 >= cols) return;
+        __nv_bfloat16* dst = C + r * ldc + col0;
+        if (col0 + 32 <= cols) {
+            uint32_t pk[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+                pk[j] = *reinterpret_cast<const uint32_t*>(&b2);
+            }
+            uint4* d4 = reinterpret_cast<uint4*>(dst);
+            d4[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            d4[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+            d4[2] = make_uint4(pk[8], pk[9], pk[10], pk[11]);
+            d4[3] = make_uint4(pk[12], pk[13], pk[14], pk[15]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) if (col0 + j < cols) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
+        }
+    }
+    __device__ __forceinline__ void row_end(int, int) {}
+};
+
+// C[rows x ldc] (f32) = or += acc (dW, accumulated over the token chunks).
+struct EpiAccumF32 {
+    float* C;
+    long long ldc, rows;
+    int cols, accumulate;
+    __device__ __forceinline__ void row_begin(int, int) {}
+    __device__ __forceinline__ void chunk(int m, int n, int row, int ch, uint32_t (&v)[32]) {
+        const long long r = (long long)m * kBM + row;
+        const int col0 = n * kBN + ch * 32;
+        if (r >= rows || col0 >= cols) return;
+        float* dst = C + r * ldc + col0;
+        if (col0 + 32 <= cols) {                                     // ldc is a multiple of 64: 16-byte accesses
+            float4* d4 = reinterpret_cast<float4*>(dst);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                float4 x = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                       __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+                if (accumulate) { const float4 o = d4[j]; x.x += o.x; x.y += o.y; x.z += o.z; x.w += o.w; }
+                d4[j] = x;
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (col0 + j < cols) dst[j] = (accumulate ? dst[j] : 0.0f) + __uint_as_float(v[j]);
+        }
+    }
+    __device__ __forceinline__ void row_end(int, int) {}
+};
+
+// out[c x ldo] = in[r x ldi]^T for bf16, 64 x 64 tiles through shared memory; columns r..ldo-1 of out are
+// left untouched (never read: tensor maps stop at r).
+__global__ void __launch_bounds__(256)
+transpose_bf16_kernel(const __nv_bfloat16* __restrict__ in, long long rows, long long cols, long long ldi,
+                      __nv_bfloat16* __restrict__ out, long long ldo) {
+    __shared__ __nv_bfloat16 tile[64][66];
+    const long long r0 = (long long)blockIdx.y * 64, c0 = (long long)blockIdx.x * 64;
+    const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
+    for (int i = ty; i < 64; i += 4) {
+        const long long r = r0 + i, c = c0 + tx;
+        tile[i][tx] = (r < rows && c < cols) ? in[r * ldi + c] : __float2bfloat16_rn(0.0f);
+    }
+    __syncthreads();
+    for (int i = ty; i < 64; i += 4) {
+        const long long c = c0 + i, r = r0 + tx;
+        if (c < cols && r < rows) out[c * ldo + r] = tile[tx][i];
     }
 }
 
@@ -297,12 +493,13 @@ static EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-// [rows x H] bf16 row-major; boxes of 64 columns x box_rows rows, 128B swizzle, zero fill out of bounds.
-static int make_map(CUtensorMap* map, const void* base, long long rows, int H, int box_rows) {
+// bf16 [rows x cols] with row pitch ld elements; boxes of 64 columns x box_rows rows, 128B swizzle, zero fill
+// outside [rows x cols].
+static int make_map(CUtensorMap* map, const void* base, long long rows, long long cols, long long ld, int box_rows) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return fail(DPPO_ERR_CUDA, "lmhead: cuTensorMapEncodeTiled is not available from this driver");
-    const cuuint64_t dims[2] = {(cuuint64_t)H, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)H * 2};
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
     const cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
@@ -312,11 +509,56 @@ static int make_map(CUtensorMap* map, const void* base, long long rows, int H, i
     return DPPO_OK;
 }
 
+constexpr size_t kLmDynSmem = (size_t)kStages * kStageBytes + 1024;
+
+template <class Epi, bool kRowSweep>
+static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const GemmShape& gs, const Epi& epi,
+                       int32_t* status, cudaStream_t s, const char* what) {
+    auto kernel = lm_gemm_kernel<Epi, kRowSweep>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLmDynSmem);
+    if (e != cudaSuccess) return cuda_fail(e, "lmhead: shared memory attribute");
+    const long long work = kRowSweep ? gs.n_mtiles : (long long)gs.n_mtiles * gs.n_ntiles;
+    const int grid = (int)(work < sm_count() ? work : sm_count());
+    if (grid < 1) return DPPO_OK;
+    kernel<<<grid, kLmThreads, kLmDynSmem, s>>>(ma, mb, gs, epi, status);
+    cudaError_t e2 = cudaGetLastError();
+    if (e2 != cudaSuccess) return cuda_fail(e2, what);
+    return DPPO_OK;
+}
+
+static long long round_up(long long x, long long m) { return (x + m - 1) / m * m; }
+
+struct LmWorkspace {
+    size_t terms, info, wt, ht, d, dt, total;    // byte offsets and the total
+    long long ld_v, ld_t, ld_tc;                 // pitches: vocabulary (D, Wt), tokens (ht), chunk tokens (Dt)
+};
+
+static LmWorkspace lm_layout(const dppo_lmhead_params* p, bool backward) {
+    LmWorkspace w;
+    const long long T = p->loss.T_max > 0 ? p->loss.T_max : 1;
+    auto al = [](size_t x) { return (x + 1023) & ~(size_t)1023; };
+    w.ld_v = round_up(p->loss.V, 8);
+    w.ld_t = round_up(T, 8);
+    w.ld_tc = kChunkTokens;
+    size_t off = 0;
+    w.terms = off; off += al((size_t)T * sizeof(RowTerms));
+    w.info = off;  off += al((size_t)T * sizeof(RowInfo));
+    w.wt = w.ht = w.d = w.dt = off;
+    if (backward) {
+        w.wt = off; off += al((size_t)p->H * w.ld_v * 2);
+        w.ht = off; off += al((size_t)p->H * w.ld_t * 2);
+        w.d = off;  off += al((size_t)kChunkTokens * w.ld_v * 2);
+        w.dt = off; off += al((size_t)p->loss.V * w.ld_tc * 2);
+    }
+    w.total = off;
+    return w;
+}
+
 }  // namespace dppo
 
 extern "C" size_t dppo_lmhead_workspace_bytes(const dppo_lmhead_params* p) {
-    if (!p) return 0;
-    return dppo_grpo_loss_workspace_bytes(&p->loss);
+    if (!p || p->loss.T_max < 0 || p->loss.V < 1 || p->H < 1) return 0;
+    return dppo::lm_layout(p, p->backward != 0).total;
 }
 
 extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hidden, const void* W,
@@ -334,46 +576,102 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
     if (lp.dtype != DPPO_BF16) return fail(DPPO_ERR_UNSUPPORTED, "lmhead: hidden and W must be bf16");
     if (!(lp.temperature > 0.0) || !(lp.eps_lo >= 0.0) || !(lp.eps_hi >= 0.0) || !(lp.beta == lp.beta))
         return fail(DPPO_ERR_INVALID_ARG, "lmhead: temperature must be > 0, eps >= 0, beta a number");
-    if (lp.T_max >= ((int64_t)1 << 31) - kBM) return fail(DPPO_ERR_BAD_SHAPE, "lmhead: T_max too large");
-    if (dhidden || dW) return fail(DPPO_ERR_UNSUPPORTED, "lmhead: the backward (dhidden, dW) is not built yet; pass NULL for both");
+    if (lp.T_max >= ((int64_t)1 << 31) - kChunkTokens) return fail(DPPO_ERR_BAD_SHAPE, "lmhead: T_max too large");
+    const bool backward = p->backward != 0;
+    if (backward && (!dhidden || !dW)) return fail(DPPO_ERR_INVALID_ARG, "lmhead: backward requested but dhidden / dW is NULL");
+    if (!backward && (dhidden || dW)) return fail(DPPO_ERR_INVALID_ARG, "lmhead: dhidden / dW given but params.backward is 0");
     if (!loss_out) return fail(DPPO_ERR_INVALID_ARG, "lmhead: NULL loss_out");
     if (lp.T_max > 0) {
         if (!hidden || !W || !target || !logp_old || !logp_ref || !cu_seqlens || !adv || !w)
             return fail(DPPO_ERR_INVALID_ARG, "lmhead: NULL array");
         if (lp.S_max < 1) return fail(DPPO_ERR_BAD_SHAPE, "lmhead: tokens but no sequences (S_max=0)");
-        if (((uintptr_t)hidden & 15) || ((uintptr_t)W & 15)) return fail(DPPO_ERR_MISALIGNED, "lmhead: hidden / W not 16-byte aligned");
+        if (((uintptr_t)hidden & 15) || ((uintptr_t)W & 15) || ((uintptr_t)dhidden & 15) || ((uintptr_t)dW & 15))
+            return fail(DPPO_ERR_MISALIGNED, "lmhead: hidden / W / dhidden / dW not 16-byte aligned");
     }
-    const size_t need = dppo_lmhead_workspace_bytes(p);
-    if (!workspace || workspace_bytes < need)
-        return fail(DPPO_ERR_WORKSPACE_TOO_SMALL, "lmhead: workspace %zu < %zu bytes", workspace_bytes, need);
-    if ((uintptr_t)workspace & 15) return fail(DPPO_ERR_MISALIGNED, "lmhead: workspace not 16-byte aligned");
+    const LmWorkspace lay = lm_layout(p, backward);
+    if (!workspace || workspace_bytes < lay.total)
+        return fail(DPPO_ERR_WORKSPACE_TOO_SMALL, "lmhead: workspace %zu < %zu bytes", workspace_bytes, lay.total);
+    if ((uintptr_t)workspace & 1023) return fail(DPPO_ERR_MISALIGNED, "lmhead: workspace not 1024-byte aligned");
+    char* ws = (char*)workspace;
 
-    LmArgs g;
-    LossArgs& a = g.loss;
+    LossArgs a;
     a.logits = nullptr; a.dlogits = nullptr;
     a.target = target; a.logp_old = logp_old; a.logp_ref = logp_ref;
     a.cu_seqlens = cu_seqlens; a.n_tokens_dev = n_tokens_dev; a.adv = adv; a.w = w; a.seg_map = seg_map;
-    a.logp_out = logp_out; a.lse_out = lse_out; a.terms = (RowTerms*)workspace; a.status = status;
+    a.logp_out = logp_out; a.lse_out = lse_out; a.terms = (RowTerms*)(ws + lay.terms); a.status = status;
     a.T_max = lp.T_max; a.row_bytes = 0; a.V = lp.V; a.S_max = lp.S_max; a.bf16 = 1;
     a.eps_lo = lp.eps_lo; a.eps_hi = lp.eps_hi; a.beta = lp.beta; a.temperature = lp.temperature;
     a.scale2 = (float)(1.4426950408889634 / lp.temperature);
-    g.H = p->H;
-    g.n_mtiles = (int)((lp.T_max + kBM - 1) / kBM);
-    g.n_ntiles = (lp.V + kBN - 1) / kBN;
-    g.n_ksteps = p->H / kBK;
     cudaStream_t s = (cudaStream_t)stream;
-    if (lp.T_max > 0) {
+    const int H = p->H, V = lp.V;
+    const long long T = lp.T_max;          // host-side bound; rows at or past the device-side count carry g = 0
+    if (T > 0) {
         alignas(64) CUtensorMap map_h, map_w;
-        int rc = make_map(&map_h, hidden, lp.T_max, p->H, kBM);
+        int rc = make_map(&map_h, hidden, T, H, H, kBM);
         if (rc != DPPO_OK) return rc;
-        rc = make_map(&map_w, W, lp.V, p->H, kBN);
+        rc = make_map(&map_w, W, V, H, H, kBN);
         if (rc != DPPO_OK) return rc;
-        const size_t dyn = (size_t)kStages * kStageBytes + 1024;
-        cudaError_t e = cudaFuncSetAttribute(lmhead_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
-        if (e != cudaSuccess) return cuda_fail(e, "lmhead: shared memory attribute");
-        const int grid = g.n_mtiles < sm_count() ? g.n_mtiles : sm_count();
-        lmhead_fwd_kernel<<<grid, kLmThreads, dyn, s>>>(map_h, map_w, g);
-        DPPO_CHECK_LAUNCH("lmhead forward launch");
+        RowInfo* info = (RowInfo*)(ws + lay.info);
+
+        // ---- forward: lse, logp, loss terms (and what the backward needs per row)
+        GemmShape gs = {};
+        gs.n_mtiles = (int)((T + kBM - 1) / kBM); gs.n_ntiles = (V + kBN - 1) / kBN; gs.n_ksteps = H / kBK;
+        EpiLse fwd = {};
+        fwd.a = a; fwd.info = backward ? info : nullptr;
+        rc = launch_gemm<EpiLse, true>(map_h, map_w, gs, fwd, status, s, "lmhead forward launch");
+        if (rc != DPPO_OK) return rc;
+
+        if (backward) {
+            __nv_bfloat16* Wt = (__nv_bfloat16*)(ws + lay.wt);
+            __nv_bfloat16* ht = (__nv_bfloat16*)(ws + lay.ht);
+            __nv_bfloat16* D = (__nv_bfloat16*)(ws + lay.d);
+            __nv_bfloat16* Dt = (__nv_bfloat16*)(ws + lay.dt);
+            // K-major copies of the two operands that are contracted over their row index
+            transpose_bf16_kernel<<<dim3((H + 63) / 64, (V + 63) / 64), 256, 0, s>>>(
+                (const __nv_bfloat16*)W, V, H, H, Wt, lay.ld_v);
+            transpose_bf16_kernel<<<dim3((H + 63) / 64, (unsigned)((T + 63) / 64)), 256, 0, s>>>(
+                (const __nv_bfloat16*)hidden, T, H, H, ht, lay.ld_t);
+            DPPO_CHECK_LAUNCH("lmhead transpose launch");
+            alignas(64) CUtensorMap map_wt;
+            rc = make_map(&map_wt, Wt, H, V, lay.ld_v, kBN);
+            if (rc != DPPO_OK) return rc;
+
+            for (long long t0 = 0, c = 0; t0 < T; t0 += kChunkTokens, ++c) {
+                const long long tc = (T - t0) < kChunkTokens ? (T - t0) : kChunkTokens;     // tokens in this chunk
+                // (1) dlogits of the chunk: D [tc x V] and Dt [V x tc]
+                GemmShape g1 = {};
+                g1.n_mtiles = (int)((tc + kBM - 1) / kBM); g1.n_ntiles = (V + kBN - 1) / kBN; g1.n_ksteps = H / kBK;
+                g1.a_row0 = (int)t0; g1.m_fast = 1;                                        // neighbours share the W tile
+                EpiDlogits e1 = {};
+                e1.info = info; e1.D = D; e1.Dt = Dt; e1.t0 = t0; e1.tc = tc; e1.ldd = lay.ld_v; e1.ldt = lay.ld_tc;
+                e1.V = V; e1.c = a.scale2;
+                rc = launch_gemm<EpiDlogits, false>(map_h, map_w, g1, e1, status, s, "lmhead dlogits launch");
+                if (rc != DPPO_OK) return rc;
+                // (2) dhidden[t0 : t0+tc, :] = D Wt^T          (M = tokens, N = H, K = V)
+                alignas(64) CUtensorMap map_d, map_dt, map_ht_c;
+                rc = make_map(&map_d, D, tc, V, lay.ld_v, kBM);
+                if (rc != DPPO_OK) return rc;
+                GemmShape g2 = {};
+                g2.n_mtiles = (int)((tc + kBM - 1) / kBM); g2.n_ntiles = (H + kBN - 1) / kBN; g2.n_ksteps = (V + kBK - 1) / kBK;
+                EpiStoreBf16 e2 = {};
+                e2.C = (__nv_bfloat16*)dhidden; e2.ldc = H; e2.row0 = t0; e2.rows = T; e2.cols = H;
+                rc = launch_gemm<EpiStoreBf16, false>(map_d, map_wt, g2, e2, status, s, "lmhead dhidden launch");
+                if (rc != DPPO_OK) return rc;
+                // (3) dW (+)= Dt ht[:, t0 : t0+tc]^T            (M = V, N = H, K = tokens of the chunk);
+                //     the K range must stop at the chunk, so ht gets a map of its own based at column t0
+                //     (t0 is a multiple of 8192: the base stays 16-byte aligned)
+                rc = make_map(&map_dt, Dt, V, tc, lay.ld_tc, kBM);
+                if (rc != DPPO_OK) return rc;
+                rc = make_map(&map_ht_c, ht + t0, H, tc, lay.ld_t, kBN);
+                if (rc != DPPO_OK) return rc;
+                GemmShape g3 = {};
+                g3.n_mtiles = (V + kBM - 1) / kBM; g3.n_ntiles = (H + kBN - 1) / kBN; g3.n_ksteps = (int)((tc + kBK - 1) / kBK);
+                EpiAccumF32 e3 = {};
+                e3.C = (float*)dW; e3.ldc = H; e3.rows = V; e3.cols = H; e3.accumulate = c > 0 ? 1 : 0;
+                rc = launch_gemm<EpiAccumF32, false>(map_dt, map_ht_c, g3, e3, status, s, "lmhead dW launch");
+                if (rc != DPPO_OK) return rc;
+            }
+        }
     }
     return launch_loss_reduce(a, loss_out, s);
 }

@@ -9,7 +9,7 @@ from paper_2603_04135_b200 import synth
 pytestmark = pytest.mark.gpu
 
 
-def _run(T, V, H, S, seed, n_tokens=None, tau=1.0):
+def _run(T, V, H, S, seed, n_tokens=None, tau=1.0, backward=False):
     from paper_2603_04135_b200 import binding as B
     w = synth.scaled(synth.WORKLOADS["config4_h2560"], V=V, H=H)
     hidden, W, target, lo, lr = synth.make_lmhead_inputs(w, T, seed, device="cuda")
@@ -19,18 +19,26 @@ def _run(T, V, H, S, seed, n_tokens=None, tau=1.0):
     cu = np.concatenate([[0], cuts, [T_true]]).astype(np.int32)
     S_real = len(cu) - 1
     adv = rng.normal(size=S_real).astype(np.float32); wseq = (rng.random(S_real) * 0.1).astype(np.float32)
-    prm = B.LmheadParams(B.LossParams(T, V, B.BF16, V, S_real, 0, w.eps, w.eps, w.beta, tau), H, 0)
+    prm = B.LmheadParams(B.LossParams(T, V, B.BF16, V, S_real, 0, w.eps, w.eps, w.beta, tau), H, int(backward))
     nbytes = B.lmhead_workspace_bytes(prm)
-    ws = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+    ws = torch.zeros(nbytes + 1024, dtype=torch.uint8, device="cuda")
+    ws = ws[(-ws.data_ptr()) % 1024:]
+    dh = torch.full((T, H), 7.0, dtype=torch.bfloat16, device="cuda") if backward else None
+    dW = torch.full((V, H), 7.0, dtype=torch.float32, device="cuda") if backward else None
     loss_out = torch.zeros(5, device="cuda"); logp_out = torch.zeros(T, device="cuda"); lse_out = torch.zeros(T, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     ntd = torch.tensor([T_true], dtype=torch.int32, device="cuda") if n_tokens is not None else None
     B.lmhead_grpo_loss(prm, hidden, W, target, lo, lr, torch.from_numpy(cu).cuda(), ntd, torch.from_numpy(adv).cuda(),
-                       torch.from_numpy(wseq).cuda(), None, None, None, logp_out, lse_out, loss_out, ws, nbytes, status)
+                       torch.from_numpy(wseq).cuda(), None, dh, dW, logp_out, lse_out, loss_out, ws, nbytes, status)
     torch.cuda.synchronize()
     assert status.item() == 0
-    ref = oracle.grpo_loss(synth.to_f64_numpy(hidden[:T_true]) @ synth.to_f64_numpy(W).T, target.cpu().numpy(),
-                           lo.cpu().numpy(), lr.cpu().numpy(), cu, adv, wseq, w.eps, w.eps, w.beta, tau, want_dlogits=False)
+    if backward:
+        ref = oracle.lmhead_grpo_loss(synth.to_f64_numpy(hidden[:T_true]), synth.to_f64_numpy(W), target.cpu().numpy(),
+                                      lo.cpu().numpy(), lr.cpu().numpy(), cu, adv, wseq, w.eps, w.eps, w.beta, tau)
+    else:
+        ref = oracle.grpo_loss(synth.to_f64_numpy(hidden[:T_true]) @ synth.to_f64_numpy(W).T, target.cpu().numpy(),
+                               lo.cpu().numpy(), lr.cpu().numpy(), cu, adv, wseq, w.eps, w.eps, w.beta, tau,
+                               want_dlogits=False)
     got = loss_out.cpu().numpy().astype(np.float64)
     # logits are f32 accumulations of exact bf16 products over H terms; the row sum runs in f32
     assert np.abs(lse_out.cpu().numpy()[:T_true] - ref["lse"]).max() <= 1e-4
@@ -38,6 +46,19 @@ def _run(T, V, H, S, seed, n_tokens=None, tau=1.0):
     assert abs(got[0] - ref["loss"]) <= 1e-4 * ref["abs_sum"]
     assert abs(got[1] - ref["pg"]) <= 1e-4 * ref["abs_sum"] and abs(got[2] - ref["kl"]) <= 1e-4 * ref["kl"] + 1e-9
     assert got[4] == T_true
+    if backward:
+        # dlogits are rounded to bf16 before the two gradient GEMMs (2^-9 per term, partly averaging out over
+        # the V- or T-long sums); dhidden is stored as bf16, dW as f32
+        gmax = np.abs(ref["g"]).max()
+        got_dh = dh.double().cpu().numpy()
+        assert (got_dh[T_true:] == 0).all()
+        err = np.abs(got_dh[:T_true] - ref["dhidden"])
+        bound = 2.0 ** -7 * np.abs(ref["dhidden"]).max(axis=1, keepdims=True) + 1e-6 * gmax
+        assert (err <= bound).all(), "dhidden worst ratio %.3g" % (err / bound).max()
+        got_dW = dW.double().cpu().numpy()
+        err = np.abs(got_dW - ref["dW"])
+        bound = 2.0 ** -7 * np.abs(ref["dW"]).max(axis=1, keepdims=True) + 1e-6 * gmax
+        assert (err <= bound).all(), "dW worst ratio %.3g" % (err / bound).max()
     return ref
 
 
@@ -52,10 +73,25 @@ def test_lmhead_full_vocabulary():
     _run(T=300, V=151936, H=2560, S=4, seed=5)
 
 
-def test_lmhead_backward_not_built():
+def test_lmhead_backward_small_shapes():
+    _run(T=200, V=1000, H=128, S=4, seed=11, backward=True)
+    _run(T=128, V=256, H=64, S=1, seed=12, backward=True)
+    _run(T=300, V=777, H=192, S=5, seed=14, n_tokens=259, tau=1.3, backward=True)
+    _run(T=130, V=2048, H=2560, S=3, seed=13, backward=True)
+
+
+def test_lmhead_backward_several_token_chunks():
+    _run(T=8192 + 8192 + 70, V=520, H=64, S=9, seed=15, backward=True)        # three chunks, the last one ragged
+
+
+def test_lmhead_argument_checks():
     from paper_2603_04135_b200 import binding as B
-    prm = B.LmheadParams(B.LossParams(8, 256, B.BF16, 256, 1, 0, 0.2, 0.2, 0.04, 1.0), 64, 0)
     z = torch.zeros(8 * 256, dtype=torch.bfloat16, device="cuda")
-    with pytest.raises(B.DppoError) as e:
+    prm = B.LmheadParams(B.LossParams(8, 256, B.BF16, 256, 1, 0, 0.2, 0.2, 0.04, 1.0), 64, 0)
+    with pytest.raises(B.DppoError) as e:       # gradients passed but not requested
         B.lmhead_grpo_loss(prm, z, z, z, z, z, z, None, z, z, None, z, z, None, None, z, z, 1 << 20)
-    assert e.value.code == B.ERR_UNSUPPORTED
+    assert e.value.code == B.ERR_INVALID_ARG
+    prm = B.LmheadParams(B.LossParams(8, 256, B.BF16, 256, 1, 0, 0.2, 0.2, 0.04, 1.0), 72, 0)
+    with pytest.raises(B.DppoError) as e:       # H not a multiple of 64
+        B.lmhead_grpo_loss(prm, z, z, z, z, z, z, None, z, z, None, None, None, None, None, z, z, 1 << 20)
+    assert e.value.code == B.ERR_BAD_SHAPE
