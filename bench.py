@@ -181,6 +181,46 @@ def run_reference(args):
     return 0
 
 
+def time_lmhead(T, H, V, dev, iters=3, warmup=1):
+    """Fused LM-head + loss, forward and backward (dhidden, dW), timed with CUDA events."""
+    from paper_2603_04135_b200 import binding as B
+    wl = synth.scaled(synth.WORKLOADS["config4_h2560"], V=V, H=H)
+    hidden, W, target, lo, lr = synth.make_lmhead_inputs(wl, T, 4, device=dev)
+    S = 177
+    cu = torch.from_numpy(np.linspace(0, T, S + 1).astype(np.int32)).to(dev)
+    adv = torch.from_numpy(np.random.default_rng(4).normal(size=S).astype(np.float32)).to(dev)
+    wseq = torch.full((S,), 1.0 / S, device=dev)
+    prm = B.LmheadParams(B.LossParams(T, V, B.BF16, V, S, 0, wl.eps, wl.eps, wl.beta, 1.0), H, 1)
+    nbytes = B.lmhead_workspace_bytes(prm)
+    ws = torch.zeros(nbytes + 1024, dtype=torch.uint8, device=dev)
+    ws = ws[(-ws.data_ptr()) % 1024:]
+    dh = torch.empty((T, H), dtype=torch.bfloat16, device=dev)
+    dW = torch.empty((V, H), dtype=torch.float32, device=dev)
+    loss_out = torch.zeros(5, device=dev); status = torch.zeros(1, dtype=torch.int32, device=dev)
+    times = []
+    for it in range(warmup + iters):
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record()
+        B.lmhead_grpo_loss(prm, hidden, W, target, lo, lr, cu, None, adv, wseq, None, dh, dW, None, None, loss_out,
+                           ws, nbytes, status)
+        e1.record()
+        torch.cuda.synchronize()
+        if it >= warmup:
+            times.append(e0.elapsed_time(e1))
+    assert status.item() == 0
+    ms = sum(times) / len(times)
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            peak = float(json.load(f)["bf16_tflops_sustained"]); peak_kind = "measured sustained cuBLAS bf16"
+    except Exception:
+        peak, peak_kind = 1400.0, "fallback sustained"
+    executed = 8.0 * T * V * H / ms / 1e9
+    return {"workload": "config4: bf16 hidden [%d x %d], W [%d x %d], forward + dhidden + dW" % (T, H, V, H),
+            "ms": ms, "tokens_per_s": T / ms * 1e3, "executed_tflops": executed, "model_tflops_6TVH": executed * 6 / 8,
+            "roofline": {"bound": "tensor", "achieved": executed, "peak": peak, "unit": "TFLOP/s", "frac": executed / peak,
+                         "peak_source": peak_kind, "note": "executed flops = 8 T V H: forward, dlogits recompute, dhidden, dW"}}
+
+
 # --------------------------------------------------------------------------------------- ours
 def run_ours(args):
     from paper_2603_04135_b200.step import DppoStep      # raises if libdppo.so is missing: no fallback
@@ -282,6 +322,12 @@ def run_ours(args):
     e2e_ms = t0.elapsed_time(t1) / e2e_steps
     del host_tok
 
+    # ---- the optional fused LM-head path on the same token count (Qwen3-4B width): forward + backward
+    lm = None
+    if rank == 0 and not args.no_lmhead:
+        del tok, dlogits, dev_tok
+        torch.cuda.empty_cache()
+        lm = time_lmhead(T, 2560, w.V, dev)
     # ---- max over ranks, totals over ranks
     (total_ms, loss_ms, e2e_ms), T_all = dp.combine_over_ranks([total_ms, loss_ms, e2e_ms], T, device=dev)
 
@@ -311,6 +357,8 @@ def run_ours(args):
                          "traffic_note": "ncu dram bytes of an 8192-row capture of the same kernel, scaled by rows"},
             "loss": loss_value,
         }
+        if lm is not None:
+            line["lmhead"] = lm
         if pool is not None:
             n_rows, _, times = time_oracle(w, seed, args.ref_rows, 1, 0, pool, cores)
             pool.close(); pool.join()
@@ -333,6 +381,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--ref-rows", type=int, default=2048, help="token rows in the oracle's timed sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-lmhead", action="store_true", help="skip the fused LM-head measurement")
     ap.add_argument("--no-clock-sampling", action="store_true", help="do not poll nvidia-smi during the timed region")
     args = ap.parse_args()
     if args.impl == "ours" and args.warmup < 3:
