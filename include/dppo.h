@@ -228,7 +228,7 @@ int dppo_grpo_loss_fwd_bwd(const dppo_loss_params* p, const void* logits, const 
  *   W        bf16 [V x H] row-major LM-head weight
  *   backward 0: forward only (loss_out, logp_out, lse_out; dhidden and dW must be NULL).
  *            1: also the gradients, dhidden = D W and dW = D^T hidden with D = dlogits recomputed from the
- *            same GEMM for 8192 tokens at a time into workspace scratch (bf16; never the full [T x V]);
+ *            same GEMM for 9472 tokens at a time into workspace scratch (bf16; never the full [T x V]);
  *            the workspace then also holds K-major copies of W and hidden
  *   dhidden  bf16 [T_max x H] out (rows at or past the true token count are zero)
  *   dW       f32 [V x H] out (overwritten, not accumulated into)

@@ -36,7 +36,8 @@ constexpr int kStageBytes = kStageBytesA + kStageBytesB;
 constexpr int kLmThreads = 192;
 constexpr int kTmemCols = 512;
 constexpr unsigned long long kLmWaitLimitNs = 2000000000ull;
-constexpr int kChunkTokens = 8192;       // tokens whose dlogits are held in scratch at a time
+constexpr int kChunkTokens = 9472;       // tokens whose dlogits are held in scratch at a time: 74 row tiles, so the
+                                         // dhidden GEMM of a chunk has 74 x H/256 tiles = whole waves on 148 SMs
 
 struct LmShared {
     unsigned long long full[kStages];    // TMA bytes have landed in stage s
@@ -659,7 +660,7 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
                 if (rc != DPPO_OK) return rc;
                 // (3) dW (+)= Dt ht[:, t0 : t0+tc]^T            (M = V, N = H, K = tokens of the chunk);
                 //     the K range must stop at the chunk, so ht gets a map of its own based at column t0
-                //     (t0 is a multiple of 8192: the base stays 16-byte aligned)
+                //     (t0 is a multiple of 9472 = 8 * 1184: the base stays 16-byte aligned)
                 rc = make_map(&map_dt, Dt, V, tc, lay.ld_tc, kBM);
                 if (rc != DPPO_OK) return rc;
                 rc = make_map(&map_ht_c, ht + t0, H, tc, lay.ld_t, kBN);
