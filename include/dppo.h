@@ -47,7 +47,8 @@ typedef enum {                          /* values of the device status word */
     DPPO_STATUS_BAD_LENGTH = 1,         /* pack: a retained unit has length < 1 or > L_row            */
     DPPO_STATUS_BAD_TARGET = 2,         /* loss: a target id outside [0, V)                           */
     DPPO_STATUS_TIMEOUT = 3,            /* a bounded device-side wait ran out                         */
-    DPPO_STATUS_BAD_SEGMENTS = 4        /* loss: cu_seqlens does not cover a token                    */
+    DPPO_STATUS_BAD_SEGMENTS = 4,       /* loss: cu_seqlens does not cover a token                    */
+    DPPO_STATUS_BAD_INDEX = 5           /* history: a prompt id outside the table                     */
 } dppo_status;
 
 int dppo_version(void);                 /* major*10000 + minor*100 + patch */
@@ -106,6 +107,21 @@ int dppo_prune_and_rescale(const dppo_prune_params* p, const float* adv, const f
                            uint8_t* cand_q, uint8_t* cand_o, uint8_t* keep_q, uint8_t* keep_o,
                            int32_t* n_keep_q, int32_t* n_keep_o, float* gamma_q, float* gamma_o,
                            float* w_seq, float* H_next, int32_t* status, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * History scores across epochs — Eq. 16 keeps one score H_t(q) per DATASET prompt; Algorithm 1 starts
+ * from H_0 = 0 and skips prompt pruning in the first epoch.  A batch gathers the scores of its prompts
+ * before dppo_prune_and_rescale (H_prev) and scatters H_next back afterwards: retained prompts get
+ * their fresh mean |A|, pruned ones keep their old score (the carry-forward).
+ *   H_table     f32 [N] one score per dataset prompt (caller zero-initialises it)
+ *   prompt_ids  i32 [P] dataset index of each prompt of the batch (distinct within a batch)
+ *   H_batch     f32 [P] out of gather;  H_next f32 [P] in to scatter
+ * An id outside [0, N) sets status DPPO_STATUS_BAD_INDEX (gather returns 0 for it, scatter skips it).
+ */
+int dppo_history_gather(const float* H_table, int N, const int32_t* prompt_ids, int P, float* H_batch,
+                        int32_t* status, void* stream);
+int dppo_history_scatter(float* H_table, int N, const int32_t* prompt_ids, int P, const float* H_next,
+                         int32_t* status, void* stream);
 
 /* ------------------------------------------------------------------------------------------------
  * Dense Prompt Packing — Section 4.3 (window-based greedy selection from a candidate pool W of

@@ -18,6 +18,7 @@ from .dppo_oracle import (
     prune_masks,
     rescale,
     prune_and_rescale,
+    history_epochs,
     pack_prompts,
     bf16_bits_to_f64,
     f64_to_bf16_bits,
@@ -30,7 +31,7 @@ from .dppo_oracle import (
 __all__ = [
     "philox4x32_10", "uniform53",
     "group_advantages", "completion_candidates", "prompt_candidates",
-    "draw_uniforms", "prune_masks", "rescale", "prune_and_rescale",
+    "draw_uniforms", "prune_masks", "rescale", "prune_and_rescale", "history_epochs",
     "pack_prompts", "bf16_bits_to_f64", "f64_to_bf16_bits",
     "token_logprob", "token_terms", "grpo_loss", "lmhead_grpo_loss",
 ]

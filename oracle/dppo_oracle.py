@@ -232,6 +232,25 @@ def prune_and_rescale(adv, mean_abs_adv, H_prev, r_q, r_o, seed=0, step=0,
                 w_seq=w_seq, H_next=H_next)
 
 
+def history_epochs(rewards_by_epoch, batches_by_epoch, N, G, r_q, r_o, seed=0, mode=0):
+    """Algorithm 1's outer loops for the pruning state only: H_0 = 0 for every dataset prompt; in epoch
+    t each batch (a list of dataset prompt ids) reads H_{t-1} of its prompts (no prompt pruning in the
+    first epoch), prunes, and writes H_t back (Eq. 16: fresh mean |A| for retained prompts, the old score
+    for pruned ones).  rewards_by_epoch[t] is [N, G]; draws use step = t * 1_000_000 + batch index.
+    Returns (final table float32 [N], list of per-batch results)."""
+    table = np.zeros(N, dtype=np.float32)
+    log = []
+    for t, (rewards, batches) in enumerate(zip(rewards_by_epoch, batches_by_epoch)):
+        for b, ids in enumerate(batches):
+            ids = np.asarray(ids, dtype=np.int64)
+            adv, mabs = group_advantages(np.asarray(rewards)[ids])
+            H_prev = None if t == 0 else table[ids].copy()
+            out = prune_and_rescale(adv, mabs, H_prev, r_q, r_o, seed=seed, step=t * 1000000 + b, mode=mode)
+            table[ids] = out["H_next"]
+            log.append(out)
+    return table, log
+
+
 # --------------------------------------------------------------------------
 # Step 5 — Dense Prompt Packing (Section 4.3; Algorithm 1's packing step)
 # --------------------------------------------------------------------------

@@ -16,7 +16,7 @@ if not os.path.exists(_LIB_PATH):
 lib = ctypes.CDLL(_LIB_PATH)
 
 F32, BF16 = 0, 1
-STATUS_OK, STATUS_BAD_LENGTH, STATUS_BAD_TARGET, STATUS_TIMEOUT, STATUS_BAD_SEGMENTS = 0, 1, 2, 3, 4
+STATUS_OK, STATUS_BAD_LENGTH, STATUS_BAD_TARGET, STATUS_TIMEOUT, STATUS_BAD_SEGMENTS, STATUS_BAD_INDEX = 0, 1, 2, 3, 4, 5
 ERR_INVALID_ARG, ERR_BAD_SHAPE, ERR_MISALIGNED, ERR_WORKSPACE_TOO_SMALL, ERR_UNSUPPORTED, ERR_CUDA = \
     -1, -2, -3, -4, -5, -6
 
@@ -56,6 +56,10 @@ lib.dppo_group_advantages.restype = ctypes.c_int
 lib.dppo_group_advantages.argtypes = [_vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_double, _vp, _vp, _vp, _vp]
 lib.dppo_prune_and_rescale.restype = ctypes.c_int
 lib.dppo_prune_and_rescale.argtypes = [ctypes.POINTER(PruneParams)] + [_vp] * 17
+lib.dppo_history_gather.restype = ctypes.c_int
+lib.dppo_history_gather.argtypes = [_vp, ctypes.c_int, _vp, ctypes.c_int, _vp, _vp, _vp]
+lib.dppo_history_scatter.restype = ctypes.c_int
+lib.dppo_history_scatter.argtypes = [_vp, ctypes.c_int, _vp, ctypes.c_int, _vp, _vp, _vp]
 lib.dppo_pack_workspace_bytes.restype = ctypes.c_size_t
 lib.dppo_pack_workspace_bytes.argtypes = [ctypes.POINTER(PackParams)]
 lib.dppo_pack_prompts.restype = ctypes.c_int
@@ -115,6 +119,14 @@ def prune_and_rescale(params, adv, mean_abs_adv, H_prev, u_q, u_o, cand_q, cand_
                                       _ptr(u_q), _ptr(u_o), _ptr(cand_q), _ptr(cand_o), _ptr(keep_q),
                                       _ptr(keep_o), _ptr(n_keep_q), _ptr(n_keep_o), _ptr(gamma_q),
                                       _ptr(gamma_o), _ptr(w_seq), _ptr(H_next), _ptr(status), _stream(stream)))
+
+
+def history_gather(H_table, N, prompt_ids, P, H_batch, status=None, stream=None):
+    _check(lib.dppo_history_gather(_ptr(H_table), N, _ptr(prompt_ids), P, _ptr(H_batch), _ptr(status), _stream(stream)))
+
+
+def history_scatter(H_table, N, prompt_ids, P, H_next, status=None, stream=None):
+    _check(lib.dppo_history_scatter(_ptr(H_table), N, _ptr(prompt_ids), P, _ptr(H_next), _ptr(status), _stream(stream)))
 
 
 def pack_workspace_bytes(params):

@@ -161,7 +161,47 @@ prune_and_rescale_kernel(dppo_prune_params prm, const float* __restrict__ adv,
     }
 }
 
+// History table (Eq. 16 across epochs): one score per dataset prompt; a batch reads its prompts' scores
+// before pruning and writes H_next back afterwards.
+__global__ void history_gather_kernel(const float* __restrict__ table, int N, const int32_t* __restrict__ ids, int P,
+                                      float* __restrict__ H_batch, int32_t* status) {
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= P) return;
+    const int id = ids[k];
+    if (id < 0 || id >= N) { set_status(status, DPPO_STATUS_BAD_INDEX); H_batch[k] = 0.0f; return; }
+    H_batch[k] = table[id];
+}
+
+__global__ void history_scatter_kernel(float* __restrict__ table, int N, const int32_t* __restrict__ ids, int P,
+                                       const float* __restrict__ H_next, int32_t* status) {
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= P) return;
+    const int id = ids[k];
+    if (id < 0 || id >= N) { set_status(status, DPPO_STATUS_BAD_INDEX); return; }
+    table[id] = H_next[k];
+}
+
 }  // namespace dppo
+
+extern "C" int dppo_history_gather(const float* H_table, int N, const int32_t* prompt_ids, int P, float* H_batch,
+                                   int32_t* status, void* stream) {
+    if (N < 0 || P < 0) return dppo::fail(DPPO_ERR_INVALID_ARG, "history_gather: N=%d P=%d", N, P);
+    if (P == 0) return DPPO_OK;
+    if (!H_table || !prompt_ids || !H_batch) return dppo::fail(DPPO_ERR_INVALID_ARG, "history_gather: NULL array");
+    dppo::history_gather_kernel<<<(P + 255) / 256, 256, 0, (cudaStream_t)stream>>>(H_table, N, prompt_ids, P, H_batch, status);
+    DPPO_CHECK_LAUNCH("history_gather launch");
+    return DPPO_OK;
+}
+
+extern "C" int dppo_history_scatter(float* H_table, int N, const int32_t* prompt_ids, int P, const float* H_next,
+                                    int32_t* status, void* stream) {
+    if (N < 0 || P < 0) return dppo::fail(DPPO_ERR_INVALID_ARG, "history_scatter: N=%d P=%d", N, P);
+    if (P == 0) return DPPO_OK;
+    if (!H_table || !prompt_ids || !H_next) return dppo::fail(DPPO_ERR_INVALID_ARG, "history_scatter: NULL array");
+    dppo::history_scatter_kernel<<<(P + 255) / 256, 256, 0, (cudaStream_t)stream>>>(H_table, N, prompt_ids, P, H_next, status);
+    DPPO_CHECK_LAUNCH("history_scatter launch");
+    return DPPO_OK;
+}
 
 extern "C" int dppo_prune_and_rescale(const dppo_prune_params* p, const float* adv,
                                       const float* mean_abs_adv, const float* H_prev,

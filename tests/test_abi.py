@@ -27,7 +27,9 @@ def test_every_declared_symbol_is_exported(B):
     names = declared_functions()
     assert {"dppo_version", "dppo_last_error", "dppo_group_advantages", "dppo_prune_and_rescale",
             "dppo_pack_workspace_bytes", "dppo_pack_prompts", "dppo_grpo_loss_workspace_bytes",
-            "dppo_grpo_loss_fwd_bwd"} <= set(names)
+            "dppo_grpo_loss_fwd_bwd", "dppo_pack_prompts_static", "dppo_pack_static_max_units",
+            "dppo_history_gather", "dppo_history_scatter", "dppo_lmhead_workspace_bytes",
+            "dppo_lmhead_grpo_loss"} <= set(names)
     for n in names:
         assert hasattr(B.lib, n), n
     assert B.version() >= 100

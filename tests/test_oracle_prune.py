@@ -407,3 +407,30 @@ def test_fixed_fraction_is_unbiased_with_realised_fraction_only():
         n += 1
     assert math.isclose(total / n, ell.mean(), abs_tol=2e-7)
     assert abs(total_eq18 / n - ell.mean()) > 1e-3                   # the printed factors are biased here
+
+
+# ---------------------------------------------------------------- history table across epochs (Eq. 16, Algorithm 1)
+def test_history_epochs_carry_forward_and_first_epoch():
+    N, G, P = 12, 4, 4
+    rng = np.random.default_rng(0)
+    rate = rng.random(N)
+    rewards = [(rng.random((N, G)) < rate[:, None]).astype(np.float32) for _ in range(4)]
+    batches = [[list(range(i, i + P)) for i in range(0, N, P)] for _ in range(4)]
+    batches[2] = [[0, 5, 10, 3], [1, 6, 11, 4], [2, 7, 8, 9]]            # another batching in the third epoch
+    table, log = oracle.history_epochs(rewards, batches, N, G, 0.6, 0.5, seed=9)
+    assert all(out["keep_q"].all() for out in log[:3])                     # first epoch: no prompt pruning
+    assert any((out["keep_q"] == 0).any() for out in log[3:])              # later epochs prune some prompts
+    # replay by hand: a prompt's score changes exactly when it was retained, to that epoch's mean |A|
+    H = np.zeros(N, dtype=np.float32)
+    i = 0
+    for t in range(4):
+        for ids in batches[t]:
+            out = log[i]; i += 1
+            mabs = oracle.group_advantages(rewards[t][ids])[1]
+            if t > 0:                                                      # candidates = lowest half of the scores read
+                order = sorted(range(P), key=lambda k: (H[ids[k]], k))
+                assert sorted(np.nonzero(out["cand_q"])[0]) == sorted(order[:P // 2])
+            for k, q in enumerate(ids):
+                if out["keep_q"][k]:
+                    H[q] = mabs[k]
+    assert np.array_equal(H, table)
