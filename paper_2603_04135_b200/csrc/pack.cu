@@ -18,7 +18,7 @@ struct PackWorkspace {                         // carved from the caller's works
     int32_t* slen;                             // its length
 };
 
-template <bool kLensInSmem>
+template <bool kLensInSmem, bool kStreamInSmem>
 __global__ void __launch_bounds__(32)
 pack_prompts_kernel(dppo_pack_params prm, const int32_t* __restrict__ len,
                     const uint8_t* __restrict__ keep, const int32_t* __restrict__ loss_len,
@@ -28,6 +28,9 @@ pack_prompts_kernel(dppo_pack_params prm, const int32_t* __restrict__ len,
                     PackWorkspace ws, int32_t* status) {
     __shared__ uint32_t placed[kPackMaxUnits / 32];
     __shared__ int32_t lens_smem[kLensInSmem ? kPackSmemLens : 1];
+    extern __shared__ int32_t pack_dyn[];                      // kStreamInSmem: stream[n_max], then loss tokens[n_max]
+    int32_t* stream_s = pack_dyn;
+    int32_t* sloss_s = pack_dyn + prm.n_max;
     const int lane = threadIdx.x;
     const int n_max = prm.n_max, L = prm.L_row;
 
@@ -43,7 +46,7 @@ pack_prompts_kernel(dppo_pack_params prm, const int32_t* __restrict__ len,
         const unsigned m = __ballot_sync(0xffffffffu, in);
         if (in) {
             const int pos = n + __popc(m & ((1u << lane) - 1u));
-            ws.stream[pos] = u;
+            if (kStreamInSmem) { stream_s[pos] = u; sloss_s[pos] = loss_len ? loss_len[u] : l; } else ws.stream[pos] = u;
             if (kLensInSmem) lens_smem[pos] = l; else ws.slen[pos] = l;
             bad = bad || l < 1 || l > L;
         }
@@ -95,13 +98,13 @@ pack_prompts_kernel(dppo_pack_params prm, const int32_t* __restrict__ len,
         }
         const int l = slen[pick];
         if (lane == 0) {
-            const int u = ws.stream[pick];
+            const int u = kStreamInSmem ? stream_s[pick] : ws.stream[pick];
             order[n_placed] = u;
             row_of[u] = row;
             off_in_row[u] = L - remaining;
             cu_seqlens[n_placed] = loss_cum;
             placed[pick >> 5] |= 1u << (pick & 31);
-            loss_cum += loss_len ? loss_len[u] : l;
+            loss_cum += kStreamInSmem ? sloss_s[pick] : (loss_len ? loss_len[u] : l);
         }
         loss_cum = __shfl_sync(0xffffffffu, loss_cum, 0);
         __syncwarp();
@@ -186,11 +189,16 @@ extern "C" int dppo_pack_prompts(const dppo_pack_params* p, const int32_t* len, 
     ws.stream = (int32_t*)workspace;
     ws.slen = (int32_t*)((char*)workspace + need / 2);
     cudaStream_t s = (cudaStream_t)stream;
-    if (p->n_max <= kPackSmemLens)
-        pack_prompts_kernel<true><<<1, 32, 0, s>>>(*p, len, keep, loss_len, order, row_of, off_in_row, row_fill,
-                                                   cu_seqlens, counts, ws, status);
-    else
-        pack_prompts_kernel<false><<<1, 32, 0, s>>>(*p, len, keep, loss_len, order, row_of, off_in_row, row_fill,
+    if (p->n_max <= kPackSmemLens) {
+        // batch-sized streams: the stream and its loss-token counts sit in shared memory too, so a placement
+        // costs shared-memory latency instead of two dependent global loads
+        const size_t dyn = (size_t)(p->n_max > 0 ? p->n_max : 1) * 2 * sizeof(int32_t);
+        cudaError_t e = cudaFuncSetAttribute(pack_prompts_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
+        if (e != cudaSuccess) return cuda_fail(e, "pack_prompts: shared memory attribute");
+        pack_prompts_kernel<true, true><<<1, 32, dyn, s>>>(*p, len, keep, loss_len, order, row_of, off_in_row, row_fill,
+                                                         cu_seqlens, counts, ws, status);
+    } else
+        pack_prompts_kernel<false, false><<<1, 32, 0, s>>>(*p, len, keep, loss_len, order, row_of, off_in_row, row_fill,
                                                     cu_seqlens, counts, ws, status);
     DPPO_CHECK_LAUNCH("pack_prompts launch");
     return DPPO_OK;
@@ -220,7 +228,7 @@ extern "C" int dppo_pack_prompts_static(const dppo_pack_params* p, const int32_t
     ws.stream = scratch;
     ws.slen = scratch + kPackStaticMaxUnits;
     // Nothing in the scratch has to start at zero: the kernel writes every stream slot it later reads.
-    pack_prompts_kernel<true><<<1, 32, 0, (cudaStream_t)stream>>>(*p, len, keep, loss_len, order, row_of, off_in_row,
+    pack_prompts_kernel<true, false><<<1, 32, 0, (cudaStream_t)stream>>>(*p, len, keep, loss_len, order, row_of, off_in_row,
                                                                   row_fill, cu_seqlens, counts, ws, status);
     DPPO_CHECK_LAUNCH("pack_prompts_static launch");
     return DPPO_OK;
