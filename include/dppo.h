@@ -207,6 +207,15 @@ typedef struct {
     double eps_lo, eps_hi;  /* clip range 1-eps_lo .. 1+eps_hi (the paper: both 0.2)                 */
     double beta;            /* KL coefficient                                                        */
     double temperature;     /* > 0 (the paper: 1)                                                    */
+    /* Variants for the other objectives the paper combines the method with (Section 5.2); zero / NULL
+       give Eq. 1 as printed. */
+    int32_t no_length_norm; /* 1: W = w[s] instead of w[s]/|o_s| (a token-level mean is then up to the w
+                               the caller passes)                                                    */
+    int32_t reserved2;      /* 0                                                                     */
+    const float* seq_log_ratio; /* device f32 [S_max] or NULL.  Given: every token of sequence s uses the
+                               sequence-level ratio rho = exp(seq_log_ratio[s]) (from
+                               dppo_sequence_log_ratio on the current log-probs, i.e. after a forward-only
+                               call) in place of exp(logp - logp_old); requires no_length_norm == 0     */
 } dppo_loss_params;
 
 size_t dppo_grpo_loss_workspace_bytes(const dppo_loss_params* p);
@@ -232,6 +241,14 @@ int dppo_grpo_loss_fwd_bwd(const dppo_loss_params* p, const void* logits, const 
                            const int32_t* seg_map, void* dlogits, float* logp_out, float* lse_out,
                            float* loss_out, void* workspace, size_t workspace_bytes,
                            int32_t* status, void* stream);
+
+/* Mean token log-ratio of each sequence, out[s] = mean_t (logp[t] - logp_old[t]) over cu_seqlens[s] <= t <
+ * cu_seqlens[s+1] (0 for an empty sequence): the log of the length-normalised sequence-level likelihood
+ * ratio of sequence-level objectives (Section 5.2).  logp, logp_old f32 [T]; out f32 [S_max].  Binary64
+ * accumulation in a fixed order.  Errors: INVALID_ARG.
+ */
+int dppo_sequence_log_ratio(const float* logp, const float* logp_old, const int32_t* cu_seqlens, int S_max,
+                            float* out, int32_t* status, void* stream);
 
 /* ------------------------------------------------------------------------------------------------
  * Fused LM-head + loss: the same loss as dppo_grpo_loss_fwd_bwd with the logits z = hidden W^T

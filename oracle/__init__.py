@@ -23,6 +23,7 @@ from .dppo_oracle import (
     bf16_bits_to_f64,
     f64_to_bf16_bits,
     token_logprob,
+    sequence_log_ratio,
     token_terms,
     grpo_loss,
     lmhead_grpo_loss,
@@ -33,5 +34,5 @@ __all__ = [
     "group_advantages", "completion_candidates", "prompt_candidates",
     "draw_uniforms", "prune_masks", "rescale", "prune_and_rescale", "history_epochs",
     "pack_prompts", "bf16_bits_to_f64", "f64_to_bf16_bits",
-    "token_logprob", "token_terms", "grpo_loss", "lmhead_grpo_loss",
+    "token_logprob", "sequence_log_ratio", "token_terms", "grpo_loss", "lmhead_grpo_loss",
 ]

@@ -345,7 +345,24 @@ def token_logprob(z, y, tau=1.0):
     return logp, lse
 
 
-def token_terms(logp, logp_old, logp_ref, A, eps_lo, eps_hi, beta):
+def sequence_log_ratio(logp, logp_old, cu_seqlens):
+    """Mean over a sequence's tokens of logp - logp_old: the log of the sequence-level likelihood ratio
+    with length normalisation, (pi_theta(o|q) / pi_old(o|q))^(1/|o|), used when the method is combined with a
+    sequence-level objective (Section 5.2, "Robustness Across RL Algorithms").  Empty sequences give 0."""
+    d = np.asarray(logp, dtype=np.float64) - np.asarray(logp_old, dtype=np.float64)
+    cu = np.asarray(cu_seqlens, dtype=np.int64)
+    out = np.zeros(len(cu) - 1)
+    for s in range(len(cu) - 1):
+        a, b = int(cu[s]), int(cu[s + 1])
+        if b > a:
+            acc = 0.0
+            for x in d[a:b]:
+                acc = acc + float(x)
+            out[s] = acc / (b - a)
+    return out
+
+
+def token_terms(logp, logp_old, logp_ref, A, eps_lo, eps_hi, beta, log_ratio=None):
     """Per-token pieces of the GRPO objective (Eq. 1) for advantage A:
 
       rho  = exp(logp - logp_old)                        probability ratio
@@ -354,11 +371,17 @@ def token_terms(logp, logp_old, logp_ref, A, eps_lo, eps_hi, beta):
       j    = surr - beta*kl
       dj   = d j / d logp = A*rho*[unclipped] + beta*(rho_hat - 1)
     where [unclipped] is 0 only when the clipped branch is strictly the smaller
-    one.  Returns dict of float64 arrays (clipped as bool).
+    one.  With log_ratio given, rho = exp(log_ratio) replaces the token ratio (dj is
+    then the derivative for a ratio whose log is the mean token log-ratio of the
+    sequence, times the sequence length — see grpo_loss).  Returns dict of float64
+    arrays (clipped as bool).
     """
     logp = np.asarray(logp, dtype=np.float64)
     A = np.asarray(A, dtype=np.float64)
-    rho = np.exp(logp - np.asarray(logp_old, dtype=np.float64))
+    if log_ratio is None:
+        rho = np.exp(logp - np.asarray(logp_old, dtype=np.float64))
+    else:                      # a ratio shared by the tokens of a sequence (its own log is given)
+        rho = np.exp(np.asarray(log_ratio, dtype=np.float64))
     d = np.asarray(logp_ref, dtype=np.float64) - logp
     rho_hat = np.exp(d)
     kl = rho_hat - d - 1.0
@@ -373,7 +396,7 @@ def token_terms(logp, logp_old, logp_ref, A, eps_lo, eps_hi, beta):
 
 def grpo_loss(logits, target, logp_old, logp_ref, cu_seqlens, adv_seg, w_seg,
               eps_lo=0.2, eps_hi=0.2, beta=0.04, tau=1.0, want_dlogits=True, rows=None,
-              chunk=256):
+              chunk=256, length_norm=True, seq_log_ratio=None):
     """The pruned GRPO loss and its gradient w.r.t. the logits.
 
     logits [T, V] float64 (exact values of the stored fp32/bf16 logits); target
@@ -386,7 +409,16 @@ def grpo_loss(logits, target, logp_old, logp_ref, cu_seqlens, adv_seg, w_seg,
 
     rows: optional index list; then only those rows of `logits` are given
     (logits[i] is token rows[i]) and loss sums are over those rows only.
+
+    Variants for the other objectives the paper combines the method with (Section 5.2):
+    length_norm=False drops Eq. 1's 1/|o_i| (W_t = w_seg[s]; a token-level mean is then a matter
+    of the w the caller passes).  seq_log_ratio [S] replaces the token ratio by the sequence-level
+    one, rho_s = exp(seq_log_ratio[s]) with seq_log_ratio = `sequence_log_ratio` of the current
+    log-probs; since d rho_s / d logp_t = rho_s / |o_s|, the gradient keeps the token form with rho_s
+    in place of rho_t when length_norm is on (asserted here).
     """
+    if seq_log_ratio is not None:
+        assert length_norm, "the sequence-level ratio is defined with the 1/|o| normalisation"
     logits = np.asarray(logits)
     cu = np.asarray(cu_seqlens, dtype=np.int64)
     S = len(cu) - 1
@@ -396,14 +428,15 @@ def grpo_loss(logits, target, logp_old, logp_ref, cu_seqlens, adv_seg, w_seg,
     seg = np.searchsorted(cu, tok, side="right") - 1
     seg_len = (cu[1:] - cu[:-1]).astype(np.float64)
     A = np.asarray(adv_seg, dtype=np.float64)[seg] if n else np.zeros(0)
-    W = (np.asarray(w_seg, dtype=np.float64)[seg] / seg_len[seg]) if n else np.zeros(0)
+    W = (np.asarray(w_seg, dtype=np.float64)[seg] / (seg_len[seg] if length_norm else 1.0)) if n else np.zeros(0)
     y = np.asarray(target, dtype=np.int64)[tok]
     logp = np.zeros(n); lse = np.zeros(n)
     for a in range(0, n, chunk):
         b = min(n, a + chunk)
         logp[a:b], lse[a:b] = token_logprob(np.asarray(logits[a:b], dtype=np.float64), y[a:b], tau)
     tt = token_terms(logp, np.asarray(logp_old)[tok], np.asarray(logp_ref)[tok], A,
-                     eps_lo, eps_hi, beta)
+                     eps_lo, eps_hi, beta,
+                     log_ratio=None if seq_log_ratio is None else np.asarray(seq_log_ratio, dtype=np.float64)[seg])
     g = -W * tt["dj"]
     out = dict(
         loss=-math.fsum(W * tt["j"]), pg=-math.fsum(W * tt["surr"]), kl=math.fsum(W * tt["kl"]),

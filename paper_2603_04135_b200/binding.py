@@ -42,7 +42,8 @@ class LossParams(ctypes.Structure):
     _fields_ = [("T_max", ctypes.c_int64), ("V", ctypes.c_int32), ("dtype", ctypes.c_int32),
                 ("row_stride", ctypes.c_int64), ("S_max", ctypes.c_int32), ("variant", ctypes.c_int32),
                 ("eps_lo", ctypes.c_double), ("eps_hi", ctypes.c_double), ("beta", ctypes.c_double),
-                ("temperature", ctypes.c_double)]
+                ("temperature", ctypes.c_double), ("no_length_norm", ctypes.c_int32), ("reserved2", ctypes.c_int32),
+                ("seq_log_ratio", ctypes.c_void_p)]
 
 
 class LmheadParams(ctypes.Structure):
@@ -73,6 +74,8 @@ lib.dppo_grpo_loss_fwd_bwd.restype = ctypes.c_int
 lib.dppo_grpo_loss_fwd_bwd.argtypes = [ctypes.POINTER(LossParams)] + [_vp] * 14 + [ctypes.c_size_t, _vp, _vp]
 
 
+lib.dppo_sequence_log_ratio.restype = ctypes.c_int
+lib.dppo_sequence_log_ratio.argtypes = [_vp, _vp, _vp, ctypes.c_int, _vp, _vp, _vp]
 lib.dppo_lmhead_workspace_bytes.restype = ctypes.c_size_t
 lib.dppo_lmhead_workspace_bytes.argtypes = [ctypes.POINTER(LmheadParams)]
 lib.dppo_lmhead_grpo_loss.restype = ctypes.c_int
@@ -177,3 +180,8 @@ def lmhead_grpo_loss(params, hidden, W, target, logp_old, logp_ref, cu_seqlens, 
                                      _ptr(logp_ref), _ptr(cu_seqlens), _ptr(n_tokens_dev), _ptr(adv), _ptr(w),
                                      _ptr(seg_map), _ptr(dhidden), _ptr(dW), _ptr(logp_out), _ptr(lse_out),
                                      _ptr(loss_out), _ptr(workspace), workspace_bytes, _ptr(status), _stream(stream)))
+
+
+def sequence_log_ratio(logp, logp_old, cu_seqlens, S_max, out, status=None, stream=None):
+    _check(lib.dppo_sequence_log_ratio(_ptr(logp), _ptr(logp_old), _ptr(cu_seqlens), S_max, _ptr(out), _ptr(status),
+                                       _stream(stream)))

@@ -140,6 +140,20 @@ loss_reduce_kernel(const RowTerms* __restrict__ terms, long long T_max, const in
     }
 }
 
+// One warp per sequence: lanes stride over the tokens, binary64, fixed-order tree.
+__global__ void __launch_bounds__(256)
+sequence_log_ratio_kernel(const float* __restrict__ logp, const float* __restrict__ logp_old,
+                          const int32_t* __restrict__ cu, int S, float* __restrict__ out) {
+    const int s = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (s >= S) return;
+    const int a = cu[s], b = cu[s + 1];
+    double acc = 0.0;
+    for (int t = a + lane; t < b; t += 32) acc += (double)logp[t] - (double)logp_old[t];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) out[s] = b > a ? (float)(acc / (double)(b - a)) : 0.0f;
+}
+
 int launch_rows_general(const LossArgs& a, cudaStream_t s) {
     const long long blocks = a.T_max < (long long)sm_count() * 4 ? a.T_max : (long long)sm_count() * 4;
     if (a.bf16) grpo_loss_rows_kernel<true><<<(unsigned)blocks, kRowThreads, 0, s>>>(a);
@@ -177,6 +191,8 @@ extern "C" int dppo_grpo_loss_fwd_bwd(const dppo_loss_params* p, const void* log
     if (p->row_stride < p->V) return fail(DPPO_ERR_BAD_SHAPE, "grpo_loss: row_stride %lld < V %d", (long long)p->row_stride, p->V);
     if (!(p->temperature > 0.0) || !(p->eps_lo >= 0.0) || !(p->eps_hi >= 0.0) || !(p->beta == p->beta))
         return fail(DPPO_ERR_INVALID_ARG, "grpo_loss: temperature must be > 0, eps >= 0, beta a number");
+    if (p->no_length_norm != 0 && p->no_length_norm != 1) return fail(DPPO_ERR_INVALID_ARG, "grpo_loss: no_length_norm %d", p->no_length_norm);
+    if (p->seq_log_ratio && p->no_length_norm) return fail(DPPO_ERR_INVALID_ARG, "grpo_loss: the sequence-level ratio needs the 1/|o| normalisation");
     if (p->variant < 0) return fail(DPPO_ERR_INVALID_ARG, "grpo_loss: variant %d", p->variant);
     if (p->T_max >= ((int64_t)1 << 31)) return fail(DPPO_ERR_BAD_SHAPE, "grpo_loss: T_max must be below 2^31");
     if (!loss_out) return fail(DPPO_ERR_INVALID_ARG, "grpo_loss: NULL loss_out");
@@ -202,6 +218,7 @@ extern "C" int dppo_grpo_loss_fwd_bwd(const dppo_loss_params* p, const void* log
     a.V = p->V; a.S_max = p->S_max; a.bf16 = p->dtype == DPPO_BF16 ? 1 : 0;
     a.eps_lo = p->eps_lo; a.eps_hi = p->eps_hi; a.beta = p->beta; a.temperature = p->temperature;
     a.scale2 = (float)(1.4426950408889634 / p->temperature);
+    a.seq_log_ratio = p->seq_log_ratio; a.no_length_norm = p->no_length_norm;
     cudaStream_t s = (cudaStream_t)stream;
     if (p->T_max > 0) {
         // variant: 0 picks the kernel from the shape; 1 forces the general kernel; C*10000 + threads
@@ -223,4 +240,15 @@ extern "C" int dppo_grpo_loss_fwd_bwd(const dppo_loss_params* p, const void* log
         if (rc != DPPO_OK) return rc;
     }
     return launch_loss_reduce(a, loss_out, s);
+}
+
+extern "C" int dppo_sequence_log_ratio(const float* logp, const float* logp_old, const int32_t* cu_seqlens, int S_max,
+                                       float* out, int32_t* status, void* stream) {
+    (void)status;
+    if (S_max < 0) return dppo::fail(DPPO_ERR_INVALID_ARG, "sequence_log_ratio: S_max=%d", S_max);
+    if (S_max == 0) return DPPO_OK;
+    if (!logp || !logp_old || !cu_seqlens || !out) return dppo::fail(DPPO_ERR_INVALID_ARG, "sequence_log_ratio: NULL array");
+    dppo::sequence_log_ratio_kernel<<<(S_max + 7) / 8, 256, 0, (cudaStream_t)stream>>>(logp, logp_old, cu_seqlens, S_max, out);
+    DPPO_CHECK_LAUNCH("sequence_log_ratio launch");
+    return DPPO_OK;
 }

@@ -36,6 +36,8 @@ struct LossArgs {
     long long row_bytes;
     int V, S_max, bf16;
     double eps_lo, eps_hi, beta, temperature;
+    const float* seq_log_ratio;   // nullable: sequence-level ratio, indexed by sequence position
+    int no_length_norm;
     float scale2;            // log2(e) / temperature as the f32 both passes multiply by
 };
 
@@ -89,6 +91,8 @@ struct RowInputs {
     double W;                // w[seq] / |o_seq|
     double zy;               // z[y] / temperature
     double logp_old, logp_ref;
+    double seq_lr;           // log of the sequence-level ratio (used when use_seq)
+    int use_seq;
     int y;
     int state;               // 0 ok, else the dppo_status to report (row adds nothing, dlogits zero)
 };
@@ -96,7 +100,8 @@ struct RowInputs {
 // load_zy = false: the caller supplies z[y] itself (the fused LM-head has no logits in memory).
 __device__ __forceinline__ void row_inputs_from_segment(const LossArgs& a, long long t, int seg, RowInputs& in,
                                                         bool load_zy = true) {
-    in.A = in.W = in.zy = in.logp_old = in.logp_ref = 0.0;
+    in.A = in.W = in.zy = in.logp_old = in.logp_ref = in.seq_lr = 0.0;
+    in.use_seq = 0;
     in.y = a.target[t];
     in.state = 0;
     const long long seg_lo = a.cu_seqlens[seg], seg_hi = a.cu_seqlens[seg + 1];
@@ -104,7 +109,8 @@ __device__ __forceinline__ void row_inputs_from_segment(const LossArgs& a, long 
     if (in.y < 0 || in.y >= a.V) { in.state = DPPO_STATUS_BAD_TARGET; return; }
     const int idx = a.seg_map ? a.seg_map[seg] : seg;
     in.A = (double)a.adv[idx];
-    in.W = (double)a.w[idx] / (double)(seg_hi - seg_lo);
+    in.W = a.no_length_norm ? (double)a.w[idx] : (double)a.w[idx] / (double)(seg_hi - seg_lo);
+    if (a.seq_log_ratio) { in.use_seq = 1; in.seq_lr = (double)a.seq_log_ratio[seg]; }
     if (load_zy)
         in.zy = (double)(a.bf16 ? Elems<true>::load1(a.logits + t * a.row_bytes, in.y)
                                 : Elems<false>::load1(a.logits + t * a.row_bytes, in.y)) / a.temperature;
@@ -155,7 +161,7 @@ __device__ __forceinline__ RowScalars row_finish(const LossArgs& a, long long t,
     } else {
         const double A = in.A, W = in.W;
         const double logp = in.zy - lse;
-        const double rho = exp(logp - in.logp_old);
+        const double rho = in.use_seq ? exp(in.seq_lr) : exp(logp - in.logp_old);
         const double d = in.logp_ref - logp;
         const double rho_hat = exp(d);
         const double kl = rho_hat - d - 1.0;

@@ -577,6 +577,8 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
     if (lp.dtype != DPPO_BF16) return fail(DPPO_ERR_UNSUPPORTED, "lmhead: hidden and W must be bf16");
     if (!(lp.temperature > 0.0) || !(lp.eps_lo >= 0.0) || !(lp.eps_hi >= 0.0) || !(lp.beta == lp.beta))
         return fail(DPPO_ERR_INVALID_ARG, "lmhead: temperature must be > 0, eps >= 0, beta a number");
+    if ((lp.no_length_norm != 0 && lp.no_length_norm != 1) || (lp.seq_log_ratio && lp.no_length_norm))
+        return fail(DPPO_ERR_INVALID_ARG, "lmhead: no_length_norm / seq_log_ratio");
     if (lp.T_max >= ((int64_t)1 << 31) - kChunkTokens) return fail(DPPO_ERR_BAD_SHAPE, "lmhead: T_max too large");
     const bool backward = p->backward != 0;
     if (backward && (!dhidden || !dW)) return fail(DPPO_ERR_INVALID_ARG, "lmhead: backward requested but dhidden / dW is NULL");
@@ -603,6 +605,7 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
     a.T_max = lp.T_max; a.row_bytes = 0; a.V = lp.V; a.S_max = lp.S_max; a.bf16 = 1;
     a.eps_lo = lp.eps_lo; a.eps_hi = lp.eps_hi; a.beta = lp.beta; a.temperature = lp.temperature;
     a.scale2 = (float)(1.4426950408889634 / lp.temperature);
+    a.seq_log_ratio = lp.seq_log_ratio; a.no_length_norm = lp.no_length_norm;
     cudaStream_t s = (cudaStream_t)stream;
     const int H = p->H, V = lp.V;
     const long long T = lp.T_max;          // host-side bound; rows at or past the device-side count carry g = 0

@@ -177,7 +177,8 @@ def test_pack_dataset_scale_and_bad_length():
 
 # ------------------------------------------------------------------------------------------- steps 6-8
 def _loss_case(V, dtype, T, S, seed, sigma_noise=0.05, logit_sigma=2.0, tau=1.0, pad=0, in_place=False,
-               forward_only=False, n_tokens=None, beta=0.04, eps=(0.2, 0.2), variant=0):
+               forward_only=False, n_tokens=None, beta=0.04, eps=(0.2, 0.2), variant=0, no_length_norm=False,
+               seq_ratio=False):
     """Runs dppo_grpo_loss_fwd_bwd on a random case and compares everything with the oracle."""
     from paper_2603_04135_b200 import binding as B
     w = synth.scaled(synth.WORKLOADS["config0"], V=V, dtype=dtype, logit_sigma=logit_sigma)
@@ -206,16 +207,34 @@ def _loss_case(V, dtype, T, S, seed, sigma_noise=0.05, logit_sigma=2.0, tau=1.0,
     loss_out = torch.zeros(5, device="cuda"); logp_out = torch.zeros(T, device="cuda"); lse_out = torch.zeros(T, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     ntd = torch.tensor([T_true], dtype=torch.int32, device="cuda") if n_tokens is not None else None
-    B.grpo_loss_fwd_bwd(prm, buf, tok.target, tok.logp_old, tok.logp_ref, torch.from_numpy(cu_pad).cuda(), ntd,
+    d_cu = torch.from_numpy(cu_pad).cuda()
+    prm.no_length_norm = int(no_length_norm)
+    slr_dev = None
+    if seq_ratio:
+        # sequence-level ratio: a forward-only sweep gives the current log-probs, their mean log-ratio per
+        # sequence goes back in as a per-sequence input of the second sweep
+        B.grpo_loss_fwd_bwd(prm, buf, tok.target, tok.logp_old, tok.logp_ref, d_cu, ntd, torch.from_numpy(adv).cuda(),
+                            torch.from_numpy(wseq).cuda(), torch.from_numpy(seg_map).cuda(), None, logp_out, None,
+                            loss_out, ws, nbytes, status)
+        slr_dev = torch.full((S_max,), 9.0, device="cuda")
+        B.sequence_log_ratio(logp_out, tok.logp_old, d_cu, S_max, slr_dev)
+        prm.seq_log_ratio = slr_dev.data_ptr()
+    B.grpo_loss_fwd_bwd(prm, buf, tok.target, tok.logp_old, tok.logp_ref, d_cu, ntd,
                         torch.from_numpy(adv).cuda(), torch.from_numpy(wseq).cuda(), torch.from_numpy(seg_map).cuda(),
                         dl, logp_out, lse_out, loss_out, ws, nbytes, status)
     torch.cuda.synchronize()
     assert status.item() == 0
 
     z = logits_before[:T_true, :V].to(torch.float64).cpu().numpy()
+    slr = None
+    if seq_ratio:
+        lp64 = oracle.token_logprob(z, tok.target.cpu().numpy()[:T_true], tau)[0]
+        slr = oracle.sequence_log_ratio(lp64, tok.logp_old.cpu().numpy()[:T_true], cu)
+        got_slr = slr_dev.cpu().numpy()
+        assert np.abs(got_slr[:S_real] - slr).max() <= LOGP_TOL[dtype] and (got_slr[S_real:] == 0).all()
     ref = oracle.grpo_loss(z, tok.target.cpu().numpy(), tok.logp_old.cpu().numpy(), tok.logp_ref.cpu().numpy(), cu,
                            adv[seg_map][:S_real], wseq[seg_map][:S_real], eps[0], eps[1], beta, tau,
-                           want_dlogits=not forward_only)
+                           want_dlogits=not forward_only, length_norm=not no_length_norm, seq_log_ratio=slr)
     lo = loss_out.cpu().numpy().astype(np.float64)
     stable = clip_decision_is_stable(ref["rho"], eps[0], eps[1])
     assert stable.all(), "test case sits on a clip boundary; change the seed"
@@ -263,6 +282,17 @@ def test_loss_all_clip_branches(dtype):
     A, rho, cl = ref["A"], ref["rho"], ref["clipped"]
     assert (cl & (A > 0) & (rho > 1.2)).any() and (cl & (A < 0) & (rho < 0.8)).any()
     assert (~cl & (A > 0)).any() and (~cl & (A < 0)).any() and (A == 0).any()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_loss_variants_of_other_objectives(dtype):
+    # no 1/|o| normalisation (token-level aggregation is then a matter of w), sequence-level ratio
+    _loss_case(2056, dtype, T=80, S=6, seed=71, no_length_norm=True)
+    _loss_case(2056, dtype, T=80, S=6, seed=72, seq_ratio=True, sigma_noise=0.3)
+    _loss_case(2056, dtype, T=80, S=6, seed=73, seq_ratio=True, n_tokens=61)
+    if dtype == "bf16":
+        _loss_case(151936, dtype, T=40, S=3, seed=74, seq_ratio=True, variant=40256)
+        _loss_case(151936, dtype, T=40, S=3, seed=75, no_length_norm=True, variant=0)
 
 
 def test_loss_full_vocab_bf16_rows():

@@ -208,3 +208,55 @@ def test_bf16_conversions_match_torch():
     assert np.array_equal(bits, want)
     back = oracle.bf16_bits_to_f64(bits)
     assert np.array_equal(back, torch.from_numpy(want.view(np.int16)).view(torch.bfloat16).double().numpy())
+
+
+def test_variant_without_length_normalisation():
+    z, y, lo, lr, cu, adv, w = _case(T=60, seed=4)
+    logp = scipy.special.log_softmax(z, axis=1)[np.arange(len(y)), y]
+    # on policy, beta = 0: every token's surrogate is A, so the loss is -sum_s w_s A_s |o_s|
+    out = oracle.grpo_loss(z, y, logp, logp, cu, adv, w, 0.2, 0.2, 0.0, length_norm=False)
+    lens = np.diff(cu)
+    assert math.isclose(out["loss"], -float((w * adv * lens).sum()), rel_tol=1e-12)
+    # it is the normalised loss with weights w_s |o_s|
+    a = oracle.grpo_loss(z, y, lo, lr, cu, adv, w, length_norm=False)
+    b = oracle.grpo_loss(z, y, lo, lr, cu, adv, w * lens)
+    assert math.isclose(a["loss"], b["loss"], rel_tol=1e-12) and np.allclose(a["dlogits"], b["dlogits"], rtol=1e-12, atol=0)
+
+
+def test_sequence_level_ratio_variant():
+    z, y, lo, lr, cu, adv, w = _case(T=45, V=31, S=4, seed=6, sigma=0.25)
+    T = len(y)
+
+    def loss_of(zz):
+        logp = scipy.special.log_softmax(zz, axis=1)[np.arange(T), y]
+        slr = oracle.sequence_log_ratio(logp, lo, cu)
+        return oracle.grpo_loss(zz, y, lo, lr, cu, adv, w, 0.2, 0.2, 0.04, seq_log_ratio=slr, want_dlogits=False)["loss"], slr
+
+    base, slr = loss_of(z)
+    # the mean token log-ratio per sequence, against a direct numpy mean
+    logp = scipy.special.log_softmax(z, axis=1)[np.arange(T), y]
+    for s in range(len(adv)):
+        assert math.isclose(slr[s], float((logp - lo)[cu[s]:cu[s + 1]].mean()), rel_tol=1e-12, abs_tol=1e-15)
+    out = oracle.grpo_loss(z, y, lo, lr, cu, adv, w, 0.2, 0.2, 0.04, seq_log_ratio=slr)
+    assert math.isclose(out["loss"], base, rel_tol=1e-14)
+    # every token of a sequence shares the ratio
+    for s in range(len(adv)):
+        assert np.allclose(out["rho"][cu[s]:cu[s + 1]], math.exp(slr[s]), rtol=1e-13)
+    # the analytic gradient is the gradient of the whole two-stage map logits -> logp -> sequence ratio -> loss
+    rng = np.random.default_rng(2)
+    h, checked = 1e-6, 0
+    for _ in range(30):
+        t = int(rng.integers(0, T)); v = int(rng.integers(0, z.shape[1])) if rng.random() > 0.3 else int(y[t])
+        s = int(np.searchsorted(cu, t, side="right") - 1)
+        if min(abs(math.exp(slr[s]) - 0.8), abs(math.exp(slr[s]) - 1.2)) < 1e-3:
+            continue
+        zp = z.copy(); zp[t, v] += h; zm = z.copy(); zm[t, v] -= h
+        fd = (loss_of(zp)[0] - loss_of(zm)[0]) / (2 * h)
+        assert math.isclose(fd, out["dlogits"][t, v], rel_tol=1e-5, abs_tol=1e-9), (t, v)
+        checked += 1
+    assert checked > 15
+    # when every token of every sequence has the same log-ratio the two objectives coincide
+    lo2 = logp - 0.07
+    a = oracle.grpo_loss(z, y, lo2, lr, cu, adv, w)
+    b = oracle.grpo_loss(z, y, lo2, lr, cu, adv, w, seq_log_ratio=oracle.sequence_log_ratio(logp, lo2, cu))
+    assert math.isclose(a["loss"], b["loss"], rel_tol=1e-12) and np.allclose(a["dlogits"], b["dlogits"], rtol=1e-10, atol=1e-18)
