@@ -302,10 +302,31 @@ def run_ours(args):
 
     # ---- end to end: host buffers in, loss scalars out, through DppoStep.step_from_host
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
-    host_tok = {k: torch.empty(getattr(tok, k).shape, dtype=getattr(tok, k).dtype, pin_memory=True)
-                for k in ("logits", "target", "logp_old", "logp_ref")}
+    # pinned host copy of the step's inputs; when all ranks together would pin more than half of the
+    # host's memory (or pinning fails) the logits come from a pinned window that is copied repeatedly
+    logits_bytes = tok.logits.numel() * tok.logits.element_size()
+    try:
+        import psutil
+        host_total = psutil.virtual_memory().total
+    except Exception:
+        host_total = 64 << 30
+    rows_host = T
+    if world * logits_bytes > host_total // 2:
+        rows_host = max(1, int((host_total // (4 * world)) // (w.V * 2)))
+    host_buffer = "full copy of the inputs"
+    while True:
+        try:
+            host_tok = {k: torch.empty((min(rows_host, T),) + tuple(getattr(tok, k).shape[1:]), dtype=getattr(tok, k).dtype,
+                                       pin_memory=True) for k in ("logits", "target", "logp_old", "logp_ref")}
+            break
+        except RuntimeError:
+            if rows_host <= 1024:
+                raise
+            rows_host //= 2
+    if rows_host < T:
+        host_buffer = "pinned window of %d rows copied repeatedly (host memory)" % rows_host
     for k in host_tok:
-        host_tok[k].copy_(getattr(tok, k))
+        host_tok[k].copy_(getattr(tok, k)[:host_tok[k].shape[0]])
     dev_tok = {k: getattr(tok, k) for k in host_tok}
     host_batch = {"rewards": torch.from_numpy(batch.rewards.reshape(-1).copy()).pin_memory(),
                   "unit_len": torch.from_numpy(batch.unit_len.copy()).pin_memory(),
@@ -347,7 +368,7 @@ def run_ours(args):
                        "parallelism": "dp%d, independent batches" % world},
             "clocks": clocks,
             "e2e": {"value": dp.throughput(T_all, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                    "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+                    "d2h_bytes_per_step": d2h, "steps": e2e_steps, "host_buffer": host_buffer},
             "gpu_launches": 5 * args.steps,
             "roofline": {"bound": "hbm", "kernel": "grpo loss sweep (rows kernel + its 1-block reduction)",
                          "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,

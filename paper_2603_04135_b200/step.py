@@ -109,7 +109,8 @@ class DppoStep:
 
         batch_host: dict with pinned tensors rewards, unit_len, loss_len and optionally H_prev.
         token_host / dev_tokens: dicts with logits, target, logp_old, logp_ref (host source, device
-        destination).  Returns (loss_out as a host tensor, bytes copied host->device, bytes device->host).
+        destination).  A host tensor with fewer rows than its destination is treated as a window that is
+        copied repeatedly (same bytes over the bus, for hosts that cannot pin the whole input).  Returns (loss_out as a host tensor, bytes copied host->device, bytes device->host).
         """
         h2d = 0
         for name in ("rewards", "unit_len", "loss_len"):
@@ -120,8 +121,16 @@ class DppoStep:
             self.H_prev.copy_(batch_host["H_prev"], non_blocking=True)
             h2d += batch_host["H_prev"].numel() * 4
         for name in ("logits", "target", "logp_old", "logp_ref"):
-            dev_tokens[name].copy_(token_host[name], non_blocking=True)
-            h2d += token_host[name].numel() * token_host[name].element_size()
+            src, dst = token_host[name], dev_tokens[name]
+            if src.shape[0] >= dst.shape[0]:
+                dst.copy_(src[:dst.shape[0]], non_blocking=True)
+            else:
+                # the pinned host buffer is a window of `src.shape[0]` rows (host memory is short): the
+                # same number of bytes crosses the bus, window by window
+                for a in range(0, dst.shape[0], src.shape[0]):
+                    b = min(dst.shape[0], a + src.shape[0])
+                    dst[a:b].copy_(src[:b - a], non_blocking=True)
+            h2d += dst.numel() * dst.element_size()
         self.prune_pack(seed, step)
         self.loss(dev_tokens["logits"], dev_tokens["target"], dev_tokens["logp_old"], dev_tokens["logp_ref"], dlogits)
         out = self.loss_out.cpu()                         # device -> host read of the result; synchronises
