@@ -274,6 +274,8 @@ typedef struct {
     dppo_loss_params loss;
     int32_t H;
     int32_t backward;
+    int32_t variant;        /* 0: CTA pairs (cta_group::2) share each B tile; 1: one CTA per tile (tuning aid) */
+    int32_t reserved;       /* 0 */
 } dppo_lmhead_params;
 
 size_t dppo_lmhead_workspace_bytes(const dppo_lmhead_params* p);

@@ -273,6 +273,189 @@ lm_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
 }
 
+// ---- the GEMM core on CTA pairs (cta_group::2) -------------------------------------------------------
+// Two CTAs of a cluster share one 256 x 256 tile: each loads its own 128 rows of A and HALF of the B tile
+// (128 rows), the leader's MMA thread issues tcgen05.mma.cta_group::2 (M = 256) which reads both halves of B
+// from the two CTAs' shared memory and writes each CTA's 128 rows into that CTA's tensor memory.  Per SM
+// and K slab this is 32 KB of operands instead of 48 KB for the same flops.  TMA loads signal the
+// leader's `full` barrier (no multicast); tcgen05.commit is multicast to both CTAs' barriers; both
+// epilogues report to the leader's `acc_empty`.
+constexpr int kStages2 = 6;
+constexpr int kHalfBN = kBN / 2;
+constexpr int kStageBytesB2 = kHalfBN * kBK * 2;             // 16 KB
+constexpr int kStageBytes2 = kStageBytesA + kStageBytesB2;   // 32 KB per CTA
+constexpr uint32_t kIdesc2 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+constexpr uint32_t kPeerMask = 0xFEFFFFFFu;                  // shared::cluster address of the pair's leader (rank bit cleared)
+
+struct LmShared2 {
+    unsigned long long full[kStages2];
+    unsigned long long empty[kStages2];
+    unsigned long long acc_full[2];
+    unsigned long long acc_empty[2];     // the leader's copy counts 8 arrivals: 4 epilogue warps x 2 CTAs
+    uint32_t tmem_base;
+    int abort;
+};
+
+template <bool kRowSweep>
+__device__ __forceinline__ bool pair_tile_of(const GemmShape& gs, uint32_t j, int& m2, int& n) {
+    const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+    const int n_m2 = (gs.n_mtiles + 1) >> 1;
+    if (kRowSweep) {
+        m2 = pair + (int)(j / (uint32_t)gs.n_ntiles) * npairs;
+        n = (int)(j % (uint32_t)gs.n_ntiles);
+        return m2 < n_m2;
+    }
+    const long long id = (long long)pair + (long long)j * npairs;
+    if (id >= (long long)n_m2 * gs.n_ntiles) return false;
+    if (gs.m_fast) { m2 = (int)(id % n_m2); n = (int)(id / n_m2); }
+    else           { m2 = (int)(id / gs.n_ntiles); n = (int)(id % gs.n_ntiles); }
+    return true;
+}
+
+__device__ __forceinline__ void lm_cluster_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+template <class Epi, bool kRowSweep>
+__global__ void __launch_bounds__(kLmThreads, 1)
+lm_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                const GemmShape gs, Epi epi, int32_t* status) {
+    extern __shared__ unsigned char lm_raw[];
+    __shared__ LmShared2 sh;
+    const uint32_t tiles = (lm_smem_u32(lm_raw) + 1023u) & ~1023u;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    uint32_t rank;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+    const bool leader = rank == 0;
+    volatile int* abort_flag = &sh.abort;
+
+    if (tid == 0) {
+        sh.abort = 0;
+        for (int s = 0; s < kStages2; ++s) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(lm_smem_u32(&sh.full[s])));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(lm_smem_u32(&sh.empty[s])));
+        }
+        for (int b = 0; b < 2; ++b) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(lm_smem_u32(&sh.acc_full[b])));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 8;" :: "r"(lm_smem_u32(&sh.acc_empty[b])));
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {                                                     // both CTAs, same warp, same destination
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                     :: "r"(lm_smem_u32(&sh.tmem_base)), "r"((uint32_t)kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    lm_cluster_sync();                                                   // the peer's barriers and tensor memory exist
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = sh.tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer (both CTAs)
+        if (lane == 0) {
+            uint32_t it = 0;
+            int m2, n;
+            for (uint32_t j = 0; pair_tile_of<kRowSweep>(gs, j, m2, n) && !*abort_flag; ++j) {
+                const int m = 2 * m2 + (int)rank;
+                for (int k = 0; k < gs.n_ksteps; ++k, ++it) {
+                    const uint32_t s = it % kStages2, use = it / kStages2;
+                    if (use > 0 && !lm_wait(lm_smem_u32(&sh.empty[s]), (use - 1) & 1, abort_flag)) break;
+                    const uint32_t bar_local = lm_smem_u32(&sh.full[s]);
+                    const uint32_t bar = bar_local & kPeerMask;           // the leader's barrier collects both CTAs' bytes
+                    const uint32_t dst_a = tiles + s * kStageBytes2, dst_b = dst_a + kStageBytesA;
+                    if (leader)
+                        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar_local), "r"((uint32_t)(2 * kStageBytes2)) : "memory");
+                    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                                 :: "r"(dst_a), "l"(&map_a), "r"(bar), "r"(k * kBK), "r"(gs.a_row0 + m * kBM) : "memory");
+                    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                                 :: "r"(dst_b), "l"(&map_b), "r"(bar), "r"(k * kBK), "r"(n * kBN + (int)rank * kHalfBN) : "memory");
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (lane == 0 && leader) {
+            uint32_t it = 0;
+            int m2, n;
+            for (uint32_t j = 0; pair_tile_of<kRowSweep>(gs, j, m2, n) && !*abort_flag; ++j) {
+                const uint32_t b = j & 1, use_b = j >> 1;
+                if (use_b > 0 && !lm_wait(lm_smem_u32(&sh.acc_empty[b]), (use_b - 1) & 1, abort_flag)) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t d_tmem = tmem_base + b * kBN;
+                bool ok = true;
+                for (int k = 0; k < gs.n_ksteps; ++k, ++it) {
+                    const uint32_t s = it % kStages2, use = it / kStages2;
+                    if (!lm_wait(lm_smem_u32(&sh.full[s]), use & 1, abort_flag)) { ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t sa = tiles + s * kStageBytes2, sb = sa + kStageBytesA;
+                    const uint64_t da = lm_smem_desc(sa), db = lm_smem_desc(sb);
+#pragma unroll
+                    for (int kk = 0; kk < kBK / 16; ++kk) {
+                        const uint32_t accumulate = (k > 0 || kk > 0) ? 1u : 0u;
+                        asm volatile("{\n\t.reg .pred p;\n\t"
+                                     "setp.ne.b32 p, %4, 0;\n\t"
+                                     "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                                     :: "r"(d_tmem), "l"(da + (uint64_t)(kk * 2)), "l"(db + (uint64_t)(kk * 2)),
+                                        "r"(kIdesc2), "r"(accumulate) : "memory");
+                    }
+                    // frees this stage in BOTH CTAs once the MMAs issued so far have read it
+                    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                                 :: "r"(lm_smem_u32(&sh.empty[s])), "h"((unsigned short)3) : "memory");
+                }
+                if (!ok) break;
+                asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                             :: "r"(lm_smem_u32(&sh.acc_full[b])), "h"((unsigned short)3) : "memory");
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        int m2, n;
+        for (uint32_t j = 0; pair_tile_of<kRowSweep>(gs, j, m2, n); ++j) {
+            const int m = 2 * m2 + (int)rank;
+            const uint32_t b = j & 1, use_b = j >> 1;
+            if (!kRowSweep || n == 0) epi.row_begin(m, row);
+            if (!__all_sync(0xffffffffu, lm_wait(lm_smem_u32(&sh.acc_full[b]), use_b & 1, abort_flag))) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + b * kBN;
+#pragma unroll 1
+            for (int ch = 0; ch < kBN / 32; ++ch) {
+                uint32_t v[32];
+                asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                             "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                             "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                             : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                               "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+                               "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+                               "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                             : "r"(taddr + (uint32_t)(ch * 32)) : "memory");
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                epi.chunk(m, n, row, ch, v);
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0)                                               // the leader's MMA thread waits for all 8 warps
+                asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" :: "r"(lm_smem_u32(&sh.acc_empty[b]) & kPeerMask) : "memory");
+            if (!kRowSweep || n == gs.n_ntiles - 1) epi.row_end(m, row);
+        }
+    }
+
+    // ---- common exit: both CTAs are done with tensor memory and with each other's barriers, then free
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    lm_cluster_sync();
+    if (tid == 0 && sh.abort) set_status(status, DPPO_STATUS_TIMEOUT);
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
+    }
+}
+
 // ---- epilogues ------------------------------------------------------------------------------------
 struct RowInfo {             // what the backward needs from the forward, per token
     float lse2_hi, lse2_lo;  // base-2 log-sum-exp of z * scale2
@@ -527,6 +710,41 @@ static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const GemmS
     return DPPO_OK;
 }
 
+constexpr size_t kLmDynSmem2 = (size_t)kStages2 * kStageBytes2 + 1024;
+
+// CTA-pair version: `mb_half` is B's tensor map with 128-row boxes.
+template <class Epi, bool kRowSweep>
+static int launch_gemm2(const CUtensorMap& ma, const CUtensorMap& mb_half, const GemmShape& gs, const Epi& epi,
+                        int32_t* status, cudaStream_t s, const char* what) {
+    auto kernel = lm_gemm2_kernel<Epi, kRowSweep>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLmDynSmem2);
+    if (e != cudaSuccess) return cuda_fail(e, "lmhead: shared memory attribute");
+    const long long n_m2 = (gs.n_mtiles + 1) / 2;
+    const long long work = kRowSweep ? n_m2 : n_m2 * gs.n_ntiles;
+    const long long max_pairs = sm_count() / 2;
+    const int pairs = (int)(work < max_pairs ? work : max_pairs);
+    if (pairs < 1) return DPPO_OK;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1);
+    cfg.blockDim = dim3(kLmThreads, 1, 1);
+    cfg.dynamicSmemBytes = kLmDynSmem2;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, kernel, ma, mb_half, gs, epi, status);
+    if (e != cudaSuccess) return cuda_fail(e, what);
+    return DPPO_OK;
+}
+
+template <class Epi, bool kRowSweep>
+static int run_gemm(bool pair, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mb_half, const GemmShape& gs,
+                    const Epi& epi, int32_t* status, cudaStream_t s, const char* what) {
+    return pair ? launch_gemm2<Epi, kRowSweep>(ma, mb_half, gs, epi, status, s, what)
+                : launch_gemm<Epi, kRowSweep>(ma, mb, gs, epi, status, s, what);
+}
+
 static long long round_up(long long x, long long m) { return (x + m - 1) / m * m; }
 
 struct LmWorkspace {
@@ -580,6 +798,7 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
     if ((lp.no_length_norm != 0 && lp.no_length_norm != 1) || (lp.seq_log_ratio && lp.no_length_norm))
         return fail(DPPO_ERR_INVALID_ARG, "lmhead: no_length_norm / seq_log_ratio");
     if (lp.T_max >= ((int64_t)1 << 31) - kChunkTokens) return fail(DPPO_ERR_BAD_SHAPE, "lmhead: T_max too large");
+    if (p->variant != 0 && p->variant != 1) return fail(DPPO_ERR_INVALID_ARG, "lmhead: variant %d", p->variant);
     const bool backward = p->backward != 0;
     if (backward && (!dhidden || !dW)) return fail(DPPO_ERR_INVALID_ARG, "lmhead: backward requested but dhidden / dW is NULL");
     if (!backward && (dhidden || dW)) return fail(DPPO_ERR_INVALID_ARG, "lmhead: dhidden / dW given but params.backward is 0");
@@ -610,10 +829,13 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
     const int H = p->H, V = lp.V;
     const long long T = lp.T_max;          // host-side bound; rows at or past the device-side count carry g = 0
     if (T > 0) {
-        alignas(64) CUtensorMap map_h, map_w;
+        const bool pair = p->variant != 1;     // CTA pairs sharing the B tile unless the single-CTA core is forced
+        alignas(64) CUtensorMap map_h, map_w, map_w_half;
         int rc = make_map(&map_h, hidden, T, H, H, kBM);
         if (rc != DPPO_OK) return rc;
         rc = make_map(&map_w, W, V, H, H, kBN);
+        if (rc != DPPO_OK) return rc;
+        rc = make_map(&map_w_half, W, V, H, H, kHalfBN);
         if (rc != DPPO_OK) return rc;
         RowInfo* info = (RowInfo*)(ws + lay.info);
 
@@ -622,7 +844,7 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
         gs.n_mtiles = (int)((T + kBM - 1) / kBM); gs.n_ntiles = (V + kBN - 1) / kBN; gs.n_ksteps = H / kBK;
         EpiLse fwd = {};
         fwd.a = a; fwd.info = backward ? info : nullptr;
-        rc = launch_gemm<EpiLse, true>(map_h, map_w, gs, fwd, status, s, "lmhead forward launch");
+        rc = run_gemm<EpiLse, true>(pair, map_h, map_w, map_w_half, gs, fwd, status, s, "lmhead forward launch");
         if (rc != DPPO_OK) return rc;
 
         if (backward) {
@@ -636,8 +858,10 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
             transpose_bf16_kernel<<<dim3((H + 63) / 64, (unsigned)((T + 63) / 64)), 256, 0, s>>>(
                 (const __nv_bfloat16*)hidden, T, H, H, ht, lay.ld_t);
             DPPO_CHECK_LAUNCH("lmhead transpose launch");
-            alignas(64) CUtensorMap map_wt;
+            alignas(64) CUtensorMap map_wt, map_wt_half;
             rc = make_map(&map_wt, Wt, H, V, lay.ld_v, kBN);
+            if (rc != DPPO_OK) return rc;
+            rc = make_map(&map_wt_half, Wt, H, V, lay.ld_v, kHalfBN);
             if (rc != DPPO_OK) return rc;
 
             for (long long t0 = 0, c = 0; t0 < T; t0 += kChunkTokens, ++c) {
@@ -649,17 +873,17 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
                 EpiDlogits e1 = {};
                 e1.info = info; e1.D = D; e1.Dt = Dt; e1.t0 = t0; e1.tc = tc; e1.ldd = lay.ld_v; e1.ldt = lay.ld_tc;
                 e1.V = V; e1.c = a.scale2;
-                rc = launch_gemm<EpiDlogits, false>(map_h, map_w, g1, e1, status, s, "lmhead dlogits launch");
+                rc = run_gemm<EpiDlogits, false>(pair, map_h, map_w, map_w_half, g1, e1, status, s, "lmhead dlogits launch");
                 if (rc != DPPO_OK) return rc;
                 // (2) dhidden[t0 : t0+tc, :] = D Wt^T          (M = tokens, N = H, K = V)
-                alignas(64) CUtensorMap map_d, map_dt, map_ht_c;
+                alignas(64) CUtensorMap map_d, map_dt, map_ht_c, map_ht_c_half;
                 rc = make_map(&map_d, D, tc, V, lay.ld_v, kBM);
                 if (rc != DPPO_OK) return rc;
                 GemmShape g2 = {};
                 g2.n_mtiles = (int)((tc + kBM - 1) / kBM); g2.n_ntiles = (H + kBN - 1) / kBN; g2.n_ksteps = (V + kBK - 1) / kBK;
                 EpiStoreBf16 e2 = {};
                 e2.C = (__nv_bfloat16*)dhidden; e2.ldc = H; e2.row0 = t0; e2.rows = T; e2.cols = H;
-                rc = launch_gemm<EpiStoreBf16, false>(map_d, map_wt, g2, e2, status, s, "lmhead dhidden launch");
+                rc = run_gemm<EpiStoreBf16, false>(pair, map_d, map_wt, map_wt_half, g2, e2, status, s, "lmhead dhidden launch");
                 if (rc != DPPO_OK) return rc;
                 // (3) dW (+)= Dt ht[:, t0 : t0+tc]^T            (M = V, N = H, K = tokens of the chunk);
                 //     the K range must stop at the chunk, so ht gets a map of its own based at column t0
@@ -668,11 +892,13 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
                 if (rc != DPPO_OK) return rc;
                 rc = make_map(&map_ht_c, ht + t0, H, tc, lay.ld_t, kBN);
                 if (rc != DPPO_OK) return rc;
+                rc = make_map(&map_ht_c_half, ht + t0, H, tc, lay.ld_t, kHalfBN);
+                if (rc != DPPO_OK) return rc;
                 GemmShape g3 = {};
                 g3.n_mtiles = (V + kBM - 1) / kBM; g3.n_ntiles = (H + kBN - 1) / kBN; g3.n_ksteps = (int)((tc + kBK - 1) / kBK);
                 EpiAccumF32 e3 = {};
                 e3.C = (float*)dW; e3.ldc = H; e3.rows = V; e3.cols = H; e3.accumulate = c > 0 ? 1 : 0;
-                rc = launch_gemm<EpiAccumF32, false>(map_dt, map_ht_c, g3, e3, status, s, "lmhead dW launch");
+                rc = run_gemm<EpiAccumF32, false>(pair, map_dt, map_ht_c, map_ht_c_half, g3, e3, status, s, "lmhead dW launch");
                 if (rc != DPPO_OK) return rc;
             }
         }

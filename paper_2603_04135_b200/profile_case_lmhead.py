@@ -22,6 +22,7 @@ def main():
     ap.add_argument("--iters", type=int, default=3)
     ap.add_argument("--seqs", type=int, default=32)
     ap.add_argument("--backward", action="store_true", help="also dhidden and dW")
+    ap.add_argument("--variant", type=int, default=0, help="0: CTA pairs, 1: one CTA per tile")
     args = ap.parse_args()
     w = synth.scaled(synth.WORKLOADS["config4_h2560"], V=args.vocab, H=args.hidden)
     T, S = args.tokens, args.seqs
@@ -29,7 +30,7 @@ def main():
     cu = torch.from_numpy(np.linspace(0, T, S + 1).astype(np.int32)).cuda()
     adv = torch.from_numpy(np.random.default_rng(0).normal(size=S).astype(np.float32)).cuda()
     wseq = torch.full((S,), 1.0 / S, device="cuda")
-    prm = B.LmheadParams(B.LossParams(T, w.V, B.BF16, w.V, S, 0, w.eps, w.eps, w.beta, 1.0), w.H, int(args.backward))
+    prm = B.LmheadParams(B.LossParams(T, w.V, B.BF16, w.V, S, 0, w.eps, w.eps, w.beta, 1.0), w.H, int(args.backward), args.variant)
     nbytes = B.lmhead_workspace_bytes(prm)
     ws = torch.zeros(nbytes + 1024, dtype=torch.uint8, device="cuda")
     ws = ws[(-ws.data_ptr()) % 1024:]

@@ -9,7 +9,7 @@ from paper_2603_04135_b200 import synth
 pytestmark = pytest.mark.gpu
 
 
-def _run(T, V, H, S, seed, n_tokens=None, tau=1.0, backward=False):
+def _run(T, V, H, S, seed, n_tokens=None, tau=1.0, backward=False, variant=0):
     from paper_2603_04135_b200 import binding as B
     w = synth.scaled(synth.WORKLOADS["config4_h2560"], V=V, H=H)
     hidden, W, target, lo, lr = synth.make_lmhead_inputs(w, T, seed, device="cuda")
@@ -19,7 +19,7 @@ def _run(T, V, H, S, seed, n_tokens=None, tau=1.0, backward=False):
     cu = np.concatenate([[0], cuts, [T_true]]).astype(np.int32)
     S_real = len(cu) - 1
     adv = rng.normal(size=S_real).astype(np.float32); wseq = (rng.random(S_real) * 0.1).astype(np.float32)
-    prm = B.LmheadParams(B.LossParams(T, V, B.BF16, V, S_real, 0, w.eps, w.eps, w.beta, tau), H, int(backward))
+    prm = B.LmheadParams(B.LossParams(T, V, B.BF16, V, S_real, 0, w.eps, w.eps, w.beta, tau), H, int(backward), variant)
     nbytes = B.lmhead_workspace_bytes(prm)
     ws = torch.zeros(nbytes + 1024, dtype=torch.uint8, device="cuda")
     ws = ws[(-ws.data_ptr()) % 1024:]
@@ -62,26 +62,31 @@ def _run(T, V, H, S, seed, n_tokens=None, tau=1.0, backward=False):
     return ref
 
 
-def test_lmhead_small_shapes():
-    _run(T=200, V=1000, H=128, S=4, seed=1)             # ragged token tile, ragged vocabulary tile
-    _run(T=128, V=256, H=64, S=1, seed=2)               # exactly one tile, one K slab
-    _run(T=130, V=4096, H=4096, S=3, seed=3)            # the wider hidden size
-    _run(T=300, V=777, H=192, S=5, seed=4, n_tokens=259, tau=1.3)
+@pytest.mark.parametrize("variant", [1, 0])           # single-CTA core, CTA-pair core
+def test_lmhead_small_shapes(variant):
+    _run(T=200, V=1000, H=128, S=4, seed=1, variant=variant)     # ragged token tile, ragged vocabulary tile
+    _run(T=128, V=256, H=64, S=1, seed=2, variant=variant)       # exactly one tile, one K slab
+    _run(T=130, V=4096, H=4096, S=3, seed=3, variant=variant)    # the wider hidden size
+    _run(T=300, V=777, H=192, S=5, seed=4, n_tokens=259, tau=1.3, variant=variant)
+    _run(T=700, V=300, H=512, S=2, seed=6, variant=variant)      # several token tiles, an odd number of them
 
 
-def test_lmhead_full_vocabulary():
-    _run(T=300, V=151936, H=2560, S=4, seed=5)
+@pytest.mark.parametrize("variant", [1, 0])
+def test_lmhead_full_vocabulary(variant):
+    _run(T=300, V=151936, H=2560, S=4, seed=5, variant=variant)
 
 
-def test_lmhead_backward_small_shapes():
-    _run(T=200, V=1000, H=128, S=4, seed=11, backward=True)
-    _run(T=128, V=256, H=64, S=1, seed=12, backward=True)
-    _run(T=300, V=777, H=192, S=5, seed=14, n_tokens=259, tau=1.3, backward=True)
-    _run(T=130, V=2048, H=2560, S=3, seed=13, backward=True)
+@pytest.mark.parametrize("variant", [1, 0])
+def test_lmhead_backward_small_shapes(variant):
+    _run(T=200, V=1000, H=128, S=4, seed=11, backward=True, variant=variant)
+    _run(T=128, V=256, H=64, S=1, seed=12, backward=True, variant=variant)
+    _run(T=300, V=777, H=192, S=5, seed=14, n_tokens=259, tau=1.3, backward=True, variant=variant)
+    _run(T=130, V=2048, H=2560, S=3, seed=13, backward=True, variant=variant)
 
 
-def test_lmhead_backward_several_token_chunks():
-    _run(T=9472 + 9472 + 70, V=520, H=64, S=9, seed=15, backward=True)        # three chunks, the last one ragged
+@pytest.mark.parametrize("variant", [1, 0])
+def test_lmhead_backward_several_token_chunks(variant):
+    _run(T=9472 + 9472 + 70, V=520, H=64, S=9, seed=15, backward=True, variant=variant)   # three chunks, the last ragged
 
 
 def test_lmhead_argument_checks():
