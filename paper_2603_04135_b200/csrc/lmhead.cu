@@ -137,7 +137,7 @@ __device__ __forceinline__ bool tile_of(const GemmShape& gs, uint32_t j, int& m,
 template <class Epi, bool kRowSweep>
 __global__ void __launch_bounds__(kLmThreads, 1)
 lm_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const GemmShape gs, Epi epi, int32_t* status) {
+               const GemmShape gs, const Epi epi_args, int32_t* status) {
     extern __shared__ unsigned char lm_raw[];
     __shared__ LmShared sh;
     const uint32_t tiles = (lm_smem_u32(lm_raw) + 1023u) & ~1023u;      // 1024-byte aligned ring (swizzle atoms)
@@ -234,6 +234,7 @@ lm_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // ------------------------------------------------------------------ epilogue (warps 2..5)
         const int q = warp & 3;                                          // TMEM lane quarter this warp may read
         const int row = q * 32 + lane;
+        Epi epi = epi_args;                                              // per-thread copy: its state lives in registers
         int m, n;
         for (uint32_t j = 0; tile_of<kRowSweep>(gs, j, m, n); ++j) {
             const uint32_t b = j & 1, use_b = j >> 1;
@@ -320,7 +321,7 @@ __device__ __forceinline__ void lm_cluster_sync() {
 template <class Epi, bool kRowSweep>
 __global__ void __launch_bounds__(kLmThreads, 1)
 lm_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                const GemmShape gs, Epi epi, int32_t* status) {
+                const GemmShape gs, const Epi epi_args, int32_t* status) {
     extern __shared__ unsigned char lm_raw[];
     __shared__ LmShared2 sh;
     const uint32_t tiles = (lm_smem_u32(lm_raw) + 1023u) & ~1023u;
@@ -415,6 +416,7 @@ lm_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         // ------------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
         const int q = warp & 3;
         const int row = q * 32 + lane;
+        Epi epi = epi_args;
         int m2, n;
         for (uint32_t j = 0; pair_tile_of<kRowSweep>(gs, j, m2, n); ++j) {
             const int m = 2 * m2 + (int)rank;
@@ -486,14 +488,13 @@ struct EpiLse {
         const int col0 = n * kBN + ch * 32;
         const int valid = a.V - col0;                                // columns of this chunk inside the vocabulary
         const float c = a.scale2;
-        if (y >= col0 && y < col0 + 32) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) if (j == y - col0) zy = __uint_as_float(v[j]);
-        }
+        const int yrel = y - col0;                                   // selects, not an indexed read: v stays in registers
         float cm = -INFINITY;
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
-            const float x = (j < valid) ? __uint_as_float(v[j]) * c : -INFINITY;
+            const float raw = __uint_as_float(v[j]);
+            zy = (j == yrel) ? raw : zy;
+            const float x = (j < valid) ? raw * c : -INFINITY;
             v[j] = __float_as_uint(x);
             cm = fmaxf(cm, x);
         }
