@@ -40,8 +40,8 @@ WORKLOAD_TEXT = WORKLOAD + ": P=32 G=8, response 64-1024 tokens, V=151936 bf16 l
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch over 8192 rows of this vocabulary.  Traffic
 # grows in proportion to the rows, so a launch over T rows moves T times the per-row figure.  The record
 # is tied to the kernel sources it was taken from: once they change, `traffic` is reported as null.
-TRAFFIC_CAPTURE = {"rows": 8192, "dram_bytes": 2489454000 + 2431373000,
-                   "source_sha256": "1ce2823fbf508f3b3f5c6cc11b9b6bd11e47ce727585594b64f8280f82dc51a8"}
+TRAFFIC_CAPTURE = {"rows": 8192, "dram_bytes": 2489454000 + 2432057000,
+                   "source_sha256": "8bb2c583a518e9187152d702cc663e4f083fa44ef177016e38109b659c93700e"}
 
 
 def captured_traffic_per_row():
