@@ -3,7 +3,7 @@
 // A logit row of the full vocabulary (151,936 bf16 = 297 KB) does not fit one SM's shared memory, and
 // dlogits cannot be written before the row's log-sum-exp is known.  Instead of reading the row twice,
 // a thread-block cluster of C CTAs splits it: each CTA pulls its slice into shared memory with bulk
-// async copies (no multicast), reduces (max, sum 2^x) over the slice, the C partial pairs are
+// async copies (each CTA fetches only its own slice), reduces (max, sum 2^x) over the slice, the C partial pairs are
 // exchanged through distributed shared memory, every CTA repeats the cheap scalar stage, and the
 // second pass runs out of shared memory straight into streaming global stores.  HBM traffic is the
 // algorithmic minimum: one read and one write per element.  The exponentials of the first pass are

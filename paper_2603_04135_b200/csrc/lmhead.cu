@@ -12,7 +12,7 @@
 // One GEMM core serves all four uses; operands are always K-major (transposed copies of W and hidden
 // are made once per call), only the epilogue differs.  One persistent CTA per SM:
 //   warp 0      TMA producer: 64-wide K slabs of A (128 rows) and of B (256 rows), 128B-swizzled, into
-//               a 4-stage shared-memory ring (no multicast)
+//               a 4-stage shared-memory ring (every CTA fetches its own operands)
 //   warp 1      one thread issues tcgen05.mma (M=128, N=256, K=16 x 4 per slab) into one of two
 //               256-column TMEM accumulators; tcgen05.commit releases smem stages / publishes the tile
 //   warps 2-5   epilogue: each thread owns one row of the tile and reads it 32 columns at a time with
@@ -279,7 +279,8 @@ lm_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 // (128 rows), the leader's MMA thread issues tcgen05.mma.cta_group::2 (M = 256) which reads both halves of B
 // from the two CTAs' shared memory and writes each CTA's 128 rows into that CTA's tensor memory.  Per SM
 // and K slab this is 32 KB of operands instead of 48 KB for the same flops.  TMA loads signal the
-// leader's `full` barrier (no multicast); tcgen05.commit is multicast to both CTAs' barriers; both
+// leader's `full` barrier (every CTA fetches its own operands); the tcgen05.commit arrivals go to both CTAs'
+// barriers; both
 // epilogues report to the leader's `acc_empty`.
 constexpr int kStages2 = 6;
 constexpr int kHalfBN = kBN / 2;
