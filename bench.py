@@ -41,7 +41,7 @@ WORKLOAD_TEXT = WORKLOAD + ": P=32 G=8, response 64-1024 tokens, V=151936 bf16 l
 # grows in proportion to the rows, so a launch over T rows moves T times the per-row figure.  The record
 # is tied to the kernel sources it was taken from: once they change, `traffic` is reported as null.
 TRAFFIC_CAPTURE = {"rows": 8192, "dram_bytes": 2489454000 + 2432057000,
-                   "source_sha256": "8bb2c583a518e9187152d702cc663e4f083fa44ef177016e38109b659c93700e"}
+                   "source_sha256": "bde4c42c69aab370d369790c1ee54f1c14658247a03e3259183b0b288407a890"}
 
 
 def captured_traffic_per_row():
