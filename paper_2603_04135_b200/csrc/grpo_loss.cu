@@ -109,28 +109,55 @@ __global__ void __launch_bounds__(kRowThreads) grpo_loss_rows_kernel(const LossA
 }
 
 // ---- final reduction: fixed order, binary64 ------------------------------------------------------
-constexpr int kReduceThreads = 1024;
+// Two launches.  The first cuts the rows into kReduceBlocks contiguous ranges, one block each (one
+// block alone is held to a single SM's load bandwidth); the second adds the per-block partial sums.
+// Ranges, strides and both trees depend on T only, so the result is the same on every run.
+constexpr int kReduceThreads = 256;
 
-__global__ void __launch_bounds__(kReduceThreads)
-loss_reduce_kernel(const RowTerms* __restrict__ terms, long long T_max, const int32_t* __restrict__ n_tokens_dev,
-                   float* __restrict__ loss_out) {
-    __shared__ double sh[4][kReduceThreads];
-    const long long T = n_tokens_dev ? min((long long)*n_tokens_dev, T_max) : T_max;
-    double acc[4] = {0.0, 0.0, 0.0, 0.0};
-    for (long long t = threadIdx.x; t < T; t += kReduceThreads) {
-        const RowTerms x = terms[t];
-        acc[0] += x.loss; acc[1] += x.pg; acc[2] += x.kl; acc[3] += x.clipped;
-    }
+__device__ __forceinline__ void block_tree_sum4(double (&sh)[4][kReduceThreads], double (&acc)[4], int n) {
 #pragma unroll
     for (int k = 0; k < 4; ++k) sh[k][threadIdx.x] = acc[k];
     __syncthreads();
-    for (int half = kReduceThreads / 2; half > 0; half >>= 1) {
-        if (threadIdx.x < half) {
+    for (int half = n / 2; half > 0; half >>= 1) {
+        if ((int)threadIdx.x < half) {
 #pragma unroll
             for (int k = 0; k < 4; ++k) sh[k][threadIdx.x] += sh[k][threadIdx.x + half];
         }
         __syncthreads();
     }
+}
+
+__global__ void __launch_bounds__(kReduceThreads)
+loss_partial_kernel(const RowTerms* __restrict__ terms, long long T_max, const int32_t* __restrict__ n_tokens_dev,
+                    RowTerms* __restrict__ partials) {
+    __shared__ double sh[4][kReduceThreads];
+    const long long T = n_tokens_dev ? min((long long)*n_tokens_dev, T_max) : T_max;
+    const long long per = (T + kReduceBlocks - 1) / kReduceBlocks;
+    const long long lo = min(T, per * blockIdx.x), hi = min(T, lo + per);
+    double acc[4] = {0.0, 0.0, 0.0, 0.0};
+    for (long long t = lo + threadIdx.x; t < hi; t += kReduceThreads) {
+        const RowTerms x = terms[t];
+        acc[0] += x.loss; acc[1] += x.pg; acc[2] += x.kl; acc[3] += x.clipped;
+    }
+    block_tree_sum4(sh, acc, kReduceThreads);
+    if (threadIdx.x == 0) {
+        RowTerms r; r.loss = sh[0][0]; r.pg = sh[1][0]; r.kl = sh[2][0]; r.clipped = sh[3][0];
+        partials[blockIdx.x] = r;
+    }
+}
+
+__global__ void __launch_bounds__(kReduceThreads)
+loss_final_kernel(const RowTerms* __restrict__ partials, long long T_max, const int32_t* __restrict__ n_tokens_dev,
+                  float* __restrict__ loss_out) {
+    static_assert(kReduceBlocks <= kReduceThreads && (kReduceBlocks & (kReduceBlocks - 1)) == 0, "one partial per thread");
+    __shared__ double sh[4][kReduceThreads];
+    const long long T = n_tokens_dev ? min((long long)*n_tokens_dev, T_max) : T_max;
+    double acc[4] = {0.0, 0.0, 0.0, 0.0};
+    if (threadIdx.x < kReduceBlocks) {
+        const RowTerms x = partials[threadIdx.x];
+        acc[0] = x.loss; acc[1] = x.pg; acc[2] = x.kl; acc[3] = x.clipped;
+    }
+    block_tree_sum4(sh, acc, kReduceThreads);
     if (threadIdx.x == 0) {
         loss_out[0] = (float)sh[0][0];
         loss_out[1] = (float)sh[1][0];
@@ -163,7 +190,10 @@ int launch_rows_general(const LossArgs& a, cudaStream_t s) {
 }
 
 int launch_loss_reduce(const LossArgs& a, float* loss_out, cudaStream_t s) {
-    loss_reduce_kernel<<<1, kReduceThreads, 0, s>>>(a.terms, a.T_max, a.n_tokens_dev, loss_out);
+    RowTerms* partials = loss_partials(a.terms, a.T_max);
+    loss_partial_kernel<<<kReduceBlocks, kReduceThreads, 0, s>>>(a.terms, a.T_max, a.n_tokens_dev, partials);
+    DPPO_CHECK_LAUNCH("grpo_loss partial sums launch");
+    loss_final_kernel<<<1, kReduceThreads, 0, s>>>(partials, a.T_max, a.n_tokens_dev, loss_out);
     DPPO_CHECK_LAUNCH("grpo_loss reduce launch");
     return DPPO_OK;
 }
@@ -172,8 +202,7 @@ int launch_loss_reduce(const LossArgs& a, float* loss_out, cudaStream_t s) {
 
 extern "C" size_t dppo_grpo_loss_workspace_bytes(const dppo_loss_params* p) {
     if (!p || p->T_max < 0) return 0;
-    const size_t rows = (size_t)(p->T_max > 0 ? p->T_max : 1);
-    return (rows * sizeof(dppo::RowTerms) + 255) & ~(size_t)255;
+    return dppo::loss_terms_bytes(p->T_max);
 }
 
 extern "C" int dppo_grpo_loss_fwd_bwd(const dppo_loss_params* p, const void* logits, const int32_t* target,

@@ -11,6 +11,17 @@ struct RowTerms {            // one per token row, in the caller's workspace
     double clipped;          // 1 if the clipped branch was strictly smaller
 };
 
+// The per-row terms are followed, in the same workspace, by the partial sums of the final reduction.
+constexpr int kReduceBlocks = 128;
+inline size_t loss_rows_bytes(long long T_max) {
+    const size_t rows = (size_t)(T_max > 0 ? T_max : 1);
+    return (rows * sizeof(RowTerms) + 255) & ~(size_t)255;
+}
+inline size_t loss_terms_bytes(long long T_max) { return loss_rows_bytes(T_max) + kReduceBlocks * sizeof(RowTerms); }
+inline RowTerms* loss_partials(RowTerms* terms, long long T_max) {
+    return (RowTerms*)((char*)terms + loss_rows_bytes(T_max));
+}
+
 struct RowScalars {          // what pass 2 needs from the scalar stage
     float lse2_hi, lse2_lo;  // base-2 log-sum-exp of z*scale2, split hi + lo
     float g_over_tau;        // dloss/dlogp / temperature

@@ -762,7 +762,7 @@ static LmWorkspace lm_layout(const dppo_lmhead_params* p, bool backward) {
     w.ld_t = round_up(T, 8);
     w.ld_tc = kChunkTokens;
     size_t off = 0;
-    w.terms = off; off += al((size_t)T * sizeof(RowTerms));
+    w.terms = off; off += al(loss_terms_bytes(T));
     w.info = off;  off += al((size_t)T * sizeof(RowInfo));
     w.wt = w.ht = w.d = w.dt = off;
     if (backward) {
