@@ -1,16 +1,16 @@
 // Fused LM-head + GRPO loss on the 5th-generation tensor cores.
 //
-// Forward: the logits z = hidden W^T are produced tile by tile (tcgen05.mma, accumulators in tensor
-// memory) and consumed on the spot — the row-wise log-sum-exp and the sampled token's logit are folded
-// in as each 128 x 256 tile leaves TMEM, so the [T x V] logits never exist in HBM (Eq. 1's
-// pi_theta(o_t | ...) is a log-softmax of exactly these).
+// The call walks over the tokens in chunks.  Per chunk:
+//   logits    z = hidden W^T, tile by tile (tcgen05.mma, accumulators in tensor memory).  As each 128 x 256
+//             tile leaves TMEM its per-row (max, sum of exponentials) and the sampled token's logit are kept;
+//             a backward pass also keeps the chunk's f32 logits in a bounded scratch (the [T x V] logits of
+//             the whole batch never exist; Eq. 1's pi_theta(o_t | ...) is a log-softmax of exactly these)
+//   rows      one warp per token joins the tile partials into the log-sum-exp and runs the loss's scalar stage
+//   dlogits   D = g (onehot - softmax)/tau of the chunk from the stored logits, as bf16, both ways round
+//   dhidden = D W and dW += D^T hidden: two more runs of the same GEMM core over the chunk
 //
-// Backward: dlogits D = g (onehot - softmax)/tau is recomputed from the same GEMM, one chunk of tokens at
-// a time, into a bounded bf16 scratch (never the full [T x V]); dhidden = D W and dW = D^T hidden are
-// two more runs of the same GEMM core over that chunk.
-//
-// One GEMM core serves all four uses; operands are always K-major (transposed copies of W and hidden
-// are made once per call), only the epilogue differs.  One persistent CTA per SM:
+// One GEMM core serves all three contractions; operands are always K-major (transposed copies of W and
+// hidden are made once per call), only the epilogue differs.  One persistent CTA per SM:
 //   warp 0      TMA producer: 64-wide K slabs of A (128 rows) and of B (256 rows), 128B-swizzled, into
 //               a 4-stage shared-memory ring (every CTA fetches its own operands)
 //   warp 1      one thread issues tcgen05.mma (M=128, N=256, K=16 x 4 per slab) into one of two
@@ -105,23 +105,15 @@ __device__ __forceinline__ uint64_t lm_smem_desc(uint32_t smem_addr) {
 // Instruction descriptor of kind::f16: D = f32, A = B = bf16, both K-major, N = 256, M = 128.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
 
-// What a launch of the GEMM core covers.  Tile j of a CTA is
-//   row sweep : m = blockIdx.x + (j / n_ntiles) * gridDim.x, n = j % n_ntiles   (a row block keeps its CTA)
-//   flat      : id = blockIdx.x + j * gridDim.x; m_fast ? (m = id % n_mtiles, n = id / n_mtiles)
-//                                                        : (m = id / n_ntiles, n = id % n_ntiles)
+// What a launch of the GEMM core covers.  Tile j of a CTA is id = blockIdx.x + j * gridDim.x with
+//   m_fast ? (m = id % n_mtiles, n = id / n_mtiles) : (m = id / n_ntiles, n = id % n_ntiles)
 struct GemmShape {
     int n_mtiles, n_ntiles, n_ksteps;
     int a_row0;                          // row offset added to A's TMA coordinate
     int m_fast;
 };
 
-template <bool kRowSweep>
 __device__ __forceinline__ bool tile_of(const GemmShape& gs, uint32_t j, int& m, int& n) {
-    if (kRowSweep) {
-        m = blockIdx.x + (int)(j / (uint32_t)gs.n_ntiles) * gridDim.x;
-        n = (int)(j % (uint32_t)gs.n_ntiles);
-        return m < gs.n_mtiles;
-    }
     const long long id = (long long)blockIdx.x + (long long)j * gridDim.x;
     if (id >= (long long)gs.n_mtiles * gs.n_ntiles) return false;
     if (gs.m_fast) { m = (int)(id % gs.n_mtiles); n = (int)(id / gs.n_mtiles); }
@@ -130,11 +122,11 @@ __device__ __forceinline__ bool tile_of(const GemmShape& gs, uint32_t j, int& m,
 }
 
 // ---- the GEMM core --------------------------------------------------------------------------------
-// Epi (one copy per epilogue thread = per tile row):
-//   void row_begin(int m, int row)                       row sweep: at n == 0; flat: every tile
+// Epi (one copy per epilogue thread = per tile row), called for every tile:
+//   void row_begin(int m, int n, int row)
 //   void chunk(int m, int n, int row, int ch, uint32_t (&v)[32])   32 accumulator columns (f32 bits)
-//   void row_end(int m, int row)                         row sweep: after the last n; flat: every tile
-template <class Epi, bool kRowSweep>
+//   void row_end(int m, int n, int row)
+template <class Epi>
 __global__ void __launch_bounds__(kLmThreads, 1)
 lm_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const GemmShape gs, const Epi epi_args, int32_t* status) {
@@ -172,7 +164,7 @@ lm_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (lane == 0) {
             uint32_t it = 0;                                             // slab counter over the CTA's lifetime
             int m, n;
-            for (uint32_t j = 0; tile_of<kRowSweep>(gs, j, m, n) && !*abort_flag; ++j) {
+            for (uint32_t j = 0; tile_of(gs, j, m, n) && !*abort_flag; ++j) {
                 for (int k = 0; k < gs.n_ksteps; ++k, ++it) {
                     const uint32_t s = it % kStages, use = it / kStages;
                     if (use > 0 && !lm_wait(lm_smem_u32(&sh.empty[s]), (use - 1) & 1, abort_flag)) break;
@@ -200,7 +192,7 @@ lm_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (lane == 0) {
             uint32_t it = 0;
             int m, n;
-            for (uint32_t j = 0; tile_of<kRowSweep>(gs, j, m, n) && !*abort_flag; ++j) {
+            for (uint32_t j = 0; tile_of(gs, j, m, n) && !*abort_flag; ++j) {
                 const uint32_t b = j & 1, use_b = j >> 1;
                 if (use_b > 0 && !lm_wait(lm_smem_u32(&sh.acc_empty[b]), (use_b - 1) & 1, abort_flag)) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -236,9 +228,9 @@ lm_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int row = q * 32 + lane;
         Epi epi = epi_args;                                              // per-thread copy: its state lives in registers
         int m, n;
-        for (uint32_t j = 0; tile_of<kRowSweep>(gs, j, m, n); ++j) {
+        for (uint32_t j = 0; tile_of(gs, j, m, n); ++j) {
             const uint32_t b = j & 1, use_b = j >> 1;
-            if (!kRowSweep || n == 0) epi.row_begin(m, row);
+            epi.row_begin(m, n, row);
             // warp-uniform outcome: the tcgen05.ld below must be executed by all 32 lanes together
             if (!__all_sync(0xffffffffu, lm_wait(lm_smem_u32(&sh.acc_full[b]), use_b & 1, abort_flag))) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -260,7 +252,7 @@ lm_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) lm_arrive(lm_smem_u32(&sh.acc_empty[b]));
-            if (!kRowSweep || n == gs.n_ntiles - 1) epi.row_end(m, row);
+            epi.row_end(m, n, row);
         }
     }
 
@@ -298,15 +290,9 @@ struct LmShared2 {
     int abort;
 };
 
-template <bool kRowSweep>
 __device__ __forceinline__ bool pair_tile_of(const GemmShape& gs, uint32_t j, int& m2, int& n) {
     const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
     const int n_m2 = (gs.n_mtiles + 1) >> 1;
-    if (kRowSweep) {
-        m2 = pair + (int)(j / (uint32_t)gs.n_ntiles) * npairs;
-        n = (int)(j % (uint32_t)gs.n_ntiles);
-        return m2 < n_m2;
-    }
     const long long id = (long long)pair + (long long)j * npairs;
     if (id >= (long long)n_m2 * gs.n_ntiles) return false;
     if (gs.m_fast) { m2 = (int)(id % n_m2); n = (int)(id / n_m2); }
@@ -319,7 +305,7 @@ __device__ __forceinline__ void lm_cluster_sync() {
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
-template <class Epi, bool kRowSweep>
+template <class Epi>
 __global__ void __launch_bounds__(kLmThreads, 1)
 lm_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const GemmShape gs, const Epi epi_args, int32_t* status) {
@@ -361,7 +347,7 @@ lm_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         if (lane == 0) {
             uint32_t it = 0;
             int m2, n;
-            for (uint32_t j = 0; pair_tile_of<kRowSweep>(gs, j, m2, n) && !*abort_flag; ++j) {
+            for (uint32_t j = 0; pair_tile_of(gs, j, m2, n) && !*abort_flag; ++j) {
                 const int m = 2 * m2 + (int)rank;
                 for (int k = 0; k < gs.n_ksteps; ++k, ++it) {
                     const uint32_t s = it % kStages2, use = it / kStages2;
@@ -383,7 +369,7 @@ lm_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         if (lane == 0 && leader) {
             uint32_t it = 0;
             int m2, n;
-            for (uint32_t j = 0; pair_tile_of<kRowSweep>(gs, j, m2, n) && !*abort_flag; ++j) {
+            for (uint32_t j = 0; pair_tile_of(gs, j, m2, n) && !*abort_flag; ++j) {
                 const uint32_t b = j & 1, use_b = j >> 1;
                 if (use_b > 0 && !lm_wait(lm_smem_u32(&sh.acc_empty[b]), (use_b - 1) & 1, abort_flag)) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -419,10 +405,10 @@ lm_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         const int row = q * 32 + lane;
         Epi epi = epi_args;
         int m2, n;
-        for (uint32_t j = 0; pair_tile_of<kRowSweep>(gs, j, m2, n); ++j) {
+        for (uint32_t j = 0; pair_tile_of(gs, j, m2, n); ++j) {
             const int m = 2 * m2 + (int)rank;
             const uint32_t b = j & 1, use_b = j >> 1;
-            if (!kRowSweep || n == 0) epi.row_begin(m, row);
+            epi.row_begin(m, n, row);
             if (!__all_sync(0xffffffffu, lm_wait(lm_smem_u32(&sh.acc_full[b]), use_b & 1, abort_flag))) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + b * kBN;
@@ -444,7 +430,7 @@ lm_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             __syncwarp();
             if (lane == 0)                                               // the leader's MMA thread waits for all 8 warps
                 asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" :: "r"(lm_smem_u32(&sh.acc_empty[b]) & kPeerMask) : "memory");
-            if (!kRowSweep || n == gs.n_ntiles - 1) epi.row_end(m, row);
+            epi.row_end(m, n, row);
         }
     }
 
@@ -466,30 +452,47 @@ struct RowInfo {             // what the backward needs from the forward, per to
     int y;                   // target, -1 if the row is invalid
 };
 
-// Forward: online (max, sum 2^x) over the vocabulary, z[y], then the loss's scalar stage.
-struct EpiLse {
-    LossArgs a;
-    RowInfo* info;           // nullable
+// Forward, one chunk of tokens: each 128 x 256 logits tile leaves behind, per token row, the tile's
+// (max, sum 2^(x - max)) of x = z * scale2, the sampled token's logit if it lies in the tile, and (for a
+// backward pass) the f32 logits themselves in a chunk-sized scratch.  The tiles of a row are combined
+// by lm_rows_kernel.
+struct EpiPartial {
+    float2* part;            // [chunk tokens x n_ntiles]
+    float* zy_out;           // [chunk tokens]
+    float* Z;                // [chunk tokens x ldz] f32, nullable
+    const int32_t* target;
+    const int32_t* n_tokens_dev;
+    long long T_max, t0, tc, ldz;
+    int V, n_ntiles;
+    float c;
     // per-thread state
-    RowInputs in;
-    long long T;
     float m2, s, zy;
     int y;
-    bool live;
-    __device__ __forceinline__ void row_begin(int m, int row) {
-        T = a.n_tokens_dev ? min((long long)*a.n_tokens_dev, a.T_max) : a.T_max;
-        const long long t = (long long)m * kBM + row;
-        live = t < T;
-        in.state = 0; in.y = -1;
-        if (live) row_gather(a, t, in, false);
-        y = (live && in.state == 0) ? in.y : -1;
-        m2 = -INFINITY; s = 0.0f; zy = 0.0f;
+    bool live, hit;
+    __device__ __forceinline__ void row_begin(int m, int, int row) {
+        const long long T = n_tokens_dev ? min((long long)*n_tokens_dev, T_max) : T_max;
+        const long long r = (long long)m * kBM + row;
+        live = r < tc && t0 + r < T;
+        y = live ? target[t0 + r] : -1;
+        m2 = -INFINITY; s = 0.0f; zy = 0.0f; hit = false;
     }
-    __device__ __forceinline__ void chunk(int, int n, int, int ch, uint32_t (&v)[32]) {
+    __device__ __forceinline__ void chunk(int m, int n, int row, int ch, uint32_t (&v)[32]) {
         const int col0 = n * kBN + ch * 32;
-        const int valid = a.V - col0;                                // columns of this chunk inside the vocabulary
-        const float c = a.scale2;
+        const int valid = V - col0;                                  // columns of this chunk inside the vocabulary
+        if (!live || valid <= 0) return;
+        if (Z) {
+            float* dst = Z + ((long long)m * kBM + row) * ldz + col0;
+            if (valid >= 32) {                                       // ldz is a multiple of 8: 16-byte stores
+                uint4* d4 = reinterpret_cast<uint4*>(dst);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) d4[j] = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) if (j < valid) dst[j] = __uint_as_float(v[j]);
+            }
+        }
         const int yrel = y - col0;                                   // selects, not an indexed read: v stays in registers
+        hit = hit || (yrel >= 0 && yrel < 32);
         float cm = -INFINITY;
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
@@ -508,87 +511,131 @@ struct EpiLse {
         }
         s += acc0 + acc1;
     }
-    __device__ __forceinline__ void row_end(int m, int row) {
-        const long long t = (long long)m * kBM + row;
-        if (!live) {
-            if (info && t < a.T_max) { RowInfo z; z.lse2_hi = 0.0f; z.lse2_lo = 0.0f; z.g_over_tau = 0.0f; z.y = -1; info[t] = z; }
-            return;
-        }
-        in.zy = (double)zy / a.temperature;
-        const RowScalars rs = row_finish(a, t, in, m2, s, true);
-        if (info) {
-            RowInfo ri;
-            ri.lse2_hi = rs.lse2_hi; ri.lse2_lo = rs.lse2_lo;
-            ri.g_over_tau = rs.valid ? rs.g_over_tau : 0.0f;
-            ri.y = rs.valid ? in.y : -1;
-            info[t] = ri;
-        }
+    __device__ __forceinline__ void row_end(int m, int n, int row) {
+        if (!live) return;
+        const long long r = (long long)m * kBM + row;
+        part[r * n_ntiles + n] = make_float2(m2, s);
+        if (hit) zy_out[r] = zy;
     }
 };
 
-// Backward, step 1: dlogits of a chunk of tokens, written as bf16 both ways round:
+// One warp per token of the chunk: the row's tile partials -> base-2 log-sum-exp, then the loss's scalar
+// stage (lane 0) -> per-row loss terms, logp, lse and what the backward needs.
+constexpr int kRowsWarps = 8;
+
+__global__ void __launch_bounds__(kRowsWarps * 32)
+lm_rows_kernel(const LossArgs a, const float2* __restrict__ part, const float* __restrict__ zy,
+               RowInfo* __restrict__ info, long long t0, long long tc, int n_ntiles) {
+    const long long r = (long long)blockIdx.x * kRowsWarps + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (r >= tc) return;
+    const long long t = t0 + r;
+    const long long T = a.n_tokens_dev ? min((long long)*a.n_tokens_dev, a.T_max) : a.T_max;
+    if (t >= T) {                                                    // no token here: the backward sees g = 0
+        if (lane == 0) { RowInfo z; z.lse2_hi = 0.0f; z.lse2_lo = 0.0f; z.g_over_tau = 0.0f; z.y = -1; info[t] = z; }
+        return;
+    }
+    float M = -INFINITY, S = 0.0f;
+    for (int i = lane; i < n_ntiles; i += 32) {
+        const float2 q = part[r * n_ntiles + i];                     // every tile holds a vocabulary column: q.x is finite
+        const float Mn = fmaxf(M, q.x);
+        S = (M == -INFINITY ? 0.0f : S * lm_ex2(M - Mn)) + q.y * lm_ex2(q.x - Mn);
+        M = Mn;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float Mo = __shfl_xor_sync(0xffffffffu, M, o), So = __shfl_xor_sync(0xffffffffu, S, o);
+        const float Mn = fmaxf(M, Mo);
+        S = (M == -INFINITY ? 0.0f : S * lm_ex2(M - Mn)) + (Mo == -INFINITY ? 0.0f : So * lm_ex2(Mo - Mn));
+        M = Mn;
+    }
+    if (lane == 0) {
+        RowInputs in;
+        row_gather(a, t, in, false);
+        if (in.state == 0) in.zy = (double)zy[r] / a.temperature;
+        const RowScalars rs = row_finish(a, t, in, M, S, true);
+        RowInfo ri;
+        ri.lse2_hi = rs.lse2_hi; ri.lse2_lo = rs.lse2_lo;
+        ri.g_over_tau = rs.valid ? rs.g_over_tau : 0.0f;
+        ri.y = rs.valid ? in.y : -1;
+        info[t] = ri;
+    }
+}
+
+// Backward, step 1: dlogits of the chunk from its stored logits, D = g (onehot - softmax) / tau, written
+// as bf16 both ways round:
 //   D  [chunk tokens x ldd]  (row = token)       feeds dhidden = D W
 //   Dt [V x ldt]             (row = vocabulary)  feeds dW = D^T hidden
-// Rows past the true token count get g = 0 from the forward, i.e. zeros.
-struct EpiDlogits {
-    const RowInfo* info;
-    __nv_bfloat16* D;
-    __nv_bfloat16* Dt;
-    long long t0, tc;        // first token of the chunk, tokens in the chunk
-    long long ldd, ldt;
-    int V;
-    float c;
-    RowInfo ri;
-    bool live;
-    __device__ __forceinline__ void row_begin(int m, int row) {
-        const long long r = (long long)m * kBM + row;
-        live = r < tc;
-        if (live) ri = info[t0 + r];
-        else { ri.lse2_hi = 0.0f; ri.lse2_lo = 0.0f; ri.g_over_tau = 0.0f; ri.y = -1; }
-    }
-    __device__ __forceinline__ void chunk(int m, int n, int row, int ch, uint32_t (&v)[32]) {
-        const int col0 = n * kBN + ch * 32;
-        if (col0 >= V || !live) return;
-        const long long r = (long long)m * kBM + row;                // token index inside the chunk
-        const float g = ri.g_over_tau;
+// 64 tokens x 64 vocabulary entries per block, transposed through shared memory so that both copies are
+// written in 128-byte runs.  Rows with g = 0 (no token, bad target) are written as zeros without
+// reading their logits.
+__global__ void __launch_bounds__(256)
+lm_dlogits_kernel(const float* __restrict__ Z, long long ldz, const RowInfo* __restrict__ info, long long t0,
+                  long long tc, int V, float c, __nv_bfloat16* __restrict__ D, long long ldd,
+                  __nv_bfloat16* __restrict__ Dt, long long ldt) {
+    __shared__ __nv_bfloat16 tile[64][64 + 2];                       // [token][vocabulary]; rows of 33 words
+    const long long r0 = (long long)blockIdx.y * 64;
+    const int v0 = blockIdx.x * 64;
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;          // 16 x 16 threads
+    const int col = v0 + 4 * tx;
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            const float p = lm_ex2(fmaf(__uint_as_float(v[j]), c, -ri.lse2_hi) - ri.lse2_lo);
-            float d = -g * p;
-            if (col0 + j == ri.y) d += g;
-            v[j] = __float_as_uint(d);
-        }
-        if (col0 + 32 <= V) {                                        // ldd is a multiple of 8: 16-byte stores
-            uint32_t pk[16];
+    for (int i = 0; i < 4; ++i) {
+        const int rr = ty + 16 * i;
+        const long long r = r0 + rr;
+        float d[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        if (r < tc && col < V) {
+            const RowInfo ri = info[t0 + r];
+            const float g = ri.g_over_tau;
+            if (g != 0.0f) {
+                const float* src = Z + r * ldz + col;
+                float z[4];
+                if (col + 4 <= V) { const float4 q = *reinterpret_cast<const float4*>(src); z[0] = q.x; z[1] = q.y; z[2] = q.z; z[3] = q.w; }
+                else {
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
-                pk[j] = *reinterpret_cast<const uint32_t*>(&b2);
+                    for (int j = 0; j < 4; ++j) z[j] = (col + j < V) ? src[j] : 0.0f;
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float p = lm_ex2(fmaf(z[j], c, -ri.lse2_hi) - ri.lse2_lo);
+                    d[j] = (col + j < V) ? (-g * p + ((col + j == ri.y) ? g : 0.0f)) : 0.0f;
+                }
             }
-            uint4* dst = reinterpret_cast<uint4*>(D + r * ldd + col0);
-            dst[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-            dst[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
-            dst[2] = make_uint4(pk[8], pk[9], pk[10], pk[11]);
-            dst[3] = make_uint4(pk[12], pk[13], pk[14], pk[15]);
-        } else {
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-                if (col0 + j < V) D[r * ldd + col0 + j] = __float2bfloat16_rn(__uint_as_float(v[j]));
         }
-        // transposed copy: for a fixed column the 32 lanes of a warp write 32 consecutive tokens (64 bytes)
+        const __nv_bfloat162 b01 = __floats2bfloat162_rn(d[0], d[1]), b23 = __floats2bfloat162_rn(d[2], d[3]);
+        *reinterpret_cast<__nv_bfloat162*>(&tile[rr][4 * tx]) = b01;
+        *reinterpret_cast<__nv_bfloat162*>(&tile[rr][4 * tx + 2]) = b23;
+        if (r < tc && col < V) {
+            __nv_bfloat16* dst = D + r * ldd + col;
+            if (col + 4 <= V) {                                      // ldd is a multiple of 8, col of 4: 8-byte stores
+                uint2 pk;
+                pk.x = *reinterpret_cast<const uint32_t*>(&b01); pk.y = *reinterpret_cast<const uint32_t*>(&b23);
+                *reinterpret_cast<uint2*>(dst) = pk;
+            } else {
 #pragma unroll
-        for (int j = 0; j < 32; ++j)
-            if (col0 + j < V) Dt[(long long)(col0 + j) * ldt + r] = __float2bfloat16_rn(__uint_as_float(v[j]));
+                for (int j = 0; j < 4; ++j) if (col + j < V) dst[j] = __float2bfloat16_rn(d[j]);
+            }
+        }
     }
-    __device__ __forceinline__ void row_end(int, int) {}
-};
+    __syncthreads();
+    // transposed copy: a warp writes one vocabulary row's 64 tokens (128 bytes), two per lane
+    const int lane = threadIdx.x & 31, wp = threadIdx.x >> 5;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int vv = wp + 8 * i;
+        const long long r = r0 + 2 * lane;
+        if (v0 + vv >= V || r >= tc) continue;
+        __nv_bfloat16* dst = Dt + (long long)(v0 + vv) * ldt + r;     // ldt and r are even: 4-byte stores
+        if (r + 2 <= tc) *reinterpret_cast<__nv_bfloat162*>(dst) = __halves2bfloat162(tile[2 * lane][vv], tile[2 * lane + 1][vv]);
+        else dst[0] = tile[2 * lane][vv];
+    }
+}
 
 // C[rows x ldc] = acc as bf16 (dhidden).
 struct EpiStoreBf16 {
     __nv_bfloat16* C;
     long long ldc, row0, rows;   // output row of tile row 0; rows that exist in C
     int cols;
-    __device__ __forceinline__ void row_begin(int, int) {}
+    __device__ __forceinline__ void row_begin(int, int, int) {}
     __device__ __forceinline__ void chunk(int m, int n, int row, int ch, uint32_t (&v)[32]) {
         const long long r = row0 + (long long)m * kBM + row;
         const int col0 = n * kBN + ch * 32;
@@ -611,7 +658,7 @@ struct EpiStoreBf16 {
             for (int j = 0; j < 32; ++j) if (col0 + j < cols) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
         }
     }
-    __device__ __forceinline__ void row_end(int, int) {}
+    __device__ __forceinline__ void row_end(int, int, int) {}
 };
 
 // C[rows x ldc] (f32) = or += acc (dW, accumulated over the token chunks).
@@ -619,7 +666,7 @@ struct EpiAccumF32 {
     float* C;
     long long ldc, rows;
     int cols, accumulate;
-    __device__ __forceinline__ void row_begin(int, int) {}
+    __device__ __forceinline__ void row_begin(int, int, int) {}
     __device__ __forceinline__ void chunk(int m, int n, int row, int ch, uint32_t (&v)[32]) {
         const long long r = (long long)m * kBM + row;
         const int col0 = n * kBN + ch * 32;
@@ -640,7 +687,7 @@ struct EpiAccumF32 {
                 if (col0 + j < cols) dst[j] = (accumulate ? dst[j] : 0.0f) + __uint_as_float(v[j]);
         }
     }
-    __device__ __forceinline__ void row_end(int, int) {}
+    __device__ __forceinline__ void row_end(int, int, int) {}
 };
 
 // out[c x ldo] = in[r x ldi]^T for bf16, 64 x 64 tiles through shared memory; columns r..ldo-1 of out are
@@ -697,13 +744,13 @@ static int make_map(CUtensorMap* map, const void* base, long long rows, long lon
 
 constexpr size_t kLmDynSmem = (size_t)kStages * kStageBytes + 1024;
 
-template <class Epi, bool kRowSweep>
+template <class Epi>
 static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const GemmShape& gs, const Epi& epi,
                        int32_t* status, cudaStream_t s, const char* what) {
-    auto kernel = lm_gemm_kernel<Epi, kRowSweep>;
+    auto kernel = lm_gemm_kernel<Epi>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLmDynSmem);
     if (e != cudaSuccess) return cuda_fail(e, "lmhead: shared memory attribute");
-    const long long work = kRowSweep ? gs.n_mtiles : (long long)gs.n_mtiles * gs.n_ntiles;
+    const long long work = (long long)gs.n_mtiles * gs.n_ntiles;
     const int grid = (int)(work < sm_count() ? work : sm_count());
     if (grid < 1) return DPPO_OK;
     kernel<<<grid, kLmThreads, kLmDynSmem, s>>>(ma, mb, gs, epi, status);
@@ -715,14 +762,14 @@ static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const GemmS
 constexpr size_t kLmDynSmem2 = (size_t)kStages2 * kStageBytes2 + 1024;
 
 // CTA-pair version: `mb_half` is B's tensor map with 128-row boxes.
-template <class Epi, bool kRowSweep>
+template <class Epi>
 static int launch_gemm2(const CUtensorMap& ma, const CUtensorMap& mb_half, const GemmShape& gs, const Epi& epi,
                         int32_t* status, cudaStream_t s, const char* what) {
-    auto kernel = lm_gemm2_kernel<Epi, kRowSweep>;
+    auto kernel = lm_gemm2_kernel<Epi>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLmDynSmem2);
     if (e != cudaSuccess) return cuda_fail(e, "lmhead: shared memory attribute");
     const long long n_m2 = (gs.n_mtiles + 1) / 2;
-    const long long work = kRowSweep ? n_m2 : n_m2 * gs.n_ntiles;
+    const long long work = n_m2 * gs.n_ntiles;
     const long long max_pairs = sm_count() / 2;
     const int pairs = (int)(work < max_pairs ? work : max_pairs);
     if (pairs < 1) return DPPO_OK;
@@ -740,18 +787,19 @@ static int launch_gemm2(const CUtensorMap& ma, const CUtensorMap& mb_half, const
     return DPPO_OK;
 }
 
-template <class Epi, bool kRowSweep>
+template <class Epi>
 static int run_gemm(bool pair, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mb_half, const GemmShape& gs,
                     const Epi& epi, int32_t* status, cudaStream_t s, const char* what) {
-    return pair ? launch_gemm2<Epi, kRowSweep>(ma, mb_half, gs, epi, status, s, what)
-                : launch_gemm<Epi, kRowSweep>(ma, mb, gs, epi, status, s, what);
+    return pair ? launch_gemm2<Epi>(ma, mb_half, gs, epi, status, s, what)
+                : launch_gemm<Epi>(ma, mb, gs, epi, status, s, what);
 }
 
 static long long round_up(long long x, long long m) { return (x + m - 1) / m * m; }
 
 struct LmWorkspace {
-    size_t terms, info, wt, ht, d, dt, total;    // byte offsets and the total
-    long long ld_v, ld_t, ld_tc;                 // pitches: vocabulary (D, Wt), tokens (ht), chunk tokens (Dt)
+    size_t terms, info, part, zy, wt, ht, z, d, dt, total;   // byte offsets and the total
+    long long ld_v, ld_t, ld_tc;                 // pitches: vocabulary (Z, D, Wt), tokens (ht), chunk tokens (Dt)
+    int n_ntiles;
 };
 
 static LmWorkspace lm_layout(const dppo_lmhead_params* p, bool backward) {
@@ -761,13 +809,17 @@ static LmWorkspace lm_layout(const dppo_lmhead_params* p, bool backward) {
     w.ld_v = round_up(p->loss.V, 8);
     w.ld_t = round_up(T, 8);
     w.ld_tc = kChunkTokens;
+    w.n_ntiles = (p->loss.V + kBN - 1) / kBN;
     size_t off = 0;
     w.terms = off; off += al(loss_terms_bytes(T));
     w.info = off;  off += al((size_t)T * sizeof(RowInfo));
-    w.wt = w.ht = w.d = w.dt = off;
+    w.part = off;  off += al((size_t)kChunkTokens * w.n_ntiles * sizeof(float2));
+    w.zy = off;    off += al((size_t)kChunkTokens * sizeof(float));
+    w.wt = w.ht = w.z = w.d = w.dt = off;
     if (backward) {
         w.wt = off; off += al((size_t)p->H * w.ld_v * 2);
         w.ht = off; off += al((size_t)p->H * w.ld_t * 2);
+        w.z = off;  off += al((size_t)kChunkTokens * w.ld_v * 4);
         w.d = off;  off += al((size_t)kChunkTokens * w.ld_v * 2);
         w.dt = off; off += al((size_t)p->loss.V * w.ld_tc * 2);
     }
@@ -840,69 +892,73 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
         rc = make_map(&map_w_half, W, V, H, H, kHalfBN);
         if (rc != DPPO_OK) return rc;
         RowInfo* info = (RowInfo*)(ws + lay.info);
-
-        // ---- forward: lse, logp, loss terms (and what the backward needs per row)
-        GemmShape gs = {};
-        gs.n_mtiles = (int)((T + kBM - 1) / kBM); gs.n_ntiles = (V + kBN - 1) / kBN; gs.n_ksteps = H / kBK;
-        EpiLse fwd = {};
-        fwd.a = a; fwd.info = backward ? info : nullptr;
-        rc = run_gemm<EpiLse, true>(pair, map_h, map_w, map_w_half, gs, fwd, status, s, "lmhead forward launch");
-        if (rc != DPPO_OK) return rc;
-
+        float2* part = (float2*)(ws + lay.part);
+        float* zy = (float*)(ws + lay.zy);
+        float* Z = backward ? (float*)(ws + lay.z) : nullptr;
+        __nv_bfloat16* Wt = (__nv_bfloat16*)(ws + lay.wt);
+        __nv_bfloat16* ht = (__nv_bfloat16*)(ws + lay.ht);
+        __nv_bfloat16* D = (__nv_bfloat16*)(ws + lay.d);
+        __nv_bfloat16* Dt = (__nv_bfloat16*)(ws + lay.dt);
+        alignas(64) CUtensorMap map_wt, map_wt_half;
         if (backward) {
-            __nv_bfloat16* Wt = (__nv_bfloat16*)(ws + lay.wt);
-            __nv_bfloat16* ht = (__nv_bfloat16*)(ws + lay.ht);
-            __nv_bfloat16* D = (__nv_bfloat16*)(ws + lay.d);
-            __nv_bfloat16* Dt = (__nv_bfloat16*)(ws + lay.dt);
             // K-major copies of the two operands that are contracted over their row index
             transpose_bf16_kernel<<<dim3((H + 63) / 64, (V + 63) / 64), 256, 0, s>>>(
                 (const __nv_bfloat16*)W, V, H, H, Wt, lay.ld_v);
             transpose_bf16_kernel<<<dim3((H + 63) / 64, (unsigned)((T + 63) / 64)), 256, 0, s>>>(
                 (const __nv_bfloat16*)hidden, T, H, H, ht, lay.ld_t);
             DPPO_CHECK_LAUNCH("lmhead transpose launch");
-            alignas(64) CUtensorMap map_wt, map_wt_half;
             rc = make_map(&map_wt, Wt, H, V, lay.ld_v, kBN);
             if (rc != DPPO_OK) return rc;
             rc = make_map(&map_wt_half, Wt, H, V, lay.ld_v, kHalfBN);
             if (rc != DPPO_OK) return rc;
+        }
 
-            for (long long t0 = 0, c = 0; t0 < T; t0 += kChunkTokens, ++c) {
-                const long long tc = (T - t0) < kChunkTokens ? (T - t0) : kChunkTokens;     // tokens in this chunk
-                // (1) dlogits of the chunk: D [tc x V] and Dt [V x tc]
-                GemmShape g1 = {};
-                g1.n_mtiles = (int)((tc + kBM - 1) / kBM); g1.n_ntiles = (V + kBN - 1) / kBN; g1.n_ksteps = H / kBK;
-                g1.a_row0 = (int)t0; g1.m_fast = 1;                                        // neighbours share the W tile
-                EpiDlogits e1 = {};
-                e1.info = info; e1.D = D; e1.Dt = Dt; e1.t0 = t0; e1.tc = tc; e1.ldd = lay.ld_v; e1.ldt = lay.ld_tc;
-                e1.V = V; e1.c = a.scale2;
-                rc = run_gemm<EpiDlogits, false>(pair, map_h, map_w, map_w_half, g1, e1, status, s, "lmhead dlogits launch");
-                if (rc != DPPO_OK) return rc;
-                // (2) dhidden[t0 : t0+tc, :] = D Wt^T          (M = tokens, N = H, K = V)
-                alignas(64) CUtensorMap map_d, map_dt, map_ht_c, map_ht_c_half;
-                rc = make_map(&map_d, D, tc, V, lay.ld_v, kBM);
-                if (rc != DPPO_OK) return rc;
-                GemmShape g2 = {};
-                g2.n_mtiles = (int)((tc + kBM - 1) / kBM); g2.n_ntiles = (H + kBN - 1) / kBN; g2.n_ksteps = (V + kBK - 1) / kBK;
-                EpiStoreBf16 e2 = {};
-                e2.C = (__nv_bfloat16*)dhidden; e2.ldc = H; e2.row0 = t0; e2.rows = T; e2.cols = H;
-                rc = run_gemm<EpiStoreBf16, false>(pair, map_d, map_wt, map_wt_half, g2, e2, status, s, "lmhead dhidden launch");
-                if (rc != DPPO_OK) return rc;
-                // (3) dW (+)= Dt ht[:, t0 : t0+tc]^T            (M = V, N = H, K = tokens of the chunk);
-                //     the K range must stop at the chunk, so ht gets a map of its own based at column t0
-                //     (t0 is a multiple of 9472 = 8 * 1184: the base stays 16-byte aligned)
-                rc = make_map(&map_dt, Dt, V, tc, lay.ld_tc, kBM);
-                if (rc != DPPO_OK) return rc;
-                rc = make_map(&map_ht_c, ht + t0, H, tc, lay.ld_t, kBN);
-                if (rc != DPPO_OK) return rc;
-                rc = make_map(&map_ht_c_half, ht + t0, H, tc, lay.ld_t, kHalfBN);
-                if (rc != DPPO_OK) return rc;
-                GemmShape g3 = {};
-                g3.n_mtiles = (V + kBM - 1) / kBM; g3.n_ntiles = (H + kBN - 1) / kBN; g3.n_ksteps = (int)((tc + kBK - 1) / kBK);
-                EpiAccumF32 e3 = {};
-                e3.C = (float*)dW; e3.ldc = H; e3.rows = V; e3.cols = H; e3.accumulate = c > 0 ? 1 : 0;
-                rc = run_gemm<EpiAccumF32, false>(pair, map_dt, map_ht_c, map_ht_c_half, g3, e3, status, s, "lmhead dW launch");
-                if (rc != DPPO_OK) return rc;
-            }
+        for (long long t0 = 0, c = 0; t0 < T; t0 += kChunkTokens, ++c) {
+            const long long tc = (T - t0) < kChunkTokens ? (T - t0) : kChunkTokens;     // tokens in this chunk
+            // (1) logits of the chunk, tile by tile: per-tile (max, sum) of every row, z[y], and (backward) the
+            //     f32 logits into Z [tc x V]
+            GemmShape g1 = {};
+            g1.n_mtiles = (int)((tc + kBM - 1) / kBM); g1.n_ntiles = lay.n_ntiles; g1.n_ksteps = H / kBK;
+            g1.a_row0 = (int)t0; g1.m_fast = 1;                                        // neighbours share the W tile
+            EpiPartial e1 = {};
+            e1.part = part; e1.zy_out = zy; e1.Z = Z; e1.target = target; e1.n_tokens_dev = n_tokens_dev;
+            e1.T_max = T; e1.t0 = t0; e1.tc = tc; e1.ldz = lay.ld_v; e1.V = V; e1.n_ntiles = lay.n_ntiles; e1.c = a.scale2;
+            rc = run_gemm<EpiPartial>(pair, map_h, map_w, map_w_half, g1, e1, status, s, "lmhead logits launch");
+            if (rc != DPPO_OK) return rc;
+            // (2) rows: log-sum-exp, logp, loss terms, dloss/dlogp
+            lm_rows_kernel<<<(unsigned)((tc + kRowsWarps - 1) / kRowsWarps), kRowsWarps * 32, 0, s>>>(
+                a, part, zy, info, t0, tc, lay.n_ntiles);
+            DPPO_CHECK_LAUNCH("lmhead rows launch");
+            if (!backward) continue;
+            // (3) dlogits of the chunk: D [tc x V] and Dt [V x tc]
+            lm_dlogits_kernel<<<dim3((V + 63) / 64, (unsigned)((tc + 63) / 64)), 256, 0, s>>>(
+                Z, lay.ld_v, info, t0, tc, V, a.scale2, D, lay.ld_v, Dt, lay.ld_tc);
+            DPPO_CHECK_LAUNCH("lmhead dlogits launch");
+            // (4) dhidden[t0 : t0+tc, :] = D Wt^T          (M = tokens, N = H, K = V)
+            alignas(64) CUtensorMap map_d, map_dt, map_ht_c, map_ht_c_half;
+            rc = make_map(&map_d, D, tc, V, lay.ld_v, kBM);
+            if (rc != DPPO_OK) return rc;
+            GemmShape g2 = {};
+            g2.n_mtiles = (int)((tc + kBM - 1) / kBM); g2.n_ntiles = (H + kBN - 1) / kBN; g2.n_ksteps = (V + kBK - 1) / kBK;
+            EpiStoreBf16 e2 = {};
+            e2.C = (__nv_bfloat16*)dhidden; e2.ldc = H; e2.row0 = t0; e2.rows = T; e2.cols = H;
+            rc = run_gemm<EpiStoreBf16>(pair, map_d, map_wt, map_wt_half, g2, e2, status, s, "lmhead dhidden launch");
+            if (rc != DPPO_OK) return rc;
+            // (5) dW (+)= Dt ht[:, t0 : t0+tc]^T            (M = V, N = H, K = tokens of the chunk);
+            //     the K range must stop at the chunk, so ht gets a map of its own based at column t0
+            //     (t0 is a multiple of 9472 = 8 * 1184: the base stays 16-byte aligned)
+            rc = make_map(&map_dt, Dt, V, tc, lay.ld_tc, kBM);
+            if (rc != DPPO_OK) return rc;
+            rc = make_map(&map_ht_c, ht + t0, H, tc, lay.ld_t, kBN);
+            if (rc != DPPO_OK) return rc;
+            rc = make_map(&map_ht_c_half, ht + t0, H, tc, lay.ld_t, kHalfBN);
+            if (rc != DPPO_OK) return rc;
+            GemmShape g3 = {};
+            g3.n_mtiles = (V + kBM - 1) / kBM; g3.n_ntiles = (H + kBN - 1) / kBN; g3.n_ksteps = (int)((tc + kBK - 1) / kBK);
+            EpiAccumF32 e3 = {};
+            e3.C = (float*)dW; e3.ldc = H; e3.rows = V; e3.cols = H; e3.accumulate = c > 0 ? 1 : 0;
+            rc = run_gemm<EpiAccumF32>(pair, map_dt, map_ht_c, map_ht_c_half, g3, e3, status, s, "lmhead dW launch");
+            if (rc != DPPO_OK) return rc;
         }
     }
     return launch_loss_reduce(a, loss_out, s);

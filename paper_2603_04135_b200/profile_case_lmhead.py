@@ -3,7 +3,7 @@
   python -m paper_2603_04135_b200.profile_case_lmhead --tokens 16384 --hidden 2560 --iters 3
 
 Prints the event-timed duration of each call and the tensor throughput it corresponds to
-(2*T*V*H flops for the forward projection; 8*T*V*H with --backward: forward, dlogits recompute, dhidden, dW).
+(2*T*V*H flops for the forward projection; 6*T*V*H with --backward: logits, dhidden, dW).
 """
 import argparse
 
@@ -38,7 +38,7 @@ def main():
     dW = torch.empty((w.V, w.H), dtype=torch.float32, device="cuda") if args.backward else None
     loss_out = torch.zeros(5, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    flops = (8.0 if args.backward else 2.0) * T * w.V * w.H     # forward, recompute, dhidden, dW: 2 T V H each
+    flops = (6.0 if args.backward else 2.0) * T * w.V * w.H     # logits, dhidden, dW: 2 T V H each
     for it in range(args.iters):
         e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
         e0.record()
