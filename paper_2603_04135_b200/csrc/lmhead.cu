@@ -94,16 +94,48 @@ __device__ __forceinline__ float lm_ex2(float x) {
     return y;
 }
 
-// Shared-memory matrix descriptor of a K-major, 128B-swizzled tile whose rows are 128 bytes apart:
-// start address >> 4, leading byte offset 1 (unused for swizzled K-major), stride byte offset 1024 >> 4
-// (8-row swizzle atoms), descriptor version 1 (sm_100), layout type 2 (SWIZZLE_128B).
-__device__ __forceinline__ uint64_t lm_smem_desc(uint32_t smem_addr) {
+// Shared-memory matrix descriptors (descriptor version 1 = sm_100, layout type 2 = SWIZZLE_128B; addresses and
+// offsets in 16-byte units).  Both layouts are made of 1024-byte swizzle atoms, 8 rows of 128 bytes, exactly as a
+// 128B-swizzled TMA box with a 64-element inner extent lands them:
+//   K-major   a row of the atom is 64 K-elements of one M/N index; the tile is one box of 64 K x (128 or 256)
+//             rows, so 8-row groups are 1024 bytes apart (stride offset); the leading offset is unused.  The
+//             next 16 K-elements are 32 bytes further along the row.
+//   MN-major  a row of the atom is 64 consecutive M/N indices of one K index (the operand is stored with its
+//             M/N index contiguous, i.e. it is used transposed without a transposed copy); one box holds
+//             64 K x 64 M/N = 8 atoms stacked along K, 1024 bytes apart (stride offset), and the boxes of
+//             successive 64-wide M/N blocks follow each other 8192 bytes apart (leading offset).  The next
+//             16 K-elements are two atoms = 2048 bytes further.
+constexpr int kMnBoxBytes = kBK * 64 * 2;                // 8 KB: 64 K-rows of 64 M/N elements
+__device__ __forceinline__ uint64_t lm_smem_desc_k(uint32_t smem_addr) {
     return (uint64_t)((smem_addr >> 4) & 0x3FFF) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
            ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
 }
+__device__ __forceinline__ uint64_t lm_smem_desc_mn(uint32_t smem_addr) {
+    return (uint64_t)((smem_addr >> 4) & 0x3FFF) | ((uint64_t)(kMnBoxBytes >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+template <bool kMn> __device__ __forceinline__ uint64_t lm_smem_desc(uint32_t smem_addr) {
+    return kMn ? lm_smem_desc_mn(smem_addr) : lm_smem_desc_k(smem_addr);
+}
+template <bool kMn> __host__ __device__ constexpr uint64_t lm_desc_kstep() { return kMn ? (uint64_t)(2048 >> 4) : (uint64_t)(32 >> 4); }
 
-// Instruction descriptor of kind::f16: D = f32, A = B = bf16, both K-major, N = 256, M = 128.
-constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+// Instruction descriptor of kind::f16: D = f32, A = B = bf16, N = 256, M = 128 (256 for a CTA pair); bits 15 / 16
+// say that A / B is MN-major.
+template <bool kAMn, bool kBMn, int kM> __host__ __device__ constexpr uint32_t lm_idesc() {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((kAMn ? 1u : 0u) << 15) | ((kBMn ? 1u : 0u) << 16) |
+           ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kM >> 4) << 24);
+}
+
+// One tiled TMA load (x = innermost coordinate, 16-byte aligned by construction: multiples of 64 elements).
+__device__ __forceinline__ void lm_tma_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 :: "r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+// The same from a CTA of a pair: the barrier may be the peer's (the pair's leader collects both CTAs' bytes).
+__device__ __forceinline__ void lm_tma_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 :: "r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
 
 // What a launch of the GEMM core covers.  Tile j of a CTA is id = blockIdx.x + j * gridDim.x with
 //   m_fast ? (m = id % n_mtiles, n = id / n_mtiles) : (m = id / n_ntiles, n = id % n_ntiles)
@@ -126,7 +158,7 @@ __device__ __forceinline__ bool tile_of(const GemmShape& gs, uint32_t j, int& m,
 //   void row_begin(int m, int n, int row)
 //   void chunk(int m, int n, int row, int ch, uint32_t (&v)[32])   32 accumulator columns (f32 bits)
 //   void row_end(int m, int n, int row)
-template <class Epi>
+template <class Epi, bool kAMn, bool kBMn>
 __global__ void __launch_bounds__(kLmThreads, 1)
 lm_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const GemmShape gs, const Epi epi_args, int32_t* status) {
@@ -171,10 +203,18 @@ lm_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     const uint32_t bar = lm_smem_u32(&sh.full[s]);
                     const uint32_t dst_a = tiles + s * kStageBytes, dst_b = dst_a + kStageBytesA;
                     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"((uint32_t)kStageBytes) : "memory");
-                    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-                                 :: "r"(dst_a), "l"(&map_a), "r"(bar), "r"(k * kBK), "r"(gs.a_row0 + m * kBM) : "memory");
-                    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-                                 :: "r"(dst_b), "l"(&map_b), "r"(bar), "r"(k * kBK), "r"(n * kBN) : "memory");
+                    if (!kAMn) {
+                        lm_tma_2d(dst_a, &map_a, bar, k * kBK, gs.a_row0 + m * kBM);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < kBM / 64; ++i) lm_tma_2d(dst_a + i * kMnBoxBytes, &map_a, bar, m * kBM + 64 * i, k * kBK);
+                    }
+                    if (!kBMn) {
+                        lm_tma_2d(dst_b, &map_b, bar, k * kBK, n * kBN);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < kBN / 64; ++i) lm_tma_2d(dst_b + i * kMnBoxBytes, &map_b, bar, n * kBN + 64 * i, k * kBK);
+                    }
                 }
             }
             if (*abort_flag) {
@@ -203,15 +243,15 @@ lm_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     if (!lm_wait(lm_smem_u32(&sh.full[s]), use & 1, abort_flag)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t sa = tiles + s * kStageBytes, sb = sa + kStageBytesA;
-                    const uint64_t da = lm_smem_desc(sa), db = lm_smem_desc(sb);
+                    const uint64_t da = lm_smem_desc<kAMn>(sa), db = lm_smem_desc<kBMn>(sb);
 #pragma unroll
-                    for (int kk = 0; kk < kBK / 16; ++kk) {              // 16 K elements = 32 bytes inside the swizzle row
+                    for (int kk = 0; kk < kBK / 16; ++kk) {              // 16 K elements per instruction
                         const uint32_t accumulate = (k > 0 || kk > 0) ? 1u : 0u;
                         asm volatile("{\n\t.reg .pred p;\n\t"
                                      "setp.ne.b32 p, %4, 0;\n\t"
                                      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                                     :: "r"(d_tmem), "l"(da + (uint64_t)(kk * 2)), "l"(db + (uint64_t)(kk * 2)),
-                                        "r"(kIdesc), "r"(accumulate) : "memory");
+                                     :: "r"(d_tmem), "l"(da + kk * lm_desc_kstep<kAMn>()), "l"(db + kk * lm_desc_kstep<kBMn>()),
+                                        "r"(lm_idesc<kAMn, kBMn, kBM>()), "r"(accumulate) : "memory");
                     }
                     // frees this smem stage once the MMAs issued so far have read it
                     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
@@ -278,7 +318,6 @@ constexpr int kStages2 = 6;
 constexpr int kHalfBN = kBN / 2;
 constexpr int kStageBytesB2 = kHalfBN * kBK * 2;             // 16 KB
 constexpr int kStageBytes2 = kStageBytesA + kStageBytesB2;   // 32 KB per CTA
-constexpr uint32_t kIdesc2 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
 constexpr uint32_t kPeerMask = 0xFEFFFFFFu;                  // shared::cluster address of the pair's leader (rank bit cleared)
 
 struct LmShared2 {
@@ -305,7 +344,7 @@ __device__ __forceinline__ void lm_cluster_sync() {
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
-template <class Epi>
+template <class Epi, bool kAMn, bool kBMn>
 __global__ void __launch_bounds__(kLmThreads, 1)
 lm_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const GemmShape gs, const Epi epi_args, int32_t* status) {
@@ -357,10 +396,19 @@ lm_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     const uint32_t dst_a = tiles + s * kStageBytes2, dst_b = dst_a + kStageBytesA;
                     if (leader)
                         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar_local), "r"((uint32_t)(2 * kStageBytes2)) : "memory");
-                    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-                                 :: "r"(dst_a), "l"(&map_a), "r"(bar), "r"(k * kBK), "r"(gs.a_row0 + m * kBM) : "memory");
-                    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-                                 :: "r"(dst_b), "l"(&map_b), "r"(bar), "r"(k * kBK), "r"(n * kBN + (int)rank * kHalfBN) : "memory");
+                    if (!kAMn) {
+                        lm_tma_2d_pair(dst_a, &map_a, bar, k * kBK, gs.a_row0 + m * kBM);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < kBM / 64; ++i) lm_tma_2d_pair(dst_a + i * kMnBoxBytes, &map_a, bar, m * kBM + 64 * i, k * kBK);
+                    }
+                    const int nb0 = n * kBN + (int)rank * kHalfBN;       // this CTA's half of the B tile
+                    if (!kBMn) {
+                        lm_tma_2d_pair(dst_b, &map_b, bar, k * kBK, nb0);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < kHalfBN / 64; ++i) lm_tma_2d_pair(dst_b + i * kMnBoxBytes, &map_b, bar, nb0 + 64 * i, k * kBK);
+                    }
                 }
             }
         }
@@ -380,15 +428,15 @@ lm_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     if (!lm_wait(lm_smem_u32(&sh.full[s]), use & 1, abort_flag)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t sa = tiles + s * kStageBytes2, sb = sa + kStageBytesA;
-                    const uint64_t da = lm_smem_desc(sa), db = lm_smem_desc(sb);
+                    const uint64_t da = lm_smem_desc<kAMn>(sa), db = lm_smem_desc<kBMn>(sb);
 #pragma unroll
                     for (int kk = 0; kk < kBK / 16; ++kk) {
                         const uint32_t accumulate = (k > 0 || kk > 0) ? 1u : 0u;
                         asm volatile("{\n\t.reg .pred p;\n\t"
                                      "setp.ne.b32 p, %4, 0;\n\t"
                                      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                                     :: "r"(d_tmem), "l"(da + (uint64_t)(kk * 2)), "l"(db + (uint64_t)(kk * 2)),
-                                        "r"(kIdesc2), "r"(accumulate) : "memory");
+                                     :: "r"(d_tmem), "l"(da + kk * lm_desc_kstep<kAMn>()), "l"(db + kk * lm_desc_kstep<kBMn>()),
+                                        "r"(lm_idesc<kAMn, kBMn, 2 * kBM>()), "r"(accumulate) : "memory");
                     }
                     // frees this stage in BOTH CTAs once the MMAs issued so far have read it
                     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
@@ -562,71 +610,51 @@ lm_rows_kernel(const LossArgs a, const float2* __restrict__ part, const float* _
     }
 }
 
-// Backward, step 1: dlogits of the chunk from its stored logits, D = g (onehot - softmax) / tau, written
-// as bf16 both ways round:
-//   D  [chunk tokens x ldd]  (row = token)       feeds dhidden = D W
-//   Dt [V x ldt]             (row = vocabulary)  feeds dW = D^T hidden
-// 64 tokens x 64 vocabulary entries per block, transposed through shared memory so that both copies are
-// written in 128-byte runs.  Rows with g = 0 (no token, bad target) are written as zeros without
-// reading their logits.
-__global__ void __launch_bounds__(256)
+// Backward, step 1: dlogits of the chunk from its stored logits, D = g (onehot - softmax) / tau, as bf16
+// [chunk tokens x ldd].  Both later contractions read this one copy: dhidden = D W takes it K-major, dW = D^T
+// hidden takes it MN-major.  Rows with g = 0 (no token, bad target) are written as zeros without reading
+// their logits.  One thread per 8 vocabulary entries of a row.
+constexpr int kDlogitsThreads = 256;
+
+__global__ void __launch_bounds__(kDlogitsThreads)
 lm_dlogits_kernel(const float* __restrict__ Z, long long ldz, const RowInfo* __restrict__ info, long long t0,
-                  long long tc, int V, float c, __nv_bfloat16* __restrict__ D, long long ldd,
-                  __nv_bfloat16* __restrict__ Dt, long long ldt) {
-    __shared__ __nv_bfloat16 tile[64][64 + 2];                       // [token][vocabulary]; rows of 33 words
-    const long long r0 = (long long)blockIdx.y * 64;
-    const int v0 = blockIdx.x * 64;
-    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;          // 16 x 16 threads
-    const int col = v0 + 4 * tx;
+                  int V, float c, __nv_bfloat16* __restrict__ D, long long ldd) {
+    const long long r = blockIdx.y;
+    const int col = (blockIdx.x * kDlogitsThreads + threadIdx.x) * 8;
+    if (col >= V) return;
+    const RowInfo ri = info[t0 + r];
+    const float g = ri.g_over_tau;
+    float d[8];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int rr = ty + 16 * i;
-        const long long r = r0 + rr;
-        float d[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-        if (r < tc && col < V) {
-            const RowInfo ri = info[t0 + r];
-            const float g = ri.g_over_tau;
+    for (int j = 0; j < 8; ++j) d[j] = 0.0f;
+    __nv_bfloat16* dst = D + r * ldd + col;
+    if (col + 8 <= V) {                                              // ldz, ldd and col are multiples of 8
+        if (g != 0.0f) {
+            const float4 q0 = *reinterpret_cast<const float4*>(Z + r * ldz + col);
+            const float4 q1 = *reinterpret_cast<const float4*>(Z + r * ldz + col + 4);
+            const float z[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+            const int yrel = ri.y - col;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const float p = lm_ex2(fmaf(z[j], c, -ri.lse2_hi) - ri.lse2_lo);
+                d[j] = -g * p + ((j == yrel) ? g : 0.0f);
+            }
+        }
+        const __nv_bfloat162 b0 = __floats2bfloat162_rn(d[0], d[1]), b1 = __floats2bfloat162_rn(d[2], d[3]);
+        const __nv_bfloat162 b2 = __floats2bfloat162_rn(d[4], d[5]), b3 = __floats2bfloat162_rn(d[6], d[7]);
+        uint4 pk;
+        pk.x = *reinterpret_cast<const uint32_t*>(&b0); pk.y = *reinterpret_cast<const uint32_t*>(&b1);
+        pk.z = *reinterpret_cast<const uint32_t*>(&b2); pk.w = *reinterpret_cast<const uint32_t*>(&b3);
+        *reinterpret_cast<uint4*>(dst) = pk;
+    } else {
+        for (int j = 0; col + j < V; ++j) {
+            float dj = 0.0f;
             if (g != 0.0f) {
-                const float* src = Z + r * ldz + col;
-                float z[4];
-                if (col + 4 <= V) { const float4 q = *reinterpret_cast<const float4*>(src); z[0] = q.x; z[1] = q.y; z[2] = q.z; z[3] = q.w; }
-                else {
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) z[j] = (col + j < V) ? src[j] : 0.0f;
-                }
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const float p = lm_ex2(fmaf(z[j], c, -ri.lse2_hi) - ri.lse2_lo);
-                    d[j] = (col + j < V) ? (-g * p + ((col + j == ri.y) ? g : 0.0f)) : 0.0f;
-                }
+                const float p = lm_ex2(fmaf(Z[r * ldz + col + j], c, -ri.lse2_hi) - ri.lse2_lo);
+                dj = -g * p + ((col + j == ri.y) ? g : 0.0f);
             }
+            dst[j] = __float2bfloat16_rn(dj);
         }
-        const __nv_bfloat162 b01 = __floats2bfloat162_rn(d[0], d[1]), b23 = __floats2bfloat162_rn(d[2], d[3]);
-        *reinterpret_cast<__nv_bfloat162*>(&tile[rr][4 * tx]) = b01;
-        *reinterpret_cast<__nv_bfloat162*>(&tile[rr][4 * tx + 2]) = b23;
-        if (r < tc && col < V) {
-            __nv_bfloat16* dst = D + r * ldd + col;
-            if (col + 4 <= V) {                                      // ldd is a multiple of 8, col of 4: 8-byte stores
-                uint2 pk;
-                pk.x = *reinterpret_cast<const uint32_t*>(&b01); pk.y = *reinterpret_cast<const uint32_t*>(&b23);
-                *reinterpret_cast<uint2*>(dst) = pk;
-            } else {
-#pragma unroll
-                for (int j = 0; j < 4; ++j) if (col + j < V) dst[j] = __float2bfloat16_rn(d[j]);
-            }
-        }
-    }
-    __syncthreads();
-    // transposed copy: a warp writes one vocabulary row's 64 tokens (128 bytes), two per lane
-    const int lane = threadIdx.x & 31, wp = threadIdx.x >> 5;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const int vv = wp + 8 * i;
-        const long long r = r0 + 2 * lane;
-        if (v0 + vv >= V || r >= tc) continue;
-        __nv_bfloat16* dst = Dt + (long long)(v0 + vv) * ldt + r;     // ldt and r are even: 4-byte stores
-        if (r + 2 <= tc) *reinterpret_cast<__nv_bfloat162*>(dst) = __halves2bfloat162(tile[2 * lane][vv], tile[2 * lane + 1][vv]);
-        else dst[0] = tile[2 * lane][vv];
     }
 }
 
@@ -690,25 +718,6 @@ struct EpiAccumF32 {
     __device__ __forceinline__ void row_end(int, int, int) {}
 };
 
-// out[c x ldo] = in[r x ldi]^T for bf16, 64 x 64 tiles through shared memory; columns r..ldo-1 of out are
-// left untouched (never read: tensor maps stop at r).
-__global__ void __launch_bounds__(256)
-transpose_bf16_kernel(const __nv_bfloat16* __restrict__ in, long long rows, long long cols, long long ldi,
-                      __nv_bfloat16* __restrict__ out, long long ldo) {
-    __shared__ __nv_bfloat16 tile[64][66];
-    const long long r0 = (long long)blockIdx.y * 64, c0 = (long long)blockIdx.x * 64;
-    const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
-    for (int i = ty; i < 64; i += 4) {
-        const long long r = r0 + i, c = c0 + tx;
-        tile[i][tx] = (r < rows && c < cols) ? in[r * ldi + c] : __float2bfloat16_rn(0.0f);
-    }
-    __syncthreads();
-    for (int i = ty; i < 64; i += 4) {
-        const long long c = c0 + i, r = r0 + tx;
-        if (c < cols && r < rows) out[c * ldo + r] = tile[tx][i];
-    }
-}
-
 // ---- host side -----------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -744,10 +753,10 @@ static int make_map(CUtensorMap* map, const void* base, long long rows, long lon
 
 constexpr size_t kLmDynSmem = (size_t)kStages * kStageBytes + 1024;
 
-template <class Epi>
+template <class Epi, bool kAMn, bool kBMn>
 static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const GemmShape& gs, const Epi& epi,
                        int32_t* status, cudaStream_t s, const char* what) {
-    auto kernel = lm_gemm_kernel<Epi>;
+    auto kernel = lm_gemm_kernel<Epi, kAMn, kBMn>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLmDynSmem);
     if (e != cudaSuccess) return cuda_fail(e, "lmhead: shared memory attribute");
     const long long work = (long long)gs.n_mtiles * gs.n_ntiles;
@@ -762,10 +771,10 @@ static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const GemmS
 constexpr size_t kLmDynSmem2 = (size_t)kStages2 * kStageBytes2 + 1024;
 
 // CTA-pair version: `mb_half` is B's tensor map with 128-row boxes.
-template <class Epi>
+template <class Epi, bool kAMn, bool kBMn>
 static int launch_gemm2(const CUtensorMap& ma, const CUtensorMap& mb_half, const GemmShape& gs, const Epi& epi,
                         int32_t* status, cudaStream_t s, const char* what) {
-    auto kernel = lm_gemm2_kernel<Epi>;
+    auto kernel = lm_gemm2_kernel<Epi, kAMn, kBMn>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLmDynSmem2);
     if (e != cudaSuccess) return cuda_fail(e, "lmhead: shared memory attribute");
     const long long n_m2 = (gs.n_mtiles + 1) / 2;
@@ -787,18 +796,19 @@ static int launch_gemm2(const CUtensorMap& ma, const CUtensorMap& mb_half, const
     return DPPO_OK;
 }
 
-template <class Epi>
+// An MN-major operand's map has 64 x 64 boxes whatever the tile (mb_half == mb then).
+template <class Epi, bool kAMn, bool kBMn>
 static int run_gemm(bool pair, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mb_half, const GemmShape& gs,
                     const Epi& epi, int32_t* status, cudaStream_t s, const char* what) {
-    return pair ? launch_gemm2<Epi>(ma, mb_half, gs, epi, status, s, what)
-                : launch_gemm<Epi>(ma, mb, gs, epi, status, s, what);
+    return pair ? launch_gemm2<Epi, kAMn, kBMn>(ma, mb_half, gs, epi, status, s, what)
+                : launch_gemm<Epi, kAMn, kBMn>(ma, mb, gs, epi, status, s, what);
 }
 
 static long long round_up(long long x, long long m) { return (x + m - 1) / m * m; }
 
 struct LmWorkspace {
-    size_t terms, info, part, zy, wt, ht, z, d, dt, total;   // byte offsets and the total
-    long long ld_v, ld_t, ld_tc;                 // pitches: vocabulary (Z, D, Wt), tokens (ht), chunk tokens (Dt)
+    size_t terms, info, part, zy, z, d, total;   // byte offsets and the total
+    long long ld_v;                              // pitch of Z and D (vocabulary)
     int n_ntiles;
 };
 
@@ -807,21 +817,16 @@ static LmWorkspace lm_layout(const dppo_lmhead_params* p, bool backward) {
     const long long T = p->loss.T_max > 0 ? p->loss.T_max : 1;
     auto al = [](size_t x) { return (x + 1023) & ~(size_t)1023; };
     w.ld_v = round_up(p->loss.V, 8);
-    w.ld_t = round_up(T, 8);
-    w.ld_tc = kChunkTokens;
     w.n_ntiles = (p->loss.V + kBN - 1) / kBN;
     size_t off = 0;
     w.terms = off; off += al(loss_terms_bytes(T));
     w.info = off;  off += al((size_t)T * sizeof(RowInfo));
     w.part = off;  off += al((size_t)kChunkTokens * w.n_ntiles * sizeof(float2));
     w.zy = off;    off += al((size_t)kChunkTokens * sizeof(float));
-    w.wt = w.ht = w.z = w.d = w.dt = off;
+    w.z = w.d = off;
     if (backward) {
-        w.wt = off; off += al((size_t)p->H * w.ld_v * 2);
-        w.ht = off; off += al((size_t)p->H * w.ld_t * 2);
         w.z = off;  off += al((size_t)kChunkTokens * w.ld_v * 4);
         w.d = off;  off += al((size_t)kChunkTokens * w.ld_v * 2);
-        w.dt = off; off += al((size_t)p->loss.V * w.ld_tc * 2);
     }
     w.total = off;
     return w;
@@ -895,21 +900,10 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
         float2* part = (float2*)(ws + lay.part);
         float* zy = (float*)(ws + lay.zy);
         float* Z = backward ? (float*)(ws + lay.z) : nullptr;
-        __nv_bfloat16* Wt = (__nv_bfloat16*)(ws + lay.wt);
-        __nv_bfloat16* ht = (__nv_bfloat16*)(ws + lay.ht);
         __nv_bfloat16* D = (__nv_bfloat16*)(ws + lay.d);
-        __nv_bfloat16* Dt = (__nv_bfloat16*)(ws + lay.dt);
-        alignas(64) CUtensorMap map_wt, map_wt_half;
+        alignas(64) CUtensorMap map_w_mn;                                              // W as [K = V][N = H]
         if (backward) {
-            // K-major copies of the two operands that are contracted over their row index
-            transpose_bf16_kernel<<<dim3((H + 63) / 64, (V + 63) / 64), 256, 0, s>>>(
-                (const __nv_bfloat16*)W, V, H, H, Wt, lay.ld_v);
-            transpose_bf16_kernel<<<dim3((H + 63) / 64, (unsigned)((T + 63) / 64)), 256, 0, s>>>(
-                (const __nv_bfloat16*)hidden, T, H, H, ht, lay.ld_t);
-            DPPO_CHECK_LAUNCH("lmhead transpose launch");
-            rc = make_map(&map_wt, Wt, H, V, lay.ld_v, kBN);
-            if (rc != DPPO_OK) return rc;
-            rc = make_map(&map_wt_half, Wt, H, V, lay.ld_v, kHalfBN);
+            rc = make_map(&map_w_mn, W, V, H, H, 64);
             if (rc != DPPO_OK) return rc;
         }
 
@@ -923,41 +917,38 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
             EpiPartial e1 = {};
             e1.part = part; e1.zy_out = zy; e1.Z = Z; e1.target = target; e1.n_tokens_dev = n_tokens_dev;
             e1.T_max = T; e1.t0 = t0; e1.tc = tc; e1.ldz = lay.ld_v; e1.V = V; e1.n_ntiles = lay.n_ntiles; e1.c = a.scale2;
-            rc = run_gemm<EpiPartial>(pair, map_h, map_w, map_w_half, g1, e1, status, s, "lmhead logits launch");
+            rc = run_gemm<EpiPartial, false, false>(pair, map_h, map_w, map_w_half, g1, e1, status, s, "lmhead logits launch");
             if (rc != DPPO_OK) return rc;
             // (2) rows: log-sum-exp, logp, loss terms, dloss/dlogp
             lm_rows_kernel<<<(unsigned)((tc + kRowsWarps - 1) / kRowsWarps), kRowsWarps * 32, 0, s>>>(
                 a, part, zy, info, t0, tc, lay.n_ntiles);
             DPPO_CHECK_LAUNCH("lmhead rows launch");
             if (!backward) continue;
-            // (3) dlogits of the chunk: D [tc x V] and Dt [V x tc]
-            lm_dlogits_kernel<<<dim3((V + 63) / 64, (unsigned)((tc + 63) / 64)), 256, 0, s>>>(
-                Z, lay.ld_v, info, t0, tc, V, a.scale2, D, lay.ld_v, Dt, lay.ld_tc);
+            // (3) dlogits of the chunk: D [tc x V]
+            lm_dlogits_kernel<<<dim3((unsigned)((V + 8 * kDlogitsThreads - 1) / (8 * kDlogitsThreads)), (unsigned)tc),
+                                kDlogitsThreads, 0, s>>>(Z, lay.ld_v, info, t0, V, a.scale2, D, lay.ld_v);
             DPPO_CHECK_LAUNCH("lmhead dlogits launch");
-            // (4) dhidden[t0 : t0+tc, :] = D Wt^T          (M = tokens, N = H, K = V)
-            alignas(64) CUtensorMap map_d, map_dt, map_ht_c, map_ht_c_half;
+            // (4) dhidden[t0 : t0+tc, :] = D W            (M = tokens, N = H, K = V; D K-major, W MN-major)
+            alignas(64) CUtensorMap map_d, map_d_mn, map_h_mn;
             rc = make_map(&map_d, D, tc, V, lay.ld_v, kBM);
             if (rc != DPPO_OK) return rc;
             GemmShape g2 = {};
             g2.n_mtiles = (int)((tc + kBM - 1) / kBM); g2.n_ntiles = (H + kBN - 1) / kBN; g2.n_ksteps = (V + kBK - 1) / kBK;
             EpiStoreBf16 e2 = {};
             e2.C = (__nv_bfloat16*)dhidden; e2.ldc = H; e2.row0 = t0; e2.rows = T; e2.cols = H;
-            rc = run_gemm<EpiStoreBf16>(pair, map_d, map_wt, map_wt_half, g2, e2, status, s, "lmhead dhidden launch");
+            rc = run_gemm<EpiStoreBf16, false, true>(pair, map_d, map_w_mn, map_w_mn, g2, e2, status, s, "lmhead dhidden launch");
             if (rc != DPPO_OK) return rc;
-            // (5) dW (+)= Dt ht[:, t0 : t0+tc]^T            (M = V, N = H, K = tokens of the chunk);
-            //     the K range must stop at the chunk, so ht gets a map of its own based at column t0
-            //     (t0 is a multiple of 9472 = 8 * 1184: the base stays 16-byte aligned)
-            rc = make_map(&map_dt, Dt, V, tc, lay.ld_tc, kBM);
+            // (5) dW (+)= D^T hidden[t0 : t0+tc, :]       (M = V, N = H, K = tokens of the chunk; both MN-major);
+            //     the K range stops at the chunk: both maps have tc rows and fill with zeros beyond
+            rc = make_map(&map_d_mn, D, tc, V, lay.ld_v, 64);
             if (rc != DPPO_OK) return rc;
-            rc = make_map(&map_ht_c, ht + t0, H, tc, lay.ld_t, kBN);
-            if (rc != DPPO_OK) return rc;
-            rc = make_map(&map_ht_c_half, ht + t0, H, tc, lay.ld_t, kHalfBN);
+            rc = make_map(&map_h_mn, (const __nv_bfloat16*)hidden + t0 * H, tc, H, H, 64);
             if (rc != DPPO_OK) return rc;
             GemmShape g3 = {};
             g3.n_mtiles = (V + kBM - 1) / kBM; g3.n_ntiles = (H + kBN - 1) / kBN; g3.n_ksteps = (int)((tc + kBK - 1) / kBK);
             EpiAccumF32 e3 = {};
             e3.C = (float*)dW; e3.ldc = H; e3.rows = V; e3.cols = H; e3.accumulate = c > 0 ? 1 : 0;
-            rc = run_gemm<EpiAccumF32>(pair, map_dt, map_ht_c, map_ht_c_half, g3, e3, status, s, "lmhead dW launch");
+            rc = run_gemm<EpiAccumF32, true, true>(pair, map_d_mn, map_h_mn, map_h_mn, g3, e3, status, s, "lmhead dW launch");
             if (rc != DPPO_OK) return rc;
         }
     }
