@@ -153,14 +153,57 @@ __device__ __forceinline__ bool tile_of(const GemmShape& gs, uint32_t j, int& m,
     return true;
 }
 
+// ---- epilogue output through shared memory ---------------------------------------------------------
+// An epilogue thread holds 32 consecutive f32 of ONE row, so direct stores make every warp instruction touch
+// 32 different lines.  Instead each epilogue warp stages its 32 x 32 block (4 KB, rows of 128 bytes, 16-byte
+// chunks XOR-swizzled with the row so that the staging writes are conflict-free) and lane 0 hands it to the
+// TMA unit as one tiled store -- or a tiled f32 add-reduction -- which writes whole 128-byte runs and clips
+// at the tensor's edges.  Two staging buffers per warp: the block being drained and the block being filled.
+constexpr int kStageTileBytes = 32 * 32 * 4;
+constexpr int kStageBytesEpi = 4 * 2 * kStageTileBytes;  // 4 epilogue warps x 2 buffers = 32 KB
+
+struct EpiCtx {
+    const CUtensorMap* map_c;            // f32 [rows x cols], 32 x 32 boxes, 128B swizzle
+    uint32_t stage;                      // this warp's two staging buffers (shared::cta address, 1024-aligned)
+    uint32_t toggle;
+    int lane;
+};
+
+// Block of 32 rows x 32 f32 at (column x, row y) of the tensor behind map_c; v = this lane's row.
+template <bool kAdd>
+__device__ __forceinline__ void lm_store_block(EpiCtx& ctx, const uint32_t (&v)[32], int x, int y) {
+    if (ctx.lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");   // the buffer filled two blocks ago has been read
+    __syncwarp();
+    const uint32_t buf = ctx.stage + ctx.toggle * kStageTileBytes;
+    const uint32_t rowp = buf + (uint32_t)ctx.lane * 128u;
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                     :: "r"(rowp + (uint32_t)((j ^ (ctx.lane & 7)) << 4)), "r"(v[4 * j]), "r"(v[4 * j + 1]), "r"(v[4 * j + 2]), "r"(v[4 * j + 3])
+                     : "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncwarp();
+    if (ctx.lane == 0) {
+        if (kAdd)
+            asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
+                         :: "l"(ctx.map_c), "r"(buf), "r"(x), "r"(y) : "memory");
+        else
+            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
+                         :: "l"(ctx.map_c), "r"(buf), "r"(x), "r"(y) : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    }
+    ctx.toggle ^= 1u;
+}
+
 // ---- the GEMM core --------------------------------------------------------------------------------
 // Epi (one copy per epilogue thread = per tile row), called for every tile:
 //   void row_begin(int m, int n, int row)
-//   void chunk(int m, int n, int row, int ch, uint32_t (&v)[32])   32 accumulator columns (f32 bits)
+//   void chunk(int m, int n, int row, int ch, uint32_t (&v)[32], EpiCtx& ctx)   32 accumulator columns (f32 bits)
 //   void row_end(int m, int n, int row)
 template <class Epi, bool kAMn, bool kBMn>
 __global__ void __launch_bounds__(kLmThreads, 1)
 lm_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const __grid_constant__ CUtensorMap map_c,
                const GemmShape gs, const Epi epi_args, int32_t* status) {
     extern __shared__ unsigned char lm_raw[];
     __shared__ LmShared sh;
@@ -267,6 +310,9 @@ lm_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int q = warp & 3;                                          // TMEM lane quarter this warp may read
         const int row = q * 32 + lane;
         Epi epi = epi_args;                                              // per-thread copy: its state lives in registers
+        EpiCtx ctx;
+        ctx.map_c = &map_c; ctx.stage = tiles + kStages * kStageBytes + (uint32_t)q * (2 * kStageTileBytes);
+        ctx.toggle = 0; ctx.lane = lane;
         int m, n;
         for (uint32_t j = 0; tile_of(gs, j, m, n); ++j) {
             const uint32_t b = j & 1, use_b = j >> 1;
@@ -287,13 +333,14 @@ lm_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                                "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
                              : "r"(taddr + (uint32_t)(ch * 32)) : "memory");
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                epi.chunk(m, n, row, ch, v);
+                epi.chunk(m, n, row, ch, v, ctx);
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) lm_arrive(lm_smem_u32(&sh.acc_empty[b]));
             epi.row_end(m, n, row);
         }
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // this warp's tiled stores are complete
     }
 
     // ---- common exit: nobody touches tensor memory any more, then the allocating warp frees it
@@ -347,6 +394,7 @@ __device__ __forceinline__ void lm_cluster_sync() {
 template <class Epi, bool kAMn, bool kBMn>
 __global__ void __launch_bounds__(kLmThreads, 1)
 lm_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                const __grid_constant__ CUtensorMap map_c,
                 const GemmShape gs, const Epi epi_args, int32_t* status) {
     extern __shared__ unsigned char lm_raw[];
     __shared__ LmShared2 sh;
@@ -452,6 +500,9 @@ lm_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         const int q = warp & 3;
         const int row = q * 32 + lane;
         Epi epi = epi_args;
+        EpiCtx ctx;
+        ctx.map_c = &map_c; ctx.stage = tiles + kStages2 * kStageBytes2 + (uint32_t)q * (2 * kStageTileBytes);
+        ctx.toggle = 0; ctx.lane = lane;
         int m2, n;
         for (uint32_t j = 0; pair_tile_of(gs, j, m2, n); ++j) {
             const int m = 2 * m2 + (int)rank;
@@ -472,7 +523,7 @@ lm_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                                "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
                              : "r"(taddr + (uint32_t)(ch * 32)) : "memory");
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                epi.chunk(m, n, row, ch, v);
+                epi.chunk(m, n, row, ch, v, ctx);
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
@@ -480,6 +531,7 @@ lm_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" :: "r"(lm_smem_u32(&sh.acc_empty[b]) & kPeerMask) : "memory");
             epi.row_end(m, n, row);
         }
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
 
     // ---- common exit: both CTAs are done with tensor memory and with each other's barriers, then free
@@ -507,10 +559,10 @@ struct RowInfo {             // what the backward needs from the forward, per to
 struct EpiPartial {
     float2* part;            // [chunk tokens x n_ntiles]
     float* zy_out;           // [chunk tokens]
-    float* Z;                // [chunk tokens x ldz] f32, nullable
+    int store_z;             // the kernel's output map is Z [chunk tokens x V] f32: keep the logits
     const int32_t* target;
     const int32_t* n_tokens_dev;
-    long long T_max, t0, tc, ldz;
+    long long T_max, t0, tc;
     int V, n_ntiles;
     float c;
     // per-thread state
@@ -524,21 +576,13 @@ struct EpiPartial {
         y = live ? target[t0 + r] : -1;
         m2 = -INFINITY; s = 0.0f; zy = 0.0f; hit = false;
     }
-    __device__ __forceinline__ void chunk(int m, int n, int row, int ch, uint32_t (&v)[32]) {
+    __device__ __forceinline__ void chunk(int m, int n, int row, int ch, uint32_t (&v)[32], EpiCtx& ctx) {
         const int col0 = n * kBN + ch * 32;
         const int valid = V - col0;                                  // columns of this chunk inside the vocabulary
-        if (!live || valid <= 0) return;
-        if (Z) {
-            float* dst = Z + ((long long)m * kBM + row) * ldz + col0;
-            if (valid >= 32) {                                       // ldz is a multiple of 8: 16-byte stores
-                uint4* d4 = reinterpret_cast<uint4*>(dst);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) d4[j] = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-            } else {
-#pragma unroll
-                for (int j = 0; j < 32; ++j) if (j < valid) dst[j] = __uint_as_float(v[j]);
-            }
-        }
+        if (valid <= 0) return;                                      // the same for the whole warp
+        const int y0 = m * kBM + row - ctx.lane;                     // first row of this warp's block
+        if (store_z && y0 < tc) lm_store_block<false>(ctx, v, col0, y0);   // clipped at V and at the chunk's last row
+        if (!live) return;
         const int yrel = y - col0;                                   // selects, not an indexed read: v stays in registers
         hit = hit || (yrel >= 0 && yrel < 32);
         float cm = -INFINITY;
@@ -664,7 +708,7 @@ struct EpiStoreBf16 {
     long long ldc, row0, rows;   // output row of tile row 0; rows that exist in C
     int cols;
     __device__ __forceinline__ void row_begin(int, int, int) {}
-    __device__ __forceinline__ void chunk(int m, int n, int row, int ch, uint32_t (&v)[32]) {
+    __device__ __forceinline__ void chunk(int m, int n, int row, int ch, uint32_t (&v)[32], EpiCtx&) {
         const long long r = row0 + (long long)m * kBM + row;
         const int col0 = n * kBN + ch * 32;
         if (r >= rows || col0 >= cols) return;
@@ -689,31 +733,18 @@ struct EpiStoreBf16 {
     __device__ __forceinline__ void row_end(int, int, int) {}
 };
 
-// C[rows x ldc] (f32) = or += acc (dW, accumulated over the token chunks).
+// C (f32, the tensor behind the kernel's output map) = or += acc (dW, accumulated over the token chunks; the
+// add is done by the memory system, nothing is read back).
 struct EpiAccumF32 {
-    float* C;
-    long long ldc, rows;
+    long long rows;
     int cols, accumulate;
     __device__ __forceinline__ void row_begin(int, int, int) {}
-    __device__ __forceinline__ void chunk(int m, int n, int row, int ch, uint32_t (&v)[32]) {
-        const long long r = (long long)m * kBM + row;
+    __device__ __forceinline__ void chunk(int m, int n, int row, int ch, uint32_t (&v)[32], EpiCtx& ctx) {
         const int col0 = n * kBN + ch * 32;
-        if (r >= rows || col0 >= cols) return;
-        float* dst = C + r * ldc + col0;
-        if (col0 + 32 <= cols) {                                     // ldc is a multiple of 64: 16-byte accesses
-            float4* d4 = reinterpret_cast<float4*>(dst);
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                float4 x = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
-                                       __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
-                if (accumulate) { const float4 o = d4[j]; x.x += o.x; x.y += o.y; x.z += o.z; x.w += o.w; }
-                d4[j] = x;
-            }
-        } else {
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-                if (col0 + j < cols) dst[j] = (accumulate ? dst[j] : 0.0f) + __uint_as_float(v[j]);
-        }
+        const int y0 = m * kBM + row - ctx.lane;                     // first row of this warp's block
+        if (y0 >= rows || col0 >= cols) return;                      // the same for the whole warp
+        if (accumulate) lm_store_block<true>(ctx, v, col0, y0);
+        else            lm_store_block<false>(ctx, v, col0, y0);
     }
     __device__ __forceinline__ void row_end(int, int, int) {}
 };
@@ -751,10 +782,26 @@ static int make_map(CUtensorMap* map, const void* base, long long rows, long lon
     return DPPO_OK;
 }
 
-constexpr size_t kLmDynSmem = (size_t)kStages * kStageBytes + 1024;
+// f32 [rows x cols] with row pitch ld elements as the target of the epilogue's tiled stores: 32 x 32 boxes
+// (128-byte rows), 128B swizzle.
+static int make_map_out(CUtensorMap* map, const void* base, long long rows, long long cols, long long ld) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return fail(DPPO_ERR_CUDA, "lmhead: cuTensorMapEncodeTiled is not available from this driver");
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * 4};
+    const cuuint32_t box[2] = {32, 32};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(DPPO_ERR_CUDA, "lmhead: cuTensorMapEncodeTiled (output) failed with %d", (int)r);
+    return DPPO_OK;
+}
+
+constexpr size_t kLmDynSmem = (size_t)kStages * kStageBytes + kStageBytesEpi + 1024;
 
 template <class Epi, bool kAMn, bool kBMn>
-static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const GemmShape& gs, const Epi& epi,
+static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const GemmShape& gs, const Epi& epi,
                        int32_t* status, cudaStream_t s, const char* what) {
     auto kernel = lm_gemm_kernel<Epi, kAMn, kBMn>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLmDynSmem);
@@ -762,17 +809,18 @@ static int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const GemmS
     const long long work = (long long)gs.n_mtiles * gs.n_ntiles;
     const int grid = (int)(work < sm_count() ? work : sm_count());
     if (grid < 1) return DPPO_OK;
-    kernel<<<grid, kLmThreads, kLmDynSmem, s>>>(ma, mb, gs, epi, status);
+    kernel<<<grid, kLmThreads, kLmDynSmem, s>>>(ma, mb, mc, gs, epi, status);
     cudaError_t e2 = cudaGetLastError();
     if (e2 != cudaSuccess) return cuda_fail(e2, what);
     return DPPO_OK;
 }
 
-constexpr size_t kLmDynSmem2 = (size_t)kStages2 * kStageBytes2 + 1024;
+constexpr size_t kLmDynSmem2 = (size_t)kStages2 * kStageBytes2 + kStageBytesEpi + 1024;
+static_assert(kLmDynSmem <= 232448 - 256 && kLmDynSmem2 <= 232448 - 256, "ring + staging must fit one CTA's shared memory");
 
 // CTA-pair version: `mb_half` is B's tensor map with 128-row boxes.
 template <class Epi, bool kAMn, bool kBMn>
-static int launch_gemm2(const CUtensorMap& ma, const CUtensorMap& mb_half, const GemmShape& gs, const Epi& epi,
+static int launch_gemm2(const CUtensorMap& ma, const CUtensorMap& mb_half, const CUtensorMap& mc, const GemmShape& gs, const Epi& epi,
                         int32_t* status, cudaStream_t s, const char* what) {
     auto kernel = lm_gemm2_kernel<Epi, kAMn, kBMn>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLmDynSmem2);
@@ -791,17 +839,19 @@ static int launch_gemm2(const CUtensorMap& ma, const CUtensorMap& mb_half, const
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    e = cudaLaunchKernelEx(&cfg, kernel, ma, mb_half, gs, epi, status);
+    e = cudaLaunchKernelEx(&cfg, kernel, ma, mb_half, mc, gs, epi, status);
     if (e != cudaSuccess) return cuda_fail(e, what);
     return DPPO_OK;
 }
 
-// An MN-major operand's map has 64 x 64 boxes whatever the tile (mb_half == mb then).
+// An MN-major operand's map has 64 x 64 boxes whatever the tile (mb_half == mb then).  mc: the f32 output of
+// the epilogues that store through the TMA unit (any valid map for the others).
 template <class Epi, bool kAMn, bool kBMn>
-static int run_gemm(bool pair, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mb_half, const GemmShape& gs,
+static int run_gemm(bool pair, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mb_half, const CUtensorMap& mc,
+                    const GemmShape& gs,
                     const Epi& epi, int32_t* status, cudaStream_t s, const char* what) {
-    return pair ? launch_gemm2<Epi, kAMn, kBMn>(ma, mb_half, gs, epi, status, s, what)
-                : launch_gemm<Epi, kAMn, kBMn>(ma, mb, gs, epi, status, s, what);
+    return pair ? launch_gemm2<Epi, kAMn, kBMn>(ma, mb_half, mc, gs, epi, status, s, what)
+                : launch_gemm<Epi, kAMn, kBMn>(ma, mb, mc, gs, epi, status, s, what);
 }
 
 static long long round_up(long long x, long long m) { return (x + m - 1) / m * m; }
@@ -816,17 +866,18 @@ static LmWorkspace lm_layout(const dppo_lmhead_params* p, bool backward) {
     LmWorkspace w;
     const long long T = p->loss.T_max > 0 ? p->loss.T_max : 1;
     auto al = [](size_t x) { return (x + 1023) & ~(size_t)1023; };
+    const size_t rows = (size_t)(T < kChunkTokens ? round_up(T, kBM) : kChunkTokens);   // rows of the per-chunk buffers
     w.ld_v = round_up(p->loss.V, 8);
     w.n_ntiles = (p->loss.V + kBN - 1) / kBN;
     size_t off = 0;
     w.terms = off; off += al(loss_terms_bytes(T));
     w.info = off;  off += al((size_t)T * sizeof(RowInfo));
-    w.part = off;  off += al((size_t)kChunkTokens * w.n_ntiles * sizeof(float2));
-    w.zy = off;    off += al((size_t)kChunkTokens * sizeof(float));
+    w.part = off;  off += al(rows * w.n_ntiles * sizeof(float2));
+    w.zy = off;    off += al(rows * sizeof(float));
     w.z = w.d = off;
     if (backward) {
-        w.z = off;  off += al((size_t)kChunkTokens * w.ld_v * 4);
-        w.d = off;  off += al((size_t)kChunkTokens * w.ld_v * 2);
+        w.z = off;  off += al(rows * w.ld_v * 4);
+        w.d = off;  off += al(rows * w.ld_v * 2);
     }
     w.total = off;
     return w;
@@ -902,8 +953,11 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
         float* Z = backward ? (float*)(ws + lay.z) : nullptr;
         __nv_bfloat16* D = (__nv_bfloat16*)(ws + lay.d);
         alignas(64) CUtensorMap map_w_mn;                                              // W as [K = V][N = H]
+        alignas(64) CUtensorMap map_dw;
         if (backward) {
             rc = make_map(&map_w_mn, W, V, H, H, 64);
+            if (rc != DPPO_OK) return rc;
+            rc = make_map_out(&map_dw, dW, V, H, H);
             if (rc != DPPO_OK) return rc;
         }
 
@@ -915,9 +969,14 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
             g1.n_mtiles = (int)((tc + kBM - 1) / kBM); g1.n_ntiles = lay.n_ntiles; g1.n_ksteps = H / kBK;
             g1.a_row0 = (int)t0; g1.m_fast = 1;                                        // neighbours share the W tile
             EpiPartial e1 = {};
-            e1.part = part; e1.zy_out = zy; e1.Z = Z; e1.target = target; e1.n_tokens_dev = n_tokens_dev;
-            e1.T_max = T; e1.t0 = t0; e1.tc = tc; e1.ldz = lay.ld_v; e1.V = V; e1.n_ntiles = lay.n_ntiles; e1.c = a.scale2;
-            rc = run_gemm<EpiPartial, false, false>(pair, map_h, map_w, map_w_half, g1, e1, status, s, "lmhead logits launch");
+            e1.part = part; e1.zy_out = zy; e1.store_z = backward ? 1 : 0; e1.target = target; e1.n_tokens_dev = n_tokens_dev;
+            e1.T_max = T; e1.t0 = t0; e1.tc = tc; e1.V = V; e1.n_ntiles = lay.n_ntiles; e1.c = a.scale2;
+            alignas(64) CUtensorMap map_z = map_h;
+            if (backward) {
+                rc = make_map_out(&map_z, Z, tc, V, lay.ld_v);
+                if (rc != DPPO_OK) return rc;
+            }
+            rc = run_gemm<EpiPartial, false, false>(pair, map_h, map_w, map_w_half, map_z, g1, e1, status, s, "lmhead logits launch");
             if (rc != DPPO_OK) return rc;
             // (2) rows: log-sum-exp, logp, loss terms, dloss/dlogp
             lm_rows_kernel<<<(unsigned)((tc + kRowsWarps - 1) / kRowsWarps), kRowsWarps * 32, 0, s>>>(
@@ -936,7 +995,7 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
             g2.n_mtiles = (int)((tc + kBM - 1) / kBM); g2.n_ntiles = (H + kBN - 1) / kBN; g2.n_ksteps = (V + kBK - 1) / kBK;
             EpiStoreBf16 e2 = {};
             e2.C = (__nv_bfloat16*)dhidden; e2.ldc = H; e2.row0 = t0; e2.rows = T; e2.cols = H;
-            rc = run_gemm<EpiStoreBf16, false, true>(pair, map_d, map_w_mn, map_w_mn, g2, e2, status, s, "lmhead dhidden launch");
+            rc = run_gemm<EpiStoreBf16, false, true>(pair, map_d, map_w_mn, map_w_mn, map_d, g2, e2, status, s, "lmhead dhidden launch");
             if (rc != DPPO_OK) return rc;
             // (5) dW (+)= D^T hidden[t0 : t0+tc, :]       (M = V, N = H, K = tokens of the chunk; both MN-major);
             //     the K range stops at the chunk: both maps have tc rows and fill with zeros beyond
@@ -947,8 +1006,8 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
             GemmShape g3 = {};
             g3.n_mtiles = (V + kBM - 1) / kBM; g3.n_ntiles = (H + kBN - 1) / kBN; g3.n_ksteps = (int)((tc + kBK - 1) / kBK);
             EpiAccumF32 e3 = {};
-            e3.C = (float*)dW; e3.ldc = H; e3.rows = V; e3.cols = H; e3.accumulate = c > 0 ? 1 : 0;
-            rc = run_gemm<EpiAccumF32, true, true>(pair, map_d_mn, map_h_mn, map_h_mn, g3, e3, status, s, "lmhead dW launch");
+            e3.rows = V; e3.cols = H; e3.accumulate = c > 0 ? 1 : 0;
+            rc = run_gemm<EpiAccumF32, true, true>(pair, map_d_mn, map_h_mn, map_h_mn, map_dw, g3, e3, status, s, "lmhead dW launch");
             if (rc != DPPO_OK) return rc;
         }
     }
