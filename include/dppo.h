@@ -252,19 +252,19 @@ int dppo_sequence_log_ratio(const float* logp, const float* logp_old, const int3
 
 /* ------------------------------------------------------------------------------------------------
  * Fused LM-head + loss: the same loss as dppo_grpo_loss_fwd_bwd with the logits z = hidden W^T
- * produced on the fly by the tensor cores and never written to memory (Eq. 1's pi_theta is the
- * log-softmax of exactly these logits).
+ * produced on the fly by the tensor cores; the [T x V] logits of the batch are never written to memory
+ * (Eq. 1's pi_theta is the log-softmax of exactly these logits).
  *
  *   loss     the loss parameters; dtype must be DPPO_BF16; row_stride and variant are ignored
  *   H        hidden width, a multiple of 64
  *   hidden   bf16 [T_max x H] row-major, one row per loss token in packed order
  *   W        bf16 [V x H] row-major LM-head weight
  *   backward 0: forward only (loss_out, logp_out, lse_out; dhidden and dW must be NULL).
- *            1: also the gradients, dhidden = D W and dW = D^T hidden with D = dlogits recomputed from the
- *            same GEMM for 9472 tokens at a time into workspace scratch (bf16; never the full [T x V]);
- *            the workspace then also holds K-major copies of W and hidden
+ *            1: also the gradients, dhidden = D W and dW = D^T hidden.  The tokens are taken 9472 at a time;
+ *            a chunk's f32 logits and its bf16 dlogits D live in workspace scratch (never the full [T x V])
  *   dhidden  bf16 [T_max x H] out (rows at or past the true token count are zero)
- *   dW       f32 [V x H] out (overwritten, not accumulated into)
+ *   dW       [V x H] out, f32 or (params.dW_dtype = DPPO_BF16) bf16; overwritten, not accumulated into.  It is
+ *            summed over the chunks in f32 either way (for bf16 in a workspace buffer, rounded once at the end)
  *   other arguments as in dppo_grpo_loss_fwd_bwd.  The workspace (dppo_lmhead_workspace_bytes, which
  *   depends on `backward`) must be 1024-byte aligned.
  * Errors: INVALID_ARG, BAD_SHAPE (H not a multiple of 64), MISALIGNED, UNSUPPORTED, WORKSPACE_TOO_SMALL,
@@ -275,7 +275,7 @@ typedef struct {
     int32_t H;
     int32_t backward;
     int32_t variant;        /* 0: CTA pairs (cta_group::2) share each B tile; 1: one CTA per tile (tuning aid) */
-    int32_t reserved;       /* 0 */
+    int32_t dW_dtype;       /* DPPO_F32 (0) or DPPO_BF16: element type of dW */
 } dppo_lmhead_params;
 
 size_t dppo_lmhead_workspace_bytes(const dppo_lmhead_params* p);

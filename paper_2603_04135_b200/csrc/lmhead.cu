@@ -749,6 +749,20 @@ struct EpiAccumF32 {
     __device__ __forceinline__ void row_end(int, int, int) {}
 };
 
+// out (bf16) = in (f32), 8 elements per thread; n is a multiple of 8.
+__global__ void __launch_bounds__(256)
+lm_f32_to_bf16_kernel(const float* __restrict__ in, __nv_bfloat16* __restrict__ out, long long n) {
+    const long long i = ((long long)blockIdx.x * 256 + threadIdx.x) * 8;
+    if (i >= n) return;
+    const float4 a = *reinterpret_cast<const float4*>(in + i), b = *reinterpret_cast<const float4*>(in + i + 4);
+    const __nv_bfloat162 b0 = __floats2bfloat162_rn(a.x, a.y), b1 = __floats2bfloat162_rn(a.z, a.w);
+    const __nv_bfloat162 b2 = __floats2bfloat162_rn(b.x, b.y), b3 = __floats2bfloat162_rn(b.z, b.w);
+    uint4 pk;
+    pk.x = *reinterpret_cast<const uint32_t*>(&b0); pk.y = *reinterpret_cast<const uint32_t*>(&b1);
+    pk.z = *reinterpret_cast<const uint32_t*>(&b2); pk.w = *reinterpret_cast<const uint32_t*>(&b3);
+    *reinterpret_cast<uint4*>(out + i) = pk;
+}
+
 // ---- host side -----------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -857,7 +871,7 @@ static int run_gemm(bool pair, const CUtensorMap& ma, const CUtensorMap& mb, con
 static long long round_up(long long x, long long m) { return (x + m - 1) / m * m; }
 
 struct LmWorkspace {
-    size_t terms, info, part, zy, z, d, total;   // byte offsets and the total
+    size_t terms, info, part, zy, z, d, dw32, total;   // byte offsets and the total
     long long ld_v;                              // pitch of Z and D (vocabulary)
     int n_ntiles;
 };
@@ -874,10 +888,11 @@ static LmWorkspace lm_layout(const dppo_lmhead_params* p, bool backward) {
     w.info = off;  off += al((size_t)T * sizeof(RowInfo));
     w.part = off;  off += al(rows * w.n_ntiles * sizeof(float2));
     w.zy = off;    off += al(rows * sizeof(float));
-    w.z = w.d = off;
+    w.z = w.d = w.dw32 = off;
     if (backward) {
         w.z = off;  off += al(rows * w.ld_v * 4);
         w.d = off;  off += al(rows * w.ld_v * 2);
+        if (p->dW_dtype == DPPO_BF16) { w.dw32 = off; off += al((size_t)p->loss.V * p->H * 4); }   // dW is accumulated in f32
     }
     w.total = off;
     return w;
@@ -909,6 +924,7 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
         return fail(DPPO_ERR_INVALID_ARG, "lmhead: no_length_norm / seq_log_ratio");
     if (lp.T_max >= ((int64_t)1 << 31) - kChunkTokens) return fail(DPPO_ERR_BAD_SHAPE, "lmhead: T_max too large");
     if (p->variant != 0 && p->variant != 1) return fail(DPPO_ERR_INVALID_ARG, "lmhead: variant %d", p->variant);
+    if (p->dW_dtype != DPPO_F32 && p->dW_dtype != DPPO_BF16) return fail(DPPO_ERR_INVALID_ARG, "lmhead: dW_dtype %d", p->dW_dtype);
     const bool backward = p->backward != 0;
     if (backward && (!dhidden || !dW)) return fail(DPPO_ERR_INVALID_ARG, "lmhead: backward requested but dhidden / dW is NULL");
     if (!backward && (dhidden || dW)) return fail(DPPO_ERR_INVALID_ARG, "lmhead: dhidden / dW given but params.backward is 0");
@@ -957,7 +973,7 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
         if (backward) {
             rc = make_map(&map_w_mn, W, V, H, H, 64);
             if (rc != DPPO_OK) return rc;
-            rc = make_map_out(&map_dw, dW, V, H, H);
+            rc = make_map_out(&map_dw, p->dW_dtype == DPPO_BF16 ? (void*)(ws + lay.dw32) : dW, V, H, H);
             if (rc != DPPO_OK) return rc;
         }
 
@@ -1009,6 +1025,11 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
             e3.rows = V; e3.cols = H; e3.accumulate = c > 0 ? 1 : 0;
             rc = run_gemm<EpiAccumF32, true, true>(pair, map_d_mn, map_h_mn, map_h_mn, map_dw, g3, e3, status, s, "lmhead dW launch");
             if (rc != DPPO_OK) return rc;
+        }
+        if (backward && p->dW_dtype == DPPO_BF16) {
+            const long long n = (long long)V * H;
+            lm_f32_to_bf16_kernel<<<(unsigned)((n / 8 + 255) / 256), 256, 0, s>>>((const float*)(ws + lay.dw32), (__nv_bfloat16*)dW, n);
+            DPPO_CHECK_LAUNCH("lmhead dW conversion launch");
         }
     }
     return launch_loss_reduce(a, loss_out, s);

@@ -9,7 +9,7 @@ from paper_2603_04135_b200 import synth
 pytestmark = pytest.mark.gpu
 
 
-def _run(T, V, H, S, seed, n_tokens=None, tau=1.0, backward=False, variant=0):
+def _run(T, V, H, S, seed, n_tokens=None, tau=1.0, backward=False, variant=0, dW_bf16=False):
     from paper_2603_04135_b200 import binding as B
     w = synth.scaled(synth.WORKLOADS["config4_h2560"], V=V, H=H)
     hidden, W, target, lo, lr = synth.make_lmhead_inputs(w, T, seed, device="cuda")
@@ -19,12 +19,12 @@ def _run(T, V, H, S, seed, n_tokens=None, tau=1.0, backward=False, variant=0):
     cu = np.concatenate([[0], cuts, [T_true]]).astype(np.int32)
     S_real = len(cu) - 1
     adv = rng.normal(size=S_real).astype(np.float32); wseq = (rng.random(S_real) * 0.1).astype(np.float32)
-    prm = B.LmheadParams(B.LossParams(T, V, B.BF16, V, S_real, 0, w.eps, w.eps, w.beta, tau), H, int(backward), variant)
+    prm = B.LmheadParams(B.LossParams(T, V, B.BF16, V, S_real, 0, w.eps, w.eps, w.beta, tau), H, int(backward), variant, B.BF16 if dW_bf16 else B.F32)
     nbytes = B.lmhead_workspace_bytes(prm)
     ws = torch.zeros(nbytes + 1024, dtype=torch.uint8, device="cuda")
     ws = ws[(-ws.data_ptr()) % 1024:]
     dh = torch.full((T, H), 7.0, dtype=torch.bfloat16, device="cuda") if backward else None
-    dW = torch.full((V, H), 7.0, dtype=torch.float32, device="cuda") if backward else None
+    dW = torch.full((V, H), 7.0, dtype=torch.bfloat16 if dW_bf16 else torch.float32, device="cuda") if backward else None
     loss_out = torch.zeros(5, device="cuda"); logp_out = torch.zeros(T, device="cuda"); lse_out = torch.zeros(T, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     ntd = torch.tensor([T_true], dtype=torch.int32, device="cuda") if n_tokens is not None else None
@@ -58,6 +58,8 @@ def _run(T, V, H, S, seed, n_tokens=None, tau=1.0, backward=False, variant=0):
         got_dW = dW.double().cpu().numpy()
         err = np.abs(got_dW - ref["dW"])
         bound = 2.0 ** -7 * np.abs(ref["dW"]).max(axis=1, keepdims=True) + 1e-6 * gmax
+        if dW_bf16:
+            bound = bound + 2.0 ** -8 * np.abs(ref["dW"])            # one more rounding, of the f32 sum to bf16
         assert (err <= bound).all(), "dW worst ratio %.3g" % (err / bound).max()
     return ref
 
@@ -87,6 +89,11 @@ def test_lmhead_backward_small_shapes(variant):
 @pytest.mark.parametrize("variant", [1, 0])
 def test_lmhead_backward_several_token_chunks(variant):
     _run(T=9472 + 9472 + 70, V=520, H=64, S=9, seed=15, backward=True, variant=variant)   # three chunks, the last ragged
+
+
+def test_lmhead_backward_bf16_dW():
+    _run(T=300, V=777, H=192, S=5, seed=21, n_tokens=259, backward=True, dW_bf16=True)
+    _run(T=9472 + 200, V=520, H=64, S=3, seed=22, backward=True, dW_bf16=True)   # summed over two chunks in f32, rounded once
 
 
 def test_lmhead_argument_checks():
