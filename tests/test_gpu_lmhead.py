@@ -96,6 +96,67 @@ def test_lmhead_backward_bf16_dW():
     _run(T=9472 + 200, V=520, H=64, S=3, seed=22, backward=True, dW_bf16=True)   # summed over two chunks in f32, rounded once
 
 
+def test_lmhead_full_size_sampled_tokens():
+    """The size the benchmark times (99,030 tokens, V = 151,936, H = 2560, eleven token chunks, the last ragged):
+    lse, logp and dhidden of sampled tokens against the oracle (each sampled token is given to the oracle as a
+    sequence of its own carrying its sequence's advantage and w / |o|), the exact token count, zero rows of
+    dhidden nowhere, and dW on sampled vocabulary rows for consistency with a float64 contraction of the
+    library's own logp (not a parity claim: its input comes from the CUDA path)."""
+    from paper_2603_04135_b200 import binding as B
+    free, _ = torch.cuda.mem_get_info()
+    if free < 20 << 30:
+        pytest.skip("needs 20 GB of free device memory")
+    w = synth.WORKLOADS["config4_h2560"]
+    T, V, H, S, seed = 99030, w.V, w.H, 177, 31
+    hidden, W, target, lo, lr = synth.make_lmhead_inputs(w, T, seed, device="cuda")
+    rng = np.random.default_rng(seed)
+    cu = np.concatenate([[0], np.sort(rng.choice(np.arange(1, T), size=S - 1, replace=False)), [T]]).astype(np.int32)
+    adv = rng.normal(size=S).astype(np.float32); wseq = (rng.random(S) * 0.1).astype(np.float32)
+    prm = B.LmheadParams(B.LossParams(T, V, B.BF16, V, S, 0, w.eps, w.eps, w.beta, 1.0), H, 1, 0, B.F32)
+    nbytes = B.lmhead_workspace_bytes(prm)
+    ws = torch.zeros(nbytes + 1024, dtype=torch.uint8, device="cuda"); ws = ws[(-ws.data_ptr()) % 1024:]
+    dh = torch.full((T, H), 7.0, dtype=torch.bfloat16, device="cuda")
+    dW = torch.full((V, H), 7.0, dtype=torch.float32, device="cuda")
+    loss_out = torch.zeros(5, device="cuda"); logp_out = torch.zeros(T, device="cuda"); lse_out = torch.zeros(T, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B.lmhead_grpo_loss(prm, hidden, W, target, lo, lr, torch.from_numpy(cu).cuda(), None, torch.from_numpy(adv).cuda(),
+                       torch.from_numpy(wseq).cuda(), None, dh, dW, logp_out, lse_out, loss_out, ws, nbytes, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0 and loss_out[4].item() == T
+    del ws
+    # sampled tokens: around every chunk boundary, first / last of some sequences, and random ones
+    edges = [t for c in range(0, T, 9472) for t in (c - 1, c, c + 127, c + 128) if 0 <= t < T]
+    pick = np.unique(np.concatenate([edges, cu[:12], cu[1:13] - 1, [T - 1], rng.choice(T, size=64, replace=False)])).astype(np.int64)
+    seg = np.searchsorted(cu, pick, side="right") - 1
+    seg_len = (cu[seg + 1] - cu[seg]).astype(np.float64)
+    idx = torch.from_numpy(pick).cuda()
+    ref = oracle.lmhead_grpo_loss(synth.to_f64_numpy(hidden[idx]), synth.to_f64_numpy(W), target[idx].cpu().numpy(),
+                                  lo[idx].cpu().numpy(), lr[idx].cpu().numpy(), np.arange(len(pick) + 1, dtype=np.int32),
+                                  adv[seg].astype(np.float64), wseq[seg].astype(np.float64) / seg_len, w.eps, w.eps, w.beta, 1.0)
+    assert np.abs(lse_out[idx].cpu().numpy() - ref["lse"]).max() <= 1e-4
+    assert np.abs(logp_out[idx].cpu().numpy() - ref["logp"]).max() <= 1e-4
+    gmax = np.abs(ref["g"]).max()
+    err = np.abs(dh[idx].double().cpu().numpy() - ref["dhidden"])
+    bound = 2.0 ** -7 * np.abs(ref["dhidden"]).max(axis=1, keepdims=True) + 1e-6 * gmax
+    assert (err <= bound).all(), "dhidden worst ratio %.3g" % (err / bound).max()
+    assert bool((dh.float().abs().amax(dim=1) > 0).all())                      # every token got its gradient row
+    # dW on sampled vocabulary rows: sum_t g_t (1[y_t = v] - exp(z_tv - lse_t)) h_t with g from the oracle's
+    # token terms evaluated at the library's logp
+    seg_all = np.searchsorted(cu, np.arange(T), side="right") - 1
+    terms = oracle.token_terms(logp_out.cpu().numpy(), lo.cpu().numpy(), lr.cpu().numpy(), adv[seg_all], w.eps, w.eps, w.beta)
+    Wt = wseq[seg_all].astype(np.float64) / (cu[seg_all + 1] - cu[seg_all])
+    g = torch.from_numpy(-Wt * terms["dj"]).cuda()
+    vs = torch.from_numpy(np.unique(np.concatenate([[0, 1, 127, 128, 255, 256, V - 1], rng.choice(V, size=40, replace=False)]))).cuda()
+    hd = hidden.double()
+    z = hd @ W[vs].double().T                                                    # [T x |vs|]
+    D = -g[:, None] * torch.exp(z - lse_out.double()[:, None])
+    D += g[:, None] * (target.long()[:, None] == vs[None, :]).double()
+    want = (D.T @ hd).cpu().numpy()
+    got = dW[vs].double().cpu().numpy()
+    bound = 2.0 ** -7 * np.abs(want).max(axis=1, keepdims=True) + 1e-6 * float(g.abs().max())
+    assert (np.abs(got - want) <= bound).all(), "dW worst ratio %.3g" % (np.abs(got - want) / bound).max()
+
+
 def test_lmhead_argument_checks():
     from paper_2603_04135_b200 import binding as B
     z = torch.zeros(8 * 256, dtype=torch.bfloat16, device="cuda")
