@@ -19,7 +19,8 @@
 namespace dppo {
 
 constexpr int kMaxCluster = 8;
-constexpr int kChunks = 4;                    // bulk copies (and mbarriers) per slice
+constexpr int kChunks = 1;                    // bulk copies (and mbarriers) per slice: one copy of the whole slice was
+                                              // 3.5 % faster than four (fewer waits and loop prologues per row)
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // give up on a copy after 2 s
 
 struct ClusterStatic {
@@ -58,10 +59,35 @@ __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
     const __half2 h = __floats2half2_rn(lo, hi);
     return *reinterpret_cast<const uint32_t*>(&h);
 }
-// Two fp16 exponentials -> two bf16 gradient entries e * sc.
-__device__ __forceinline__ uint32_t scale_pair(uint32_t h2, float sc) {
+// Packed f32 pairs (one instruction works on both halves of a 64-bit register pair).
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pair_of(float lo, float hi) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpair(f32x2 p, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(p)); }
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+    f32x2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+    f32x2 d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+    f32x2 d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+// Two fp16 exponentials -> two bf16 gradient entries e * sc (sc2 = the scale in both halves).
+__device__ __forceinline__ uint32_t scale_pair(uint32_t h2, f32x2 sc2) {
     const float2 e = __half22float2(*reinterpret_cast<const __half2*>(&h2));
-    const __nv_bfloat162 b = __floats2bfloat162_rn(e.x * sc, e.y * sc);
+    float lo, hi;
+    unpair(mul2(pair_of(e.x, e.y), sc2), lo, hi);
+    const __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<const uint32_t*>(&b);
 }
 
@@ -69,6 +95,14 @@ __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+// One 32-bit word = two bf16 logits -> their exponentials 2^(z c - r) as an fp16 pair; acc += the two (f32).
+__device__ __forceinline__ uint32_t exp_pair(uint32_t w, f32x2 c2, f32x2 nr2, f32x2& acc) {
+    float a, b;
+    unpair(fma2(pair_of(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u)), c2, nr2), a, b);
+    const float ea = ex2(a), eb = ex2(b);
+    acc = add2(acc, pair_of(ea, eb));
+    return pack_half2(ea, eb);
 }
 
 // The cluster barrier is used once, as a start-up handshake ("my mbarriers exist"): no data rides on it.
@@ -142,7 +176,7 @@ grpo_loss_cluster_kernel(const LossArgs a, const int C, const int vec_per_cta) {
         const int b = k * chunk_vec, e = min(nv, b + chunk_vec);
         if (e > b) {
             ok = mbar_wait(smem_u32(&st.bar[k]), 0) && ok;
-#pragma unroll 4
+#pragma unroll 2
             for (int i = b + tid; i < e; i += THREADS) {
                 const uint4 q = slice[i];
                 mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&q.x));
@@ -171,21 +205,19 @@ grpo_loss_cluster_kernel(const LossArgs a, const int C, const int vec_per_cta) {
     // ---- pass 1b: sum of 2^(z c - r) over the slice
     float s = 0.0f, etail = 0.0f;
     if (nv > 0 || ztail > -INFINITY) {
-        float s0 = 0.0f, s1 = 0.0f;
+        const f32x2 c2 = pair_of(c, c), nr2 = pair_of(-r, -r);
+        f32x2 acc0 = pair_of(0.0f, 0.0f), acc1 = acc0;
 #pragma unroll 2
         for (int i = tid; i < nv; i += THREADS) {
             const uint4 q = slice[i];
-            const float e0 = ex2(fmaf(__uint_as_float(q.x << 16), c, -r)), e1 = ex2(fmaf(__uint_as_float(q.x & 0xffff0000u), c, -r));
-            const float e2 = ex2(fmaf(__uint_as_float(q.y << 16), c, -r)), e3 = ex2(fmaf(__uint_as_float(q.y & 0xffff0000u), c, -r));
-            const float e4 = ex2(fmaf(__uint_as_float(q.z << 16), c, -r)), e5 = ex2(fmaf(__uint_as_float(q.z & 0xffff0000u), c, -r));
-            const float e6 = ex2(fmaf(__uint_as_float(q.w << 16), c, -r)), e7 = ex2(fmaf(__uint_as_float(q.w & 0xffff0000u), c, -r));
-            s0 += (e0 + e2) + (e4 + e6);
-            s1 += (e1 + e3) + (e5 + e7);
             // the exponentials replace the logits in place, as fp16 pairs: the second pass needs no exp
             uint4 h;
-            h.x = pack_half2(e0, e1); h.y = pack_half2(e2, e3); h.z = pack_half2(e4, e5); h.w = pack_half2(e6, e7);
+            h.x = exp_pair(q.x, c2, nr2, acc0); h.y = exp_pair(q.y, c2, nr2, acc1);
+            h.z = exp_pair(q.z, c2, nr2, acc0); h.w = exp_pair(q.w, c2, nr2, acc1);
             slice[i] = h;
         }
+        float s0, s1;
+        unpair(add2(acc0, acc1), s0, s1);
         s = s0 + s1;
         if (ztail > -INFINITY) { etail = ex2(fmaf(ztail, c, -r)); s += etail; }
     }
@@ -244,14 +276,15 @@ grpo_loss_cluster_kernel(const LossArgs a, const int C, const int vec_per_cta) {
         const float ng = rs.valid ? -rs.g_over_tau : 0.0f;
         // softmax = e * 2^(r - lse2) with e relative to this CTA's reference r
         const float sc = ng * ex2((r - rs.lse2_hi) - rs.lse2_lo);
+        const f32x2 sc2 = pair_of(sc, sc);
         const int y = rs.valid ? a.target[t] : -1;
         const int yvec = (y >= 0 ? (y >> 3) : -1) - v0;     // vector of the target relative to this slice
-#pragma unroll 4
+#pragma unroll 2
         for (int i = tid; i < nv; i += THREADS) {
             const uint4 q = slice[i];
             uint4 o;
-            o.x = scale_pair(q.x, sc); o.y = scale_pair(q.y, sc);
-            o.z = scale_pair(q.z, sc); o.w = scale_pair(q.w, sc);
+            o.x = scale_pair(q.x, sc2); o.y = scale_pair(q.y, sc2);
+            o.z = scale_pair(q.z, sc2); o.w = scale_pair(q.w, sc2);
             __stcs(dst + i, o);
         }
         // the one element that also carries the onehot term: the thread that stored its vector redoes it
