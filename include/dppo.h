@@ -263,8 +263,10 @@ int dppo_sequence_log_ratio(const float* logp, const float* logp_old, const int3
  *            1: also the gradients, dhidden = D W and dW = D^T hidden.  The tokens are taken 9472 at a time;
  *            a chunk's f32 logits and its bf16 dlogits D live in workspace scratch (never the full [T x V])
  *   dhidden  bf16 [T_max x H] out (rows at or past the true token count are zero)
- *   dW       [V x H] out, f32 or (params.dW_dtype = DPPO_BF16) bf16; overwritten, not accumulated into.  It is
- *            summed over the chunks in f32 either way (for bf16 in a workspace buffer, rounded once at the end)
+ *   dW       [V x H] out, f32 or (params.dW_dtype = DPPO_BF16) bf16; overwritten, or added to when
+ *            params.accumulate_dW = 1.  It is summed over the chunks in f32 either way (for bf16 in a workspace
+ *            buffer, rounded once at the end).  Each element receives one add per chunk, in stream order: the
+ *            result does not vary from run to run
  *   other arguments as in dppo_grpo_loss_fwd_bwd.  The workspace (dppo_lmhead_workspace_bytes, which
  *   depends on `backward`) must be 1024-byte aligned.
  * Errors: INVALID_ARG, BAD_SHAPE (H not a multiple of 64), MISALIGNED, UNSUPPORTED, WORKSPACE_TOO_SMALL,
@@ -276,6 +278,8 @@ typedef struct {
     int32_t backward;
     int32_t variant;        /* 0: CTA pairs (cta_group::2) share each B tile; 1: one CTA per tile (tuning aid) */
     int32_t dW_dtype;       /* DPPO_F32 (0) or DPPO_BF16: element type of dW */
+    int32_t accumulate_dW;  /* 0: dW is overwritten; 1: the gradient is added to what dW holds (micro-batches) */
+    int32_t reserved;       /* 0 */
 } dppo_lmhead_params;
 
 size_t dppo_lmhead_workspace_bytes(const dppo_lmhead_params* p);

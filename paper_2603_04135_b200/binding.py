@@ -48,7 +48,8 @@ class LossParams(ctypes.Structure):
 
 class LmheadParams(ctypes.Structure):
     _fields_ = [("loss", LossParams), ("H", ctypes.c_int32), ("backward", ctypes.c_int32), ("variant", ctypes.c_int32),
-                ("dW_dtype", ctypes.c_int32)]
+                ("dW_dtype", ctypes.c_int32),
+                ("accumulate_dW", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
 _vp = ctypes.c_void_p

@@ -763,6 +763,18 @@ lm_f32_to_bf16_kernel(const float* __restrict__ in, __nv_bfloat16* __restrict__ 
     *reinterpret_cast<uint4*>(out + i) = pk;
 }
 
+// out (f32) = in (bf16), 8 elements per thread; n is a multiple of 8.
+__global__ void __launch_bounds__(256)
+lm_bf16_to_f32_kernel(const __nv_bfloat16* __restrict__ in, float* __restrict__ out, long long n) {
+    const long long i = ((long long)blockIdx.x * 256 + threadIdx.x) * 8;
+    if (i >= n) return;
+    const uint4 q = *reinterpret_cast<const uint4*>(in + i);
+    *reinterpret_cast<float4*>(out + i) = make_float4(__uint_as_float(q.x << 16), __uint_as_float(q.x & 0xffff0000u),
+                                                       __uint_as_float(q.y << 16), __uint_as_float(q.y & 0xffff0000u));
+    *reinterpret_cast<float4*>(out + i + 4) = make_float4(__uint_as_float(q.z << 16), __uint_as_float(q.z & 0xffff0000u),
+                                                           __uint_as_float(q.w << 16), __uint_as_float(q.w & 0xffff0000u));
+}
+
 // ---- host side -----------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -925,6 +937,8 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
     if (lp.T_max >= ((int64_t)1 << 31) - kChunkTokens) return fail(DPPO_ERR_BAD_SHAPE, "lmhead: T_max too large");
     if (p->variant != 0 && p->variant != 1) return fail(DPPO_ERR_INVALID_ARG, "lmhead: variant %d", p->variant);
     if (p->dW_dtype != DPPO_F32 && p->dW_dtype != DPPO_BF16) return fail(DPPO_ERR_INVALID_ARG, "lmhead: dW_dtype %d", p->dW_dtype);
+    if ((p->accumulate_dW != 0 && p->accumulate_dW != 1) || p->reserved != 0)
+        return fail(DPPO_ERR_INVALID_ARG, "lmhead: accumulate_dW %d reserved %d", p->accumulate_dW, p->reserved);
     const bool backward = p->backward != 0;
     if (backward && (!dhidden || !dW)) return fail(DPPO_ERR_INVALID_ARG, "lmhead: backward requested but dhidden / dW is NULL");
     if (!backward && (dhidden || dW)) return fail(DPPO_ERR_INVALID_ARG, "lmhead: dhidden / dW given but params.backward is 0");
@@ -975,6 +989,11 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
             if (rc != DPPO_OK) return rc;
             rc = make_map_out(&map_dw, p->dW_dtype == DPPO_BF16 ? (void*)(ws + lay.dw32) : dW, V, H, H);
             if (rc != DPPO_OK) return rc;
+            if (p->accumulate_dW && p->dW_dtype == DPPO_BF16) {        // the f32 sum starts from the caller's bf16 dW
+                const long long n = (long long)V * H;
+                lm_bf16_to_f32_kernel<<<(unsigned)((n / 8 + 255) / 256), 256, 0, s>>>((const __nv_bfloat16*)dW, (float*)(ws + lay.dw32), n);
+                DPPO_CHECK_LAUNCH("lmhead dW conversion launch");
+            }
         }
 
         for (long long t0 = 0, c = 0; t0 < T; t0 += kChunkTokens, ++c) {
@@ -1022,7 +1041,7 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
             GemmShape g3 = {};
             g3.n_mtiles = (V + kBM - 1) / kBM; g3.n_ntiles = (H + kBN - 1) / kBN; g3.n_ksteps = (int)((tc + kBK - 1) / kBK);
             EpiAccumF32 e3 = {};
-            e3.rows = V; e3.cols = H; e3.accumulate = c > 0 ? 1 : 0;
+            e3.rows = V; e3.cols = H; e3.accumulate = (c > 0 || p->accumulate_dW) ? 1 : 0;
             rc = run_gemm<EpiAccumF32, true, true>(pair, map_d_mn, map_h_mn, map_h_mn, map_dw, g3, e3, status, s, "lmhead dW launch");
             if (rc != DPPO_OK) return rc;
         }

@@ -39,6 +39,7 @@ def test_struct_layouts_match_header(B):
     assert ctypes.sizeof(B.PruneParams) == 48
     assert ctypes.sizeof(B.PackParams) == 16
     assert ctypes.sizeof(B.LossParams) == 80 and B.LossParams.seq_log_ratio.offset == 72
+    assert ctypes.sizeof(B.LmheadParams) == 104 and B.LmheadParams.dW_dtype.offset == 92
     assert B.LossParams.row_stride.offset == 16 and B.LossParams.eps_lo.offset == 32
 
 

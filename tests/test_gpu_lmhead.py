@@ -96,6 +96,39 @@ def test_lmhead_backward_bf16_dW():
     _run(T=9472 + 200, V=520, H=64, S=3, seed=22, backward=True, dW_bf16=True)   # summed over two chunks in f32, rounded once
 
 
+@pytest.mark.parametrize("dW_bf16", [False, True])
+def test_lmhead_accumulate_dW(dW_bf16):
+    """accumulate_dW = 1 adds the gradient to what dW holds: a second call on the first call's result gives twice
+    the oracle's dW (dhidden is overwritten both times)."""
+    from paper_2603_04135_b200 import binding as B
+    T, V, H, S, seed = 9472 + 300, 520, 64, 4, 41
+    w = synth.scaled(synth.WORKLOADS["config4_h2560"], V=V, H=H)
+    hidden, W, target, lo, lr = synth.make_lmhead_inputs(w, T, seed, device="cuda")
+    rng = np.random.default_rng(seed)
+    cu = np.concatenate([[0], np.sort(rng.choice(np.arange(1, T), size=S - 1, replace=False)), [T]]).astype(np.int32)
+    adv = rng.normal(size=S).astype(np.float32); wseq = (rng.random(S) * 0.1).astype(np.float32)
+    dh = torch.zeros((T, H), dtype=torch.bfloat16, device="cuda")
+    dW = torch.full((V, H), 7.0, dtype=torch.bfloat16 if dW_bf16 else torch.float32, device="cuda")
+    loss_out = torch.zeros(5, device="cuda"); status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for acc in (0, 1):
+        prm = B.LmheadParams(B.LossParams(T, V, B.BF16, V, S, 0, w.eps, w.eps, w.beta, 1.0), H, 1, 0,
+                             B.BF16 if dW_bf16 else B.F32, acc)
+        nbytes = B.lmhead_workspace_bytes(prm)
+        ws = torch.zeros(nbytes + 1024, dtype=torch.uint8, device="cuda"); ws = ws[(-ws.data_ptr()) % 1024:]
+        B.lmhead_grpo_loss(prm, hidden, W, target, lo, lr, torch.from_numpy(cu).cuda(), None, torch.from_numpy(adv).cuda(),
+                           torch.from_numpy(wseq).cuda(), None, dh, dW, None, None, loss_out, ws, nbytes, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    ref = oracle.lmhead_grpo_loss(synth.to_f64_numpy(hidden), synth.to_f64_numpy(W), target.cpu().numpy(), lo.cpu().numpy(),
+                                  lr.cpu().numpy(), cu, adv, wseq, w.eps, w.eps, w.beta, 1.0)
+    want = 2.0 * ref["dW"]
+    bound = 2.0 * (2.0 ** -7 * np.abs(ref["dW"]).max(axis=1, keepdims=True) + 1e-6 * np.abs(ref["g"]).max())
+    if dW_bf16:
+        bound = bound + 2.0 ** -7 * np.abs(want)                 # the intermediate and the final rounding to bf16
+    err = np.abs(dW.double().cpu().numpy() - want)
+    assert (err <= bound).all(), "dW worst ratio %.3g" % (err / bound).max()
+
+
 def test_lmhead_full_size_sampled_tokens():
     """The size the benchmark times (99,030 tokens, V = 151,936, H = 2560, eleven token chunks, the last ragged):
     lse, logp and dhidden of sampled tokens against the oracle (each sampled token is given to the oracle as a
