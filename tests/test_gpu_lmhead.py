@@ -129,6 +129,61 @@ def test_lmhead_accumulate_dW(dW_bf16):
     assert (err <= bound).all(), "dW worst ratio %.3g" % (err / bound).max()
 
 
+@pytest.mark.parametrize("H", [2560, 4096])
+def test_config4_whole_path(H):
+    """The fused LM-head configuration end to end at a size the oracle finishes: advantages -> pruning with
+    probabilities 0.5 / 0.5 -> packing -> fused LM-head + loss driven by the packer's cu_seqlens, placement order
+    and device-side token count, over the full vocabulary and both hidden widths, forward and backward."""
+    from paper_2603_04135_b200 import binding as B
+    from paper_2603_04135_b200.step import DppoStep
+    from parity_util import oracle_prune_pack, assert_prune_equal, assert_pack_equal
+    V = 151936 if H == 2560 else 32768                      # the oracle's float64 dW is V x H: keep the wider case small
+    w = synth.scaled(synth.WORKLOADS["config4_h%d" % H], P=4, G=8, resp_len=("uniform", 4, 24), L_row=128, N_win=4, V=V)
+    seed = 4
+    batch = synth.make_batch(w, seed)
+    ref = oracle_prune_pack(batch, w, seed, step=2)
+    pk = ref["pack"]
+    T = pk["counts"][3]
+    assert 60 <= T <= 500
+    T_cap = int(batch.loss_len.sum())                        # buffers sized for the unpruned batch
+    st = DppoStep(w.P, w.G, w.L_row, w.N_win, w.r_q, w.r_o, w.V, w.dtype, T_cap, w.eps, w.eps, w.beta)
+    st.set_batch(batch.rewards, batch.unit_len, batch.loss_len, ref["H_prev"])
+    st.prune_pack(seed=seed, step=2)
+    assert_prune_equal(st.prune_results(), ref)
+    assert_pack_equal(st.pack_results(), pk, w.P * w.G)
+
+    hidden, W, target, lo, lr = synth.make_lmhead_inputs(w, T_cap, seed, device="cuda")
+    prm = B.LmheadParams(B.LossParams(T_cap, w.V, B.BF16, w.V, w.P * w.G, 0, w.eps, w.eps, w.beta, 1.0), H, 1, 0, B.F32)
+    nbytes = B.lmhead_workspace_bytes(prm)
+    ws = torch.zeros(nbytes + 1024, dtype=torch.uint8, device="cuda"); ws = ws[(-ws.data_ptr()) % 1024:]
+    dh = torch.full((T_cap, H), 7.0, dtype=torch.bfloat16, device="cuda")
+    dW = torch.full((w.V, H), 7.0, dtype=torch.float32, device="cuda")
+    B.lmhead_grpo_loss(prm, hidden, W, target, lo, lr, st.cu_seqlens, st.counts[3:4], st.adv, st.w_seq, st.order,
+                       dh, dW, st.logp_out, st.lse_out, st.loss_out, ws, nbytes, st.status)
+    torch.cuda.synchronize()
+    assert st.status.item() == 0
+
+    order = np.asarray(pk["order"], dtype=np.int64)
+    want = oracle.lmhead_grpo_loss(synth.to_f64_numpy(hidden[:T]), synth.to_f64_numpy(W), target.cpu().numpy()[:T],
+                                   lo.cpu().numpy()[:T], lr.cpu().numpy()[:T], np.asarray(pk["cu_seqlens"]),
+                                   ref["adv"].reshape(-1)[order], ref["prune"]["w_seq"].reshape(-1)[order],
+                                   w.eps, w.eps, w.beta, 1.0)
+    got = st.loss_out.cpu().numpy().astype(np.float64)
+    assert got[4] == T
+    assert np.abs(st.lse_out.cpu().numpy()[:T] - want["lse"]).max() <= 1e-4
+    assert np.abs(st.logp_out.cpu().numpy()[:T] - want["logp"]).max() <= 1e-4
+    assert abs(got[0] - want["loss"]) <= 1e-4 * want["abs_sum"]
+    gmax = np.abs(want["g"]).max()
+    got_dh = dh.double().cpu().numpy()
+    assert (got_dh[T:] == 0).all()                           # rows beyond the retained tokens are cleared
+    err = np.abs(got_dh[:T] - want["dhidden"])
+    bound = 2.0 ** -7 * np.abs(want["dhidden"]).max(axis=1, keepdims=True) + 1e-6 * gmax
+    assert (err <= bound).all(), "dhidden worst ratio %.3g" % (err / bound).max()
+    err = np.abs(dW.double().cpu().numpy() - want["dW"])
+    bound = 2.0 ** -7 * np.abs(want["dW"]).max(axis=1, keepdims=True) + 1e-6 * gmax
+    assert (err <= bound).all(), "dW worst ratio %.3g" % (err / bound).max()
+
+
 def test_lmhead_full_size_sampled_tokens():
     """The size the benchmark times (99,030 tokens, V = 151,936, H = 2560, eleven token chunks, the last ragged):
     lse, logp and dhidden of sampled tokens against the oracle (each sampled token is given to the oracle as a
