@@ -13,9 +13,10 @@
 namespace dppo {
 
 // ---- kernel choice for variant 0 (from measurements on B200 at V = 151,936) --------------------------
-constexpr int kClusterMinV = 16384;                 // shorter rows: the general kernel's second pass hits L1/L2
+constexpr size_t kClusterMinRowBytes = 32768;       // shorter rows: the general kernel's second pass hits L1/L2
 constexpr int kClusterAuto = 4;                     // smallest cluster tried first
 constexpr int kClusterThreads = 256;
+constexpr int kClusterThreadsF32 = 128;             // half the arithmetic per byte: fewer threads do (5.6 against 5.4 TB/s)
 constexpr size_t kClusterMaxSlice = 76 * 1024;      // slice bytes per CTA: keeps three CTAs resident per SM
 
 // ---- general kernel --------------------------------------------------------------------------------
@@ -259,10 +260,10 @@ extern "C" int dppo_grpo_loss_fwd_bwd(const dppo_loss_params* p, const void* log
             rc = launch_rows_cluster(a, p->variant / 10000, p->variant % 10000, s);
         } else {
             rc = DPPO_ERR_UNSUPPORTED;
-            if (a.bf16 && p->V >= kClusterMinV) {
-                const int nvec = p->V >> 3;
+            if ((size_t)p->V * esize >= kClusterMinRowBytes) {
+                const int nvec = p->V >> (a.bf16 ? 3 : 2);
                 for (int C = kClusterAuto; C <= 8 && rc == DPPO_ERR_UNSUPPORTED; C *= 2)
-                    if ((size_t)((nvec + C - 1) / C) * 16 <= kClusterMaxSlice) rc = launch_rows_cluster(a, C, kClusterThreads, s);
+                    if ((size_t)((nvec + C - 1) / C) * 16 <= kClusterMaxSlice) rc = launch_rows_cluster(a, C, a.bf16 ? kClusterThreads : kClusterThreadsF32, s);
             }
             if (rc == DPPO_ERR_UNSUPPORTED) rc = launch_rows_general(a, s);
         }

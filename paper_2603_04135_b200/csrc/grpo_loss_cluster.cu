@@ -11,6 +11,9 @@
 // second pass is a scale-and-convert with no exp: one MUFU op per element in total.  Several CTAs
 // per SM sit in different phases (copy in flight / reducing / storing), which is what overlaps the
 // memory system with the exp work.
+//
+// f32 rows take the same path with 4-element vectors: the exponentials replace the logits in place as f32
+// (same size, nothing to pack) and dlogits leave as f32; a full-vocabulary f32 row (594 KB) needs a cluster of 8.
 #include <cuda_fp16.h>
 
 #include "common.cuh"
@@ -105,6 +108,28 @@ __device__ __forceinline__ uint32_t exp_pair(uint32_t w, f32x2 c2, f32x2 nr2, f3
     return pack_half2(ea, eb);
 }
 
+// f32 rows: one 16-byte vector = four logits -> their exponentials 2^(z c - r), in place; acc += the four.
+__device__ __forceinline__ uint4 exp_quad(uint4 q, f32x2 c2, f32x2 nr2, f32x2& acc0, f32x2& acc1) {
+    float a, b, e0, e1;
+    unpair(fma2(pair_of(__uint_as_float(q.x), __uint_as_float(q.y)), c2, nr2), a, b);
+    e0 = ex2(a); e1 = ex2(b);
+    acc0 = add2(acc0, pair_of(e0, e1));
+    q.x = __float_as_uint(e0); q.y = __float_as_uint(e1);
+    unpair(fma2(pair_of(__uint_as_float(q.z), __uint_as_float(q.w)), c2, nr2), a, b);
+    e0 = ex2(a); e1 = ex2(b);
+    acc1 = add2(acc1, pair_of(e0, e1));
+    q.z = __float_as_uint(e0); q.w = __float_as_uint(e1);
+    return q;
+}
+__device__ __forceinline__ uint4 scale_quad(uint4 q, f32x2 sc2) {
+    float a, b;
+    unpair(mul2(pair_of(__uint_as_float(q.x), __uint_as_float(q.y)), sc2), a, b);
+    q.x = __float_as_uint(a); q.y = __float_as_uint(b);
+    unpair(mul2(pair_of(__uint_as_float(q.z), __uint_as_float(q.w)), sc2), a, b);
+    q.z = __float_as_uint(a); q.w = __float_as_uint(b);
+    return q;
+}
+
 // The cluster barrier is used once, as a start-up handshake ("my mbarriers exist"): no data rides on it.
 __device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.aligned;" ::: "memory"); }
@@ -118,9 +143,11 @@ __device__ __forceinline__ void remote_store_signal(uint32_t local_slot, uint32_
                  :: "r"(rslot), "l"(v), "r"(rbar) : "memory");
 }
 
-template <int THREADS>
+template <int THREADS, bool kF32>
 __global__ void __launch_bounds__(THREADS)
 grpo_loss_cluster_kernel(const LossArgs a, const int C, const int vec_per_cta) {
+    constexpr int kLog2PerVec = kF32 ? 2 : 3;               // elements per 16-byte vector: 4 f32 or 8 bf16
+    constexpr int kPerVec = 1 << kLog2PerVec;
     extern __shared__ __align__(128) unsigned char slice_raw[];
     __shared__ ClusterStatic st;
     uint4* slice = reinterpret_cast<uint4*>(slice_raw);
@@ -131,7 +158,7 @@ grpo_loss_cluster_kernel(const LossArgs a, const int C, const int vec_per_cta) {
     const long long T = a.n_tokens_dev ? min((long long)*a.n_tokens_dev, a.T_max) : a.T_max;
     if (t >= T) return;                                     // uniform over the cluster: nobody reaches a barrier
 
-    const int nvec = a.V >> 3;                              // whole 16-byte vectors of the row
+    const int nvec = a.V >> kLog2PerVec;                    // whole 16-byte vectors of the row
     const int v0 = rank * vec_per_cta;
     const int nv = max(0, min(vec_per_cta, nvec - v0));     // vectors of this CTA's slice
     const int chunk_vec = (nv + kChunks - 1) / kChunks;
@@ -170,6 +197,7 @@ grpo_loss_cluster_kernel(const LossArgs a, const int C, const int vec_per_cta) {
 
     // ---- pass 1a: slice maximum (packed bf16 max), chunk by chunk as the copies land
     __nv_bfloat162 mx2 = __float2bfloat162_rn(-INFINITY);
+    float mxa = -INFINITY, mxb = -INFINITY;
     bool ok = true;
 #pragma unroll
     for (int k = 0; k < kChunks; ++k) {
@@ -179,20 +207,25 @@ grpo_loss_cluster_kernel(const LossArgs a, const int C, const int vec_per_cta) {
 #pragma unroll 2
             for (int i = b + tid; i < e; i += THREADS) {
                 const uint4 q = slice[i];
-                mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&q.x));
-                mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&q.y));
-                mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&q.z));
-                mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&q.w));
+                if constexpr (kF32) {
+                    mxa = fmaxf(mxa, fmaxf(__uint_as_float(q.x), __uint_as_float(q.y)));
+                    mxb = fmaxf(mxb, fmaxf(__uint_as_float(q.z), __uint_as_float(q.w)));
+                } else {
+                    mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&q.x));
+                    mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&q.y));
+                    mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&q.z));
+                    mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&q.w));
+                }
             }
         }
     }
     if (!ok) st.failed = 1;                                 // benign race: every writer stores 1
-    float m = fmaxf(__low2float(mx2), __high2float(mx2));
+    float m = kF32 ? fmaxf(mxa, mxb) : fmaxf(__low2float(mx2), __high2float(mx2));
     // the row's ragged tail (V % 8 elements) belongs to the last CTA and is read from global memory
-    const int tail0 = nvec << 3;
+    const int tail0 = nvec << kLog2PerVec;
     float ztail = -INFINITY;
     if (rank == C - 1 && tail0 + tid < a.V) {
-        ztail = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(row)[tail0 + tid]);
+        ztail = Elems<!kF32>::load1(row, tail0 + tid);
         m = fmaxf(m, ztail);
     }
     m = warp_max(m);
@@ -210,10 +243,14 @@ grpo_loss_cluster_kernel(const LossArgs a, const int C, const int vec_per_cta) {
 #pragma unroll 2
         for (int i = tid; i < nv; i += THREADS) {
             const uint4 q = slice[i];
-            // the exponentials replace the logits in place, as fp16 pairs: the second pass needs no exp
+            // the exponentials replace the logits in place (bf16 rows: as fp16 pairs): the second pass needs no exp
             uint4 h;
-            h.x = exp_pair(q.x, c2, nr2, acc0); h.y = exp_pair(q.y, c2, nr2, acc1);
-            h.z = exp_pair(q.z, c2, nr2, acc0); h.w = exp_pair(q.w, c2, nr2, acc1);
+            if constexpr (kF32) {
+                h = exp_quad(q, c2, nr2, acc0, acc1);
+            } else {
+                h.x = exp_pair(q.x, c2, nr2, acc0); h.y = exp_pair(q.y, c2, nr2, acc1);
+                h.z = exp_pair(q.z, c2, nr2, acc0); h.w = exp_pair(q.w, c2, nr2, acc1);
+            }
             slice[i] = h;
         }
         float s0, s1;
@@ -278,33 +315,42 @@ grpo_loss_cluster_kernel(const LossArgs a, const int C, const int vec_per_cta) {
         const float sc = ng * ex2((r - rs.lse2_hi) - rs.lse2_lo);
         const f32x2 sc2 = pair_of(sc, sc);
         const int y = rs.valid ? a.target[t] : -1;
-        const int yvec = (y >= 0 ? (y >> 3) : -1) - v0;     // vector of the target relative to this slice
+        const int yvec = (y >= 0 ? (y >> kLog2PerVec) : -1) - v0;   // vector of the target relative to this slice
 #pragma unroll 2
         for (int i = tid; i < nv; i += THREADS) {
             const uint4 q = slice[i];
             uint4 o;
-            o.x = scale_pair(q.x, sc2); o.y = scale_pair(q.y, sc2);
-            o.z = scale_pair(q.z, sc2); o.w = scale_pair(q.w, sc2);
+            if constexpr (kF32) {
+                o = scale_quad(q, sc2);
+            } else {
+                o.x = scale_pair(q.x, sc2); o.y = scale_pair(q.y, sc2);
+                o.z = scale_pair(q.z, sc2); o.w = scale_pair(q.w, sc2);
+            }
             __stcs(dst + i, o);
         }
         // the one element that also carries the onehot term: the thread that stored its vector redoes it
         if (yvec >= 0 && yvec < nv && (yvec % THREADS) == tid) {
-            const uint32_t word = reinterpret_cast<const uint32_t*>(slice + yvec)[(y & 7) >> 1];
-            const float2 e = __half22float2(*reinterpret_cast<const __half2*>(&word));
-            const float ey = (y & 1) ? e.y : e.x;
-            reinterpret_cast<__nv_bfloat16*>(drow)[y] = __float2bfloat16_rn(fmaf(ey, sc, -ng));
+            if constexpr (kF32) {
+                const float ey = reinterpret_cast<const float*>(slice + yvec)[y & 3];
+                reinterpret_cast<float*>(drow)[y] = fmaf(ey, sc, -ng);
+            } else {
+                const uint32_t word = reinterpret_cast<const uint32_t*>(slice + yvec)[(y & 7) >> 1];
+                const float2 e = __half22float2(*reinterpret_cast<const __half2*>(&word));
+                const float ey = (y & 1) ? e.y : e.x;
+                reinterpret_cast<__nv_bfloat16*>(drow)[y] = __float2bfloat16_rn(fmaf(ey, sc, -ng));
+            }
         }
         if (rank == C - 1 && tail0 + tid < a.V) {
             const int v = tail0 + tid;
-            reinterpret_cast<__nv_bfloat16*>(drow)[v] = __float2bfloat16_rn(sc * etail - (v == y ? ng : 0.0f));
+            Elems<!kF32>::store1(drow, v, sc * etail - (v == y ? ng : 0.0f));
         }
     }
 }
 
 // ---- host side ---------------------------------------------------------------------------------------
-template <int THREADS>
+template <int THREADS, bool kF32>
 static int launch_cluster_t(const LossArgs& a, int C, int vec_per_cta, size_t dyn_bytes, cudaStream_t s) {
-    auto kernel = grpo_loss_cluster_kernel<THREADS>;
+    auto kernel = grpo_loss_cluster_kernel<THREADS, kF32>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_bytes);
     if (e != cudaSuccess) { cudaGetLastError(); return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: %zu bytes of shared memory refused", dyn_bytes); }
     cudaLaunchConfig_t cfg = {};
@@ -325,20 +371,29 @@ static int launch_cluster_t(const LossArgs& a, int C, int vec_per_cta, size_t dy
 }
 
 int launch_rows_cluster(const LossArgs& a, int C, int threads, cudaStream_t s) {
-    if (!a.bf16) return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: bf16 rows only");
     if (C != 2 && C != 4 && C != 8) return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: cluster size %d", C);
-    if ((a.V & 7) >= threads) return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: tail");
+    const int log2_per_vec = a.bf16 ? 3 : 2;
+    if ((a.V & ((1 << log2_per_vec) - 1)) >= threads) return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: tail");
     if (a.T_max * C >= (1ll << 31)) return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: grid too large");
-    const int nvec = a.V >> 3;
+    const int nvec = a.V >> log2_per_vec;
     const int vec_per_cta = (nvec + C - 1) / C;
     const size_t dyn_bytes = (size_t)(vec_per_cta > 0 ? vec_per_cta : 1) * 16;
     if (dyn_bytes > 220 * 1024) return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: slice of %zu bytes exceeds shared memory", dyn_bytes);
     if (dyn_bytes / kChunks + 16 >= (1u << 20)) return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: chunk too large");
-    switch (threads) {
-        case 128: return launch_cluster_t<128>(a, C, vec_per_cta, dyn_bytes, s);
-        case 256: return launch_cluster_t<256>(a, C, vec_per_cta, dyn_bytes, s);
-        case 512: return launch_cluster_t<512>(a, C, vec_per_cta, dyn_bytes, s);
-        case 1024: return launch_cluster_t<1024>(a, C, vec_per_cta, dyn_bytes, s);
+    if (a.bf16) {
+        switch (threads) {
+            case 128: return launch_cluster_t<128, false>(a, C, vec_per_cta, dyn_bytes, s);
+            case 256: return launch_cluster_t<256, false>(a, C, vec_per_cta, dyn_bytes, s);
+            case 512: return launch_cluster_t<512, false>(a, C, vec_per_cta, dyn_bytes, s);
+            case 1024: return launch_cluster_t<1024, false>(a, C, vec_per_cta, dyn_bytes, s);
+        }
+    } else {
+        switch (threads) {
+            case 128: return launch_cluster_t<128, true>(a, C, vec_per_cta, dyn_bytes, s);
+            case 256: return launch_cluster_t<256, true>(a, C, vec_per_cta, dyn_bytes, s);
+            case 512: return launch_cluster_t<512, true>(a, C, vec_per_cta, dyn_bytes, s);
+            case 1024: return launch_cluster_t<1024, true>(a, C, vec_per_cta, dyn_bytes, s);
+        }
     }
     return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: %d threads", threads);
 }

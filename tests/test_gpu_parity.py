@@ -331,11 +331,32 @@ def test_loss_cluster_kernel_variants(C):
     _loss_case(65536, "bf16", T=700, S=7, seed=61, variant=v)
 
 
+@pytest.mark.parametrize("C", [2, 4, 8])
+def test_loss_cluster_kernel_f32_rows(C):
+    # the same kernel on f32 rows (4-element vectors, f32 exponentials in place, f32 dlogits)
+    v = C * 10000 + 256
+    if C >= 4:
+        for threads in (128, 256, 512):
+            _loss_case(151936, "f32", T=11, S=3, seed=140 + C, variant=C * 10000 + threads)
+        _loss_case(151936 - 5, "f32", T=7, S=2, seed=150 + C, variant=v, pad=1)         # tail of 3 elements, padded stride
+        _loss_case(151936, "f32", T=9, S=2, seed=151 + C, variant=v, in_place=True)
+        _loss_case(151936, "f32", T=9, S=2, seed=153 + C, variant=v, n_tokens=5, tau=1.3)
+    _loss_case(65536, "f32", T=40, S=4, seed=152 + C, variant=v, forward_only=True)
+    _loss_case(4099, "f32", T=33, S=4, seed=154 + C, variant=v)
+    _loss_case(12, "f32", T=33, S=4, seed=155 + C, variant=v)                           # 3 vectors: most slices are empty
+    _loss_case(3, "f32", T=20, S=2, seed=156 + C, variant=v)                            # tail only
+    _loss_case(65536, "f32", T=200, S=7, seed=157 + C, variant=v, sigma_noise=0.3)
+    _loss_case(1024, "f32", T=40, S=3, seed=158 + C, variant=v, logit_sigma=40.0, centre_on_oracle=True)
+
+
 def test_loss_auto_dispatch_matches_forced_kernels():
     # variant 0 on a long bf16 row takes the cluster kernel; outputs agree with the general kernel's
     a = _loss_case(151936, "bf16", T=11, S=2, seed=60, variant=0)
     b = _loss_case(151936, "bf16", T=11, S=2, seed=60, variant=1)
     assert a["loss"] == b["loss"]                                                # same oracle case both times
+    _loss_case(151936, "f32", T=11, S=2, seed=61, variant=0)                     # f32: cluster of 8
+    _loss_case(151936, "f32", T=11, S=2, seed=61, variant=1)
+    _loss_case(40000, "f32", T=30, S=2, seed=62, variant=0)                      # f32: cluster of 4
 
 
 def test_loss_wide_dynamic_range():
