@@ -40,8 +40,8 @@ WORKLOAD_TEXT = WORKLOAD + ": P=32 G=8, response 64-1024 tokens, V=151936 bf16 l
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch over 8192 rows of this vocabulary.  Traffic
 # grows in proportion to the rows, so a launch over T rows moves T times the per-row figure.  The record
 # is tied to the kernel sources it was taken from: once they change, `traffic` is reported as null.
-TRAFFIC_CAPTURE = {"rows": 8192, "dram_bytes": 2489447000 + 2431674000,
-                   "source_sha256": "fe76e9147401febb14965f4ac6ab9757a923f31946c68319afc3105a0fbd9641"}
+TRAFFIC_CAPTURE = {"rows": 8192, "dram_bytes": 2489492000 + 2431635000,
+                   "source_sha256": "5721e4e06dc57767a99e0d57761c440ba557d4fe4253af4ab08d0946f5a0e33c"}
 
 
 def captured_traffic_per_row():
