@@ -238,7 +238,10 @@ grpo_loss_cluster_kernel(const LossArgs a, const int C, const int vec_per_cta) {
     // ---- pass 1b: sum of 2^(z c - r) over the slice
     float s = 0.0f, etail = 0.0f;
     if (nv > 0 || ztail > -INFINITY) {
-        const f32x2 c2 = pair_of(c, c), nr2 = pair_of(-r, -r);
+        // a slice of nothing but -inf (a masked part of the vocabulary) has r = -inf: any finite offset gives its
+        // exponentials the value 0 they must have, where -r would give NaN
+        const float nr = r > -INFINITY ? -r : 0.0f;
+        const f32x2 c2 = pair_of(c, c), nr2 = pair_of(nr, nr);
         f32x2 acc0 = pair_of(0.0f, 0.0f), acc1 = acc0;
 #pragma unroll 2
         for (int i = tid; i < nv; i += THREADS) {

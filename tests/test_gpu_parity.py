@@ -178,7 +178,7 @@ def test_pack_dataset_scale_and_bad_length():
 # ------------------------------------------------------------------------------------------- steps 6-8
 def _loss_case(V, dtype, T, S, seed, sigma_noise=0.05, logit_sigma=2.0, tau=1.0, pad=0, in_place=False,
                forward_only=False, n_tokens=None, beta=0.04, eps=(0.2, 0.2), variant=0, no_length_norm=False,
-               seq_ratio=False, centre_on_oracle=False):
+               seq_ratio=False, centre_on_oracle=False, neg_inf_cols=None):
     """Runs dppo_grpo_loss_fwd_bwd on a random case and compares everything with the oracle.
     centre_on_oracle: old / reference log-probs = the oracle's current log-prob + noise (for logits whose
     log-sum-exp is far from the Gaussian closed form the generator centres on)."""
@@ -186,6 +186,13 @@ def _loss_case(V, dtype, T, S, seed, sigma_noise=0.05, logit_sigma=2.0, tau=1.0,
     w = synth.scaled(synth.WORKLOADS["config0"], V=V, dtype=dtype, logit_sigma=logit_sigma)
     tok = synth.make_token_inputs(w, T, seed, device="cuda", sigma_old=sigma_noise, sigma_ref=2 * sigma_noise)
     rng = np.random.default_rng(seed)
+    if neg_inf_cols is not None:
+        # a masked part of the vocabulary: logits of -inf (probability zero), never sampled
+        lo_c, hi_c = neg_inf_cols
+        tok.logits[:, lo_c:hi_c] = float("-inf")
+        hit = (tok.target >= lo_c) & (tok.target < hi_c)
+        tok.target[hit] = 0 if lo_c > 0 else hi_c
+        centre_on_oracle = True
     if centre_on_oracle:
         lp = oracle.token_logprob(tok.logits.to(torch.float64).cpu().numpy(), tok.target.cpu().numpy(), tau)[0]
         tok.logp_old = torch.from_numpy((lp + sigma_noise * rng.normal(size=T)).astype(np.float32)).cuda()
@@ -366,6 +373,19 @@ def test_loss_wide_dynamic_range():
     _loss_case(151936, "bf16", T=8, S=2, seed=91, logit_sigma=30.0, variant=1, centre_on_oracle=True)
     _loss_case(1024, "f32", T=40, S=3, seed=92, logit_sigma=40.0, centre_on_oracle=True)
     _loss_case(4099, "bf16", T=40, S=3, seed=93, logit_sigma=0.0)                # every logit equal: lse = ln V
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_loss_masked_vocabulary(dtype):
+    # -inf logits: a few columns, a whole slice of the cluster kernel (37,984 elements of a bf16 row over 4 CTAs,
+    # 18,992 of an f32 row over 8), the padded end of the vocabulary
+    V = 151936
+    _loss_case(V, dtype, T=6, S=2, seed=201, neg_inf_cols=(1000, 3000))
+    _loss_case(V, dtype, T=6, S=2, seed=202, neg_inf_cols=(37984, 75968))
+    _loss_case(V, dtype, T=6, S=2, seed=203, neg_inf_cols=(0, 37984))
+    _loss_case(V, dtype, T=6, S=2, seed=204, neg_inf_cols=(151669, V))
+    _loss_case(V, dtype, T=6, S=2, seed=205, neg_inf_cols=(37984, 75968), variant=1)
+    _loss_case(4099, dtype, T=20, S=2, seed=206, neg_inf_cols=(100, 4099))
 
 
 @pytest.mark.parametrize("variant", [0, 1])
