@@ -261,7 +261,7 @@ int dppo_sequence_log_ratio(const float* logp, const float* logp_old, const int3
  *   W        bf16 [V x H] row-major LM-head weight
  *   backward 0: forward only (loss_out, logp_out, lse_out; dhidden and dW must be NULL).
  *            1: also the gradients, dhidden = D W and dW = D^T hidden.  The tokens are taken 9472 at a time;
- *            a chunk's f32 logits and its bf16 dlogits D live in workspace scratch (never the full [T x V])
+ *            a chunk's exponentials (fp16) and its bf16 dlogits D live in workspace scratch (never the full [T x V])
  *   dhidden  bf16 [T_max x H] out (rows at or past the true token count are zero)
  *   dW       [V x H] out, f32 or (params.dW_dtype = DPPO_BF16) bf16; overwritten, or added to when
  *            params.accumulate_dW = 1.  It is summed over the chunks in f32 either way (for bf16 in a workspace

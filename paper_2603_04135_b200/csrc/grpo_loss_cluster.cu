@@ -147,7 +147,6 @@ template <int THREADS, bool kF32>
 __global__ void __launch_bounds__(THREADS)
 grpo_loss_cluster_kernel(const LossArgs a, const int C, const int vec_per_cta) {
     constexpr int kLog2PerVec = kF32 ? 2 : 3;               // elements per 16-byte vector: 4 f32 or 8 bf16
-    constexpr int kPerVec = 1 << kLog2PerVec;
     extern __shared__ __align__(128) unsigned char slice_raw[];
     __shared__ ClusterStatic st;
     uint4* slice = reinterpret_cast<uint4*>(slice_raw);

@@ -3,15 +3,18 @@
 // The call walks over the tokens in chunks.  Per chunk:
 //   logits    z = hidden W^T, tile by tile (tcgen05.mma, accumulators in tensor memory).  As each 128 x 256
 //             tile leaves TMEM its per-row (max, sum of exponentials) and the sampled token's logit are kept;
-//             a backward pass also keeps the chunk's f32 logits in a bounded scratch (the [T x V] logits of
-//             the whole batch never exist; Eq. 1's pi_theta(o_t | ...) is a log-softmax of exactly these)
+//             a backward pass also keeps the exponentials themselves, relative to the tile's row maxima, as
+//             fp16 in a bounded scratch (the [T x V] logits never exist in memory, not even for one chunk;
+//             Eq. 1's pi_theta(o_t | ...) is a log-softmax of exactly these f32 accumulators)
 //   rows      one warp per token joins the tile partials into the log-sum-exp and runs the loss's scalar stage
-//   dlogits   D = g (onehot - softmax)/tau of the chunk from the stored logits, as bf16, both ways round
+//   dlogits   D = g (onehot - softmax)/tau of the chunk as bf16: the stored exponentials times one factor per
+//             (token, tile), no second exp
 //   dhidden = D W and dW += D^T hidden: two more runs of the same GEMM core over the chunk
 //
-// One GEMM core serves all three contractions; operands are always K-major (transposed copies of W and
-// hidden are made once per call), only the epilogue differs.  One persistent CTA per SM:
-//   warp 0      TMA producer: 64-wide K slabs of A (128 rows) and of B (256 rows), 128B-swizzled, into
+// One GEMM core serves all three contractions; an operand is K-major or MN-major as stored (W, hidden and D
+// are never copied transposed), only the epilogue differs.  One persistent CTA per SM, by default paired with
+// its neighbour (cta_group::2, see lm_gemm2_kernel); in the single-CTA form:
+//   warp 0      TMA producer: 64-deep K slabs of A (128 rows) and of B (256 rows), 128B-swizzled, into
 //               a 4-stage shared-memory ring (every CTA fetches its own operands)
 //   warp 1      one thread issues tcgen05.mma (M=128, N=256, K=16 x 4 per slab) into one of two
 //               256-column TMEM accumulators; tcgen05.commit releases smem stages / publishes the tile
@@ -20,6 +23,7 @@
 // Every wait is bounded; on a timeout the CTA records DPPO_STATUS_TIMEOUT, leaves its loops, frees its
 // tensor memory and returns.
 #include <cuda.h>
+#include <cuda_fp16.h>
 
 #include "common.cuh"
 #include "grpo_loss.cuh"
@@ -195,6 +199,44 @@ __device__ __forceinline__ void lm_store_block(EpiCtx& ctx, const uint32_t (&v)[
     ctx.toggle ^= 1u;
 }
 
+// The same staging for 2-byte elements: a block of 32 rows x 64 fp16 (again rows of 128 bytes) is filled in two
+// halves, 32 columns each (h = this lane's row of the half, 16 words of two fp16); the second half sends it.
+__device__ __forceinline__ void lm_store_half_block(EpiCtx& ctx, const uint32_t (&h)[16], int half, int x, int y) {
+    if (half == 0) {
+        if (ctx.lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");   // the buffer filled two blocks ago has been read
+        __syncwarp();
+    }
+    const uint32_t buf = ctx.stage + ctx.toggle * kStageTileBytes;
+    const uint32_t rowp = buf + (uint32_t)ctx.lane * 128u;
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                     :: "r"(rowp + (uint32_t)(((4 * half + j) ^ (ctx.lane & 7)) << 4)), "r"(h[4 * j]), "r"(h[4 * j + 1]), "r"(h[4 * j + 2]), "r"(h[4 * j + 3])
+                     : "memory");
+    if (half == 0) return;
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncwarp();
+    if (ctx.lane == 0) {
+        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
+                     :: "l"(ctx.map_c), "r"(buf), "r"(x), "r"(y) : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    }
+    ctx.toggle ^= 1u;
+}
+
+// 32 consecutive f32 columns of this thread's TMEM lane (its tile row) into registers.
+__device__ __forceinline__ void lm_tmem_load32(uint32_t (&v)[32], uint32_t taddr) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                   "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+                   "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+                   "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                 : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
 // ---- the GEMM core --------------------------------------------------------------------------------
 // Epi (one copy per epilogue thread = per tile row), called for every tile:
 //   void row_begin(int m, int n, int row)
@@ -321,18 +363,18 @@ lm_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (!__all_sync(0xffffffffu, lm_wait(lm_smem_u32(&sh.acc_full[b]), use_b & 1, abort_flag))) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + b * kBN;
+            if constexpr (Epi::kTwoPass) {                               // a first look at the whole tile (its row maxima)
+#pragma unroll 1
+                for (int ch = 0; ch < kBN / 32; ++ch) {
+                    uint32_t v[32];
+                    lm_tmem_load32(v, taddr + (uint32_t)(ch * 32));
+                    epi.scan(m, n, row, ch, v);
+                }
+            }
 #pragma unroll 1
             for (int ch = 0; ch < kBN / 32; ++ch) {
                 uint32_t v[32];
-                asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-                             "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-                             "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-                             : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-                               "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-                               "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-                               "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-                             : "r"(taddr + (uint32_t)(ch * 32)) : "memory");
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                lm_tmem_load32(v, taddr + (uint32_t)(ch * 32));
                 epi.chunk(m, n, row, ch, v, ctx);
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -511,18 +553,18 @@ lm_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             if (!__all_sync(0xffffffffu, lm_wait(lm_smem_u32(&sh.acc_full[b]), use_b & 1, abort_flag))) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + b * kBN;
+            if constexpr (Epi::kTwoPass) {                               // a first look at the whole tile (its row maxima)
+#pragma unroll 1
+                for (int ch = 0; ch < kBN / 32; ++ch) {
+                    uint32_t v[32];
+                    lm_tmem_load32(v, taddr + (uint32_t)(ch * 32));
+                    epi.scan(m, n, row, ch, v);
+                }
+            }
 #pragma unroll 1
             for (int ch = 0; ch < kBN / 32; ++ch) {
                 uint32_t v[32];
-                asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-                             "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-                             "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-                             : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-                               "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-                               "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-                               "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-                             : "r"(taddr + (uint32_t)(ch * 32)) : "memory");
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                lm_tmem_load32(v, taddr + (uint32_t)(ch * 32));
                 epi.chunk(m, n, row, ch, v, ctx);
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -553,13 +595,12 @@ struct RowInfo {             // what the backward needs from the forward, per to
 };
 
 // Forward, one chunk of tokens: each 128 x 256 logits tile leaves behind, per token row, the tile's
-// (max, sum 2^(x - max)) of x = z * scale2, the sampled token's logit if it lies in the tile, and (for a
-// backward pass) the f32 logits themselves in a chunk-sized scratch.  The tiles of a row are combined
-// by lm_rows_kernel.
+// (max, sum 2^(x - max)) of x = z * scale2 and the sampled token's logit if it lies in the tile.  The tiles of a
+// row are combined by lm_rows_kernel.  This form keeps nothing else (forward-only calls).
 struct EpiPartial {
+    static constexpr bool kTwoPass = false;
     float2* part;            // [chunk tokens x n_ntiles]
     float* zy_out;           // [chunk tokens]
-    int store_z;             // the kernel's output map is Z [chunk tokens x V] f32: keep the logits
     const int32_t* target;
     const int32_t* n_tokens_dev;
     long long T_max, t0, tc;
@@ -579,10 +620,7 @@ struct EpiPartial {
     __device__ __forceinline__ void chunk(int m, int n, int row, int ch, uint32_t (&v)[32], EpiCtx& ctx) {
         const int col0 = n * kBN + ch * 32;
         const int valid = V - col0;                                  // columns of this chunk inside the vocabulary
-        if (valid <= 0) return;                                      // the same for the whole warp
-        const int y0 = m * kBM + row - ctx.lane;                     // first row of this warp's block
-        if (store_z && y0 < tc) lm_store_block<false>(ctx, v, col0, y0);   // clipped at V and at the chunk's last row
-        if (!live) return;
+        if (valid <= 0 || !live) return;
         const int yrel = y - col0;                                   // selects, not an indexed read: v stays in registers
         hit = hit || (yrel >= 0 && yrel < 32);
         float cm = -INFINITY;
@@ -607,6 +645,76 @@ struct EpiPartial {
         if (!live) return;
         const long long r = (long long)m * kBM + row;
         part[r * n_ntiles + n] = make_float2(m2, s);
+        if (hit) zy_out[r] = zy;
+    }
+};
+
+// The same for a call with a backward pass: the tile is read out of tensor memory twice.  The first look takes
+// each row's maximum over the tile's 256 columns (and picks up the sampled token's logit); the second forms the
+// exponentials e = 2^(x - max) ONCE, adds them up for the log-sum-exp and keeps them, as fp16, in a chunk-sized
+// scratch E [chunk tokens x V]: softmax = e * 2^(max - lse2), so the backward scales them (no second exp) and
+// the f32 logits are never written out.  e lies in (0, 1]; fp16 keeps 11 bits of it down to 2^-14 of the tile's
+// largest term, far below what the bf16 dlogits resolve.
+struct EpiPartialExp {
+    static constexpr bool kTwoPass = true;
+    float2* part;            // [chunk tokens x n_ntiles]
+    float* zy_out;           // [chunk tokens]
+    const int32_t* target;
+    const int32_t* n_tokens_dev;
+    long long T_max, t0, tc;
+    int V, n_ntiles;
+    float c;
+    // per-thread state
+    float mraw, s, zy;
+    int y;
+    bool live, hit;
+    __device__ __forceinline__ void row_begin(int m, int, int row) {
+        const long long T = n_tokens_dev ? min((long long)*n_tokens_dev, T_max) : T_max;
+        const long long r = (long long)m * kBM + row;
+        live = r < tc && t0 + r < T;
+        y = live ? target[t0 + r] : -1;
+        mraw = -INFINITY; s = 0.0f; zy = 0.0f; hit = false;
+    }
+    __device__ __forceinline__ void scan(int, int n, int, int ch, const uint32_t (&v)[32]) {
+        const int col0 = n * kBN + ch * 32;
+        const int valid = V - col0;
+        if (valid <= 0) return;
+        const int yrel = y - col0;
+        hit = hit || (yrel >= 0 && yrel < 32);
+        float a0 = -INFINITY, a1 = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < 32; j += 2) {
+            const float r0 = __uint_as_float(v[j]), r1 = __uint_as_float(v[j + 1]);
+            zy = (j == yrel) ? r0 : zy;
+            zy = (j + 1 == yrel) ? r1 : zy;
+            a0 = fmaxf(a0, (j < valid) ? r0 : -INFINITY);
+            a1 = fmaxf(a1, (j + 1 < valid) ? r1 : -INFINITY);
+        }
+        mraw = fmaxf(mraw, fmaxf(a0, a1));
+    }
+    __device__ __forceinline__ void chunk(int m, int n, int row, int ch, uint32_t (&v)[32], EpiCtx& ctx) {
+        const int col0 = n * kBN + ch * 32;
+        const int valid = V - col0;
+        const int y0 = m * kBM + row - ctx.lane;                     // first row of this warp's block
+        if (y0 >= tc || V - (col0 & ~63) <= 0) return;               // nothing of this 64-column block exists (whole warp)
+        const float nm2 = -(mraw * c);                               // c > 0: the maximum of x = raw * c is mraw * c
+        uint32_t h[16];
+        float acc0 = 0.0f, acc1 = 0.0f;
+#pragma unroll
+        for (int j = 0; j < 32; j += 2) {
+            const float e0 = (j < valid) ? lm_ex2(fmaf(__uint_as_float(v[j]), c, nm2)) : 0.0f;
+            const float e1 = (j + 1 < valid) ? lm_ex2(fmaf(__uint_as_float(v[j + 1]), c, nm2)) : 0.0f;
+            acc0 += e0; acc1 += e1;
+            const __half2 p = __floats2half2_rn(e0, e1);
+            h[j >> 1] = *reinterpret_cast<const uint32_t*>(&p);
+        }
+        s += acc0 + acc1;
+        lm_store_half_block(ctx, h, ch & 1, col0 & ~63, y0);        // clipped at V and at the chunk's last row
+    }
+    __device__ __forceinline__ void row_end(int m, int n, int row) {
+        if (!live) return;
+        const long long r = (long long)m * kBM + row;
+        part[r * n_ntiles + n] = make_float2(mraw * c, s);
         if (hit) zy_out[r] = zy;
     }
 };
@@ -654,15 +762,16 @@ lm_rows_kernel(const LossArgs a, const float2* __restrict__ part, const float* _
     }
 }
 
-// Backward, step 1: dlogits of the chunk from its stored logits, D = g (onehot - softmax) / tau, as bf16
-// [chunk tokens x ldd].  Both later contractions read this one copy: dhidden = D W takes it K-major, dW = D^T
-// hidden takes it MN-major.  Rows with g = 0 (no token, bad target) are written as zeros without reading
-// their logits.  One thread per 8 vocabulary entries of a row.
+// Backward, step 1: dlogits of the chunk from the stored exponentials, D = g (onehot - softmax) / tau with
+// softmax = e * 2^(tile max - lse2), as bf16 [chunk tokens x ldd].  Both later contractions read this one copy:
+// dhidden = D W takes it K-major, dW = D^T hidden takes it MN-major.  Rows with g = 0 (no token, bad target) are
+// written as zeros without reading their exponentials.  One thread per 8 vocabulary entries of a row (8 divides
+// the tile width, so a thread's entries share one tile maximum).
 constexpr int kDlogitsThreads = 256;
 
 __global__ void __launch_bounds__(kDlogitsThreads)
-lm_dlogits_kernel(const float* __restrict__ Z, long long ldz, const RowInfo* __restrict__ info, long long t0,
-                  int V, float c, __nv_bfloat16* __restrict__ D, long long ldd) {
+lm_dlogits_kernel(const __half* __restrict__ E, long long lde, const float2* __restrict__ part, int n_ntiles,
+                  const RowInfo* __restrict__ info, long long t0, int V, __nv_bfloat16* __restrict__ D, long long ldd) {
     const long long r = blockIdx.y;
     const int col = (blockIdx.x * kDlogitsThreads + threadIdx.x) * 8;
     if (col >= V) return;
@@ -672,17 +781,19 @@ lm_dlogits_kernel(const float* __restrict__ Z, long long ldz, const RowInfo* __r
 #pragma unroll
     for (int j = 0; j < 8; ++j) d[j] = 0.0f;
     __nv_bfloat16* dst = D + r * ldd + col;
-    if (col + 8 <= V) {                                              // ldz, ldd and col are multiples of 8
+    float f = 0.0f;                                                  // g * 2^(tile max - lse2)
+    if (g != 0.0f) f = g * lm_ex2((part[r * n_ntiles + col / kBN].x - ri.lse2_hi) - ri.lse2_lo);
+    if (col + 8 <= V) {                                              // lde, ldd and col are multiples of 8
         if (g != 0.0f) {
-            const float4 q0 = *reinterpret_cast<const float4*>(Z + r * ldz + col);
-            const float4 q1 = *reinterpret_cast<const float4*>(Z + r * ldz + col + 4);
-            const float z[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+            const uint4 q = *reinterpret_cast<const uint4*>(E + r * lde + col);
+            const float2 e0 = __half22float2(*reinterpret_cast<const __half2*>(&q.x));
+            const float2 e1 = __half22float2(*reinterpret_cast<const __half2*>(&q.y));
+            const float2 e2 = __half22float2(*reinterpret_cast<const __half2*>(&q.z));
+            const float2 e3 = __half22float2(*reinterpret_cast<const __half2*>(&q.w));
+            const float e[8] = {e0.x, e0.y, e1.x, e1.y, e2.x, e2.y, e3.x, e3.y};
             const int yrel = ri.y - col;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const float p = lm_ex2(fmaf(z[j], c, -ri.lse2_hi) - ri.lse2_lo);
-                d[j] = -g * p + ((j == yrel) ? g : 0.0f);
-            }
+            for (int j = 0; j < 8; ++j) d[j] = fmaf(-f, e[j], (j == yrel) ? g : 0.0f);
         }
         const __nv_bfloat162 b0 = __floats2bfloat162_rn(d[0], d[1]), b1 = __floats2bfloat162_rn(d[2], d[3]);
         const __nv_bfloat162 b2 = __floats2bfloat162_rn(d[4], d[5]), b3 = __floats2bfloat162_rn(d[6], d[7]);
@@ -693,10 +804,7 @@ lm_dlogits_kernel(const float* __restrict__ Z, long long ldz, const RowInfo* __r
     } else {
         for (int j = 0; col + j < V; ++j) {
             float dj = 0.0f;
-            if (g != 0.0f) {
-                const float p = lm_ex2(fmaf(Z[r * ldz + col + j], c, -ri.lse2_hi) - ri.lse2_lo);
-                dj = -g * p + ((col + j == ri.y) ? g : 0.0f);
-            }
+            if (g != 0.0f) dj = fmaf(-f, __half2float(E[r * lde + col + j]), (col + j == ri.y) ? g : 0.0f);
             dst[j] = __float2bfloat16_rn(dj);
         }
     }
@@ -704,6 +812,7 @@ lm_dlogits_kernel(const float* __restrict__ Z, long long ldz, const RowInfo* __r
 
 // C[rows x ldc] = acc as bf16 (dhidden).
 struct EpiStoreBf16 {
+    static constexpr bool kTwoPass = false;
     __nv_bfloat16* C;
     long long ldc, row0, rows;   // output row of tile row 0; rows that exist in C
     int cols;
@@ -736,6 +845,7 @@ struct EpiStoreBf16 {
 // C (f32, the tensor behind the kernel's output map) = or += acc (dW, accumulated over the token chunks; the
 // add is done by the memory system, nothing is read back).
 struct EpiAccumF32 {
+    static constexpr bool kTwoPass = false;
     long long rows;
     int cols, accumulate;
     __device__ __forceinline__ void row_begin(int, int, int) {}
@@ -824,6 +934,22 @@ static int make_map_out(CUtensorMap* map, const void* base, long long rows, long
     return DPPO_OK;
 }
 
+// fp16 [rows x cols] with row pitch ld elements as the target of the half-block stores: boxes of 64 columns x 32
+// rows (128-byte rows), 128B swizzle.
+static int make_map_out_f16(CUtensorMap* map, const void* base, long long rows, long long cols, long long ld) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return fail(DPPO_ERR_CUDA, "lmhead: cuTensorMapEncodeTiled is not available from this driver");
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    const cuuint32_t box[2] = {64, 32};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(DPPO_ERR_CUDA, "lmhead: cuTensorMapEncodeTiled (exponentials) failed with %d", (int)r);
+    return DPPO_OK;
+}
+
 constexpr size_t kLmDynSmem = (size_t)kStages * kStageBytes + kStageBytesEpi + 1024;
 
 template <class Epi, bool kAMn, bool kBMn>
@@ -884,7 +1010,7 @@ static long long round_up(long long x, long long m) { return (x + m - 1) / m * m
 
 struct LmWorkspace {
     size_t terms, info, part, zy, z, d, dw32, total;   // byte offsets and the total
-    long long ld_v;                              // pitch of Z and D (vocabulary)
+    long long ld_v;                              // pitch of E and D (vocabulary)
     int n_ntiles;
 };
 
@@ -902,7 +1028,7 @@ static LmWorkspace lm_layout(const dppo_lmhead_params* p, bool backward) {
     w.zy = off;    off += al(rows * sizeof(float));
     w.z = w.d = w.dw32 = off;
     if (backward) {
-        w.z = off;  off += al(rows * w.ld_v * 4);
+        w.z = off;  off += al(rows * w.ld_v * 2);
         w.d = off;  off += al(rows * w.ld_v * 2);
         if (p->dW_dtype == DPPO_BF16) { w.dw32 = off; off += al((size_t)p->loss.V * p->H * 4); }   // dW is accumulated in f32
     }
@@ -980,7 +1106,7 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
         RowInfo* info = (RowInfo*)(ws + lay.info);
         float2* part = (float2*)(ws + lay.part);
         float* zy = (float*)(ws + lay.zy);
-        float* Z = backward ? (float*)(ws + lay.z) : nullptr;
+        __half* E = backward ? (__half*)(ws + lay.z) : nullptr;
         __nv_bfloat16* D = (__nv_bfloat16*)(ws + lay.d);
         alignas(64) CUtensorMap map_w_mn;                                              // W as [K = V][N = H]
         alignas(64) CUtensorMap map_dw;
@@ -999,19 +1125,24 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
         for (long long t0 = 0, c = 0; t0 < T; t0 += kChunkTokens, ++c) {
             const long long tc = (T - t0) < kChunkTokens ? (T - t0) : kChunkTokens;     // tokens in this chunk
             // (1) logits of the chunk, tile by tile: per-tile (max, sum) of every row, z[y], and (backward) the
-            //     f32 logits into Z [tc x V]
+            //     exponentials relative to the tile maxima, as fp16, into E [tc x V]
             GemmShape g1 = {};
             g1.n_mtiles = (int)((tc + kBM - 1) / kBM); g1.n_ntiles = lay.n_ntiles; g1.n_ksteps = H / kBK;
             g1.a_row0 = (int)t0; g1.m_fast = 1;                                        // neighbours share the W tile
-            EpiPartial e1 = {};
-            e1.part = part; e1.zy_out = zy; e1.store_z = backward ? 1 : 0; e1.target = target; e1.n_tokens_dev = n_tokens_dev;
-            e1.T_max = T; e1.t0 = t0; e1.tc = tc; e1.V = V; e1.n_ntiles = lay.n_ntiles; e1.c = a.scale2;
-            alignas(64) CUtensorMap map_z = map_h;
             if (backward) {
-                rc = make_map_out(&map_z, Z, tc, V, lay.ld_v);
+                EpiPartialExp e1 = {};
+                e1.part = part; e1.zy_out = zy; e1.target = target; e1.n_tokens_dev = n_tokens_dev;
+                e1.T_max = T; e1.t0 = t0; e1.tc = tc; e1.V = V; e1.n_ntiles = lay.n_ntiles; e1.c = a.scale2;
+                alignas(64) CUtensorMap map_e;
+                rc = make_map_out_f16(&map_e, E, tc, V, lay.ld_v);
                 if (rc != DPPO_OK) return rc;
+                rc = run_gemm<EpiPartialExp, false, false>(pair, map_h, map_w, map_w_half, map_e, g1, e1, status, s, "lmhead logits launch");
+            } else {
+                EpiPartial e1 = {};
+                e1.part = part; e1.zy_out = zy; e1.target = target; e1.n_tokens_dev = n_tokens_dev;
+                e1.T_max = T; e1.t0 = t0; e1.tc = tc; e1.V = V; e1.n_ntiles = lay.n_ntiles; e1.c = a.scale2;
+                rc = run_gemm<EpiPartial, false, false>(pair, map_h, map_w, map_w_half, map_h, g1, e1, status, s, "lmhead logits launch");
             }
-            rc = run_gemm<EpiPartial, false, false>(pair, map_h, map_w, map_w_half, map_z, g1, e1, status, s, "lmhead logits launch");
             if (rc != DPPO_OK) return rc;
             // (2) rows: log-sum-exp, logp, loss terms, dloss/dlogp
             lm_rows_kernel<<<(unsigned)((tc + kRowsWarps - 1) / kRowsWarps), kRowsWarps * 32, 0, s>>>(
@@ -1020,7 +1151,7 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
             if (!backward) continue;
             // (3) dlogits of the chunk: D [tc x V]
             lm_dlogits_kernel<<<dim3((unsigned)((V + 8 * kDlogitsThreads - 1) / (8 * kDlogitsThreads)), (unsigned)tc),
-                                kDlogitsThreads, 0, s>>>(Z, lay.ld_v, info, t0, V, a.scale2, D, lay.ld_v);
+                                kDlogitsThreads, 0, s>>>(E, lay.ld_v, part, lay.n_ntiles, info, t0, V, D, lay.ld_v);
             DPPO_CHECK_LAUNCH("lmhead dlogits launch");
             // (4) dhidden[t0 : t0+tc, :] = D W            (M = tokens, N = H, K = V; D K-major, W MN-major)
             alignas(64) CUtensorMap map_d, map_d_mn, map_h_mn;
