@@ -768,44 +768,60 @@ lm_rows_kernel(const LossArgs a, const float2* __restrict__ part, const float* _
 // written as zeros without reading their exponentials.  One thread per 8 vocabulary entries of a row (8 divides
 // the tile width, so a thread's entries share one tile maximum).
 constexpr int kDlogitsThreads = 256;
+constexpr int kDlogitsVecs = 4;              // 16-byte vectors per thread, a block's width apart: their loads overlap
+
+__device__ __forceinline__ uint4 lm_dlogits_vec(uint4 q, float f, float g, int yrel) {
+    const float2 e0 = __half22float2(*reinterpret_cast<const __half2*>(&q.x));
+    const float2 e1 = __half22float2(*reinterpret_cast<const __half2*>(&q.y));
+    const float2 e2 = __half22float2(*reinterpret_cast<const __half2*>(&q.z));
+    const float2 e3 = __half22float2(*reinterpret_cast<const __half2*>(&q.w));
+    const float e[8] = {e0.x, e0.y, e1.x, e1.y, e2.x, e2.y, e3.x, e3.y};
+    float d[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) d[j] = fmaf(-f, e[j], (j == yrel) ? g : 0.0f);
+    const __nv_bfloat162 b0 = __floats2bfloat162_rn(d[0], d[1]), b1 = __floats2bfloat162_rn(d[2], d[3]);
+    const __nv_bfloat162 b2 = __floats2bfloat162_rn(d[4], d[5]), b3 = __floats2bfloat162_rn(d[6], d[7]);
+    uint4 pk;
+    pk.x = *reinterpret_cast<const uint32_t*>(&b0); pk.y = *reinterpret_cast<const uint32_t*>(&b1);
+    pk.z = *reinterpret_cast<const uint32_t*>(&b2); pk.w = *reinterpret_cast<const uint32_t*>(&b3);
+    return pk;
+}
 
 __global__ void __launch_bounds__(kDlogitsThreads)
 lm_dlogits_kernel(const __half* __restrict__ E, long long lde, const float2* __restrict__ part, int n_ntiles,
                   const RowInfo* __restrict__ info, long long t0, int V, __nv_bfloat16* __restrict__ D, long long ldd) {
     const long long r = blockIdx.y;
-    const int col = (blockIdx.x * kDlogitsThreads + threadIdx.x) * 8;
-    if (col >= V) return;
+    const int col0 = (blockIdx.x * kDlogitsVecs * kDlogitsThreads + threadIdx.x) * 8;
     const RowInfo ri = info[t0 + r];
     const float g = ri.g_over_tau;
-    float d[8];
+    const __half* erow = E + r * lde;
+    __nv_bfloat16* drow = D + r * ldd;
+    uint4 q[kDlogitsVecs];
+    float mx[kDlogitsVecs];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) d[j] = 0.0f;
-    __nv_bfloat16* dst = D + r * ldd + col;
-    float f = 0.0f;                                                  // g * 2^(tile max - lse2)
-    if (g != 0.0f) f = g * lm_ex2((part[r * n_ntiles + col / kBN].x - ri.lse2_hi) - ri.lse2_lo);
-    if (col + 8 <= V) {                                              // lde, ldd and col are multiples of 8
-        if (g != 0.0f) {
-            const uint4 q = *reinterpret_cast<const uint4*>(E + r * lde + col);
-            const float2 e0 = __half22float2(*reinterpret_cast<const __half2*>(&q.x));
-            const float2 e1 = __half22float2(*reinterpret_cast<const __half2*>(&q.y));
-            const float2 e2 = __half22float2(*reinterpret_cast<const __half2*>(&q.z));
-            const float2 e3 = __half22float2(*reinterpret_cast<const __half2*>(&q.w));
-            const float e[8] = {e0.x, e0.y, e1.x, e1.y, e2.x, e2.y, e3.x, e3.y};
-            const int yrel = ri.y - col;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) d[j] = fmaf(-f, e[j], (j == yrel) ? g : 0.0f);
+    for (int i = 0; i < kDlogitsVecs; ++i) {                         // lde, ldd and the columns are multiples of 8
+        const int col = col0 + i * kDlogitsThreads * 8;
+        q[i] = make_uint4(0u, 0u, 0u, 0u);
+        mx[i] = 0.0f;
+        if (g != 0.0f && col + 8 <= V) {
+            q[i] = __ldcs(reinterpret_cast<const uint4*>(erow + col));
+            mx[i] = part[r * n_ntiles + col / kBN].x;                // the same tile for the whole warp
         }
-        const __nv_bfloat162 b0 = __floats2bfloat162_rn(d[0], d[1]), b1 = __floats2bfloat162_rn(d[2], d[3]);
-        const __nv_bfloat162 b2 = __floats2bfloat162_rn(d[4], d[5]), b3 = __floats2bfloat162_rn(d[6], d[7]);
-        uint4 pk;
-        pk.x = *reinterpret_cast<const uint32_t*>(&b0); pk.y = *reinterpret_cast<const uint32_t*>(&b1);
-        pk.z = *reinterpret_cast<const uint32_t*>(&b2); pk.w = *reinterpret_cast<const uint32_t*>(&b3);
-        *reinterpret_cast<uint4*>(dst) = pk;
-    } else {
-        for (int j = 0; col + j < V; ++j) {
-            float dj = 0.0f;
-            if (g != 0.0f) dj = fmaf(-f, __half2float(E[r * lde + col + j]), (col + j == ri.y) ? g : 0.0f);
-            dst[j] = __float2bfloat16_rn(dj);
+    }
+#pragma unroll
+    for (int i = 0; i < kDlogitsVecs; ++i) {
+        const int col = col0 + i * kDlogitsThreads * 8;
+        if (col >= V) break;
+        const float f = g != 0.0f ? g * lm_ex2((mx[i] - ri.lse2_hi) - ri.lse2_lo) : 0.0f;   // g * 2^(tile max - lse2)
+        if (col + 8 <= V) {
+            *reinterpret_cast<uint4*>(drow + col) = lm_dlogits_vec(q[i], f, g, ri.y - col);
+        } else {                                                     // the row's ragged end, element by element
+            const float ft = g != 0.0f ? g * lm_ex2((part[r * n_ntiles + col / kBN].x - ri.lse2_hi) - ri.lse2_lo) : 0.0f;
+            for (int j = 0; col + j < V; ++j) {
+                float dj = 0.0f;
+                if (g != 0.0f) dj = fmaf(-ft, __half2float(erow[col + j]), (col + j == ri.y) ? g : 0.0f);
+                drow[col + j] = __float2bfloat16_rn(dj);
+            }
         }
     }
 }
@@ -1150,7 +1166,7 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
             DPPO_CHECK_LAUNCH("lmhead rows launch");
             if (!backward) continue;
             // (3) dlogits of the chunk: D [tc x V]
-            lm_dlogits_kernel<<<dim3((unsigned)((V + 8 * kDlogitsThreads - 1) / (8 * kDlogitsThreads)), (unsigned)tc),
+            lm_dlogits_kernel<<<dim3((unsigned)((V + 8 * kDlogitsVecs * kDlogitsThreads - 1) / (8 * kDlogitsVecs * kDlogitsThreads)), (unsigned)tc),
                                 kDlogitsThreads, 0, s>>>(E, lay.ld_v, part, lay.n_ntiles, info, t0, V, D, lay.ld_v);
             DPPO_CHECK_LAUNCH("lmhead dlogits launch");
             // (4) dhidden[t0 : t0+tc, :] = D W            (M = tokens, N = H, K = V; D K-major, W MN-major)
