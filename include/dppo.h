@@ -21,6 +21,8 @@
  *    are recorded in the caller's `status` word (device int32, first error wins, caller zeroes it)
  *    as a positive dppo_status; the kernel then finishes without trapping.
  *  - Every output is a deterministic function of the inputs (no floating-point atomics).
+ *  - Each entry point that enqueues work opens an NVTX range of its own name around its host side, so
+ *    its launches are grouped under it in a timeline profiler.
  */
 #ifndef DPPO_H_
 #define DPPO_H_

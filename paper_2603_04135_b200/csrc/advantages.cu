@@ -46,6 +46,7 @@ __global__ void group_advantages_kernel(const float* __restrict__ rewards, int P
 
 extern "C" int dppo_group_advantages(const float* rewards, int P, int G, int std_ddof, double std_eps,
                                      float* adv, float* mean_abs_adv, int32_t* status, void* stream) {
+    dppo::NvtxRange nvtx_range("dppo_group_advantages");
     (void)status;
     if (P < 0 || G < 1) return dppo::fail(DPPO_ERR_INVALID_ARG, "group_advantages: P=%d G=%d", P, G);
     if (std_ddof != 0 && std_ddof != 1)

@@ -6,6 +6,8 @@
 #include <stdarg.h>
 #include <stdio.h>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "dppo.h"
 
 namespace dppo {
@@ -20,6 +22,15 @@ int sm_count();                                    // SMs of the current device 
         cudaError_t e__ = cudaGetLastError();                          \
         if (e__ != cudaSuccess) return ::dppo::cuda_fail(e__, what);   \
     } while (0)
+
+// ---- host: a named NVTX range around each entry point's host work (its launches show under it in a timeline
+// tool; a few nanoseconds when no tool is attached)
+struct NvtxRange {
+    explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+    ~NvtxRange() { nvtxRangePop(); }
+    NvtxRange(const NvtxRange&) = delete;
+    NvtxRange& operator=(const NvtxRange&) = delete;
+};
 
 // ---- device: status word ---------------------------------------------------------------------------
 __device__ __forceinline__ void set_status(int32_t* status, int32_t code) {

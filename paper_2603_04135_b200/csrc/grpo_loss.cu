@@ -213,6 +213,7 @@ extern "C" int dppo_grpo_loss_fwd_bwd(const dppo_loss_params* p, const void* log
                                       void* dlogits, float* logp_out, float* lse_out, float* loss_out,
                                       void* workspace, size_t workspace_bytes, int32_t* status,
                                       void* stream) {
+    dppo::NvtxRange nvtx_range("dppo_grpo_loss_fwd_bwd");
     using namespace dppo;
     if (!p) return fail(DPPO_ERR_INVALID_ARG, "grpo_loss: NULL params");
     if (p->T_max < 0 || p->V < 1 || p->S_max < 0)
@@ -274,6 +275,7 @@ extern "C" int dppo_grpo_loss_fwd_bwd(const dppo_loss_params* p, const void* log
 
 extern "C" int dppo_sequence_log_ratio(const float* logp, const float* logp_old, const int32_t* cu_seqlens, int S_max,
                                        float* out, int32_t* status, void* stream) {
+    dppo::NvtxRange nvtx_range("dppo_sequence_log_ratio");
     (void)status;
     if (S_max < 0) return dppo::fail(DPPO_ERR_INVALID_ARG, "sequence_log_ratio: S_max=%d", S_max);
     if (S_max == 0) return DPPO_OK;

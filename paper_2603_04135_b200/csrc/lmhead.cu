@@ -1065,6 +1065,7 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
                                      const float* w, const int32_t* seg_map, void* dhidden, void* dW,
                                      float* logp_out, float* lse_out, float* loss_out, void* workspace,
                                      size_t workspace_bytes, int32_t* status, void* stream) {
+    dppo::NvtxRange nvtx_range("dppo_lmhead_grpo_loss");
     using namespace dppo;
     if (!p) return fail(DPPO_ERR_INVALID_ARG, "lmhead: NULL params");
     const dppo_loss_params& lp = p->loss;

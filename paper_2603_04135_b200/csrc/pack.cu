@@ -171,6 +171,7 @@ extern "C" int dppo_pack_prompts(const dppo_pack_params* p, const int32_t* len, 
                                  int32_t* off_in_row, int32_t* row_fill, int32_t* cu_seqlens,
                                  int32_t* counts, void* workspace, size_t workspace_bytes,
                                  int32_t* status, void* stream) {
+    dppo::NvtxRange nvtx_range("dppo_pack_prompts");
     using namespace dppo;
     if (!p) return fail(DPPO_ERR_INVALID_ARG, "pack_prompts: NULL params");
     if (p->n_max < 0 || p->L_row < 1 || p->N_win < 1 || (p->policy != 0 && p->policy != 1))
@@ -210,6 +211,7 @@ extern "C" int dppo_pack_prompts_static(const dppo_pack_params* p, const int32_t
                                         const int32_t* loss_len, int32_t* order, int32_t* row_of,
                                         int32_t* off_in_row, int32_t* row_fill, int32_t* cu_seqlens,
                                         int32_t* counts, int32_t* status, void* stream) {
+    dppo::NvtxRange nvtx_range("dppo_pack_prompts_static");
     using namespace dppo;
     if (!p) return fail(DPPO_ERR_INVALID_ARG, "pack_prompts_static: NULL params");
     if (p->n_max < 0 || p->L_row < 1 || p->N_win < 1 || (p->policy != 0 && p->policy != 1))

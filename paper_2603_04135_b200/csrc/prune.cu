@@ -185,6 +185,7 @@ __global__ void history_scatter_kernel(float* __restrict__ table, int N, const i
 
 extern "C" int dppo_history_gather(const float* H_table, int N, const int32_t* prompt_ids, int P, float* H_batch,
                                    int32_t* status, void* stream) {
+    dppo::NvtxRange nvtx_range("dppo_history_gather");
     if (N < 0 || P < 0) return dppo::fail(DPPO_ERR_INVALID_ARG, "history_gather: N=%d P=%d", N, P);
     if (P == 0) return DPPO_OK;
     if (!H_table || !prompt_ids || !H_batch) return dppo::fail(DPPO_ERR_INVALID_ARG, "history_gather: NULL array");
@@ -195,6 +196,7 @@ extern "C" int dppo_history_gather(const float* H_table, int N, const int32_t* p
 
 extern "C" int dppo_history_scatter(float* H_table, int N, const int32_t* prompt_ids, int P, const float* H_next,
                                     int32_t* status, void* stream) {
+    dppo::NvtxRange nvtx_range("dppo_history_scatter");
     if (N < 0 || P < 0) return dppo::fail(DPPO_ERR_INVALID_ARG, "history_scatter: N=%d P=%d", N, P);
     if (P == 0) return DPPO_OK;
     if (!H_table || !prompt_ids || !H_next) return dppo::fail(DPPO_ERR_INVALID_ARG, "history_scatter: NULL array");
@@ -210,6 +212,7 @@ extern "C" int dppo_prune_and_rescale(const dppo_prune_params* p, const float* a
                                       int32_t* n_keep_q, int32_t* n_keep_o, float* gamma_q,
                                       float* gamma_o, float* w_seq, float* H_next, int32_t* status,
                                       void* stream) {
+    dppo::NvtxRange nvtx_range("dppo_prune_and_rescale");
     (void)status;
     if (!p) return dppo::fail(DPPO_ERR_INVALID_ARG, "prune_and_rescale: NULL params");
     if (p->P < 0 || p->G < 1) return dppo::fail(DPPO_ERR_INVALID_ARG, "prune_and_rescale: P=%d G=%d", p->P, p->G);
