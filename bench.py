@@ -221,6 +221,47 @@ def time_lmhead(T, H, V, dev, iters=3, warmup=1):
                          "peak_source": peak_kind, "note": "executed flops = 6 T V H: logits, dhidden, dW (a chunk's exponentials are kept as fp16, nothing is recomputed)"}}
 
 
+# --------------------------------------------------------------------------------------- pruning / packing sweep
+def run_prune_pack_sweep(args):
+    """The pruning / packing sweep shape (32 x 8 completions, log-normal lengths, rows of 8192): for every
+    (r_q, r_o, N_win) cell the valid-token density of the packed rows against per-sequence padding to the longest
+    retained unit, the device time of advantages + prune + pack (CUDA events, median of 20) and the oracle's time
+    for the same three steps on one host core.  Prints one JSON line; not part of the default run."""
+    import oracle
+    from paper_2603_04135_b200.step import DppoStep
+    torch.cuda.set_device(0)
+    w = synth.WORKLOADS["config2"]
+    batch = synth.make_batch(w, 2)
+    cells = []
+    for r_q in (0.0, 0.25, 0.5):
+        for r_o in (0.0, 0.25, 0.5):
+            for N_win in (4, 16, 64):
+                st = DppoStep(w.P, w.G, w.L_row, N_win, r_q, r_o, 1, "bf16", 1, w.eps, w.eps, w.beta)
+                H_prev = oracle.group_advantages(batch.rewards_prev)[1]
+                st.set_batch(batch.rewards, batch.unit_len, batch.loss_len, H_prev)
+                times = []
+                for it in range(25):
+                    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+                    e0.record(); st.prune_pack(seed=2, step=11); e1.record()
+                    torch.cuda.synchronize()
+                    if it >= 5:
+                        times.append(e0.elapsed_time(e1) * 1e3)
+                n_units, n_rows, tokens, _ = (int(x) for x in st.counts.cpu().numpy())
+                keep = st.keep_o.cpu().numpy() == 1
+                t0 = time.perf_counter()
+                for _ in range(5):
+                    adv, mabs = oracle.group_advantages(batch.rewards)
+                    pr = oracle.prune_and_rescale(adv, mabs, H_prev, r_q, r_o, seed=2, step=11)
+                    oracle.pack_prompts(batch.unit_len, w.L_row, N_win, keep=pr["keep_o"].reshape(-1), loss_len=batch.loss_len)
+                cpu_us = (time.perf_counter() - t0) / 5 * 1e6
+                cells.append({"r_q": r_q, "r_o": r_o, "N_win": N_win, "units": n_units, "rows": n_rows, "tokens": tokens,
+                              "density_packed": tokens / (n_rows * w.L_row) if n_rows else None,
+                              "density_padded": tokens / (n_units * int(batch.unit_len[keep].max())) if n_units else None,
+                              "gpu_us": statistics.median(times), "oracle_us_1core": cpu_us})
+    print(json.dumps({"sweep": "config2: P=32 G=8, log-normal lengths, L_row=8192; advantages + prune + pack", "cells": cells}))
+    return 0
+
+
 # --------------------------------------------------------------------------------------- ours
 def run_ours(args):
     from paper_2603_04135_b200.step import DppoStep      # raises if libdppo.so is missing: no fallback
@@ -404,7 +445,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-lmhead", action="store_true", help="skip the fused LM-head measurement")
     ap.add_argument("--no-clock-sampling", action="store_true", help="do not poll nvidia-smi during the timed region")
+    ap.add_argument("--prune-pack-sweep", action="store_true",
+                    help="instead of the benchmark: density and timing table of the pruning / packing sweep shape")
     args = ap.parse_args()
+    if args.prune_pack_sweep:
+        sys.exit(run_prune_pack_sweep(args))
     if args.impl == "ours" and args.warmup < 3:
         args.warmup = 3
     sys.exit(run_reference(args) if args.impl == "reference" else run_ours(args))
