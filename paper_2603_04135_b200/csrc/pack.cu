@@ -68,6 +68,78 @@ pack_prompts_kernel(dppo_pack_params prm, const int32_t* __restrict__ len,
 
     // ---- greedy placement
     int n_placed = 0, lo = 0, row = 0, remaining = L, loss_cum = 0;
+    if (kStreamInSmem && prm.policy == 0) {
+        // Batch-sized streams, first-fit: as long as the pool lies within 64 stream positions from `base` (a
+        // multiple of 32 at or below the oldest unplaced unit), lane i keeps positions base + i and base + 32 + i
+        // in registers (length, unit index, loss tokens) and the two placed-masks are warp-uniform registers.  A
+        // placement is then ballot -> ffs -> two shuffles, with no shared-memory round trip on its dependent
+        // chain.  A wider pool (large N_win, or many later units placed over a waiting one) leaves this loop for
+        // the general one below, which continues from the same state.
+        int base = 0;
+        int lenA, lenB, uA, uB, lsA, lsB;
+        uint32_t pA = 0u, pB = 0u;
+        auto load_block = [&](int b0, int& len_r, int& u_r, int& ls_r) {
+            const int j = b0 + lane;
+            const bool in = j < n;
+            len_r = in ? lens_smem[j] : 0x7fffffff;
+            u_r = in ? stream_s[j] : -1;
+            ls_r = in ? sloss_s[j] : 0;
+        };
+        load_block(0, lenA, uA, lsA);
+        load_block(32, lenB, uB, lsB);
+        while (n_placed < n) {
+            const int fetched = min(n, prm.N_win + n_placed);
+            if (fetched - base > 64) break;
+            const int jA = base + lane, jB = jA + 32;
+            bool in_b = false;
+            unsigned m = __ballot_sync(0xffffffffu, jA >= lo && jA < fetched && !((pA >> lane) & 1u) && lenA <= remaining);
+            if (!m) {
+                in_b = true;
+                m = __ballot_sync(0xffffffffu, jB >= lo && jB < fetched && !((pB >> lane) & 1u) && lenB <= remaining);
+            }
+            if (!m) {                                            // nothing in W fits: close the row
+                if (lane == 0) row_fill[row] = L - remaining;
+                ++row;
+                remaining = L;
+                continue;
+            }
+            const int src = __ffs(m) - 1;
+            const int l = __shfl_sync(0xffffffffu, in_b ? lenB : lenA, src);
+            const int ls = __shfl_sync(0xffffffffu, in_b ? lsB : lsA, src);
+            if (lane == src) {                                   // the lane that holds the unit writes its placement
+                const int u = in_b ? uB : uA;
+                order[n_placed] = u;
+                row_of[u] = row;
+                off_in_row[u] = L - remaining;
+                cu_seqlens[n_placed] = loss_cum;
+            }
+            if (in_b) pB |= 1u << src; else pA |= 1u << src;
+            loss_cum += ls;
+            remaining -= l;
+            ++n_placed;
+            if (base + (in_b ? 32 : 0) + src == lo) {            // the oldest unit went: next unplaced position
+                ++lo;
+                if (lo < base + 32) {
+                    const uint32_t w = ~pA & (0xffffffffu << (lo - base));
+                    lo = w ? base + __ffs(w) - 1 : base + 32;
+                }
+                if (lo >= base + 32 && lo < base + 64) {
+                    const uint32_t w = ~pB & (0xffffffffu << (lo - base - 32));
+                    lo = w ? base + 32 + __ffs(w) - 1 : base + 64;
+                }
+                lo = min(lo, n);
+                while (lo >= base + 32 && lo < n) {              // block A is used up: slide the window by 32
+                    if (lane == 0) placed[base >> 5] = pA;
+                    base += 32;
+                    lenA = lenB; uA = uB; lsA = lsB; pA = pB;
+                    load_block(base + 32, lenB, uB, lsB);
+                    pB = 0u;
+                }
+            }
+        }
+        if (lane == 0) { placed[base >> 5] = pA; placed[(base >> 5) + 1] = pB; }   // state for the general loop
+        __syncwarp();
+    }
     while (n_placed < n) {
         const int fetched = min(n, prm.N_win + n_placed);       // stream positions that have entered W
         int pick = -1;
