@@ -56,3 +56,30 @@ def test_epochs_with_history_table_match_oracle(mode):
     status.zero_()
     B.history_scatter(table, N, bad, 4, out, status)
     assert status.item() == B.STATUS_BAD_INDEX
+
+
+@pytest.mark.parametrize("b,r", [(0.5, 0.7), (0.5, 0.9), (0.5, 0.5)])
+def test_prompt_rescaling_second_moment_matches_theorem_d1(b, r):
+    """Appendix D.3's closed form for the variance inflation of prompt-level rescaling, E_{q ~ pruned}[gamma(q)^2] =
+    (1 - b r)(1 - (1 - b) r)/(1 - r), on the library's gamma_q: explicit draws retain exactly the expected number of
+    candidates, so |S^q|/P = 1 - b r and the mean of gamma_q^2 over the retained prompts is the closed form."""
+    from paper_2603_04135_b200 import binding as B
+    P, G = 40, 2
+    n_cand = P // 2                                          # the library takes floor(P/2) candidates: b = 0.5
+    n_keep_c = round(n_cand * (1 - r))
+    H = np.arange(P, dtype=np.float32)                       # prompts 0 .. n_cand-1 rank lowest
+    u_q = np.full(P, 0.999); u_q[n_keep_c:n_cand] = 0.0      # the last candidates are pruned
+    f32 = dict(dtype=torch.float32, device="cuda"); i32 = dict(dtype=torch.int32, device="cuda"); u8 = dict(dtype=torch.uint8, device="cuda")
+    adv = torch.zeros(P * G, **f32); mabs = torch.zeros(P, **f32)
+    cand_q = torch.zeros(P, **u8); cand_o = torch.zeros(P * G, **u8); keep_q = torch.zeros(P, **u8); keep_o = torch.zeros(P * G, **u8)
+    nq = torch.zeros(1, **i32); no = torch.zeros(P, **i32)
+    gq = torch.zeros(P, **f32); go = torch.zeros(P * G, **f32); ws = torch.zeros(P * G, **f32); H_next = torch.zeros(P, **f32)
+    prm = B.PruneParams(P, G, r, 0.0, 0, 0, 0, 0)
+    B.prune_and_rescale(prm, adv, mabs, torch.from_numpy(H).cuda(), torch.from_numpy(u_q).cuda(),
+                        torch.ones(P * G, dtype=torch.float64, device="cuda"), cand_q, cand_o, keep_q, keep_o, nq, no,
+                        gq, go, ws, H_next)
+    kept = keep_q.cpu().numpy() == 1
+    assert cand_q.cpu().numpy()[:n_cand].all() and kept.sum() == P - n_cand + n_keep_c
+    factor = float((gq.cpu().numpy()[kept].astype(np.float64) ** 2).mean())
+    closed = (1 - b * r) * (1 - (1 - b) * r) / (1 - r)
+    assert abs(factor - closed) <= 1e-6 * closed
