@@ -385,11 +385,13 @@ def run_ours(args):
     del host_tok
 
     # ---- the optional fused LM-head path on the same token count (Qwen3-4B width): forward + backward
-    lm = None
+    lm = lm_wide = None
     if rank == 0 and not args.no_lmhead:
         del tok, dlogits, dev_tok
         torch.cuda.empty_cache()
         lm = time_lmhead(T, 2560, w.V, dev)
+        torch.cuda.empty_cache()
+        lm_wide = time_lmhead(T, 4096, w.V, dev)
     # ---- max over ranks, totals over ranks
     (total_ms, loss_ms, e2e_ms), T_all = dp.combine_over_ranks([total_ms, loss_ms, e2e_ms], T, device=dev)
 
@@ -421,6 +423,7 @@ def run_ours(args):
         }
         if lm is not None:
             line["lmhead"] = lm
+            line["lmhead_h4096"] = lm_wide
         if pool is not None:
             n_rows, _, times = time_oracle(w, seed, args.ref_rows, 1, 0, pool, cores)
             pool.close(); pool.join()
