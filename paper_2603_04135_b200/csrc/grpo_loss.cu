@@ -12,12 +12,25 @@
 
 namespace dppo {
 
-// ---- kernel choice for variant 0 (from measurements on B200 at V = 151,936) --------------------------
-constexpr size_t kClusterMinRowBytes = 32768;       // shorter rows: the general kernel's second pass hits L1/L2
-constexpr int kClusterAuto = 4;                     // smallest cluster tried first
-constexpr int kClusterThreads = 256;
-constexpr int kClusterThreadsF32 = 128;             // half the arithmetic per byte: fewer threads do (5.6 against 5.4 TB/s)
-constexpr size_t kClusterMaxSlice = 76 * 1024;      // slice bytes per CTA: keeps three CTAs resident per SM
+// ---- kernel choice for variant 0 (from sweeps on B200 over rows of 2 KB to 594 KB, both dtypes) -------------
+// Every row that fits goes to the shared-memory kernel, split over the smallest cluster whose slices stay at a size
+// that keeps enough CTAs per SM in flight: the whole row in one CTA up to 44 KB (five CTAs per SM), two CTAs up to
+// 55 KB slices (four per SM), else four or eight CTAs with slices up to 76 KB (three per SM).  Measured at rows of
+// 32 / 64 / 128 KB: 6.7 / 6.5 / 6.4 TB/s with 1 / 2 / 4 CTAs against 2.8 / 3.5 / 3.7 TB/s for the general kernel
+// and 2.6 / 4.4 / 6.4 with four CTAs throughout.  Below about 8 KB per row the grid's launch rate (one CTA per row,
+// about 250 rows per microsecond) is the limit, still three times the general kernel's rate.
+constexpr size_t kSliceMax1 = 44 * 1024;
+constexpr size_t kSliceMax2 = 55 * 1024;
+constexpr size_t kSliceMax48 = 76 * 1024;
+constexpr int kClusterThreads = 256;                // bf16 slices above 16 KB
+constexpr int kClusterThreadsSmall = 128;           // bf16 slices up to 16 KB, and f32 rows (half the arithmetic per byte)
+
+static int auto_cluster_size(int nvec) {
+    const size_t limit[4] = {kSliceMax1, kSliceMax2, kSliceMax48, kSliceMax48};
+    for (int i = 0, C = 1; i < 4; ++i, C *= 2)
+        if ((size_t)((nvec + C - 1) / C) * 16 <= limit[i]) return C;
+    return 0;                                       // longer rows: the general kernel
+}
 
 // ---- general kernel --------------------------------------------------------------------------------
 constexpr int kRowThreads = 512;
@@ -261,10 +274,12 @@ extern "C" int dppo_grpo_loss_fwd_bwd(const dppo_loss_params* p, const void* log
             rc = launch_rows_cluster(a, p->variant / 10000, p->variant % 10000, s);
         } else {
             rc = DPPO_ERR_UNSUPPORTED;
-            if ((size_t)p->V * esize >= kClusterMinRowBytes) {
-                const int nvec = p->V >> (a.bf16 ? 3 : 2);
-                for (int C = kClusterAuto; C <= 8 && rc == DPPO_ERR_UNSUPPORTED; C *= 2)
-                    if ((size_t)((nvec + C - 1) / C) * 16 <= kClusterMaxSlice) rc = launch_rows_cluster(a, C, a.bf16 ? kClusterThreads : kClusterThreadsF32, s);
+            const int nvec = p->V >> (a.bf16 ? 3 : 2);
+            const int C = auto_cluster_size(nvec);
+            if (C > 0) {
+                const size_t slice = (size_t)((nvec + C - 1) / C) * 16;
+                const int threads = (a.bf16 && slice > 16 * 1024) ? kClusterThreads : kClusterThreadsSmall;
+                rc = launch_rows_cluster(a, C, threads, s);
             }
             if (rc == DPPO_ERR_UNSUPPORTED) rc = launch_rows_general(a, s);
         }

@@ -373,7 +373,7 @@ static int launch_cluster_t(const LossArgs& a, int C, int vec_per_cta, size_t dy
 }
 
 int launch_rows_cluster(const LossArgs& a, int C, int threads, cudaStream_t s) {
-    if (C != 2 && C != 4 && C != 8) return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: cluster size %d", C);
+    if (C != 1 && C != 2 && C != 4 && C != 8) return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: cluster size %d", C);
     const int log2_per_vec = a.bf16 ? 3 : 2;
     if ((a.V & ((1 << log2_per_vec) - 1)) >= threads) return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: tail");
     if (a.T_max * C >= (1ll << 31)) return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: grid too large");
