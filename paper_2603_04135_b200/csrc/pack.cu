@@ -11,7 +11,9 @@
 namespace dppo {
 
 constexpr int kPackMaxUnits = 65536;           // bitmask of 2048 words in shared memory
-constexpr int kPackSmemLens = 8192;            // stream lengths cached in shared memory up to this n_max
+constexpr int kPackSmemLens = 8192;            // stream lengths in a static shared array up to this n_max (stream in global)
+constexpr int kPackSmemAll = 16384;            // stream, lengths and loss tokens all in dynamic shared memory up to this
+                                               // n_max (192 KB): covers a dataset of 7.5-8.5 k prompts packed at set-up
 
 struct PackWorkspace {                         // carved from the caller's workspace, all i32 [n_max]
     int32_t* stream;                           // unit index of stream position j
@@ -27,10 +29,11 @@ pack_prompts_kernel(dppo_pack_params prm, const int32_t* __restrict__ len,
                     int32_t* __restrict__ cu_seqlens, int32_t* __restrict__ counts,
                     PackWorkspace ws, int32_t* status) {
     __shared__ uint32_t placed[kPackMaxUnits / 32];
-    __shared__ int32_t lens_smem[kLensInSmem ? kPackSmemLens : 1];
-    extern __shared__ int32_t pack_dyn[];                      // kStreamInSmem: stream[n_max], then loss tokens[n_max]
+    __shared__ int32_t lens_static[(kLensInSmem && !kStreamInSmem) ? kPackSmemLens : 1];
+    extern __shared__ int32_t pack_dyn[];                      // kStreamInSmem: stream, loss tokens, lengths, [n_max] each
     int32_t* stream_s = pack_dyn;
     int32_t* sloss_s = pack_dyn + prm.n_max;
+    int32_t* lens_smem = kStreamInSmem ? pack_dyn + 2 * prm.n_max : lens_static;
     const int lane = threadIdx.x;
     const int n_max = prm.n_max, L = prm.L_row;
 
@@ -262,10 +265,10 @@ extern "C" int dppo_pack_prompts(const dppo_pack_params* p, const int32_t* len, 
     ws.stream = (int32_t*)workspace;
     ws.slen = (int32_t*)((char*)workspace + need / 2);
     cudaStream_t s = (cudaStream_t)stream;
-    if (p->n_max <= kPackSmemLens) {
+    if (p->n_max <= kPackSmemAll) {
         // batch-sized streams: the stream and its loss-token counts sit in shared memory too, so a placement
         // costs shared-memory latency instead of two dependent global loads
-        const size_t dyn = (size_t)(p->n_max > 0 ? p->n_max : 1) * 2 * sizeof(int32_t);
+        const size_t dyn = (size_t)(p->n_max > 0 ? p->n_max : 1) * 3 * sizeof(int32_t);
         cudaError_t e = cudaFuncSetAttribute(pack_prompts_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
         if (e != cudaSuccess) return cuda_fail(e, "pack_prompts: shared memory attribute");
         pack_prompts_kernel<true, true><<<1, 32, dyn, s>>>(*p, len, keep, loss_len, order, row_of, off_in_row, row_fill,
