@@ -205,7 +205,7 @@ typedef struct {
     int64_t row_stride;     /* elements between consecutive rows (>= V; bytes a multiple of 16)      */
     int32_t S_max;          /* cu_seqlens has S_max+1 entries, non-decreasing, last >= true T        */
     int32_t variant;        /* 0: the library picks the kernel.  Tuning aid: 1 forces the general two-pass
-                               kernel, C*10000+threads the shared-memory kernel with C = 1, 2, 4 or 8
+                               kernel, 2 the warp-per-row kernel (rows up to 8 KB), C*10000+threads the shared-memory kernel with C = 1, 2, 4 or 8
                                CTAs per row and 128 / 256 / 512 / 1024 threads per CTA               */
     double eps_lo, eps_hi;  /* clip range 1-eps_lo .. 1+eps_hi (the paper: both 0.2)                 */
     double beta;            /* KL coefficient                                                        */

@@ -18,12 +18,18 @@ namespace dppo {
 // 55 KB slices (four per SM), else four or eight CTAs with slices up to 76 KB (three per SM).  Measured at rows of
 // 32 / 64 / 128 KB: 6.7 / 6.5 / 6.4 TB/s with 1 / 2 / 4 CTAs against 2.8 / 3.5 / 3.7 TB/s for the general kernel
 // and 2.6 / 4.4 / 6.4 with four CTAs throughout.  Below about 8 KB per row the grid's launch rate (one CTA per row,
-// about 250 rows per microsecond) is the limit, still three times the general kernel's rate.
+// about 250 rows per microsecond) is the limit: those rows go to the warp-per-row kernel (2 KB rows: 3.3-3.6 TB/s
+// against 1.0).
 constexpr size_t kSliceMax1 = 44 * 1024;
 constexpr size_t kSliceMax2 = 55 * 1024;
 constexpr size_t kSliceMax48 = 76 * 1024;
 constexpr int kClusterThreads = 256;                // bf16 slices above 16 KB
 constexpr int kClusterThreadsSmall = 128;           // bf16 slices up to 16 KB, and f32 rows (half the arithmetic per byte)
+
+// Short rows: one warp per row, the row in registers (grpo_loss_warp.cu).
+int launch_rows_warp(const LossArgs& a, cudaStream_t s);
+constexpr int kWarpRowMaxVecBf16 = 256;             // bf16 rows of up to 4 KB, f32 rows of up to 8 KB (an 8 KB bf16 row is
+constexpr int kWarpRowMaxVecF32 = 512;              // as fast in one CTA of the shared-memory kernel: 3.4 TB/s)
 
 static int auto_cluster_size(int nvec) {
     const size_t limit[4] = {kSliceMax1, kSliceMax2, kSliceMax48, kSliceMax48};
@@ -270,13 +276,17 @@ extern "C" int dppo_grpo_loss_fwd_bwd(const dppo_loss_params* p, const void* log
         int rc;
         if (p->variant == 1) {
             rc = launch_rows_general(a, s);
+        } else if (p->variant == 2) {
+            rc = launch_rows_warp(a, s);
         } else if (p->variant >= 10000) {
             rc = launch_rows_cluster(a, p->variant / 10000, p->variant % 10000, s);
         } else {
             rc = DPPO_ERR_UNSUPPORTED;
             const int nvec = p->V >> (a.bf16 ? 3 : 2);
             const int C = auto_cluster_size(nvec);
-            if (C > 0) {
+            if (nvec <= (a.bf16 ? kWarpRowMaxVecBf16 : kWarpRowMaxVecF32)) {
+                rc = launch_rows_warp(a, s);
+            } else if (C > 0) {
                 const size_t slice = (size_t)((nvec + C - 1) / C) * 16;
                 const int threads = (a.bf16 && slice > 16 * 1024) ? kClusterThreads : kClusterThreadsSmall;
                 rc = launch_rows_cluster(a, C, threads, s);

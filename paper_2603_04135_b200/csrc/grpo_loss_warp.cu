@@ -1,0 +1,211 @@
+// Loss sweep for short rows (up to 8 KB): one WARP per row, the row held in registers.
+//
+// With one CTA per row a short row costs more to launch than to process (the grid's launch rate, about 250 CTAs
+// per microsecond, caps 2 KB rows at 1 TB/s).  Here persistent warps walk over the rows: a lane loads up to
+// kVPL 16-byte vectors of the row straight into registers (coalesced, 512 bytes per warp instruction), the row
+// maximum and the sum of exponentials are warp reductions, lane 0 runs the scalar stage, and the stored
+// exponentials are scaled into dlogits from the same registers.  HBM sees one read and one write per element
+// and nothing goes through shared memory.  The arithmetic per element is the shared-memory kernel's: packed bf16
+// maximum, 2^(z c - r) once, kept as fp16 pairs (bf16 rows) or f32 (f32 rows), then a scale.
+#include <cuda_fp16.h>
+
+#include "common.cuh"
+#include "grpo_loss.cuh"
+
+namespace dppo {
+namespace warprow {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+// Two bf16 logits in one word -> their exponentials 2^(z c + nr) as an fp16 pair; s += the two.
+__device__ __forceinline__ uint32_t exp_pair(uint32_t w, float c, float nr, float& s0, float& s1) {
+    const float e0 = ex2(fmaf(__uint_as_float(w << 16), c, nr));
+    const float e1 = ex2(fmaf(__uint_as_float(w & 0xffff0000u), c, nr));
+    s0 += e0; s1 += e1;
+    const __half2 h = __floats2half2_rn(e0, e1);
+    return *reinterpret_cast<const uint32_t*>(&h);
+}
+// Two fp16 exponentials -> two bf16 gradient entries e * sc.
+__device__ __forceinline__ uint32_t scale_pair(uint32_t h2, float sc) {
+    const float2 e = __half22float2(*reinterpret_cast<const __half2*>(&h2));
+    const __nv_bfloat162 b = __floats2bfloat162_rn(e.x * sc, e.y * sc);
+    return *reinterpret_cast<const uint32_t*>(&b);
+}
+__device__ __forceinline__ uint32_t exp_f32(uint32_t w, float c, float nr, float& s) {
+    const float e = ex2(fmaf(__uint_as_float(w), c, nr));
+    s += e;
+    return __float_as_uint(e);
+}
+
+// The binary64 scalar stage as a call of its own: its registers are then not the whole kernel's, which is what
+// lets more warps (rows in flight) share an SM.
+__device__ __noinline__ RowScalars finish_row(const LossArgs& a, long long t, const RowInputs& in, float ref2, float sum2) {
+    return row_finish(a, t, in, ref2, sum2, true);
+}
+
+}  // namespace warprow
+
+using namespace warprow;
+
+// Resident CTAs per SM the register allocation aims at: more rows in flight for the short forms.
+template <bool kF32, int kVPL> constexpr int min_ctas() { return kVPL <= 4 ? 4 : kVPL == 8 ? 3 : kF32 ? 2 : 1; }
+
+template <bool kF32, int kVPL>
+__global__ void __launch_bounds__(kThreads, min_ctas<kF32, kVPL>())
+grpo_loss_warp_kernel(const LossArgs a) {
+    constexpr int kLog2PerVec = kF32 ? 2 : 3;               // elements per 16-byte vector: 4 f32 or 8 bf16
+    constexpr uint32_t kPad = kF32 ? 0xFF800000u : 0xFF80FF80u;   // -inf: adds nothing to the maximum or the sum
+    const int lane = threadIdx.x & 31;
+    const long long warp0 = (long long)blockIdx.x * kWarps + (threadIdx.x >> 5);
+    const long long n_warps = (long long)gridDim.x * kWarps;
+    const long long T = a.n_tokens_dev ? min((long long)*a.n_tokens_dev, a.T_max) : a.T_max;
+    const int nvec = a.V >> kLog2PerVec;
+    const int tail0 = nvec << kLog2PerVec;                  // the ragged tail: one element per lane
+    const bool has_tail = tail0 + lane < a.V;
+    const float c = a.scale2;
+
+    for (long long t = warp0; t < T; t += n_warps) {
+        const char* row = a.logits + t * a.row_bytes;
+        const uint4* rowv = reinterpret_cast<const uint4*>(row);
+        uint4 d[kVPL];
+#pragma unroll
+        for (int j = 0; j < kVPL; ++j) {
+            const int i = lane + 32 * j;
+            d[j] = i < nvec ? __ldcs(rowv + i) : make_uint4(kPad, kPad, kPad, kPad);
+        }
+        const float ztail = has_tail ? Elems<!kF32>::load1(row, tail0 + lane) : -INFINITY;
+        RowInputs in;                                       // filled by lane 0 while the loads are in flight
+        row_gather_warp(a, t, lane, in);
+
+        // ---- row maximum
+        float m = ztail;
+        if constexpr (kF32) {
+#pragma unroll
+            for (int j = 0; j < kVPL; ++j)
+                m = fmaxf(m, fmaxf(fmaxf(__uint_as_float(d[j].x), __uint_as_float(d[j].y)),
+                                   fmaxf(__uint_as_float(d[j].z), __uint_as_float(d[j].w))));
+        } else {
+            __nv_bfloat162 mx2 = __float2bfloat162_rn(-INFINITY);
+#pragma unroll
+            for (int j = 0; j < kVPL; ++j) {
+                mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&d[j].x));
+                mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&d[j].y));
+                mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&d[j].z));
+                mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&d[j].w));
+            }
+            m = fmaxf(m, fmaxf(__low2float(mx2), __high2float(mx2)));
+        }
+        m = warp_max(m);
+        const float r = m * c;                              // -inf only if the whole row is -inf
+        const float nr = r > -INFINITY ? -r : 0.0f;
+
+        // ---- exponentials 2^(z c - r) in place, and their sum
+        float s0 = 0.0f, s1 = 0.0f;
+#pragma unroll
+        for (int j = 0; j < kVPL; ++j) {
+            if constexpr (kF32) {
+                d[j].x = exp_f32(d[j].x, c, nr, s0); d[j].y = exp_f32(d[j].y, c, nr, s1);
+                d[j].z = exp_f32(d[j].z, c, nr, s0); d[j].w = exp_f32(d[j].w, c, nr, s1);
+            } else {
+                d[j].x = exp_pair(d[j].x, c, nr, s0, s1); d[j].y = exp_pair(d[j].y, c, nr, s0, s1);
+                d[j].z = exp_pair(d[j].z, c, nr, s0, s1); d[j].w = exp_pair(d[j].w, c, nr, s0, s1);
+            }
+        }
+        const float etail = ztail > -INFINITY ? ex2(fmaf(ztail, c, nr)) : 0.0f;
+        const float s = warp_sum(s0 + s1 + etail);
+
+        // ---- scalar stage (lane 0), broadcast of what the stores need
+        RowScalars rs;
+        rs.lse2_hi = 0.0f; rs.lse2_lo = 0.0f; rs.g_over_tau = 0.0f; rs.valid = false;
+        int y = -1;
+        if (lane == 0) {
+            rs = finish_row(a, t, in, r, s);
+            y = rs.valid ? in.y : -1;
+        }
+        const float lse2_hi = __shfl_sync(0xffffffffu, rs.lse2_hi, 0), lse2_lo = __shfl_sync(0xffffffffu, rs.lse2_lo, 0);
+        const float ng = -__shfl_sync(0xffffffffu, rs.valid ? rs.g_over_tau : 0.0f, 0);
+        y = __shfl_sync(0xffffffffu, y, 0);
+
+        // ---- dlogits = g/tau (onehot - 2^(z c - lse2)) from the registers
+        if (a.dlogits) {
+            char* drow = a.dlogits + t * a.row_bytes;
+            uint4* dst = reinterpret_cast<uint4*>(drow);
+            const float sc = ng * ex2((r - lse2_hi) - lse2_lo);
+#pragma unroll
+            for (int j = 0; j < kVPL; ++j) {
+                const int i = lane + 32 * j;
+                if (i < nvec) {
+                    uint4 o;
+                    if constexpr (kF32) {
+                        o.x = __float_as_uint(__uint_as_float(d[j].x) * sc); o.y = __float_as_uint(__uint_as_float(d[j].y) * sc);
+                        o.z = __float_as_uint(__uint_as_float(d[j].z) * sc); o.w = __float_as_uint(__uint_as_float(d[j].w) * sc);
+                    } else {
+                        o.x = scale_pair(d[j].x, sc); o.y = scale_pair(d[j].y, sc);
+                        o.z = scale_pair(d[j].z, sc); o.w = scale_pair(d[j].w, sc);
+                    }
+                    __stcs(dst + i, o);
+                }
+            }
+            // the one element that also carries the onehot term: the lane that stored its vector redoes it
+            const int yvec = y >= 0 ? (y >> kLog2PerVec) : -1;
+            if (yvec >= 0 && yvec < nvec && (yvec & 31) == lane) {
+                const int jy = yvec >> 5;
+                const int wy = kF32 ? (y & 3) : ((y & 7) >> 1);
+                uint32_t word = 0;
+#pragma unroll
+                for (int j = 0; j < kVPL; ++j) {
+                    const uint32_t wj = wy == 0 ? d[j].x : wy == 1 ? d[j].y : wy == 2 ? d[j].z : d[j].w;
+                    word = j == jy ? wj : word;             // selects: d stays in registers
+                }
+                if constexpr (kF32) {
+                    reinterpret_cast<float*>(drow)[y] = fmaf(__uint_as_float(word), sc, -ng);
+                } else {
+                    const float2 e = __half22float2(*reinterpret_cast<const __half2*>(&word));
+                    reinterpret_cast<__nv_bfloat16*>(drow)[y] = __float2bfloat16_rn(fmaf((y & 1) ? e.y : e.x, sc, -ng));
+                }
+            }
+            if (has_tail) {
+                const int v = tail0 + lane;
+                Elems<!kF32>::store1(drow, v, sc * etail - (v == y ? ng : 0.0f));
+            }
+        }
+    }
+}
+
+// ---- host side ---------------------------------------------------------------------------------------
+template <bool kF32, int kVPL>
+static int launch_warp_t(const LossArgs& a, cudaStream_t s) {
+    auto kernel = grpo_loss_warp_kernel<kF32, kVPL>;
+    int per_sm = 0;
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, 0);
+    if (e != cudaSuccess || per_sm < 1) { cudaGetLastError(); return fail(DPPO_ERR_UNSUPPORTED, "warp-per-row kernel does not fit this device"); }
+    const long long want = (a.T_max + kWarps - 1) / kWarps;
+    const long long cap = (long long)sm_count() * per_sm;
+    kernel<<<(unsigned)(want < cap ? want : cap), kThreads, 0, s>>>(a);
+    DPPO_CHECK_LAUNCH("grpo_loss warp-per-row launch");
+    return DPPO_OK;
+}
+
+template <bool kF32>
+static int launch_warp_dtype(const LossArgs& a, int vpl, cudaStream_t s) {
+    if (vpl <= 2) return launch_warp_t<kF32, 2>(a, s);
+    if (vpl <= 4) return launch_warp_t<kF32, 4>(a, s);
+    if (vpl <= 8) return launch_warp_t<kF32, 8>(a, s);
+    return launch_warp_t<kF32, 16>(a, s);
+}
+
+// Rows of up to 512 vectors (8 KB).  DPPO_ERR_UNSUPPORTED (nothing launched) for longer rows.
+int launch_rows_warp(const LossArgs& a, cudaStream_t s) {
+    const int nvec = a.V >> (a.bf16 ? 3 : 2);
+    if (nvec > 32 * 16) return fail(DPPO_ERR_UNSUPPORTED, "warp-per-row kernel: rows of %d vectors exceed %d", nvec, 32 * 16);
+    const int vpl = (nvec + 31) / 32;
+    return a.bf16 ? launch_warp_dtype<false>(a, vpl, s) : launch_warp_dtype<true>(a, vpl, s);
+}
+
+}  // namespace dppo

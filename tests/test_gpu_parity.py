@@ -357,6 +357,24 @@ def test_loss_cluster_kernel_f32_rows(C):
     _loss_case(1024, "f32", T=40, S=3, seed=158 + C, variant=v, logit_sigma=40.0, centre_on_oracle=True)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_loss_warp_per_row_kernel(dtype):
+    # short rows, one warp per row with the row in registers (forced): every vectors-per-lane form, ragged ends,
+    # fewer rows than warps and many more, in place, forward only, masked columns
+    v = 2
+    for V, seed in [(1, 300), (5, 301), (8, 302), (100, 303), (256, 304), (1000, 305), (1024, 306), (2047, 307)]:
+        _loss_case(V, dtype, T=67, S=5, seed=seed, variant=v)
+    big = 4096 if dtype == "bf16" else 2048                                      # 16 vectors per lane
+    _loss_case(big, dtype, T=40, S=3, seed=310, variant=v)
+    _loss_case(1536, dtype, T=5000, S=40, seed=311, variant=v)                   # several rows per warp
+    _loss_case(1024, dtype, T=50, S=4, seed=312, variant=v, in_place=True)
+    _loss_case(1024, dtype, T=50, S=4, seed=313, variant=v, forward_only=True)
+    _loss_case(1000, dtype, T=50, S=4, seed=314, variant=v, n_tokens=37, tau=1.7, pad=8)
+    _loss_case(1024, dtype, T=20, S=2, seed=315, variant=v, neg_inf_cols=(100, 1024))
+    _loss_case(1024, dtype, T=40, S=3, seed=316, variant=v, logit_sigma=40.0, centre_on_oracle=True)
+    _loss_case(2040, dtype, T=80, S=6, seed=317, variant=v, seq_ratio=True, sigma_noise=0.3)
+
+
 def test_loss_auto_dispatch_matches_forced_kernels():
     # variant 0 on a long bf16 row takes the cluster kernel; outputs agree with the general kernel's
     a = _loss_case(151936, "bf16", T=11, S=2, seed=60, variant=0)
