@@ -440,6 +440,19 @@ def test_loss_is_bit_reproducible(variant):
                            b.view(torch.int16) if b.dtype == torch.bfloat16 else b.view(torch.int32))
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_loss_kernel_choice_boundaries(dtype):
+    # row lengths on both sides of every switch of the library's kernel choice: warp per row -> one CTA -> two ->
+    # four -> eight CTAs -> general kernel (limits in 16-byte vectors: 256 or 512, 2816, 7040, 19456, 38912)
+    per_vec = 8 if dtype == "bf16" else 4
+    warp_max = 256 if dtype == "bf16" else 512
+    seed = 400
+    for nvec in (warp_max, 2816, 7040, 19456, 38912):
+        for V in (nvec * per_vec, nvec * per_vec + per_vec, nvec * per_vec + 3):
+            seed += 1
+            _loss_case(V, dtype, T=5, S=2, seed=seed, variant=0)
+
+
 def test_loss_bad_target_and_empty():
     from paper_2603_04135_b200 import binding as B
     V, T = 512, 8
