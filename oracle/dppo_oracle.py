@@ -460,7 +460,7 @@ def grpo_loss(logits, target, logp_old, logp_ref, cu_seqlens, adv_seg, w_seg,
 # Step 9 — the same loss with the LM-head projection in front
 # --------------------------------------------------------------------------
 def lmhead_grpo_loss(hidden, W_head, target, logp_old, logp_ref, cu_seqlens, adv_seg, w_seg,
-                     eps_lo=0.2, eps_hi=0.2, beta=0.04, tau=1.0):
+                     eps_lo=0.2, eps_hi=0.2, beta=0.04, tau=1.0, length_norm=True, seq_log_ratio=None):
     """logits = hidden @ W_head^T (float64 accumulation of the exact bf16 inputs),
     then `grpo_loss`; dhidden = D @ W_head and dW = D^T @ hidden with D the
     float64 dlogits."""
@@ -468,7 +468,8 @@ def lmhead_grpo_loss(hidden, W_head, target, logp_old, logp_ref, cu_seqlens, adv
     Wm = np.asarray(W_head, dtype=np.float64)
     z = h @ Wm.T
     out = grpo_loss(z, target, logp_old, logp_ref, cu_seqlens, adv_seg, w_seg,
-                    eps_lo, eps_hi, beta, tau, want_dlogits=True)
+                    eps_lo, eps_hi, beta, tau, want_dlogits=True, length_norm=length_norm,
+                    seq_log_ratio=seq_log_ratio)
     D = out["dlogits"]
     out["dhidden"] = D @ Wm
     out["dW"] = D.T @ h

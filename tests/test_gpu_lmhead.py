@@ -184,6 +184,56 @@ def test_config4_whole_path(H):
     assert (err <= bound).all(), "dW worst ratio %.3g" % (err / bound).max()
 
 
+@pytest.mark.parametrize("mode", ["no_length_norm", "seq_ratio"])
+def test_lmhead_loss_variants(mode):
+    """The objectives of Section 5.2 through the fused path: weights without the 1/|o| factor, and the
+    sequence-level ratio (a forward-only call gives the current log-probs, their per-sequence mean log-ratio goes
+    back in for the call with gradients)."""
+    from paper_2603_04135_b200 import binding as B
+    T, V, H, S, seed = 300, 1000, 128, 5, 51
+    w = synth.scaled(synth.WORKLOADS["config4_h2560"], V=V, H=H, sigma_old=0.3)
+    hidden, W, target, lo, lr = synth.make_lmhead_inputs(w, T, seed, device="cuda")
+    rng = np.random.default_rng(seed)
+    cu = np.concatenate([[0], np.sort(rng.choice(np.arange(1, T), size=S - 1, replace=False)), [T]]).astype(np.int32)
+    adv = rng.normal(size=S).astype(np.float32); wseq = (rng.random(S) * 0.1).astype(np.float32)
+    d_cu = torch.from_numpy(cu).cuda(); d_adv = torch.from_numpy(adv).cuda(); d_w = torch.from_numpy(wseq).cuda()
+    loss_out = torch.zeros(5, device="cuda"); logp_out = torch.zeros(T, device="cuda"); lse_out = torch.zeros(T, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    fwd = B.LmheadParams(B.LossParams(T, V, B.BF16, V, S, 0, w.eps, w.eps, w.beta, 1.0), H, 0)
+    bwd = B.LmheadParams(B.LossParams(T, V, B.BF16, V, S, 0, w.eps, w.eps, w.beta, 1.0), H, 1, 0, B.F32)
+    nbytes = max(B.lmhead_workspace_bytes(fwd), B.lmhead_workspace_bytes(bwd))
+    ws = torch.zeros(nbytes + 1024, dtype=torch.uint8, device="cuda"); ws = ws[(-ws.data_ptr()) % 1024:]
+    slr = None
+    if mode == "seq_ratio":
+        B.lmhead_grpo_loss(fwd, hidden, W, target, lo, lr, d_cu, None, d_adv, d_w, None, None, None, logp_out, None, loss_out,
+                           ws, nbytes, status)
+        slr_dev = torch.zeros(S, device="cuda")
+        B.sequence_log_ratio(logp_out, lo, d_cu, S, slr_dev)
+        bwd.loss.seq_log_ratio = slr_dev.data_ptr()
+        z = synth.to_f64_numpy(hidden) @ synth.to_f64_numpy(W).T
+        slr = oracle.sequence_log_ratio(oracle.token_logprob(z, target.cpu().numpy())[0], lo.cpu().numpy(), cu)
+        assert np.abs(slr_dev.cpu().numpy() - slr).max() <= 1e-4
+    else:
+        bwd.loss.no_length_norm = 1
+    dh = torch.zeros((T, H), dtype=torch.bfloat16, device="cuda"); dW = torch.zeros((V, H), device="cuda")
+    B.lmhead_grpo_loss(bwd, hidden, W, target, lo, lr, d_cu, None, d_adv, d_w, None, dh, dW, logp_out, lse_out, loss_out,
+                       ws, nbytes, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    ref = oracle.lmhead_grpo_loss(synth.to_f64_numpy(hidden), synth.to_f64_numpy(W), target.cpu().numpy(), lo.cpu().numpy(),
+                                  lr.cpu().numpy(), cu, adv, wseq, w.eps, w.eps, w.beta, 1.0,
+                                  length_norm=(mode != "no_length_norm"), seq_log_ratio=slr)
+    got = loss_out.cpu().numpy().astype(np.float64)
+    assert abs(got[0] - ref["loss"]) <= 1e-4 * ref["abs_sum"]
+    gmax = np.abs(ref["g"]).max()
+    err = np.abs(dh.double().cpu().numpy() - ref["dhidden"])
+    bound = 2.0 ** -7 * np.abs(ref["dhidden"]).max(axis=1, keepdims=True) + 1e-6 * gmax
+    assert (err <= bound).all(), "dhidden worst ratio %.3g" % (err / bound).max()
+    err = np.abs(dW.double().cpu().numpy() - ref["dW"])
+    bound = 2.0 ** -7 * np.abs(ref["dW"]).max(axis=1, keepdims=True) + 1e-6 * gmax
+    assert (err <= bound).all(), "dW worst ratio %.3g" % (err / bound).max()
+
+
 def test_lmhead_full_size_sampled_tokens():
     """The size the benchmark times (99,030 tokens, V = 151,936, H = 2560, eleven token chunks, the last ragged):
     lse, logp and dhidden of sampled tokens against the oracle (each sampled token is given to the oracle as a
