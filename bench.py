@@ -264,6 +264,9 @@ def run_prune_pack_sweep(args):
 
 # --------------------------------------------------------------------------------------- ours
 def run_ours(args):
+    if not os.path.exists(os.path.join(ROOT, "paper_2603_04135_b200", "libdppo.so")):
+        from paper_2603_04135_b200 import build          # a checkout without the built library: compile it in-tree
+        build.build_library()
     from paper_2603_04135_b200.step import DppoStep      # raises if libdppo.so is missing: no fallback
     from paper_2603_04135_b200 import dp
 
