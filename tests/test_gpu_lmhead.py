@@ -74,6 +74,15 @@ def test_lmhead_small_shapes(variant):
 
 
 @pytest.mark.parametrize("variant", [1, 0])
+def test_lmhead_edge_shapes(variant):
+    # one token, one vocabulary entry, one more than a tile in each direction, fewer tokens than a tile
+    for kw in [dict(T=1, V=8, H=64, S=1, seed=61), dict(T=5, V=300, H=64, S=2, seed=62), dict(T=2, V=1, H=64, S=1, seed=63),
+               dict(T=129, V=257, H=128, S=3, seed=64), dict(T=64, V=65, H=64, S=2, seed=65)]:
+        _run(backward=False, variant=variant, **kw)
+        _run(backward=True, variant=variant, **kw)
+
+
+@pytest.mark.parametrize("variant", [1, 0])
 def test_lmhead_full_vocabulary(variant):
     _run(T=300, V=151936, H=2560, S=4, seed=5, variant=variant)
 
