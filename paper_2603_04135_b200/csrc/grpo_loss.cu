@@ -23,8 +23,8 @@ namespace dppo {
 constexpr size_t kSliceMax1 = 44 * 1024;
 constexpr size_t kSliceMax2 = 55 * 1024;
 constexpr size_t kSliceMax48 = 76 * 1024;
-constexpr int kClusterThreads = 256;                // bf16 slices above 16 KB
-constexpr int kClusterThreadsSmall = 128;           // bf16 slices up to 16 KB, and f32 rows (half the arithmetic per byte)
+constexpr int kClusterThreads = 256;                // bf16 slices above 16 KB, f32 slices above 64 KB
+constexpr int kClusterThreadsSmall = 128;           // shorter slices (f32 has half the arithmetic per byte)
 
 // Short rows: one warp per row, the row in registers (grpo_loss_warp.cu).
 int launch_rows_warp(const LossArgs& a, cudaStream_t s);
@@ -288,7 +288,8 @@ extern "C" int dppo_grpo_loss_fwd_bwd(const dppo_loss_params* p, const void* log
                 rc = launch_rows_warp(a, s);
             } else if (C > 0) {
                 const size_t slice = (size_t)((nvec + C - 1) / C) * 16;
-                const int threads = (a.bf16 && slice > 16 * 1024) ? kClusterThreads : kClusterThreadsSmall;
+                // 256 threads for bf16 slices above 16 KB and f32 slices above 64 KB, else 128
+                const int threads = slice > (a.bf16 ? 16u : 64u) * 1024 ? kClusterThreads : kClusterThreadsSmall;
                 rc = launch_rows_cluster(a, C, threads, s);
             }
             if (rc == DPPO_ERR_UNSUPPORTED) rc = launch_rows_general(a, s);
