@@ -40,8 +40,8 @@ WORKLOAD_TEXT = WORKLOAD + ": P=32 G=8, response 64-1024 tokens, V=151936 bf16 l
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch over 8192 rows of this vocabulary.  Traffic
 # grows in proportion to the rows, so a launch over T rows moves T times the per-row figure.  The record
 # is tied to the kernel sources it was taken from: once they change, `traffic` is reported as null.
-TRAFFIC_CAPTURE = {"rows": 8192, "dram_bytes": 2489447000 + 2430915000,
-                   "source_sha256": "bf45720255b1adf4d114cecb3cecddea188b91b21e6ff7a59bec44316a22e05c"}
+TRAFFIC_CAPTURE = {"rows": 8192, "dram_bytes": 2489504000 + 2431640000,
+                   "source_sha256": "e9560dea6352e68770f24457c44a0df5462c8a9da2d58d5ba39d42e571b97d3b"}
 
 
 def captured_traffic_per_row():

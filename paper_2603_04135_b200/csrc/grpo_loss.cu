@@ -26,8 +26,6 @@ constexpr size_t kSliceMax48 = 76 * 1024;
 constexpr int kClusterThreads = 256;                // bf16 slices above 16 KB, f32 slices above 64 KB
 constexpr int kClusterThreadsSmall = 128;           // shorter slices (f32 has half the arithmetic per byte)
 
-// Short rows: one warp per row, the row in registers (grpo_loss_warp.cu).
-int launch_rows_warp(const LossArgs& a, cudaStream_t s);
 constexpr int kWarpRowMaxVecBf16 = 256;             // bf16 rows of up to 4 KB, f32 rows of up to 8 KB (an 8 KB bf16 row is
 constexpr int kWarpRowMaxVecF32 = 512;              // as fast in one CTA of the shared-memory kernel: 3.4 TB/s)
 

@@ -207,6 +207,9 @@ int launch_rows_general(const LossArgs& a, cudaStream_t s);
 // Cluster kernel: the row is split over `cluster` CTAs that keep their slice in shared memory.
 // Returns DPPO_ERR_UNSUPPORTED (nothing launched) when the shape or the device cannot take it.
 int launch_rows_cluster(const LossArgs& a, int cluster, int threads, cudaStream_t s);
+// Short rows (up to 512 16-byte vectors): one warp per row, the row in registers (grpo_loss_warp.cu).
+// Returns DPPO_ERR_UNSUPPORTED (nothing launched) for longer rows.
+int launch_rows_warp(const LossArgs& a, cudaStream_t s);
 int launch_loss_reduce(const LossArgs& a, float* loss_out, cudaStream_t s);
 
 }  // namespace dppo
