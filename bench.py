@@ -209,6 +209,20 @@ def time_lmhead(T, H, V, dev, iters=3, warmup=1):
             times.append(e0.elapsed_time(e1))
     assert status.item() == 0
     ms = sum(times) / len(times)
+    # forward only (loss, log-probs, lse; no scratch kept): 2 T V H flops
+    prm_f = B.LmheadParams(B.LossParams(T, V, B.BF16, V, S, 0, wl.eps, wl.eps, wl.beta, 1.0), H, 0)
+    times_f = []
+    for it in range(warmup + iters):
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record()
+        B.lmhead_grpo_loss(prm_f, hidden, W, target, lo, lr, cu, None, adv, wseq, None, None, None, None, None, loss_out,
+                           ws, nbytes, status)
+        e1.record()
+        torch.cuda.synchronize()
+        if it >= warmup:
+            times_f.append(e0.elapsed_time(e1))
+    assert status.item() == 0
+    ms_f = sum(times_f) / len(times_f)
     try:
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
             peak = float(json.load(f)["bf16_tflops_sustained"]); peak_kind = "measured sustained cuBLAS bf16"
@@ -217,6 +231,8 @@ def time_lmhead(T, H, V, dev, iters=3, warmup=1):
     executed = 6.0 * T * V * H / ms / 1e9
     return {"workload": "config4: bf16 hidden [%d x %d], W [%d x %d], forward + dhidden + dW" % (T, H, V, H),
             "ms": ms, "tokens_per_s": T / ms * 1e3, "executed_tflops": executed, "model_tflops_6TVH": executed,
+            "forward_only": {"ms": ms_f, "tokens_per_s": T / ms_f * 1e3, "executed_tflops_2TVH": 2.0 * T * V * H / ms_f / 1e9,
+                             "frac_of_peak": 2.0 * T * V * H / ms_f / 1e9 / peak},
             "roofline": {"bound": "tensor", "achieved": executed, "peak": peak, "unit": "TFLOP/s", "frac": executed / peak,
                          "peak_source": peak_kind, "note": "executed flops = 6 T V H: logits, dhidden, dW (a chunk's exponentials are kept as fp16, nothing is recomputed)"}}
 
