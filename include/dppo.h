@@ -13,7 +13,9 @@
  *    dppo_last_error() gives the message of the calling thread's last failure.
  *  - Unless a parameter says "host", array pointers are DEVICE pointers owned by the caller.  The
  *    library allocates no memory and keeps no state between calls; scratch comes from a caller
- *    workspace sized by the matching *_workspace_bytes() (a pure host function).
+ *    workspace sized by the matching *_workspace_bytes() (a pure host function).  The one exception is
+ *    dppo_pack_prompts_static, whose scratch is an array inside the library that all its calls on a device
+ *    share (see there).
  *  - Work is enqueued on `stream` (a cudaStream_t passed as void*); there is no host
  *    synchronisation inside.  Outputs are valid once the stream reaches that point.
  *  - Host-visible arguments are validated before anything is launched.  Problems only the device
@@ -206,7 +208,12 @@ typedef struct {
     int32_t S_max;          /* cu_seqlens has S_max+1 entries, non-decreasing, last >= true T        */
     int32_t variant;        /* 0: the library picks the kernel.  Tuning aid: 1 forces the general two-pass
                                kernel, 2 the warp-per-row kernel (rows up to 8 KB), C*10000+threads the shared-memory kernel with C = 1, 2, 4 or 8
-                               CTAs per row and 128 / 256 / 512 / 1024 threads per CTA               */
+                               CTAs per row and 128 / 256 / 512 / 1024 threads per CTA.
+                               Self-test of the bounded waits: 1000000 + (0 or a C*10000+threads code) runs the
+                               shared-memory kernel with every CTA expecting one exchange message more than is
+                               ever sent and a wait limit of 1 ms: every row then ends as a timed-out row does
+                               (status DPPO_STATUS_TIMEOUT; the row's dlogits, logp_out, lse_out and loss terms
+                               are zero) and nothing hangs                                           */
     double eps_lo, eps_hi;  /* clip range 1-eps_lo .. 1+eps_hi (the paper: both 0.2)                 */
     double beta;            /* KL coefficient                                                        */
     double temperature;     /* > 0 (the paper: 1)                                                    */
@@ -245,6 +252,22 @@ int dppo_grpo_loss_fwd_bwd(const dppo_loss_params* p, const void* logits, const 
                            float* loss_out, void* workspace, size_t workspace_bytes,
                            int32_t* status, void* stream);
 
+/* Which kernel a dppo_grpo_loss_fwd_bwd call with these parameters runs on the current device (a host-side query:
+ * it makes the same choice and the same device checks as the call and launches nothing).  Rows of up to 4 KB (bf16)
+ * or 8 KB (f32) go to the warp-per-row kernel, rows that fit eight shared-memory slices to the shared-memory
+ * kernel, longer ones to the general two-pass kernel.  fell_back = 1 says that the device refused the kernel the
+ * row length asked for (its shared memory or cluster size) and the slower general kernel runs instead.
+ * Errors: INVALID_ARG; UNSUPPORTED when params.variant forces a kernel that cannot take the shape.
+ */
+typedef enum { DPPO_KERNEL_GENERAL = 0, DPPO_KERNEL_WARP = 1, DPPO_KERNEL_SHARED = 2 } dppo_loss_kernel;
+typedef struct {
+    int32_t kernel;         /* dppo_loss_kernel                                                      */
+    int32_t ctas_per_row;   /* cluster size of the shared-memory kernel, else 1                      */
+    int32_t threads;        /* threads that work on one row at a time in each CTA                    */
+    int32_t fell_back;      /* 1: general kernel in place of the one the row length asked for        */
+} dppo_loss_kernel_choice;
+int dppo_grpo_loss_kernel_choice(const dppo_loss_params* p, dppo_loss_kernel_choice* out);
+
 /* Mean token log-ratio of each sequence, out[s] = mean_t (logp[t] - logp_old[t]) over cu_seqlens[s] <= t <
  * cu_seqlens[s+1] (0 for an empty sequence): the log of the length-normalised sequence-level likelihood
  * ratio of sequence-level objectives (Section 5.2).  logp, logp_old f32 [T]; out f32 [S_max].  Binary64
@@ -279,7 +302,11 @@ typedef struct {
     dppo_loss_params loss;
     int32_t H;
     int32_t backward;
-    int32_t variant;        /* 0: CTA pairs (cta_group::2) share each B tile; 1: one CTA per tile (tuning aid) */
+    int32_t variant;        /* 0: CTA pairs (cta_group::2) share each B tile; 1: one CTA per tile (tuning aid).
+                               100 / 101: the same two with the self-test of the bounded waits: the first pipeline
+                               stage of every CTA expects 16 bytes more than are ever copied and the wait limit
+                               is 1 ms, so every CTA gives up, frees its tensor memory and returns; the call
+                               reports DPPO_STATUS_TIMEOUT and its other outputs are unspecified    */
     int32_t dW_dtype;       /* DPPO_F32 (0) or DPPO_BF16: element type of dW */
     int32_t accumulate_dW;  /* 0: dW is overwritten; 1: the gradient is added to what dW holds (micro-batches) */
     int32_t reserved;       /* 0 */

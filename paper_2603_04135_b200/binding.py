@@ -46,6 +46,17 @@ class LossParams(ctypes.Structure):
                 ("seq_log_ratio", ctypes.c_void_p)]
 
 
+class LossKernelChoice(ctypes.Structure):
+    _fields_ = [("kernel", ctypes.c_int32), ("ctas_per_row", ctypes.c_int32), ("threads", ctypes.c_int32),
+                ("fell_back", ctypes.c_int32)]
+
+
+KERNEL_GENERAL, KERNEL_WARP, KERNEL_SHARED = 0, 1, 2
+KERNEL_NAMES = {KERNEL_GENERAL: "general two-pass", KERNEL_WARP: "warp per row", KERNEL_SHARED: "shared memory"}
+LOSS_WAIT_SELF_TEST = 1000000      # added to dppo_loss_params.variant
+LMHEAD_WAIT_SELF_TEST = 100        # added to dppo_lmhead_params.variant
+
+
 class LmheadParams(ctypes.Structure):
     _fields_ = [("loss", LossParams), ("H", ctypes.c_int32), ("backward", ctypes.c_int32), ("variant", ctypes.c_int32),
                 ("dW_dtype", ctypes.c_int32),
@@ -76,6 +87,8 @@ lib.dppo_grpo_loss_fwd_bwd.restype = ctypes.c_int
 lib.dppo_grpo_loss_fwd_bwd.argtypes = [ctypes.POINTER(LossParams)] + [_vp] * 14 + [ctypes.c_size_t, _vp, _vp]
 
 
+lib.dppo_grpo_loss_kernel_choice.restype = ctypes.c_int
+lib.dppo_grpo_loss_kernel_choice.argtypes = [ctypes.POINTER(LossParams), ctypes.POINTER(LossKernelChoice)]
 lib.dppo_sequence_log_ratio.restype = ctypes.c_int
 lib.dppo_sequence_log_ratio.argtypes = [_vp, _vp, _vp, ctypes.c_int, _vp, _vp, _vp]
 lib.dppo_lmhead_workspace_bytes.restype = ctypes.c_size_t
@@ -170,6 +183,13 @@ def grpo_loss_fwd_bwd(params, logits, target, logp_old, logp_ref, cu_seqlens, n_
                                       _ptr(seg_map), _ptr(dlogits), _ptr(logp_out), _ptr(lse_out),
                                       _ptr(loss_out), _ptr(workspace), workspace_bytes, _ptr(status),
                                       _stream(stream)))
+
+
+def grpo_loss_kernel_choice(params):
+    """The kernel dppo_grpo_loss_fwd_bwd runs for these parameters on the current device, as a LossKernelChoice."""
+    out = LossKernelChoice()
+    _check(lib.dppo_grpo_loss_kernel_choice(ctypes.byref(params), ctypes.byref(out)))
+    return out
 
 
 def lmhead_workspace_bytes(params):

@@ -38,6 +38,8 @@ static int auto_cluster_size(int nvec) {
 
 // ---- general kernel --------------------------------------------------------------------------------
 constexpr int kRowThreads = 512;
+LossArgs loss_args_from_params(const dppo_loss_params* p);
+int run_rows(LossArgs a, int variant, cudaStream_t s, bool launch, dppo_loss_kernel_choice* choice);
 
 template <bool kBf16>
 __global__ void __launch_bounds__(kRowThreads) grpo_loss_rows_kernel(const LossArgs a) {
@@ -54,8 +56,11 @@ __global__ void __launch_bounds__(kRowThreads) grpo_loss_rows_kernel(const LossA
         const char* row = a.logits + t * a.row_bytes;
         const uint4* rowv = reinterpret_cast<const uint4*>(row);
 
-        // pass 1: running raw maximum m, reference r = m c, sum of 2^(z c - r)
-        float m = -INFINITY, r = -INFINITY, s = 0.0f;
+        // pass 1: running raw maximum m, reference r = m c, sum of 2^(z c - r).  While a thread has seen nothing
+        // but -inf (a masked start of the vocabulary) its reference is still -inf: the offset added to z c is then
+        // 0, not -r = +inf, so that those elements add 2^(-inf) = 0 (and not the NaN of -inf + inf) and s is a
+        // clean 0 when the first finite maximum arrives.
+        float m = -INFINITY, r = -INFINITY, nr = 0.0f, s = 0.0f;
         for (int i = tid; i < nvec; i += kRowThreads) {
             float f[VW];
             E::unpack(rowv[i], f);
@@ -64,20 +69,20 @@ __global__ void __launch_bounds__(kRowThreads) grpo_loss_rows_kernel(const LossA
             for (int e = 1; e < VW; ++e) mx = fmaxf(mx, f[e]);
             if (mx > m) {
                 const float r_new = mx * c;
-                s *= exp2f(r - r_new);                       // 0 when r is still -inf
-                m = mx; r = r_new;
+                s *= exp2f(r - r_new);                       // s is 0 while r is still -inf
+                m = mx; r = r_new; nr = -r_new;
             }
 #pragma unroll
-            for (int e = 0; e < VW; ++e) s += exp2f(fmaf(f[e], c, -r));
+            for (int e = 0; e < VW; ++e) s += exp2f(fmaf(f[e], c, nr));
         }
         for (int v = nvec * VW + tid; v < a.V; v += kRowThreads) {      // ragged tail
             const float z = E::load1(row, v);
             if (z > m) {
                 const float r_new = z * c;
                 s *= exp2f(r - r_new);
-                m = z; r = r_new;
+                m = z; r = r_new; nr = -r_new;
             }
-            s += exp2f(fmaf(z, c, -r));
+            s += exp2f(fmaf(z, c, nr));
         }
         // combine (r, s) pairs: warp, then block
         float R = warp_max(r);
@@ -216,6 +221,74 @@ int launch_loss_reduce(const LossArgs& a, float* loss_out, cudaStream_t s) {
     return DPPO_OK;
 }
 
+// The shape-dependent part of the kernel arguments (pointers are filled in by the caller).
+LossArgs loss_args_from_params(const dppo_loss_params* p) {
+    LossArgs a = {};
+    const size_t esize = p->dtype == DPPO_BF16 ? 2 : 4;
+    a.T_max = p->T_max; a.row_bytes = (long long)p->row_stride * (long long)esize;
+    a.V = p->V; a.S_max = p->S_max; a.bf16 = p->dtype == DPPO_BF16 ? 1 : 0;
+    a.eps_lo = p->eps_lo; a.eps_hi = p->eps_hi; a.beta = p->beta; a.temperature = p->temperature;
+    a.scale2 = (float)(1.4426950408889634 / p->temperature);
+    a.seq_log_ratio = p->seq_log_ratio; a.no_length_norm = p->no_length_norm;
+    a.wait_limit_ns = kDefaultWaitLimitNs; a.test_extra_tx = 0;
+    return a;
+}
+
+// Picks the row kernel for `variant` and launches it (launch = true) or only runs the checks a launch would make.
+// variant: 0 picks the kernel from the shape; 1 forces the general kernel; 2 the warp-per-row kernel;
+// C*10000 + threads forces the shared-memory kernel with C CTAs per row (a tuning aid; unsupported shapes are an
+// error); kSelfTestVariant + one of those runs the self-test of the bounded waits on the shared-memory kernel.
+// choice (nullable) receives what was taken; fell_back = 1 when the device refused the kernel the shape asked for
+// and the general kernel took over.
+constexpr int kSelfTestVariant = 1000000;
+
+int run_rows(LossArgs a, int variant, cudaStream_t s, bool launch, dppo_loss_kernel_choice* choice) {
+    dppo_loss_kernel_choice ch = {DPPO_KERNEL_GENERAL, 1, kRowThreads, 0};
+    const bool self_test = variant >= kSelfTestVariant;
+    if (self_test) {
+        variant -= kSelfTestVariant;
+        a.wait_limit_ns = kSelfTestWaitLimitNs;
+        a.test_extra_tx = 8;
+    }
+    int rc;
+    if (variant == 1) {
+        rc = launch ? launch_rows_general(a, s) : DPPO_OK;
+    } else if (variant == 2) {
+        ch.kernel = DPPO_KERNEL_WARP; ch.threads = 32;
+        rc = launch_rows_warp(a, s, launch);
+    } else if (variant >= 10000) {
+        ch.kernel = DPPO_KERNEL_SHARED; ch.ctas_per_row = variant / 10000; ch.threads = variant % 10000;
+        rc = launch_rows_cluster(a, ch.ctas_per_row, ch.threads, s, launch);
+    } else if (variant == 0) {
+        rc = DPPO_ERR_UNSUPPORTED;
+        const int nvec = a.V >> (a.bf16 ? 3 : 2);
+        const int C = auto_cluster_size(nvec);
+        bool refused = false;
+        if (nvec <= (a.bf16 ? kWarpRowMaxVecBf16 : kWarpRowMaxVecF32)) {
+            ch.kernel = DPPO_KERNEL_WARP; ch.threads = 32;
+            rc = launch_rows_warp(a, s, launch);
+            refused = rc == DPPO_ERR_UNSUPPORTED;
+        } else if (C > 0) {
+            const size_t slice = (size_t)((nvec + C - 1) / C) * 16;
+            // 256 threads for bf16 slices above 16 KB and f32 slices above 64 KB, else 128
+            const int threads = slice > (a.bf16 ? 16u : 64u) * 1024 ? kClusterThreads : kClusterThreadsSmall;
+            ch.kernel = DPPO_KERNEL_SHARED; ch.ctas_per_row = C; ch.threads = threads;
+            rc = launch_rows_cluster(a, C, threads, s, launch);
+            refused = rc == DPPO_ERR_UNSUPPORTED;
+        }
+        if (rc == DPPO_ERR_UNSUPPORTED) {                  // too long for eight slices, or refused by this device
+            ch.kernel = DPPO_KERNEL_GENERAL; ch.ctas_per_row = 1; ch.threads = kRowThreads; ch.fell_back = refused ? 1 : 0;
+            rc = launch ? launch_rows_general(a, s) : DPPO_OK;
+        }
+    } else {
+        rc = fail(DPPO_ERR_INVALID_ARG, "grpo_loss: variant %d", variant);
+    }
+    if (rc == DPPO_OK && self_test && ch.kernel != DPPO_KERNEL_SHARED)
+        return fail(DPPO_ERR_UNSUPPORTED, "grpo_loss: the wait self-test runs on the shared-memory kernel only");
+    if (choice) *choice = ch;
+    return rc;
+}
+
 }  // namespace dppo
 
 extern "C" size_t dppo_grpo_loss_workspace_bytes(const dppo_loss_params* p) {
@@ -257,44 +330,26 @@ extern "C" int dppo_grpo_loss_fwd_bwd(const dppo_loss_params* p, const void* log
         return fail(DPPO_ERR_WORKSPACE_TOO_SMALL, "grpo_loss: workspace %zu < %zu bytes", workspace_bytes, need);
     if ((uintptr_t)workspace & 15) return fail(DPPO_ERR_MISALIGNED, "grpo_loss: workspace not 16-byte aligned");
 
-    LossArgs a;
+    LossArgs a = loss_args_from_params(p);
     a.logits = (const char*)logits; a.dlogits = (char*)dlogits;
     a.target = target; a.logp_old = logp_old; a.logp_ref = logp_ref;
     a.cu_seqlens = cu_seqlens; a.n_tokens_dev = n_tokens_dev; a.adv = adv; a.w = w; a.seg_map = seg_map;
     a.logp_out = logp_out; a.lse_out = lse_out; a.terms = (RowTerms*)workspace; a.status = status;
-    a.T_max = p->T_max; a.row_bytes = (long long)p->row_stride * (long long)esize;
-    a.V = p->V; a.S_max = p->S_max; a.bf16 = p->dtype == DPPO_BF16 ? 1 : 0;
-    a.eps_lo = p->eps_lo; a.eps_hi = p->eps_hi; a.beta = p->beta; a.temperature = p->temperature;
-    a.scale2 = (float)(1.4426950408889634 / p->temperature);
-    a.seq_log_ratio = p->seq_log_ratio; a.no_length_norm = p->no_length_norm;
     cudaStream_t s = (cudaStream_t)stream;
     if (p->T_max > 0) {
-        // variant: 0 picks the kernel from the shape; 1 forces the general kernel; C*10000 + threads
-        // forces the cluster kernel with C CTAs per row (a tuning aid; unsupported shapes are an error)
-        int rc;
-        if (p->variant == 1) {
-            rc = launch_rows_general(a, s);
-        } else if (p->variant == 2) {
-            rc = launch_rows_warp(a, s);
-        } else if (p->variant >= 10000) {
-            rc = launch_rows_cluster(a, p->variant / 10000, p->variant % 10000, s);
-        } else {
-            rc = DPPO_ERR_UNSUPPORTED;
-            const int nvec = p->V >> (a.bf16 ? 3 : 2);
-            const int C = auto_cluster_size(nvec);
-            if (nvec <= (a.bf16 ? kWarpRowMaxVecBf16 : kWarpRowMaxVecF32)) {
-                rc = launch_rows_warp(a, s);
-            } else if (C > 0) {
-                const size_t slice = (size_t)((nvec + C - 1) / C) * 16;
-                // 256 threads for bf16 slices above 16 KB and f32 slices above 64 KB, else 128
-                const int threads = slice > (a.bf16 ? 16u : 64u) * 1024 ? kClusterThreads : kClusterThreadsSmall;
-                rc = launch_rows_cluster(a, C, threads, s);
-            }
-            if (rc == DPPO_ERR_UNSUPPORTED) rc = launch_rows_general(a, s);
-        }
+        const int rc = run_rows(a, p->variant, s, true, nullptr);
         if (rc != DPPO_OK) return rc;
     }
     return launch_loss_reduce(a, loss_out, s);
+}
+
+extern "C" int dppo_grpo_loss_kernel_choice(const dppo_loss_params* p, dppo_loss_kernel_choice* out) {
+    using namespace dppo;
+    if (!p || !out) return fail(DPPO_ERR_INVALID_ARG, "grpo_loss_kernel_choice: NULL argument");
+    if (p->V < 1 || p->T_max < 0 || (p->dtype != DPPO_F32 && p->dtype != DPPO_BF16) || p->variant < 0 || !(p->temperature > 0.0))
+        return fail(DPPO_ERR_INVALID_ARG, "grpo_loss_kernel_choice: V=%d T_max=%lld dtype=%d variant=%d", p->V,
+                    (long long)p->T_max, p->dtype, p->variant);
+    return run_rows(loss_args_from_params(p), p->variant, nullptr, false, out);
 }
 
 extern "C" int dppo_sequence_log_ratio(const float* logp, const float* logp_old, const int32_t* cu_seqlens, int S_max,

@@ -50,7 +50,12 @@ struct LossArgs {
     const float* seq_log_ratio;   // nullable: sequence-level ratio, indexed by sequence position
     int no_length_norm;
     float scale2;            // log2(e) / temperature as the f32 both passes multiply by
+    unsigned long long wait_limit_ns;   // bound of every device-side wait (on %globaltimer)
+    int test_extra_tx;       // 0; the self-test of the bounded waits announces this many bytes that never arrive
 };
+
+constexpr unsigned long long kDefaultWaitLimitNs = 2000000000ull;   // give up on a copy or a peer after 2 s
+constexpr unsigned long long kSelfTestWaitLimitNs = 1000000ull;     // the self-test's waits run out after 1 ms
 
 // ---- 16-byte vectors ------------------------------------------------------------------------------
 template <bool kBf16> struct Elems;
@@ -206,10 +211,11 @@ __device__ __forceinline__ RowScalars row_scalar_stage(const LossArgs& a, long l
 int launch_rows_general(const LossArgs& a, cudaStream_t s);
 // Cluster kernel: the row is split over `cluster` CTAs that keep their slice in shared memory.
 // Returns DPPO_ERR_UNSUPPORTED (nothing launched) when the shape or the device cannot take it.
-int launch_rows_cluster(const LossArgs& a, int cluster, int threads, cudaStream_t s);
+// launch = false: run the checks only (shape, shared memory, cluster fit) and launch nothing.
+int launch_rows_cluster(const LossArgs& a, int cluster, int threads, cudaStream_t s, bool launch = true);
 // Short rows (up to 512 16-byte vectors): one warp per row, the row in registers (grpo_loss_warp.cu).
 // Returns DPPO_ERR_UNSUPPORTED (nothing launched) for longer rows.
-int launch_rows_warp(const LossArgs& a, cudaStream_t s);
+int launch_rows_warp(const LossArgs& a, cudaStream_t s, bool launch = true);
 int launch_loss_reduce(const LossArgs& a, float* loss_out, cudaStream_t s);
 
 }  // namespace dppo

@@ -24,7 +24,8 @@ namespace dppo {
 constexpr int kMaxCluster = 8;
 constexpr int kChunks = 1;                    // bulk copies (and mbarriers) per slice: one copy of the whole slice was
                                               // 3.5 % faster than four (fewer waits and loop prologues per row)
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // give up on a copy after 2 s
+constexpr unsigned long long kSettleNs = 20000ull;            // after a failed exchange: time for remote stores already
+                                                              // issued by the peers to land before this CTA leaves
 
 struct ClusterStatic {
     unsigned long long bar[kChunks];          // one mbarrier per bulk copy of the slice
@@ -45,7 +46,7 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 
 // Bounded wait on phase `parity` of an mbarrier; false when the limit ran out.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned long long limit_ns) {
     const unsigned long long t0 = global_ns();
     for (;;) {
         uint32_t done;
@@ -54,7 +55,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
                      "selp.u32 %0, 1, 0, p;\n\t}"
                      : "=r"(done) : "r"(bar), "r"(parity) : "memory");
         if (done) return true;
-        if (global_ns() - t0 > kWaitLimitNs) return false;
+        if (global_ns() - t0 > limit_ns) return false;
     }
 }
 
@@ -130,9 +131,12 @@ __device__ __forceinline__ uint4 scale_quad(uint4 q, f32x2 sc2) {
     return q;
 }
 
-// The cluster barrier is used once, as a start-up handshake ("my mbarriers exist"): no data rides on it.
+// The cluster barrier is used once on the way in, as a start-up handshake ("my mbarriers exist"): no data rides on
+// it.  Only a CTA whose exchange failed uses it a second time, on the way out (see the end of the kernel).
 __device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 
 // 8-byte store into CTA `rank`'s shared memory that also signals that CTA's mbarrier (8 bytes of tx).
 __device__ __forceinline__ void remote_store_signal(uint32_t local_slot, uint32_t local_bar, int rank, unsigned long long v) {
@@ -172,8 +176,10 @@ grpo_loss_cluster_kernel(const LossArgs a, const int C, const int vec_per_cta) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(&st.bar[k])));
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(&st.xbar)));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        // the exchange expects one 8-byte pair from each CTA of the cluster (its own included)
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(smem_u32(&st.xbar)), "r"(8u * C) : "memory");
+        // the exchange expects one 8-byte pair from each CTA of the cluster (its own included); the self-test of the
+        // bounded waits announces one pair more than will ever be sent, so that every CTA's wait runs out
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                     :: "r"(smem_u32(&st.xbar)), "r"(8u * (uint32_t)C + (uint32_t)a.test_extra_tx) : "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 #pragma unroll
         for (int k = 0; k < kChunks; ++k) {
@@ -202,7 +208,10 @@ grpo_loss_cluster_kernel(const LossArgs a, const int C, const int vec_per_cta) {
     for (int k = 0; k < kChunks; ++k) {
         const int b = k * chunk_vec, e = min(nv, b + chunk_vec);
         if (e > b) {
-            ok = mbar_wait(smem_u32(&st.bar[k]), 0) && ok;
+            bool landed = mbar_wait(smem_u32(&st.bar[k]), 0, a.wait_limit_ns);
+            // a copy that is late: one more bounded chance to land before anything else happens to this CTA's
+            // shared memory (the row is reported as failed either way)
+            if (!landed) { mbar_wait(smem_u32(&st.bar[k]), 0, a.wait_limit_ns); ok = false; }
 #pragma unroll 2
             for (int i = b + tid; i < e; i += THREADS) {
                 const uint4 q = slice[i];
@@ -277,7 +286,7 @@ grpo_loss_cluster_kernel(const LossArgs a, const int C, const int vec_per_cta) {
             remote_store_signal(smem_u32(&st.x[rank]), smem_u32(&st.xbar), lane, v);
         }
         if (lane == 0) {
-            const bool arrived = mbar_wait(smem_u32(&st.xbar), 0);
+            const bool arrived = mbar_wait(smem_u32(&st.xbar), 0, a.wait_limit_ns);
             float R = -INFINITY;
             bool failed = !arrived;
             for (int k = 0; k < C && arrived; ++k) {
@@ -300,6 +309,7 @@ grpo_loss_cluster_kernel(const LossArgs a, const int C, const int vec_per_cta) {
                 }
                 RowScalars bad; bad.lse2_hi = 0.0f; bad.lse2_lo = 0.0f; bad.g_over_tau = 0.0f; bad.valid = false;
                 st.row = bad;
+                st.failed = arrived ? 1 : 2;                 // 2: this CTA's own wait for the pairs ran out
             } else {
                 st.row = row_finish(a, t, st.in, R, S, rank == 0);
             }
@@ -313,8 +323,9 @@ grpo_loss_cluster_kernel(const LossArgs a, const int C, const int vec_per_cta) {
         char* drow = a.dlogits + t * a.row_bytes;
         uint4* dst = reinterpret_cast<uint4*>(drow) + v0;
         const float ng = rs.valid ? -rs.g_over_tau : 0.0f;
-        // softmax = e * 2^(r - lse2) with e relative to this CTA's reference r
-        const float sc = ng * ex2((r - rs.lse2_hi) - rs.lse2_lo);
+        // softmax = e * 2^(r - lse2) with e relative to this CTA's reference r (a row that failed has no lse2: its
+        // gradient is written as zeros)
+        const float sc = st.failed ? 0.0f : ng * ex2((r - rs.lse2_hi) - rs.lse2_lo);
         const f32x2 sc2 = pair_of(sc, sc);
         const int y = rs.valid ? a.target[t] : -1;
         const int yvec = (y >= 0 ? (y >> kLog2PerVec) : -1) - v0;   // vector of the target relative to this slice
@@ -347,36 +358,69 @@ grpo_loss_cluster_kernel(const LossArgs a, const int C, const int vec_per_cta) {
             Elems<!kF32>::store1(drow, v, sc * etail - (v == y ? ng : 0.0f));
         }
     }
+
+    // ---- way out after a failed exchange.  A CTA that has received all C pairs knows that every peer is done
+    //      writing into its shared memory and simply returns.  A CTA whose own wait ran out does not: a slow peer
+    //      could still send its pair, and that remote store must not land in shared memory that already belongs to
+    //      another CTA.  It therefore waits on the cluster barrier, which completes once every peer has either
+    //      arrived here as well (it failed too) or exited (it sends before it can exit), and then lets stores that
+    //      are already under way settle.  Every wait before this point is bounded, so every peer gets that far.
+    if (st.failed == 2) {                                   // written before the block barrier above: uniform
+        cluster_arrive_release();
+        cluster_wait_acquire();
+        const unsigned long long t0 = global_ns();
+        while (global_ns() - t0 < kSettleNs) { }
+    }
 }
 
 // ---- host side ---------------------------------------------------------------------------------------
+constexpr size_t kClusterSmemMax = 220 * 1024;            // largest slice a CTA may hold
+
+// The dynamic shared-memory limit of an instantiation is raised once per device to the largest slice any launch
+// may ask for (a per-call value could be lowered by another host thread between this thread's set and its launch).
 template <int THREADS, bool kF32>
-static int launch_cluster_t(const LossArgs& a, int C, int vec_per_cta, size_t dyn_bytes, cudaStream_t s) {
+static int cluster_prepare_t(int C, size_t dyn_bytes, cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, bool check_fit) {
     auto kernel = grpo_loss_cluster_kernel<THREADS, kF32>;
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_bytes);
-    if (e != cudaSuccess) { cudaGetLastError(); return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: %zu bytes of shared memory refused", dyn_bytes); }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(a.T_max * C), 1, 1);
-    cfg.blockDim = dim3(THREADS, 1, 1);
-    cfg.dynamicSmemBytes = dyn_bytes;
-    cfg.stream = s;
-    cudaLaunchAttribute attr[2];
+    static bool raised[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); dev = -1; }
+    if (dev < 0 || !raised[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kClusterSmemMax);
+        if (e != cudaSuccess) { cudaGetLastError(); return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: %zu bytes of shared memory refused", kClusterSmemMax); }
+        if (dev >= 0) raised[dev] = true;
+    }
+    cfg->blockDim = dim3(THREADS, 1, 1);
+    cfg->dynamicSmemBytes = dyn_bytes;
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = (unsigned)C; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     attr[1].id = cudaLaunchAttributeClusterSchedulingPolicyPreference;
     // clusters handed to whichever GPC has room rather than spread evenly: 5 % faster on eight-CTA clusters (f32
     // rows of the full vocabulary), 2.5 % on four while the board is below its power limit
     attr[1].val.clusterSchedulingPolicyPreference = cudaClusterSchedulingPolicyLoadBalancing;
-    cfg.attrs = attr; cfg.numAttrs = 2;
-    int max_clusters = 0;
-    e = cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &cfg);
-    if (e != cudaSuccess || max_clusters < 1) { cudaGetLastError(); return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: cluster of %d CTAs does not fit this device", C); }
-    e = cudaLaunchKernelEx(&cfg, kernel, a, C, vec_per_cta);
+    cfg->attrs = attr; cfg->numAttrs = 2;
+    if (check_fit) {
+        int max_clusters = 0;
+        cudaError_t e = cudaOccupancyMaxActiveClusters(&max_clusters, kernel, cfg);
+        if (e != cudaSuccess || max_clusters < 1) { cudaGetLastError(); return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: cluster of %d CTAs does not fit this device", C); }
+    }
+    return DPPO_OK;
+}
+
+// launch = false: only the checks a launch would make (used by the kernel-choice query).
+template <int THREADS, bool kF32>
+static int launch_cluster_t(const LossArgs& a, int C, int vec_per_cta, size_t dyn_bytes, cudaStream_t s, bool launch) {
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[2];
+    cfg.gridDim = dim3((unsigned)((a.T_max > 0 ? a.T_max : 1) * C), 1, 1);
+    cfg.stream = s;
+    const int rc = cluster_prepare_t<THREADS, kF32>(C, dyn_bytes, &cfg, attr, true);
+    if (rc != DPPO_OK || !launch) return rc;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, grpo_loss_cluster_kernel<THREADS, kF32>, a, C, vec_per_cta);
     if (e != cudaSuccess) return cuda_fail(e, "grpo_loss cluster launch");
     return DPPO_OK;
 }
 
-int launch_rows_cluster(const LossArgs& a, int C, int threads, cudaStream_t s) {
+int launch_rows_cluster(const LossArgs& a, int C, int threads, cudaStream_t s, bool launch) {
     if (C != 1 && C != 2 && C != 4 && C != 8) return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: cluster size %d", C);
     const int log2_per_vec = a.bf16 ? 3 : 2;
     if ((a.V & ((1 << log2_per_vec) - 1)) >= threads) return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: tail");
@@ -384,21 +428,21 @@ int launch_rows_cluster(const LossArgs& a, int C, int threads, cudaStream_t s) {
     const int nvec = a.V >> log2_per_vec;
     const int vec_per_cta = (nvec + C - 1) / C;
     const size_t dyn_bytes = (size_t)(vec_per_cta > 0 ? vec_per_cta : 1) * 16;
-    if (dyn_bytes > 220 * 1024) return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: slice of %zu bytes exceeds shared memory", dyn_bytes);
+    if (dyn_bytes > kClusterSmemMax) return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: slice of %zu bytes exceeds shared memory", dyn_bytes);
     if (dyn_bytes / kChunks + 16 >= (1u << 20)) return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: chunk too large");
     if (a.bf16) {
         switch (threads) {
-            case 128: return launch_cluster_t<128, false>(a, C, vec_per_cta, dyn_bytes, s);
-            case 256: return launch_cluster_t<256, false>(a, C, vec_per_cta, dyn_bytes, s);
-            case 512: return launch_cluster_t<512, false>(a, C, vec_per_cta, dyn_bytes, s);
-            case 1024: return launch_cluster_t<1024, false>(a, C, vec_per_cta, dyn_bytes, s);
+            case 128: return launch_cluster_t<128, false>(a, C, vec_per_cta, dyn_bytes, s, launch);
+            case 256: return launch_cluster_t<256, false>(a, C, vec_per_cta, dyn_bytes, s, launch);
+            case 512: return launch_cluster_t<512, false>(a, C, vec_per_cta, dyn_bytes, s, launch);
+            case 1024: return launch_cluster_t<1024, false>(a, C, vec_per_cta, dyn_bytes, s, launch);
         }
     } else {
         switch (threads) {
-            case 128: return launch_cluster_t<128, true>(a, C, vec_per_cta, dyn_bytes, s);
-            case 256: return launch_cluster_t<256, true>(a, C, vec_per_cta, dyn_bytes, s);
-            case 512: return launch_cluster_t<512, true>(a, C, vec_per_cta, dyn_bytes, s);
-            case 1024: return launch_cluster_t<1024, true>(a, C, vec_per_cta, dyn_bytes, s);
+            case 128: return launch_cluster_t<128, true>(a, C, vec_per_cta, dyn_bytes, s, launch);
+            case 256: return launch_cluster_t<256, true>(a, C, vec_per_cta, dyn_bytes, s, launch);
+            case 512: return launch_cluster_t<512, true>(a, C, vec_per_cta, dyn_bytes, s, launch);
+            case 1024: return launch_cluster_t<1024, true>(a, C, vec_per_cta, dyn_bytes, s, launch);
         }
     }
     return fail(DPPO_ERR_UNSUPPORTED, "cluster kernel: %d threads", threads);

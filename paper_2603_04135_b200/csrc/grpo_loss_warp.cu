@@ -180,11 +180,12 @@ grpo_loss_warp_kernel(const LossArgs a) {
 
 // ---- host side ---------------------------------------------------------------------------------------
 template <bool kF32, int kVPL>
-static int launch_warp_t(const LossArgs& a, cudaStream_t s) {
+static int launch_warp_t(const LossArgs& a, cudaStream_t s, bool launch) {
     auto kernel = grpo_loss_warp_kernel<kF32, kVPL>;
     int per_sm = 0;
     cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, 0);
     if (e != cudaSuccess || per_sm < 1) { cudaGetLastError(); return fail(DPPO_ERR_UNSUPPORTED, "warp-per-row kernel does not fit this device"); }
+    if (!launch) return DPPO_OK;
     const long long want = (a.T_max + kWarps - 1) / kWarps;
     const long long cap = (long long)sm_count() * per_sm;
     kernel<<<(unsigned)(want < cap ? want : cap), kThreads, 0, s>>>(a);
@@ -193,19 +194,19 @@ static int launch_warp_t(const LossArgs& a, cudaStream_t s) {
 }
 
 template <bool kF32>
-static int launch_warp_dtype(const LossArgs& a, int vpl, cudaStream_t s) {
-    if (vpl <= 2) return launch_warp_t<kF32, 2>(a, s);
-    if (vpl <= 4) return launch_warp_t<kF32, 4>(a, s);
-    if (vpl <= 8) return launch_warp_t<kF32, 8>(a, s);
-    return launch_warp_t<kF32, 16>(a, s);
+static int launch_warp_dtype(const LossArgs& a, int vpl, cudaStream_t s, bool launch) {
+    if (vpl <= 2) return launch_warp_t<kF32, 2>(a, s, launch);
+    if (vpl <= 4) return launch_warp_t<kF32, 4>(a, s, launch);
+    if (vpl <= 8) return launch_warp_t<kF32, 8>(a, s, launch);
+    return launch_warp_t<kF32, 16>(a, s, launch);
 }
 
 // Rows of up to 512 vectors (8 KB).  DPPO_ERR_UNSUPPORTED (nothing launched) for longer rows.
-int launch_rows_warp(const LossArgs& a, cudaStream_t s) {
+int launch_rows_warp(const LossArgs& a, cudaStream_t s, bool launch) {
     const int nvec = a.V >> (a.bf16 ? 3 : 2);
     if (nvec > 32 * 16) return fail(DPPO_ERR_UNSUPPORTED, "warp-per-row kernel: rows of %d vectors exceed %d", nvec, 32 * 16);
     const int vpl = (nvec + 31) / 32;
-    return a.bf16 ? launch_warp_dtype<false>(a, vpl, s) : launch_warp_dtype<true>(a, vpl, s);
+    return a.bf16 ? launch_warp_dtype<false>(a, vpl, s, launch) : launch_warp_dtype<true>(a, vpl, s, launch);
 }
 
 }  // namespace dppo

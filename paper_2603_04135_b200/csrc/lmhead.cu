@@ -39,9 +39,22 @@ constexpr int kStageBytesB = kBN * kBK * 2;                  // 32 KB
 constexpr int kStageBytes = kStageBytesA + kStageBytesB;
 constexpr int kLmThreads = 192;
 constexpr int kTmemCols = 512;
-constexpr unsigned long long kLmWaitLimitNs = 2000000000ull;
 constexpr int kChunkTokens = 9472;       // tokens whose dlogits are held in scratch at a time: 74 row tiles, so the
                                          // dhidden GEMM of a chunk has 74 x H/256 tiles = whole waves on 148 SMs
+constexpr int kMaxChunkTokens = 1 << 16;
+
+// Launch-shape choices of the call, by hidden width (from sweeps on B200 at 99,030 tokens, V = 151,936).
+struct LmTune {
+    int chunk_tokens;                    // a multiple of 256 (whole row-tile pairs)
+    int group_logits;                    // column tiles per group of the logits launch (0: all row tiles of two column tiles at a time)
+    int group_dw;                        // the same for the dW launch (0: all column tiles of a few row tiles at a time)
+    int hints;                           // two bits per operand load (kHint...): logits A, B; dhidden A, B; dW A, B
+};
+static LmTune lm_tune(int H) {
+    (void)H;
+    LmTune t = {kChunkTokens, 0, 0, 0};
+    return t;
+}
 
 struct LmShared {
     unsigned long long full[kStages];    // TMA bytes have landed in stage s
@@ -70,12 +83,12 @@ __device__ __forceinline__ bool lm_try(uint32_t bar, uint32_t parity) {
 }
 
 // Bounded wait; also leaves when another role has raised the abort flag.
-__device__ __forceinline__ bool lm_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool lm_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned long long limit_ns) {
     const unsigned long long t0 = lm_global_ns();
     for (;;) {
         if (lm_try(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (lm_global_ns() - t0 > kLmWaitLimitNs) { *abort_flag = 1; return false; }
+        if (lm_global_ns() - t0 > limit_ns) { *abort_flag = 1; return false; }
     }
 }
 
@@ -130,31 +143,69 @@ template <bool kAMn, bool kBMn, int kM> __host__ __device__ constexpr uint32_t l
            ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kM >> 4) << 24);
 }
 
-// One tiled TMA load (x = innermost coordinate, 16-byte aligned by construction: multiples of 64 elements).
-__device__ __forceinline__ void lm_tma_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-                 :: "r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
-}
-// The same from a CTA of a pair: the barrier may be the peer's (the pair's leader collects both CTAs' bytes).
-__device__ __forceinline__ void lm_tma_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
-    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-                 :: "r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+// L2 eviction policy of an operand's loads: a tile that other CTAs (or later waves) will ask for again is kept
+// (evict_last), one that is streamed through once makes room first (evict_first).
+enum { kHintNone = 0, kHintEvictFirst = 1, kHintEvictLast = 2 };
+__device__ __forceinline__ uint64_t lm_l2_policy(int hint) {
+    uint64_t pol = 0;
+    if (hint == kHintEvictFirst) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    else if (hint == kHintEvictLast) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
 }
 
-// What a launch of the GEMM core covers.  Tile j of a CTA is id = blockIdx.x + j * gridDim.x with
-//   m_fast ? (m = id % n_mtiles, n = id / n_mtiles) : (m = id / n_ntiles, n = id % n_ntiles)
+// One tiled TMA load (x = innermost coordinate, 16-byte aligned by construction: multiples of 64 elements).
+// pol = 0: no hint.
+__device__ __forceinline__ void lm_tma_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, uint64_t pol) {
+    if (pol)
+        asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+                     :: "r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "l"(pol) : "memory");
+    else
+        asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                     :: "r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+// The same from a CTA of a pair: the barrier may be the peer's (the pair's leader collects both CTAs' bytes).
+__device__ __forceinline__ void lm_tma_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, uint64_t pol) {
+    if (pol)
+        asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+                     :: "r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "l"(pol) : "memory");
+    else
+        asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                     :: "r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+
+// What a launch of the GEMM core covers, and the order in which its tiles are handed out.  Work item j of a CTA
+// (or CTA pair) is id = its index + j * (number of CTAs or pairs); ids are laid over the n_m x n_ntiles grid of
+// work items (n_m = row tiles, or row-tile pairs for CTA pairs) as
+//   group == 0:  m_fast ? (m = id % n_m, n = id / n_m) : (m = id / n_ntiles, n = id % n_ntiles)
+//   group  > 0:  column tiles are taken `group` at a time; within a group the ids sweep over all m with n fastest.
+//                The CTAs that run together then share `group` B tiles and about (CTAs / group) A tiles: a working
+//                set that fits L2 whatever the size of A, and every B tile is fetched from HBM once per launch.
 struct GemmShape {
     int n_mtiles, n_ntiles, n_ksteps;
     int a_row0;                          // row offset added to A's TMA coordinate
     int m_fast;
+    int group;
+    int hint_a, hint_b;                  // L2 eviction hints of the operand loads (kHint...)
+    unsigned long long wait_limit_ns;    // bound of every wait on a pipeline barrier
+    int test_extra_tx;                   // 0; self-test of the bounded waits: bytes the first stage expects but never gets
 };
 
-__device__ __forceinline__ bool tile_of(const GemmShape& gs, uint32_t j, int& m, int& n) {
-    const long long id = (long long)blockIdx.x + (long long)j * gridDim.x;
-    if (id >= (long long)gs.n_mtiles * gs.n_ntiles) return false;
-    if (gs.m_fast) { m = (int)(id % gs.n_mtiles); n = (int)(id / gs.n_mtiles); }
-    else           { m = (int)(id / gs.n_ntiles); n = (int)(id % gs.n_ntiles); }
+__device__ __forceinline__ bool tile_from_id(const GemmShape& gs, long long id, int n_m, int& m, int& n) {
+    if (id >= (long long)n_m * gs.n_ntiles) return false;
+    if (gs.group > 0) {
+        const long long per_group = (long long)gs.group * n_m;
+        const int grp = (int)(id / per_group);
+        const int local = (int)(id - (long long)grp * per_group);
+        const int n0 = grp * gs.group;
+        const int width = min(gs.group, gs.n_ntiles - n0);         // the last group may be narrower
+        m = local / width; n = n0 + local % width;
+    } else if (gs.m_fast) { m = (int)(id % n_m); n = (int)(id / n_m); }
+    else                  { m = (int)(id / gs.n_ntiles); n = (int)(id % gs.n_ntiles); }
     return true;
+}
+
+__device__ __forceinline__ bool tile_of(const GemmShape& gs, uint32_t j, int& m, int& n) {
+    return tile_from_id(gs, (long long)blockIdx.x + (long long)j * gridDim.x, gs.n_mtiles, m, n);
 }
 
 // ---- epilogue output through shared memory ---------------------------------------------------------
@@ -279,26 +330,28 @@ lm_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
+            const uint64_t pol_a = lm_l2_policy(gs.hint_a), pol_b = lm_l2_policy(gs.hint_b);
             uint32_t it = 0;                                             // slab counter over the CTA's lifetime
             int m, n;
             for (uint32_t j = 0; tile_of(gs, j, m, n) && !*abort_flag; ++j) {
                 for (int k = 0; k < gs.n_ksteps; ++k, ++it) {
                     const uint32_t s = it % kStages, use = it / kStages;
-                    if (use > 0 && !lm_wait(lm_smem_u32(&sh.empty[s]), (use - 1) & 1, abort_flag)) break;
+                    if (use > 0 && !lm_wait(lm_smem_u32(&sh.empty[s]), (use - 1) & 1, abort_flag, gs.wait_limit_ns)) break;
                     const uint32_t bar = lm_smem_u32(&sh.full[s]);
                     const uint32_t dst_a = tiles + s * kStageBytes, dst_b = dst_a + kStageBytesA;
-                    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"((uint32_t)kStageBytes) : "memory");
+                    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                                 :: "r"(bar), "r"((uint32_t)kStageBytes + (it == 0 ? (uint32_t)gs.test_extra_tx : 0u)) : "memory");
                     if (!kAMn) {
-                        lm_tma_2d(dst_a, &map_a, bar, k * kBK, gs.a_row0 + m * kBM);
+                        lm_tma_2d(dst_a, &map_a, bar, k * kBK, gs.a_row0 + m * kBM, pol_a);
                     } else {
 #pragma unroll
-                        for (int i = 0; i < kBM / 64; ++i) lm_tma_2d(dst_a + i * kMnBoxBytes, &map_a, bar, m * kBM + 64 * i, k * kBK);
+                        for (int i = 0; i < kBM / 64; ++i) lm_tma_2d(dst_a + i * kMnBoxBytes, &map_a, bar, m * kBM + 64 * i, k * kBK, pol_a);
                     }
                     if (!kBMn) {
-                        lm_tma_2d(dst_b, &map_b, bar, k * kBK, n * kBN);
+                        lm_tma_2d(dst_b, &map_b, bar, k * kBK, n * kBN, pol_b);
                     } else {
 #pragma unroll
-                        for (int i = 0; i < kBN / 64; ++i) lm_tma_2d(dst_b + i * kMnBoxBytes, &map_b, bar, n * kBN + 64 * i, k * kBK);
+                        for (int i = 0; i < kBN / 64; ++i) lm_tma_2d(dst_b + i * kMnBoxBytes, &map_b, bar, n * kBN + 64 * i, k * kBK, pol_b);
                     }
                 }
             }
@@ -308,7 +361,7 @@ lm_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 const uint32_t pending = it < (uint32_t)kStages ? it : (uint32_t)kStages;
                 for (uint32_t i = 0; i < pending; ++i) {
                     const uint32_t i2 = it - 1 - i;
-                    lm_wait_plain(lm_smem_u32(&sh.full[i2 % kStages]), (i2 / kStages) & 1, 200000000ull);
+                    lm_wait_plain(lm_smem_u32(&sh.full[i2 % kStages]), (i2 / kStages) & 1, gs.wait_limit_ns);
                 }
             }
         }
@@ -319,13 +372,13 @@ lm_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             int m, n;
             for (uint32_t j = 0; tile_of(gs, j, m, n) && !*abort_flag; ++j) {
                 const uint32_t b = j & 1, use_b = j >> 1;
-                if (use_b > 0 && !lm_wait(lm_smem_u32(&sh.acc_empty[b]), (use_b - 1) & 1, abort_flag)) break;
+                if (use_b > 0 && !lm_wait(lm_smem_u32(&sh.acc_empty[b]), (use_b - 1) & 1, abort_flag, gs.wait_limit_ns)) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t d_tmem = tmem_base + b * kBN;
                 bool ok = true;
                 for (int k = 0; k < gs.n_ksteps; ++k, ++it) {
                     const uint32_t s = it % kStages, use = it / kStages;
-                    if (!lm_wait(lm_smem_u32(&sh.full[s]), use & 1, abort_flag)) { ok = false; break; }
+                    if (!lm_wait(lm_smem_u32(&sh.full[s]), use & 1, abort_flag, gs.wait_limit_ns)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t sa = tiles + s * kStageBytes, sb = sa + kStageBytesA;
                     const uint64_t da = lm_smem_desc<kAMn>(sa), db = lm_smem_desc<kBMn>(sb);
@@ -360,7 +413,7 @@ lm_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const uint32_t b = j & 1, use_b = j >> 1;
             epi.row_begin(m, n, row);
             // warp-uniform outcome: the tcgen05.ld below must be executed by all 32 lanes together
-            if (!__all_sync(0xffffffffu, lm_wait(lm_smem_u32(&sh.acc_full[b]), use_b & 1, abort_flag))) break;
+            if (!__all_sync(0xffffffffu, lm_wait(lm_smem_u32(&sh.acc_full[b]), use_b & 1, abort_flag, gs.wait_limit_ns))) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + b * kBN;
             if constexpr (Epi::kTwoPass) {                               // a first look at the whole tile (its row maxima)
@@ -420,12 +473,7 @@ struct LmShared2 {
 
 __device__ __forceinline__ bool pair_tile_of(const GemmShape& gs, uint32_t j, int& m2, int& n) {
     const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
-    const int n_m2 = (gs.n_mtiles + 1) >> 1;
-    const long long id = (long long)pair + (long long)j * npairs;
-    if (id >= (long long)n_m2 * gs.n_ntiles) return false;
-    if (gs.m_fast) { m2 = (int)(id % n_m2); n = (int)(id / n_m2); }
-    else           { m2 = (int)(id / gs.n_ntiles); n = (int)(id % gs.n_ntiles); }
-    return true;
+    return tile_from_id(gs, (long long)pair + (long long)j * npairs, (gs.n_mtiles + 1) >> 1, m2, n);
 }
 
 __device__ __forceinline__ void lm_cluster_sync() {
@@ -474,31 +522,43 @@ lm_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs)
         if (lane == 0) {
+            const uint64_t pol_a = lm_l2_policy(gs.hint_a), pol_b = lm_l2_policy(gs.hint_b);
             uint32_t it = 0;
             int m2, n;
             for (uint32_t j = 0; pair_tile_of(gs, j, m2, n) && !*abort_flag; ++j) {
                 const int m = 2 * m2 + (int)rank;
                 for (int k = 0; k < gs.n_ksteps; ++k, ++it) {
                     const uint32_t s = it % kStages2, use = it / kStages2;
-                    if (use > 0 && !lm_wait(lm_smem_u32(&sh.empty[s]), (use - 1) & 1, abort_flag)) break;
+                    if (use > 0 && !lm_wait(lm_smem_u32(&sh.empty[s]), (use - 1) & 1, abort_flag, gs.wait_limit_ns)) break;
                     const uint32_t bar_local = lm_smem_u32(&sh.full[s]);
                     const uint32_t bar = bar_local & kPeerMask;           // the leader's barrier collects both CTAs' bytes
                     const uint32_t dst_a = tiles + s * kStageBytes2, dst_b = dst_a + kStageBytesA;
                     if (leader)
-                        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar_local), "r"((uint32_t)(2 * kStageBytes2)) : "memory");
+                        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                                     :: "r"(bar_local), "r"((uint32_t)(2 * kStageBytes2) + (it == 0 ? (uint32_t)gs.test_extra_tx : 0u)) : "memory");
                     if (!kAMn) {
-                        lm_tma_2d_pair(dst_a, &map_a, bar, k * kBK, gs.a_row0 + m * kBM);
+                        lm_tma_2d_pair(dst_a, &map_a, bar, k * kBK, gs.a_row0 + m * kBM, pol_a);
                     } else {
 #pragma unroll
-                        for (int i = 0; i < kBM / 64; ++i) lm_tma_2d_pair(dst_a + i * kMnBoxBytes, &map_a, bar, m * kBM + 64 * i, k * kBK);
+                        for (int i = 0; i < kBM / 64; ++i) lm_tma_2d_pair(dst_a + i * kMnBoxBytes, &map_a, bar, m * kBM + 64 * i, k * kBK, pol_a);
                     }
                     const int nb0 = n * kBN + (int)rank * kHalfBN;       // this CTA's half of the B tile
                     if (!kBMn) {
-                        lm_tma_2d_pair(dst_b, &map_b, bar, k * kBK, nb0);
+                        lm_tma_2d_pair(dst_b, &map_b, bar, k * kBK, nb0, pol_b);
                     } else {
 #pragma unroll
-                        for (int i = 0; i < kHalfBN / 64; ++i) lm_tma_2d_pair(dst_b + i * kMnBoxBytes, &map_b, bar, nb0 + 64 * i, k * kBK);
+                        for (int i = 0; i < kHalfBN / 64; ++i) lm_tma_2d_pair(dst_b + i * kMnBoxBytes, &map_b, bar, nb0 + 64 * i, k * kBK, pol_b);
                     }
+                }
+            }
+            if (*abort_flag && leader) {
+                // leaving early: the leader's `full` barriers count the copies of both CTAs, so the leader gives the
+                // copies still in flight a bounded chance to land; its peer cannot leave before it (the cluster
+                // barrier on the way out), so neither CTA's shared memory goes away under a copy
+                const uint32_t pending = it < (uint32_t)kStages2 ? it : (uint32_t)kStages2;
+                for (uint32_t i = 0; i < pending; ++i) {
+                    const uint32_t i2 = it - 1 - i;
+                    lm_wait_plain(lm_smem_u32(&sh.full[i2 % kStages2]), (i2 / kStages2) & 1, gs.wait_limit_ns);
                 }
             }
         }
@@ -509,13 +569,13 @@ lm_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             int m2, n;
             for (uint32_t j = 0; pair_tile_of(gs, j, m2, n) && !*abort_flag; ++j) {
                 const uint32_t b = j & 1, use_b = j >> 1;
-                if (use_b > 0 && !lm_wait(lm_smem_u32(&sh.acc_empty[b]), (use_b - 1) & 1, abort_flag)) break;
+                if (use_b > 0 && !lm_wait(lm_smem_u32(&sh.acc_empty[b]), (use_b - 1) & 1, abort_flag, gs.wait_limit_ns)) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t d_tmem = tmem_base + b * kBN;
                 bool ok = true;
                 for (int k = 0; k < gs.n_ksteps; ++k, ++it) {
                     const uint32_t s = it % kStages2, use = it / kStages2;
-                    if (!lm_wait(lm_smem_u32(&sh.full[s]), use & 1, abort_flag)) { ok = false; break; }
+                    if (!lm_wait(lm_smem_u32(&sh.full[s]), use & 1, abort_flag, gs.wait_limit_ns)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t sa = tiles + s * kStageBytes2, sb = sa + kStageBytesA;
                     const uint64_t da = lm_smem_desc<kAMn>(sa), db = lm_smem_desc<kBMn>(sb);
@@ -550,7 +610,7 @@ lm_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             const int m = 2 * m2 + (int)rank;
             const uint32_t b = j & 1, use_b = j >> 1;
             epi.row_begin(m, n, row);
-            if (!__all_sync(0xffffffffu, lm_wait(lm_smem_u32(&sh.acc_full[b]), use_b & 1, abort_flag))) break;
+            if (!__all_sync(0xffffffffu, lm_wait(lm_smem_u32(&sh.acc_full[b]), use_b & 1, abort_flag, gs.wait_limit_ns))) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + b * kBN;
             if constexpr (Epi::kTwoPass) {                               // a first look at the whole tile (its row maxima)
@@ -1034,7 +1094,8 @@ static LmWorkspace lm_layout(const dppo_lmhead_params* p, bool backward) {
     LmWorkspace w;
     const long long T = p->loss.T_max > 0 ? p->loss.T_max : 1;
     auto al = [](size_t x) { return (x + 1023) & ~(size_t)1023; };
-    const size_t rows = (size_t)(T < kChunkTokens ? round_up(T, kBM) : kChunkTokens);   // rows of the per-chunk buffers
+    const int chunk = lm_tune(p->H).chunk_tokens;
+    const size_t rows = (size_t)(T < chunk ? round_up(T, kBM) : chunk);   // rows of the per-chunk buffers
     w.ld_v = round_up(p->loss.V, 8);
     w.n_ntiles = (p->loss.V + kBN - 1) / kBN;
     size_t off = 0;
@@ -1077,8 +1138,9 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
         return fail(DPPO_ERR_INVALID_ARG, "lmhead: temperature must be > 0, eps >= 0, beta a number");
     if ((lp.no_length_norm != 0 && lp.no_length_norm != 1) || (lp.seq_log_ratio && lp.no_length_norm))
         return fail(DPPO_ERR_INVALID_ARG, "lmhead: no_length_norm / seq_log_ratio");
-    if (lp.T_max >= ((int64_t)1 << 31) - kChunkTokens) return fail(DPPO_ERR_BAD_SHAPE, "lmhead: T_max too large");
-    if (p->variant != 0 && p->variant != 1) return fail(DPPO_ERR_INVALID_ARG, "lmhead: variant %d", p->variant);
+    if (lp.T_max >= ((int64_t)1 << 31) - kMaxChunkTokens) return fail(DPPO_ERR_BAD_SHAPE, "lmhead: T_max too large");
+    if (p->variant != 0 && p->variant != 1 && p->variant != 100 && p->variant != 101)
+        return fail(DPPO_ERR_INVALID_ARG, "lmhead: variant %d", p->variant);
     if (p->dW_dtype != DPPO_F32 && p->dW_dtype != DPPO_BF16) return fail(DPPO_ERR_INVALID_ARG, "lmhead: dW_dtype %d", p->dW_dtype);
     if ((p->accumulate_dW != 0 && p->accumulate_dW != 1) || p->reserved != 0)
         return fail(DPPO_ERR_INVALID_ARG, "lmhead: accumulate_dW %d reserved %d", p->accumulate_dW, p->reserved);
@@ -1108,11 +1170,16 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
     a.eps_lo = lp.eps_lo; a.eps_hi = lp.eps_hi; a.beta = lp.beta; a.temperature = lp.temperature;
     a.scale2 = (float)(1.4426950408889634 / lp.temperature);
     a.seq_log_ratio = lp.seq_log_ratio; a.no_length_norm = lp.no_length_norm;
+    a.wait_limit_ns = kDefaultWaitLimitNs; a.test_extra_tx = 0;
     cudaStream_t s = (cudaStream_t)stream;
     const int H = p->H, V = lp.V;
     const long long T = lp.T_max;          // host-side bound; rows at or past the device-side count carry g = 0
     if (T > 0) {
-        const bool pair = p->variant != 1;     // CTA pairs sharing the B tile unless the single-CTA core is forced
+        const bool pair = p->variant % 100 != 1;   // CTA pairs sharing the B tile unless the single-CTA core is forced
+        const bool self_test = p->variant >= 100;  // every CTA's first pipeline wait runs out (see dppo_lmhead_params.variant)
+        GemmShape gs0 = {};
+        gs0.wait_limit_ns = self_test ? kSelfTestWaitLimitNs : kDefaultWaitLimitNs;
+        gs0.test_extra_tx = self_test ? 16 : 0;
         alignas(64) CUtensorMap map_h, map_w, map_w_half;
         int rc = make_map(&map_h, hidden, T, H, H, kBM);
         if (rc != DPPO_OK) return rc;
@@ -1139,13 +1206,16 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
             }
         }
 
-        for (long long t0 = 0, c = 0; t0 < T; t0 += kChunkTokens, ++c) {
-            const long long tc = (T - t0) < kChunkTokens ? (T - t0) : kChunkTokens;     // tokens in this chunk
+        const LmTune tune = lm_tune(H);
+        const long long chunk = tune.chunk_tokens;
+        for (long long t0 = 0, c = 0; t0 < T; t0 += chunk, ++c) {
+            const long long tc = (T - t0) < chunk ? (T - t0) : chunk;                   // tokens in this chunk
             // (1) logits of the chunk, tile by tile: per-tile (max, sum) of every row, z[y], and (backward) the
             //     exponentials relative to the tile maxima, as fp16, into E [tc x V]
-            GemmShape g1 = {};
+            GemmShape g1 = gs0;
             g1.n_mtiles = (int)((tc + kBM - 1) / kBM); g1.n_ntiles = lay.n_ntiles; g1.n_ksteps = H / kBK;
             g1.a_row0 = (int)t0; g1.m_fast = 1;                                        // neighbours share the W tile
+            g1.group = tune.group_logits; g1.hint_a = tune.hints & 3; g1.hint_b = (tune.hints >> 2) & 3;
             if (backward) {
                 EpiPartialExp e1 = {};
                 e1.part = part; e1.zy_out = zy; e1.target = target; e1.n_tokens_dev = n_tokens_dev;
@@ -1174,8 +1244,9 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
             alignas(64) CUtensorMap map_d, map_d_mn, map_h_mn;
             rc = make_map(&map_d, D, tc, V, lay.ld_v, kBM);
             if (rc != DPPO_OK) return rc;
-            GemmShape g2 = {};
+            GemmShape g2 = gs0;
             g2.n_mtiles = (int)((tc + kBM - 1) / kBM); g2.n_ntiles = (H + kBN - 1) / kBN; g2.n_ksteps = (V + kBK - 1) / kBK;
+            g2.hint_a = (tune.hints >> 4) & 3; g2.hint_b = (tune.hints >> 6) & 3;
             EpiStoreBf16 e2 = {};
             e2.C = (__nv_bfloat16*)dhidden; e2.ldc = H; e2.row0 = t0; e2.rows = T; e2.cols = H;
             rc = run_gemm<EpiStoreBf16, false, true>(pair, map_d, map_w_mn, map_w_mn, map_d, g2, e2, status, s, "lmhead dhidden launch");
@@ -1186,8 +1257,9 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
             if (rc != DPPO_OK) return rc;
             rc = make_map(&map_h_mn, (const __nv_bfloat16*)hidden + t0 * H, tc, H, H, 64);
             if (rc != DPPO_OK) return rc;
-            GemmShape g3 = {};
+            GemmShape g3 = gs0;
             g3.n_mtiles = (V + kBM - 1) / kBM; g3.n_ntiles = (H + kBN - 1) / kBN; g3.n_ksteps = (int)((tc + kBK - 1) / kBK);
+            g3.group = tune.group_dw; g3.hint_a = (tune.hints >> 8) & 3; g3.hint_b = (tune.hints >> 10) & 3;
             EpiAccumF32 e3 = {};
             e3.rows = V; e3.cols = H; e3.accumulate = (c > 0 || p->accumulate_dW) ? 1 : 0;
             rc = run_gemm<EpiAccumF32, true, true>(pair, map_d_mn, map_h_mn, map_h_mn, map_dw, g3, e3, status, s, "lmhead dW launch");

@@ -7,6 +7,7 @@ All arithmetic happens inside libdppo.
 import torch
 
 from . import binding as B
+from . import dp
 
 
 class DppoStep:
@@ -19,7 +20,7 @@ class DppoStep:
     """
 
     def __init__(self, P, G, L_row, N_win, r_q, r_o, V, dtype, T_max, eps_lo=0.2, eps_hi=0.2, beta=0.04,
-                 temperature=1.0, mode=0, reverse=0, policy=0, std_ddof=0, std_eps=1e-6, device="cuda"):
+                 temperature=1.0, mode=0, reverse=0, policy=0, std_ddof=0, std_eps=1e-6, device="cuda", group=None):
         if not torch.cuda.is_available():
             raise RuntimeError("DppoStep needs a CUDA device: libdppo has no CPU path")
         self.P, self.G, self.n = P, G, P * G
@@ -28,6 +29,8 @@ class DppoStep:
         self.std_ddof, self.std_eps = std_ddof, std_eps
         dev = torch.device(device)
         self.device = dev
+        self.group = group                       # torch.distributed process group of the data-parallel ranks (or None)
+        self.H_table = None                      # dataset-wide history scores, owned by run_epochs
         n = self.n
         f32 = dict(dtype=torch.float32, device=dev)
         i32 = dict(dtype=torch.int32, device=dev)
@@ -135,6 +138,72 @@ class DppoStep:
         self.loss(dev_tokens["logits"], dev_tokens["target"], dev_tokens["logp_old"], dev_tokens["logp_ref"], dlogits)
         out = self.loss_out.cpu()                         # device -> host read of the result; synchronises
         return out, h2d, out.numel() * 4
+
+    # -- several ranks ---------------------------------------------------------------------------
+    def shard(self, world, rank):
+        """This rank's contiguous range of the packed rows of the last prune_pack (reads the packer's
+        outputs: synchronises).  See dp.shard_rows."""
+        n_units = int(self.counts[0].item())
+        order = self.order[:n_units].long()
+        return dp.shard_rows(self.row_of[order].cpu().tolist(), self.cu_seqlens.cpu().tolist(), n_units, world, rank)
+
+    def loss_shard(self, shard, logits, target, logp_old, logp_ref, dlogits=None, row_stride=None):
+        """Loss sweep over one rank's share of the packed rows: `logits` (and the other per-token inputs) hold the
+        tokens [tok_lo, tok_hi) of the batch, in packed order.  The sequence weights are those of the WHOLE batch,
+        so the five scalars of all ranks add up to the batch's (all_reduce_loss)."""
+        lo, hi = shard["seq_lo"], shard["seq_hi"]
+        T_r = shard["tok_hi"] - shard["tok_lo"]
+        prm = B.LossParams.from_buffer_copy(self.loss_params)
+        prm.T_max, prm.S_max = T_r, max(hi - lo, 1)
+        prm.row_stride = self.V if row_stride is None else row_stride
+        cu_local = (self.cu_seqlens[lo:hi + 1] - shard["tok_lo"]).contiguous() if hi > lo else self.cu_seqlens[:2] * 0
+        seg_map = self.order[lo:max(hi, lo + 1)].contiguous()
+        B.grpo_loss_fwd_bwd(prm, logits, target, logp_old, logp_ref, cu_local, None, self.adv, self.w_seq, seg_map,
+                            dlogits, self.logp_out, self.lse_out, self.loss_out, self.loss_ws, self.loss_ws_bytes,
+                            self.status)
+
+    def all_reduce_loss(self, average=False):
+        """Combines loss_out over the ranks of `group` (a no-op for a single process); see dp.all_reduce_loss."""
+        return dp.all_reduce_loss(self.loss_out, self.group, average)
+
+    # -- several epochs ----------------------------------------------------------------------------
+    def run_epochs(self, n_prompts, batches_by_epoch, rewards_fn, seed, lengths_fn=None, on_batch=None):
+        """Algorithm 1's outer loops around the small steps, with the dataset-wide history table of Eq. 16.
+
+        The table H (one score per dataset prompt, zero at the start) lives on the device and is owned by this
+        object (self.H_table).  For batch b of epoch t (a list of P dataset prompt ids): gather the prompts'
+        scores -> advantages -> candidate sets, masks and weights (no prompt pruning in the first epoch; the
+        generator's step word is t * 1,000,000 + b) -> scatter the updated scores back (retained prompts get their
+        fresh mean |A|, pruned ones keep the old score) -> pack the retained completions.  Every step is a library
+        call on the current stream; nothing is read back unless `on_batch` does.
+
+        rewards_fn(t, ids) -> float32 [P, G] rewards of those prompts in epoch t (host array)
+        lengths_fn(t, ids) -> (unit_len, loss_len) int32 [P*G] each, or None to skip the packing step
+        on_batch(t, b, self)  called after each batch with the results in this object's buffers
+        Returns self.H_table.
+        """
+        self.H_table = torch.zeros(n_prompts, dtype=torch.float32, device=self.device)
+        ids_dev = torch.zeros(self.P, dtype=torch.int32, device=self.device)
+        for t, batches in enumerate(batches_by_epoch):
+            for b, ids in enumerate(batches):
+                if len(ids) != self.P:
+                    raise ValueError("a batch must hold P = %d prompt ids, got %d" % (self.P, len(ids)))
+                ids_dev.copy_(torch.as_tensor(ids, dtype=torch.int32), non_blocking=False)
+                self.rewards.copy_(torch.as_tensor(rewards_fn(t, ids), dtype=torch.float32).reshape(-1))
+                if lengths_fn is not None:
+                    unit_len, loss_len = lengths_fn(t, ids)
+                    self.unit_len.copy_(torch.as_tensor(unit_len, dtype=torch.int32).reshape(-1))
+                    self.loss_len.copy_(torch.as_tensor(loss_len, dtype=torch.int32).reshape(-1))
+                B.history_gather(self.H_table, n_prompts, ids_dev, self.P, self.H_prev, self.status)
+                self.has_history = t > 0
+                self.advantages()
+                self.prune(seed, t * 1000000 + b)
+                B.history_scatter(self.H_table, n_prompts, ids_dev, self.P, self.H_next, self.status)
+                if lengths_fn is not None:
+                    self.pack()
+                if on_batch is not None:
+                    on_batch(t, b, self)
+        return self.H_table
 
     # -- results -----------------------------------------------------------------------------------
     def n_tokens(self):

@@ -29,7 +29,7 @@ def test_every_declared_symbol_is_exported(B):
             "dppo_pack_workspace_bytes", "dppo_pack_prompts", "dppo_grpo_loss_workspace_bytes",
             "dppo_grpo_loss_fwd_bwd", "dppo_pack_prompts_static", "dppo_pack_static_max_units",
             "dppo_history_gather", "dppo_history_scatter", "dppo_lmhead_workspace_bytes",
-            "dppo_lmhead_grpo_loss", "dppo_sequence_log_ratio"} <= set(names)
+            "dppo_lmhead_grpo_loss", "dppo_sequence_log_ratio", "dppo_grpo_loss_kernel_choice"} <= set(names)
     for n in names:
         assert hasattr(B.lib, n), n
     assert B.version() >= 100
@@ -37,7 +37,7 @@ def test_every_declared_symbol_is_exported(B):
 
 def test_struct_layouts_match_header(B):
     assert ctypes.sizeof(B.PruneParams) == 48
-    assert ctypes.sizeof(B.PackParams) == 16
+    assert ctypes.sizeof(B.PackParams) == 16 and ctypes.sizeof(B.LossKernelChoice) == 16
     assert ctypes.sizeof(B.LossParams) == 80 and B.LossParams.seq_log_ratio.offset == 72
     assert ctypes.sizeof(B.LmheadParams) == 104 and B.LmheadParams.dW_dtype.offset == 92
     assert B.LossParams.row_stride.offset == 16 and B.LossParams.eps_lo.offset == 32

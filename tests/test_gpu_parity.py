@@ -409,6 +409,10 @@ def test_loss_masked_vocabulary(dtype):
     _loss_case(V, dtype, T=6, S=2, seed=204, neg_inf_cols=(151669, V))
     _loss_case(V, dtype, T=6, S=2, seed=205, neg_inf_cols=(37984, 75968), variant=1)
     _loss_case(4099, dtype, T=20, S=2, seed=206, neg_inf_cols=(100, 4099))
+    # the general two-pass kernel with a masked START of the vocabulary: threads whose first elements are all -inf
+    _loss_case(V, dtype, T=6, S=2, seed=207, neg_inf_cols=(0, 37984), variant=1)
+    _loss_case(4099, dtype, T=20, S=2, seed=208, neg_inf_cols=(0, 100), variant=1)
+    _loss_case(4099, dtype, T=20, S=2, seed=209, neg_inf_cols=(0, 4090), variant=1)      # only the ragged end is finite
 
 
 @pytest.mark.parametrize("variant", [0, 1])
@@ -451,6 +455,31 @@ def test_loss_kernel_choice_boundaries(dtype):
         for V in (nvec * per_vec, nvec * per_vec + per_vec, nvec * per_vec + 3):
             seed += 1
             _loss_case(V, dtype, T=5, S=2, seed=seed, variant=0)
+
+
+def test_loss_kernel_choice_query():
+    # the host-side query names the kernel a call takes, for every branch of the choice
+    from paper_2603_04135_b200 import binding as B
+
+    def choice(V, dtype, variant=0):
+        esz = 2 if dtype == B.BF16 else 4
+        stride = -(-V * esz // 16) * 16 // esz
+        c = B.grpo_loss_kernel_choice(B.LossParams(64, V, dtype, stride, 4, variant, 0.2, 0.2, 0.04, 1.0))
+        return (c.kernel, c.ctas_per_row, c.threads, c.fell_back)
+
+    assert choice(1024, B.BF16) == (B.KERNEL_WARP, 1, 32, 0)
+    assert choice(2048, B.F32) == (B.KERNEL_WARP, 1, 32, 0)
+    assert choice(8192, B.BF16) == (B.KERNEL_SHARED, 1, 128, 0)
+    assert choice(16384, B.BF16) == (B.KERNEL_SHARED, 1, 256, 0)
+    assert choice(32768, B.BF16) == (B.KERNEL_SHARED, 2, 256, 0)
+    assert choice(151936, B.BF16) == (B.KERNEL_SHARED, 4, 256, 0)        # the benchmark's rows
+    assert choice(151936, B.F32) == (B.KERNEL_SHARED, 8, 256, 0)
+    assert choice(400000, B.BF16) == (B.KERNEL_GENERAL, 1, 512, 0)       # too long for eight slices: not a fall-back
+    assert choice(151936, B.BF16, variant=1)[0] == B.KERNEL_GENERAL
+    assert choice(151936, B.BF16, variant=80128) == (B.KERNEL_SHARED, 8, 128, 0)
+    with pytest.raises(B.DppoError) as e:
+        choice(151936, B.F32, variant=10256)                              # one CTA cannot hold 594 KB
+    assert e.value.code == B.ERR_UNSUPPORTED
 
 
 def test_loss_bad_target_and_empty():
