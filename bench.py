@@ -11,6 +11,12 @@ bf16 logits over a 151,936-token vocabulary, pruning probabilities 0.25 / 0.25).
 N > 1 is launched with torch.distributed.run, one rank per GPU; every rank works on its own batch
 (no data-path collective) and rank 0 reports the whole-job throughput with the max time over ranks.
 `--impl reference` times the float64 CPU oracle on the host cores instead (rank 0 only).
+
+Side modes (each prints its own lines and is not part of the default run):
+  --prune-pack-sweep            density / timing table of the pruning and packing sweep shape
+  --profile-case loss           a self-contained run of the loss sweep for timing and profiler captures
+                                (--rows --vocab --dtype --iters --in-place --full-call --back-to-back --variant)
+  --profile-case lmhead         the same for the fused LM-head (--tokens --hidden --vocab --iters --backward --variant)
 """
 import argparse
 import json
@@ -36,7 +42,7 @@ WORKLOAD = "config3"
 WORKLOAD_TEXT = WORKLOAD + ": P=32 G=8, response 64-1024 tokens, V=151936 bf16 logits, r_q=r_o=0.25, L_row=8192, N_win=16"
 
 
-# DRAM traffic of the dominant kernel from its last ncu capture (profiles/loss_sweep_cluster_kernel.md):
+# DRAM traffic of the dominant kernel from its last ncu capture:
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch over 8192 rows of this vocabulary.  Traffic
 # grows in proportion to the rows, so a launch over T rows moves T times the per-row figure.  The record
 # is tied to the kernel sources it was taken from: once they change, `traffic` is reported as null.
@@ -181,60 +187,161 @@ def run_reference(args):
     return 0
 
 
-def time_lmhead(T, H, V, dev, iters=3, warmup=1):
-    """Fused LM-head + loss, forward and backward (dhidden, dW), timed with CUDA events."""
+def bf16_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["bf16_tflops_sustained"]), "measured sustained cuBLAS bf16"
+    except Exception:
+        return 1400.0, "fallback sustained"
+
+
+def time_lmhead(H, dev, gpu_index, iters=10, warmup=3, sample_clocks=True):
+    """The fused LM-head configuration as stated: a batch of 64 prompts x 8 completions (64-1024 response tokens)
+    goes through advantages -> pruning with probabilities 0.5 / 0.5 -> packing, and the fused LM-head + loss runs on
+    the retained tokens with the packer's cu_seqlens, placement order and device-side token count and the
+    library's own advantages and sequence weights.  Forward + backward (dhidden, dW) and forward only, each timed
+    with CUDA events over `iters` calls after `warmup`, with the clocks sampled during the timed calls."""
     from paper_2603_04135_b200 import binding as B
-    wl = synth.scaled(synth.WORKLOADS["config4_h2560"], V=V, H=H)
-    hidden, W, target, lo, lr = synth.make_lmhead_inputs(wl, T, 4, device=dev)
-    S = 177
-    cu = torch.from_numpy(np.linspace(0, T, S + 1).astype(np.int32)).to(dev)
-    adv = torch.from_numpy(np.random.default_rng(4).normal(size=S).astype(np.float32)).to(dev)
-    wseq = torch.full((S,), 1.0 / S, device=dev)
-    prm = B.LmheadParams(B.LossParams(T, V, B.BF16, V, S, 0, wl.eps, wl.eps, wl.beta, 1.0), H, 1)
-    nbytes = B.lmhead_workspace_bytes(prm)
+    from paper_2603_04135_b200.step import DppoStep
+    w = synth.WORKLOADS["config4_h%d" % H]
+    seed = 4
+    batch = synth.make_batch(w, seed)
+    T_cap = int(batch.loss_len.sum())
+    st = DppoStep(w.P, w.G, w.L_row, w.N_win, w.r_q, w.r_o, w.V, w.dtype, T_cap, w.eps, w.eps, w.beta, device=dev)
+    prev = torch.from_numpy(batch.rewards_prev.reshape(-1).copy()).to(dev)
+    H_prev = torch.zeros(w.P, device=dev); scratch = torch.zeros(w.P * w.G, device=dev)
+    st.advantages(rewards=prev, adv=scratch, mean_abs_adv=H_prev)          # history scores: the earlier epoch's mean |A|
+    st.set_batch(batch.rewards, batch.unit_len, batch.loss_len, H_prev)
+    st.prune_pack(seed=seed, step=1)
+    T = st.n_tokens()
+    S = int(st.counts[0].item())
+    assert st.status.item() == 0 and 0 < T <= T_cap
+    hidden, W, target, lo, lr = synth.make_lmhead_inputs(w, T, seed, device=dev)   # exactly the retained tokens
+    V = w.V
+
+    def params(backward):
+        return B.LmheadParams(B.LossParams(T, V, B.BF16, V, w.P * w.G, 0, w.eps, w.eps, w.beta, 1.0), H, backward)
+
+    nbytes = max(B.lmhead_workspace_bytes(params(1)), B.lmhead_workspace_bytes(params(0)))
     ws = torch.zeros(nbytes + 1024, dtype=torch.uint8, device=dev)
     ws = ws[(-ws.data_ptr()) % 1024:]
     dh = torch.empty((T, H), dtype=torch.bfloat16, device=dev)
     dW = torch.empty((V, H), dtype=torch.float32, device=dev)
-    loss_out = torch.zeros(5, device=dev); status = torch.zeros(1, dtype=torch.int32, device=dev)
-    times = []
-    for it in range(warmup + iters):
+
+    def timed(backward):
+        prm = params(backward)
+        sampler = ClockSampler(gpu_index)
+        times = []
+        for it in range(warmup + iters):
+            if it == warmup and sample_clocks:
+                torch.cuda.synchronize()
+                sampler.start()
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+            e0.record()
+            B.lmhead_grpo_loss(prm, hidden, W, target, lo, lr, st.cu_seqlens, st.counts[3:4], st.adv, st.w_seq, st.order,
+                               dh if backward else None, dW if backward else None, None, None, st.loss_out, ws, nbytes,
+                               st.status)
+            e1.record()
+            times.append((e0, e1))
+        torch.cuda.synchronize()
+        clocks = sampler.stop() if sample_clocks else None
+        assert st.status.item() == 0 and st.loss_out[4].item() == T
+        ms = [a.elapsed_time(b) for a, b in times[warmup:]]
+        return sum(ms) / len(ms), min(ms), clocks
+
+    ms, ms_min, clocks = timed(1)
+    ms_f, ms_f_min, clocks_f = timed(0)
+    peak, peak_kind = bf16_peak()
+    executed = 6.0 * T * V * H / ms / 1e9
+    fwd = 2.0 * T * V * H / ms_f / 1e9
+    return {"config": {"workload": "config4_h%d: P=%d G=%d, response 64-1024 tokens, pruning probabilities r_q=r_o=%.2f "
+                                   "(retention 0.5 / 0.5) through prune -> pack; bf16 hidden [%d x %d], W [%d x %d]"
+                                   % (H, w.P, w.G, w.r_q, T, H, V, H),
+                       "valid_tokens": T, "sequences_retained": S, "unpruned_tokens": T_cap,
+                       "calls_timed": iters, "warmup": warmup},
+            "ms": ms, "ms_min": ms_min, "tokens_per_s": T / ms * 1e3, "executed_tflops": executed, "model_tflops_6TVH": executed,
+            "clocks": clocks,
+            "forward_only": {"ms": ms_f, "ms_min": ms_f_min, "tokens_per_s": T / ms_f * 1e3, "executed_tflops_2TVH": fwd,
+                             "frac_of_peak": fwd / peak, "clocks": clocks_f},
+            "roofline": {"bound": "tensor", "achieved": executed, "peak": peak, "unit": "TFLOP/s", "frac": executed / peak,
+                         "peak_source": peak_kind,
+                         "note": "executed flops = 6 T V H: logits, dhidden, dW (a chunk's exponentials are kept as bf16, nothing is recomputed)"}}
+
+
+# --------------------------------------------------------------------------------------- profile cases
+def run_profile_case(args):
+    """A small, self-contained run of one entry point for timing and profiler captures: prints the event-timed
+    duration of each call.  `loss`: dppo_grpo_loss_fwd_bwd on --rows token rows of the large-vocabulary workload
+    (bf16 logits, V = 151,936: 2.5 GB in + 2.5 GB out at 8192 rows, well above L2 yet small enough for a multi-pass
+    capture).  `lmhead`: dppo_lmhead_grpo_loss on --tokens tokens (2 T V H flops forward, 6 T V H with --backward)."""
+    from paper_2603_04135_b200 import binding as B
+    torch.cuda.set_device(0)
+    rng = np.random.default_rng(0)
+    if args.profile_case == "loss":
+        w = synth.scaled(synth.WORKLOADS["config3"], V=args.vocab, dtype=args.dtype)
+        T, S = args.rows, args.seqs
+        tok = synth.make_token_inputs(w, T, 0, device="cuda")
+        cu = torch.from_numpy(np.linspace(0, T, S + 1).astype(np.int32)).cuda()
+        adv = torch.from_numpy(rng.normal(size=S).astype(np.float32)).cuda()
+        wseq = torch.full((S,), 1.0 / S, device="cuda")
+        dl = tok.logits if args.in_place else torch.empty_like(tok.logits)
+        prm = B.LossParams(T, w.V, B.BF16 if args.dtype == "bf16" else B.F32, w.V, S, args.variant, w.eps, w.eps, w.beta, 1.0)
+        ch = B.grpo_loss_kernel_choice(prm)
+        print("kernel: %s, %d CTA(s) per row, %d threads%s" % (B.KERNEL_NAMES[ch.kernel], ch.ctas_per_row, ch.threads,
+                                                                  " (fell back)" if ch.fell_back else ""))
+        nbytes = B.grpo_loss_workspace_bytes(prm)
+        ws = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+        loss_out = torch.zeros(5, device="cuda"); status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        esize = 2 if args.dtype == "bf16" else 4
+        ntd = seg_map = logp_out = lse_out = None
+        if args.full_call:      # everything the training step passes: device token count, seg_map, logp / lse outputs
+            ntd = torch.tensor([T], dtype=torch.int32, device="cuda")
+            seg_map = torch.arange(S, dtype=torch.int32, device="cuda")
+            logp_out = torch.zeros(T, device="cuda"); lse_out = torch.zeros(T, device="cuda")
+        events = []
+        for it in range(args.iters):
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+            e0.record()
+            B.grpo_loss_fwd_bwd(prm, tok.logits, tok.target, tok.logp_old, tok.logp_ref, cu, ntd, adv, wseq, seg_map,
+                                None if args.forward_only else dl, logp_out, lse_out, loss_out, ws, nbytes, status)
+            e1.record()
+            events.append((e0, e1))
+            if not args.back_to_back:
+                torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        per_row = (1 if args.forward_only else 2) * w.V * esize
+        for it, (e0, e1) in enumerate(events):
+            ms = e0.elapsed_time(e1)
+            print("iter %d: %.3f ms  %.1f GB/s algorithmic  loss %.6g  status %d" % (
+                it, ms, T * per_row / ms / 1e6, loss_out[0].item(), status.item()))
+        assert status.item() == 0
+        return 0
+    w = synth.scaled(synth.WORKLOADS["config4_h2560"], V=args.vocab, H=args.hidden)
+    T, S = args.tokens, args.seqs
+    hidden, W, target, lo, lr = synth.make_lmhead_inputs(w, T, 0, device="cuda")
+    cu = torch.from_numpy(np.linspace(0, T, S + 1).astype(np.int32)).cuda()
+    adv = torch.from_numpy(rng.normal(size=S).astype(np.float32)).cuda()
+    wseq = torch.full((S,), 1.0 / S, device="cuda")
+    prm = B.LmheadParams(B.LossParams(T, w.V, B.BF16, w.V, S, 0, w.eps, w.eps, w.beta, 1.0), w.H, int(args.backward), args.variant)
+    nbytes = B.lmhead_workspace_bytes(prm)
+    ws = torch.zeros(nbytes + 1024, dtype=torch.uint8, device="cuda")
+    ws = ws[(-ws.data_ptr()) % 1024:]
+    dh = torch.empty((T, w.H), dtype=torch.bfloat16, device="cuda") if args.backward else None
+    dW = torch.empty((w.V, w.H), dtype=torch.float32, device="cuda") if args.backward else None
+    loss_out = torch.zeros(5, device="cuda"); status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    flops = (6.0 if args.backward else 2.0) * T * w.V * w.H          # logits, dhidden, dW: 2 T V H each
+    for it in range(args.iters):
         e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
         e0.record()
         B.lmhead_grpo_loss(prm, hidden, W, target, lo, lr, cu, None, adv, wseq, None, dh, dW, None, None, loss_out,
                            ws, nbytes, status)
         e1.record()
         torch.cuda.synchronize()
-        if it >= warmup:
-            times.append(e0.elapsed_time(e1))
+        ms = e0.elapsed_time(e1)
+        print("iter %d: %.3f ms  %.1f TFLOP/s executed  %.0f tokens/s  loss %.6g  status %d" % (
+            it, ms, flops / ms / 1e9, T / ms * 1e3, loss_out[0].item(), status.item()))
     assert status.item() == 0
-    ms = sum(times) / len(times)
-    # forward only (loss, log-probs, lse; no scratch kept): 2 T V H flops
-    prm_f = B.LmheadParams(B.LossParams(T, V, B.BF16, V, S, 0, wl.eps, wl.eps, wl.beta, 1.0), H, 0)
-    times_f = []
-    for it in range(warmup + iters):
-        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
-        e0.record()
-        B.lmhead_grpo_loss(prm_f, hidden, W, target, lo, lr, cu, None, adv, wseq, None, None, None, None, None, loss_out,
-                           ws, nbytes, status)
-        e1.record()
-        torch.cuda.synchronize()
-        if it >= warmup:
-            times_f.append(e0.elapsed_time(e1))
-    assert status.item() == 0
-    ms_f = sum(times_f) / len(times_f)
-    try:
-        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
-            peak = float(json.load(f)["bf16_tflops_sustained"]); peak_kind = "measured sustained cuBLAS bf16"
-    except Exception:
-        peak, peak_kind = 1400.0, "fallback sustained"
-    executed = 6.0 * T * V * H / ms / 1e9
-    return {"workload": "config4: bf16 hidden [%d x %d], W [%d x %d], forward + dhidden + dW" % (T, H, V, H),
-            "ms": ms, "tokens_per_s": T / ms * 1e3, "executed_tflops": executed, "model_tflops_6TVH": executed,
-            "forward_only": {"ms": ms_f, "tokens_per_s": T / ms_f * 1e3, "executed_tflops_2TVH": 2.0 * T * V * H / ms_f / 1e9,
-                             "frac_of_peak": 2.0 * T * V * H / ms_f / 1e9 / peak},
-            "roofline": {"bound": "tensor", "achieved": executed, "peak": peak, "unit": "TFLOP/s", "frac": executed / peak,
-                         "peak_source": peak_kind, "note": "executed flops = 6 T V H: logits, dhidden, dW (a chunk's exponentials are kept as fp16, nothing is recomputed)"}}
+    return 0
 
 
 # --------------------------------------------------------------------------------------- pruning / packing sweep
@@ -360,6 +467,52 @@ def run_ours(args):
     assert st.status.item() == 0
     loss_value = float(st.loss_out[0].item())
 
+    # ---- the same kernel in its other modes (rank 0 of a single-GPU run; a few calls each, CUDA events)
+    modes = None
+    if rank == 0 and world == 1 and not args.no_modes:
+        from paper_2603_04135_b200 import binding as B
+
+        def timed_calls(fn, n=5, warm=2):
+            evs = []
+            for it in range(warm + n):
+                a_, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a_.record(); fn(); b_.record()
+                evs.append((a_, b_))
+            torch.cuda.synchronize()
+            assert st.status.item() == 0
+            return sum(x.elapsed_time(y) for x, y in evs[warm:]) / n
+
+        slr = torch.zeros(w.P * w.G, device=dev)
+
+        def seq_ratio_step():
+            # sequence-level ratio: a forward-only sweep for the current log-probs, their per-sequence mean
+            # log-ratio, then the gradient sweep with that ratio (the logits are read twice)
+            st.loss_params.seq_log_ratio = None
+            st.loss(tok.logits, tok.target, tok.logp_old, tok.logp_ref, None)
+            B.sequence_log_ratio(st.logp_out, tok.logp_old, st.cu_seqlens, w.P * w.G, slr, st.status)
+            st.loss_params.seq_log_ratio = slr.data_ptr()
+            st.loss(tok.logits, tok.target, tok.logp_old, tok.logp_ref, dlogits)
+            st.loss_params.seq_log_ratio = None
+
+        peak_m, _ = measured_peaks()
+        vb = w.V * 2
+        modes = {}
+        for name, fn, bytes_per_token in (
+                ("forward_only", lambda: st.loss(tok.logits, tok.target, tok.logp_old, tok.logp_ref, None), vb),
+                ("seq_ratio", seq_ratio_step, 3 * vb),
+                ("in_place", lambda: st.loss(dlogits, tok.target, tok.logp_old, tok.logp_ref, dlogits), 2 * vb)):
+            if name == "in_place":
+                dlogits.copy_(tok.logits)                     # the in-place form overwrites its input
+            ms_mode = timed_calls(fn)
+            gbs = T * bytes_per_token / (ms_mode / 1e3) / 1e9
+            modes[name] = {"ms": ms_mode, "algorithmic_bytes_per_token": bytes_per_token, "achieved_gbs": gbs,
+                           "frac": gbs / peak_m, "tokens_per_s": T / ms_mode * 1e3}
+        modes["in_place"]["note"] = "dlogits written over the logits; after the first call the input is the previous gradient"
+        modes["seq_ratio"]["note"] = "forward-only sweep + per-sequence mean log-ratio + gradient sweep: two reads, one write"
+        ch = B.grpo_loss_kernel_choice(st.loss_params)
+        modes["kernel_choice"] = {"kernel": B.KERNEL_NAMES[ch.kernel], "ctas_per_row": ch.ctas_per_row, "threads": ch.threads,
+                                  "fell_back_to_general_kernel": bool(ch.fell_back)}
+
     # ---- end to end: host buffers in, loss scalars out, through DppoStep.step_from_host
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
     # pinned host copy of the step's inputs; when all ranks together would pin more than half of the
@@ -408,9 +561,9 @@ def run_ours(args):
     if rank == 0 and not args.no_lmhead:
         del tok, dlogits, dev_tok
         torch.cuda.empty_cache()
-        lm = time_lmhead(T, 2560, w.V, dev)
+        lm = time_lmhead(2560, dev, local_rank, sample_clocks=not args.no_clock_sampling)
         torch.cuda.empty_cache()
-        lm_wide = time_lmhead(T, 4096, w.V, dev)
+        lm_wide = time_lmhead(4096, dev, local_rank, sample_clocks=not args.no_clock_sampling)
     # ---- max over ranks, totals over ranks
     (total_ms, loss_ms, e2e_ms), T_all = dp.combine_over_ranks([total_ms, loss_ms, e2e_ms], T, device=dev)
 
@@ -440,6 +593,9 @@ def run_ours(args):
                          "traffic_note": "ncu dram bytes of an 8192-row capture of the same kernel, scaled by rows"},
             "loss": loss_value,
         }
+        if modes is not None:
+            line["roofline"]["kernel_choice"] = modes.pop("kernel_choice")
+            line["loss_sweep_modes"] = modes
         if lm is not None:
             line["lmhead"] = lm
             line["lmhead_h4096"] = lm_wide
@@ -466,12 +622,29 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=2048, help="token rows in the oracle's timed sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-lmhead", action="store_true", help="skip the fused LM-head measurement")
+    ap.add_argument("--no-modes", action="store_true", help="skip the forward-only / in-place / sequence-ratio timings")
+    ap.add_argument("--profile-case", choices=["loss", "lmhead"], help="instead of the benchmark: a small self-contained run")
+    ap.add_argument("--rows", type=int, default=8192)
+    ap.add_argument("--tokens", type=int, default=16384)
+    ap.add_argument("--hidden", type=int, default=2560)
+    ap.add_argument("--vocab", type=int, default=151936)
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"])
+    ap.add_argument("--iters", type=int, default=3)
+    ap.add_argument("--seqs", type=int, default=16)
+    ap.add_argument("--variant", type=int, default=0, help="kernel variant of the profile case (see include/dppo.h)")
+    ap.add_argument("--in-place", action="store_true")
+    ap.add_argument("--forward-only", action="store_true")
+    ap.add_argument("--full-call", action="store_true")
+    ap.add_argument("--back-to-back", action="store_true", help="enqueue all iterations before synchronising")
+    ap.add_argument("--backward", action="store_true", help="lmhead profile case: also dhidden and dW")
     ap.add_argument("--no-clock-sampling", action="store_true", help="do not poll nvidia-smi during the timed region")
     ap.add_argument("--prune-pack-sweep", action="store_true",
                     help="instead of the benchmark: density and timing table of the pruning / packing sweep shape")
     args = ap.parse_args()
     if args.prune_pack_sweep:
         sys.exit(run_prune_pack_sweep(args))
+    if args.profile_case:
+        sys.exit(run_profile_case(args))
     if args.impl == "ours" and args.warmup < 3:
         args.warmup = 3
     sys.exit(run_reference(args) if args.impl == "reference" else run_ours(args))

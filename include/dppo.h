@@ -52,7 +52,9 @@ typedef enum {                          /* values of the device status word */
     DPPO_STATUS_BAD_TARGET = 2,         /* loss: a target id outside [0, V)                           */
     DPPO_STATUS_TIMEOUT = 3,            /* a bounded device-side wait ran out                         */
     DPPO_STATUS_BAD_SEGMENTS = 4,       /* loss: cu_seqlens does not cover a token                    */
-    DPPO_STATUS_BAD_INDEX = 5           /* history: a prompt id outside the table                     */
+    DPPO_STATUS_BAD_INDEX = 5,          /* history: a prompt id outside the table                     */
+    DPPO_STATUS_RANGE = 6               /* fused LM-head backward: a sampled token whose log-prob under the
+                                           current policy is below about -66 (see dppo_lmhead_grpo_loss)  */
 } dppo_status;
 
 int dppo_version(void);                 /* major*10000 + minor*100 + patch */
@@ -150,8 +152,10 @@ size_t dppo_pack_workspace_bytes(const dppo_pack_params* p);
  *              n_units repeat the total, so the array is non-decreasing over its whole length
  *   counts     i32 [4] out: n_units, n_rows, total tokens, total loss tokens
  * A retained unit with length < 1 or > L_row sets status DPPO_STATUS_BAD_LENGTH and packs nothing
- * (counts = 0).  Errors: INVALID_ARG, BAD_SHAPE (n_max above the limit the workspace query
- * reports as 0 bytes), WORKSPACE_TOO_SMALL.
+ * (counts = 0); so does a stream whose tokens add up to 2^31 or more (the counts are i32).  The limit is
+ * n_max <= 2,097,152 units (a dataset-sized stream, packed once at set-up; one warp places about a million units
+ * per second).  Errors: INVALID_ARG, BAD_SHAPE (n_max above the limit: the workspace query reports 0 bytes),
+ * WORKSPACE_TOO_SMALL.
  */
 int dppo_pack_prompts(const dppo_pack_params* p, const int32_t* len, const uint8_t* keep,
                       const int32_t* loss_len, int32_t* order, int32_t* row_of, int32_t* off_in_row,
@@ -163,7 +167,7 @@ int dppo_pack_prompts(const dppo_pack_params* p, const int32_t* len, const uint8
  * sake of callers, not of the method.)
  *
  * Same operation, same arguments and same results as dppo_pack_prompts, minus `workspace`: the
- * scratch is a fixed 64 KB array inside the library's device image.  It is meant for callers that
+ * scratch is a fixed 32 KB array inside the library's device image.  It is meant for callers that
  * have no way to hand over device scratch at the point of the call: host code that is given only
  * its input and output buffers by a framework and owns no allocator, or a training loop whose
  * device memory is entirely reserved by a pool, where a cudaMalloc would fail or would stall every
@@ -171,10 +175,12 @@ int dppo_pack_prompts(const dppo_pack_params* p, const int32_t* len, const uint8
  * allocation).
  *
  *  - Limit: n_max <= dppo_pack_static_max_units() (8192 units); larger requests return
- *    DPPO_ERR_BAD_SHAPE and launch nothing.  Every GPU that loads the library holds the 64 KB until
+ *    DPPO_ERR_BAD_SHAPE and launch nothing.  Every GPU that loads the library holds the 32 KB until
  *    the process ends, used or not.
  *  - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
  *    that device current) and caches it; make that first call before starting any stream capture.
+ *    The cached address belongs to the device's context at that time: after cudaDeviceReset (or any
+ *    other way of replacing that context) this entry point must not be used again in the process.
  *  - All calls on a device share the one array.  It keeps whatever the previous call left there;
  *    the kernel never reads a slot before writing it, so nothing needs clearing.  Two calls whose
  *    kernels can overlap on the GPU (different streams, no ordering between them) race on it:
@@ -286,8 +292,13 @@ int dppo_sequence_log_ratio(const float* logp, const float* logp_old, const int3
  *   hidden   bf16 [T_max x H] row-major, one row per loss token in packed order
  *   W        bf16 [V x H] row-major LM-head weight
  *   backward 0: forward only (loss_out, logp_out, lse_out; dhidden and dW must be NULL).
- *            1: also the gradients, dhidden = D W and dW = D^T hidden.  The tokens are taken 9472 at a time;
- *            a chunk's exponentials (fp16) and its bf16 dlogits D live in workspace scratch (never the full [T x V])
+ *            1: also the gradients, dhidden = D W and dW = D^T hidden with D = dlogits.  The tokens are taken 9472
+ *            at a time.  A chunk's exponentials are kept in workspace scratch as bf16, relative to each row's own
+ *            reference, the sampled token's logit (never the full [T x V], and never the logits themselves); D is
+ *            that scratch times one factor per row, so the two contractions read the scratch directly and no
+ *            dlogits array is formed.  The reference bounds the representable rows: a sampled token whose log-prob
+ *            under the current policy is below about -66 sets status DPPO_STATUS_RANGE; that row adds nothing to
+ *            the loss and its gradient is zero
  *   dhidden  bf16 [T_max x H] out (rows at or past the true token count are zero)
  *   dW       [V x H] out, f32 or (params.dW_dtype = DPPO_BF16) bf16; overwritten, or added to when
  *            params.accumulate_dW = 1.  It is summed over the chunks in f32 either way (for bf16 in a workspace
@@ -296,7 +307,7 @@ int dppo_sequence_log_ratio(const float* logp, const float* logp_old, const int3
  *   other arguments as in dppo_grpo_loss_fwd_bwd.  The workspace (dppo_lmhead_workspace_bytes, which
  *   depends on `backward`) must be 1024-byte aligned.
  * Errors: INVALID_ARG, BAD_SHAPE (H not a multiple of 64), MISALIGNED, UNSUPPORTED, WORKSPACE_TOO_SMALL,
- * CUDA (tensor-map creation).  Device status: BAD_TARGET, BAD_SEGMENTS, TIMEOUT.
+ * CUDA (tensor-map creation).  Device status: BAD_TARGET, BAD_SEGMENTS, RANGE, TIMEOUT.
  */
 typedef struct {
     dppo_loss_params loss;

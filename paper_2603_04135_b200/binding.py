@@ -16,7 +16,8 @@ if not os.path.exists(_LIB_PATH):
 lib = ctypes.CDLL(_LIB_PATH)
 
 F32, BF16 = 0, 1
-STATUS_OK, STATUS_BAD_LENGTH, STATUS_BAD_TARGET, STATUS_TIMEOUT, STATUS_BAD_SEGMENTS, STATUS_BAD_INDEX = 0, 1, 2, 3, 4, 5
+STATUS_OK, STATUS_BAD_LENGTH, STATUS_BAD_TARGET, STATUS_TIMEOUT, STATUS_BAD_SEGMENTS, STATUS_BAD_INDEX, STATUS_RANGE = \
+    0, 1, 2, 3, 4, 5, 6
 ERR_INVALID_ARG, ERR_BAD_SHAPE, ERR_MISALIGNED, ERR_WORKSPACE_TOO_SMALL, ERR_UNSUPPORTED, ERR_CUDA = \
     -1, -2, -3, -4, -5, -6
 

@@ -70,7 +70,19 @@ grpo_loss_warp_kernel(const LossArgs a) {
     const bool has_tail = tail0 + lane < a.V;
     const float c = a.scale2;
 
-    for (long long t = warp0; t < T; t += n_warps) {
+    // Every warp takes a CONTIGUOUS range of rows.  Consecutive tokens mostly belong to the same sequence, so the
+    // sequence's scalars (bounds, advantage, weight) stay in registers from row to row and the search of cu_seqlens
+    // runs only when a row leaves the current sequence; the sampled token's logit is taken out of the registers
+    // that hold the row.  What is left on a row's dependent chain is one round trip: its vectors and its three
+    // per-token scalars, all issued together, while the next row is already on its way into L2.
+    const long long per_warp = (T + n_warps - 1) / n_warps;
+    const long long t_begin = min(T, warp0 * per_warp), t_end = min(T, t_begin + per_warp);
+    long long seg_lo = 0, seg_hi = 0;                       // empty: the first row looks its sequence up
+    __shared__ double seg_scalars[kWarps][3];               // the cached sequence's advantage, weight, log-ratio: read
+    double* seg = seg_scalars[threadIdx.x >> 5];            // once per row, so they need not occupy registers
+    bool seg_ok = false;
+
+    for (long long t = t_begin; t < t_end; ++t) {
         const char* row = a.logits + t * a.row_bytes;
         const uint4* rowv = reinterpret_cast<const uint4*>(row);
         uint4 d[kVPL];
@@ -80,8 +92,70 @@ grpo_loss_warp_kernel(const LossArgs a) {
             d[j] = i < nvec ? __ldcs(rowv + i) : make_uint4(kPad, kPad, kPad, kPad);
         }
         const float ztail = has_tail ? Elems<!kF32>::load1(row, tail0 + lane) : -INFINITY;
-        RowInputs in;                                       // filled by lane 0 while the loads are in flight
-        row_gather_warp(a, t, lane, in);
+        const int y_in = a.target[t];                       // the same address in every lane: one broadcast load each
+        const float lp_old = a.logp_old[t], lp_ref = a.logp_ref[t];
+        if (t + 1 < t_end) {                                // the next row's lines towards L2 (128 bytes per lane and step)
+            const char* nxt = row + a.row_bytes;
+            for (int off = lane * 128; off < (nvec << 4); off += 32 * 128)
+                asm volatile("prefetch.global.L2 [%0];" :: "l"(nxt + off));
+        }
+        if (t < seg_lo || t >= seg_hi) {                    // the row is outside the cached sequence: look it up
+            seg_ok = false;
+            if (a.S_max >= 1) {
+                int lo = 0, hi = a.S_max;
+                while (hi - lo > 1) {                       // 32 probes per round trip; cu_seqlens is non-decreasing
+                    const int step = (hi - lo + 31) >> 5;
+                    const long long idx = (long long)lo + (long long)(lane + 1) * step;
+                    const bool le = idx < hi && (long long)a.cu_seqlens[idx] <= t;
+                    const int n = __popc(__ballot_sync(0xffffffffu, le));
+                    lo += n * step;
+                    hi = min(hi, lo + step);
+                }
+                seg_lo = a.cu_seqlens[lo]; seg_hi = a.cu_seqlens[lo + 1];
+                if (t >= seg_lo && t < seg_hi) {
+                    seg_ok = true;
+                    const int idx = a.seg_map ? a.seg_map[lo] : lo;
+                    if (lane == 0) {
+                        seg[0] = (double)a.adv[idx];
+                        seg[1] = a.no_length_norm ? (double)a.w[idx] : (double)a.w[idx] / (double)(seg_hi - seg_lo);
+                        seg[2] = a.seq_log_ratio ? (double)a.seq_log_ratio[lo] : 0.0;
+                    }
+                    __syncwarp();
+                } else {
+                    seg_lo = seg_hi = 0;                    // no sequence covers this row: the next row searches again
+                }
+            }
+        }
+        // the sampled token's logit out of the registers: the lane and vector that hold element y_in
+        float zy_f = 0.0f;
+        const bool y_ok = y_in >= 0 && y_in < a.V;
+        if (y_ok) {
+            if (y_in >= tail0) {
+                zy_f = __shfl_sync(0xffffffffu, ztail, y_in - tail0);
+            } else {
+                const int yv = y_in >> kLog2PerVec, jy = yv >> 5;
+                const int wy = kF32 ? (y_in & 3) : ((y_in & 7) >> 1);
+                uint32_t word = 0;
+#pragma unroll
+                for (int j = 0; j < kVPL; ++j) {
+                    const uint32_t wj = wy == 0 ? d[j].x : wy == 1 ? d[j].y : wy == 2 ? d[j].z : d[j].w;
+                    word = j == jy ? wj : word;             // selects: d stays in registers
+                }
+                word = __shfl_sync(0xffffffffu, word, yv & 31);
+                zy_f = kF32 ? __uint_as_float(word) : __uint_as_float((y_in & 1) ? (word & 0xffff0000u) : (word << 16));
+            }
+        }
+        RowInputs in;
+        in.A = in.W = in.zy = in.logp_old = in.logp_ref = in.seq_lr = 0.0;
+        in.use_seq = 0; in.y = y_in; in.state = 0;
+        if (!seg_ok) in.state = DPPO_STATUS_BAD_SEGMENTS;
+        else if (!y_ok) in.state = DPPO_STATUS_BAD_TARGET;
+        else {
+            in.A = seg[0]; in.W = seg[1];
+            if (a.seq_log_ratio) { in.use_seq = 1; in.seq_lr = seg[2]; }
+            in.zy = (double)zy_f / a.temperature;
+            in.logp_old = (double)lp_old; in.logp_ref = (double)lp_ref;
+        }
 
         // ---- row maximum
         float m = ztail;

@@ -25,6 +25,8 @@
 #include <cuda.h>
 #include <cuda_fp16.h>
 
+#include <algorithm>
+
 #include "common.cuh"
 #include "grpo_loss.cuh"
 
@@ -45,14 +47,22 @@ constexpr int kMaxChunkTokens = 1 << 16;
 
 // Launch-shape choices of the call, by hidden width (from sweeps on B200 at 99,030 tokens, V = 151,936).
 struct LmTune {
-    int chunk_tokens;                    // a multiple of 256 (whole row-tile pairs)
+    int chunk_tokens;                    // tokens whose dlogits are held at a time (a multiple of 256: whole row-tile pairs)
+    int sub_tokens;                      // the logits, dlogits and dW launches take a chunk in pieces of about this size
     int group_logits;                    // column tiles per group of the logits launch (0: all row tiles of two column tiles at a time)
     int group_dw;                        // the same for the dW launch (0: all column tiles of a few row tiles at a time)
-    int hints;                           // two bits per operand load (kHint...): logits A, B; dhidden A, B; dW A, B
+    int hints;                           // two bits each (kHint...): loads of logits A, B; dhidden A, B; dW A, B; then the
+                                         // stores of the exponentials and the add-reductions of dW
 };
 static LmTune lm_tune(int H) {
-    (void)H;
-    LmTune t = {kChunkTokens, 0, 0, 0};
+    // The hidden rows of a piece are re-read by every wave of the logits and dW launches and should stay in L2
+    // between them: a piece holds at most about 48 MB of them (9472 rows at H = 2560: one piece per chunk; H = 4096:
+    // two pieces of 4864 and 4608 rows, 288 ms against 300 ms for the whole call).  Chunks of 18,944 tokens, pieces of
+    // a third or a quarter of a chunk, grouped tile orders and eviction hints on the loads or on the stores of the
+    // exponentials and of dW were all measured within 1 % of this choice or slower.
+    LmTune t = {kChunkTokens, kChunkTokens, 0, 0, 0};
+    const long long rows_48mb = (48500000ll / (2ll * (H > 0 ? H : 1))) / 256 * 256;
+    if (rows_48mb < kChunkTokens) t.sub_tokens = (int)(rows_48mb < 256 ? 256 : rows_48mb);
     return t;
 }
 
@@ -186,6 +196,7 @@ struct GemmShape {
     int m_fast;
     int group;
     int hint_a, hint_b;                  // L2 eviction hints of the operand loads (kHint...)
+    int hint_c;                          // and of the epilogue's tiled stores / add-reductions
     unsigned long long wait_limit_ns;    // bound of every wait on a pipeline barrier
     int test_extra_tx;                   // 0; self-test of the bounded waits: bytes the first stage expects but never gets
 };
@@ -219,6 +230,7 @@ constexpr int kStageBytesEpi = 4 * 2 * kStageTileBytes;  // 4 epilogue warps x 2
 
 struct EpiCtx {
     const CUtensorMap* map_c;            // f32 [rows x cols], 32 x 32 boxes, 128B swizzle
+    uint64_t pol;                        // L2 eviction policy of the tiled stores (0: none)
     uint32_t stage;                      // this warp's two staging buffers (shared::cta address, 1024-aligned)
     uint32_t toggle;
     int lane;
@@ -239,12 +251,21 @@ __device__ __forceinline__ void lm_store_block(EpiCtx& ctx, const uint32_t (&v)[
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncwarp();
     if (ctx.lane == 0) {
-        if (kAdd)
-            asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
-                         :: "l"(ctx.map_c), "r"(buf), "r"(x), "r"(y) : "memory");
-        else
-            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
-                         :: "l"(ctx.map_c), "r"(buf), "r"(x), "r"(y) : "memory");
+        if (kAdd) {
+            if (ctx.pol)
+                asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;"
+                             :: "l"(ctx.map_c), "r"(buf), "r"(x), "r"(y), "l"(ctx.pol) : "memory");
+            else
+                asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
+                             :: "l"(ctx.map_c), "r"(buf), "r"(x), "r"(y) : "memory");
+        } else {
+            if (ctx.pol)
+                asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;"
+                             :: "l"(ctx.map_c), "r"(buf), "r"(x), "r"(y), "l"(ctx.pol) : "memory");
+            else
+                asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
+                             :: "l"(ctx.map_c), "r"(buf), "r"(x), "r"(y) : "memory");
+        }
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
     }
     ctx.toggle ^= 1u;
@@ -268,8 +289,12 @@ __device__ __forceinline__ void lm_store_half_block(EpiCtx& ctx, const uint32_t 
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncwarp();
     if (ctx.lane == 0) {
-        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
-                     :: "l"(ctx.map_c), "r"(buf), "r"(x), "r"(y) : "memory");
+        if (ctx.pol)
+            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;"
+                         :: "l"(ctx.map_c), "r"(buf), "r"(x), "r"(y), "l"(ctx.pol) : "memory");
+        else
+            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
+                         :: "l"(ctx.map_c), "r"(buf), "r"(x), "r"(y) : "memory");
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
     }
     ctx.toggle ^= 1u;
@@ -406,7 +431,8 @@ lm_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int row = q * 32 + lane;
         Epi epi = epi_args;                                              // per-thread copy: its state lives in registers
         EpiCtx ctx;
-        ctx.map_c = &map_c; ctx.stage = tiles + kStages * kStageBytes + (uint32_t)q * (2 * kStageTileBytes);
+        ctx.map_c = &map_c; ctx.pol = lm_l2_policy(gs.hint_c);
+        ctx.stage = tiles + kStages * kStageBytes + (uint32_t)q * (2 * kStageTileBytes);
         ctx.toggle = 0; ctx.lane = lane;
         int m, n;
         for (uint32_t j = 0; tile_of(gs, j, m, n); ++j) {
@@ -603,7 +629,8 @@ lm_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         const int row = q * 32 + lane;
         Epi epi = epi_args;
         EpiCtx ctx;
-        ctx.map_c = &map_c; ctx.stage = tiles + kStages2 * kStageBytes2 + (uint32_t)q * (2 * kStageTileBytes);
+        ctx.map_c = &map_c; ctx.pol = lm_l2_policy(gs.hint_c);
+        ctx.stage = tiles + kStages2 * kStageBytes2 + (uint32_t)q * (2 * kStageTileBytes);
         ctx.toggle = 0; ctx.lane = lane;
         int m2, n;
         for (uint32_t j = 0; pair_tile_of(gs, j, m2, n); ++j) {
@@ -650,7 +677,8 @@ lm_gemm2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 // ---- epilogues ------------------------------------------------------------------------------------
 struct RowInfo {             // what the backward needs from the forward, per token
     float lse2_hi, lse2_lo;  // base-2 log-sum-exp of z * scale2
-    float g_over_tau;        // dloss/dlogp / temperature (0 for rows that add nothing)
+    float f;                 // dlogits[t, v] = -f * E'[t, v]: f = (dloss/dlogp / temperature) * 2^(ref - lse2); 0 for rows
+                             // that add nothing (no token, bad target, out of range)
     int y;                   // target, -1 if the row is invalid
 };
 
@@ -709,23 +737,35 @@ struct EpiPartial {
     }
 };
 
-// The same for a call with a backward pass: the tile is read out of tensor memory twice.  The first look takes
-// each row's maximum over the tile's 256 columns (and picks up the sampled token's logit); the second forms the
-// exponentials e = 2^(x - max) ONCE, adds them up for the log-sum-exp and keeps them, as fp16, in a chunk-sized
-// scratch E [chunk tokens x V]: softmax = e * 2^(max - lse2), so the backward scales them (no second exp) and
-// the f32 logits are never written out.  e lies in (0, 1]; fp16 keeps 11 bits of it down to 2^-14 of the tile's
-// largest term, far below what the bf16 dlogits resolve.
-struct EpiPartialExp {
-    static constexpr bool kTwoPass = true;
-    float2* part;            // [chunk tokens x n_ntiles]
-    float* zy_out;           // [chunk tokens]
+// The same for a call with a backward pass.  The exponentials are formed ONCE, relative to a per-row reference
+// that is known before the GEMM starts: the sampled token's own logit (ref2[t] = scale2 * hidden[t] . W[y_t],
+// one dot product per token, see lm_ref_kernel).  e = 2^(x - ref2) is added up for the log-sum-exp and kept, as
+// bf16, in a chunk-sized scratch E' [chunk tokens x V]; the f32 logits are never written out.  Because the
+// reference is the same for a whole row, softmax = e * 2^(ref2 - lse2) is a ROW scaling of E', and so is the
+// gradient: with the one entry E'[t, y_t] replaced by e_y - 2^(lse2 - ref2) (lm_rows_ref_kernel),
+//     dlogits[t, :] = -f_t * E'[t, :],   f_t = (dloss/dlogp / temperature) * 2^(ref2 - lse2).
+// The two gradient contractions therefore read E' itself: dhidden = -diag(f) (E' W) scales the accumulator rows
+// in its epilogue, dW = E'^T (-diag(f) hidden) takes pre-scaled hidden rows.  No dlogits pass, no second copy.
+// The row maximum is never below the sampled token's logit, so e >= 1 for the largest entry; bf16 has the exponent
+// range of f32, and the exponent is clamped at 100 so that sums of V such entries times weights stay far from the
+// f32 overflow in the two contractions.  A row counts as in range while its sum stays below 2^96, i.e. while its
+// sampled token has a log-prob above about -66 (any token a sampler could have drawn); rows beyond that are
+// reported by the rows kernel and get a zero gradient.
+constexpr float kMaxExp2 = 100.0f;
+constexpr float kMaxRowSum = 7.9e28f;        // 2^96
+
+struct EpiExpRef {
+    static constexpr bool kTwoPass = false;
+    float* sums;             // [piece tokens x n_ntiles] sum of e over the tile's columns
+    float* zy_out;           // [piece tokens]
+    const float* ref2;       // [T] the rows' references
     const int32_t* target;
     const int32_t* n_tokens_dev;
     long long T_max, t0, tc;
     int V, n_ntiles;
     float c;
     // per-thread state
-    float mraw, s, zy;
+    float nref, s, zy;
     int y;
     bool live, hit;
     __device__ __forceinline__ void row_begin(int m, int, int row) {
@@ -733,51 +773,68 @@ struct EpiPartialExp {
         const long long r = (long long)m * kBM + row;
         live = r < tc && t0 + r < T;
         y = live ? target[t0 + r] : -1;
-        mraw = -INFINITY; s = 0.0f; zy = 0.0f; hit = false;
+        nref = live ? -ref2[t0 + r] : 0.0f;
+        s = 0.0f; zy = 0.0f; hit = false;
     }
-    __device__ __forceinline__ void scan(int, int n, int, int ch, const uint32_t (&v)[32]) {
+    __device__ __forceinline__ void chunk(int m, int n, int row, int ch, uint32_t (&v)[32], EpiCtx& ctx) {
         const int col0 = n * kBN + ch * 32;
-        const int valid = V - col0;
-        if (valid <= 0) return;
+        const int valid = live ? V - col0 : 0;                       // rows without a token are written as zeros
+        const int y0 = m * kBM + row - ctx.lane;                     // first row of this warp's block
+        if (y0 >= tc || V - (col0 & ~63) <= 0) return;               // nothing of this 64-column block exists (whole warp)
         const int yrel = y - col0;
         hit = hit || (yrel >= 0 && yrel < 32);
-        float a0 = -INFINITY, a1 = -INFINITY;
+        uint32_t h[16];
+        float acc0 = 0.0f, acc1 = 0.0f;
 #pragma unroll
         for (int j = 0; j < 32; j += 2) {
             const float r0 = __uint_as_float(v[j]), r1 = __uint_as_float(v[j + 1]);
             zy = (j == yrel) ? r0 : zy;
             zy = (j + 1 == yrel) ? r1 : zy;
-            a0 = fmaxf(a0, (j < valid) ? r0 : -INFINITY);
-            a1 = fmaxf(a1, (j + 1 < valid) ? r1 : -INFINITY);
-        }
-        mraw = fmaxf(mraw, fmaxf(a0, a1));
-    }
-    __device__ __forceinline__ void chunk(int m, int n, int row, int ch, uint32_t (&v)[32], EpiCtx& ctx) {
-        const int col0 = n * kBN + ch * 32;
-        const int valid = V - col0;
-        const int y0 = m * kBM + row - ctx.lane;                     // first row of this warp's block
-        if (y0 >= tc || V - (col0 & ~63) <= 0) return;               // nothing of this 64-column block exists (whole warp)
-        const float nm2 = -(mraw * c);                               // c > 0: the maximum of x = raw * c is mraw * c
-        uint32_t h[16];
-        float acc0 = 0.0f, acc1 = 0.0f;
-#pragma unroll
-        for (int j = 0; j < 32; j += 2) {
-            const float e0 = (j < valid) ? lm_ex2(fmaf(__uint_as_float(v[j]), c, nm2)) : 0.0f;
-            const float e1 = (j + 1 < valid) ? lm_ex2(fmaf(__uint_as_float(v[j + 1]), c, nm2)) : 0.0f;
+            const float e0 = (j < valid) ? lm_ex2(fminf(fmaf(r0, c, nref), kMaxExp2)) : 0.0f;
+            const float e1 = (j + 1 < valid) ? lm_ex2(fminf(fmaf(r1, c, nref), kMaxExp2)) : 0.0f;
             acc0 += e0; acc1 += e1;
-            const __half2 p = __floats2half2_rn(e0, e1);
+            const __nv_bfloat162 p = __floats2bfloat162_rn(e0, e1);
             h[j >> 1] = *reinterpret_cast<const uint32_t*>(&p);
         }
         s += acc0 + acc1;
-        lm_store_half_block(ctx, h, ch & 1, col0 & ~63, y0);        // clipped at V and at the chunk's last row
+        lm_store_half_block(ctx, h, ch & 1, col0 & ~63, y0);        // clipped at V and at the piece's last row
     }
     __device__ __forceinline__ void row_end(int m, int n, int row) {
         if (!live) return;
         const long long r = (long long)m * kBM + row;
-        part[r * n_ntiles + n] = make_float2(mraw * c, s);
+        sums[r * n_ntiles + n] = s;
         if (hit) zy_out[r] = zy;
     }
 };
+
+// The rows' references for a backward call: ref2[t] = scale2 * (hidden[t] . W[y_t]) in f32, one warp per token
+// (0 for a row without a token or with a target outside the vocabulary).  It only has to be NEAR the logit the
+// tensor cores will produce for that entry: any value works as a reference, the log-prob itself uses the GEMM's.
+__global__ void __launch_bounds__(256)
+lm_ref_kernel(const __nv_bfloat16* __restrict__ hidden, const __nv_bfloat16* __restrict__ W, const int32_t* __restrict__ target,
+              const int32_t* __restrict__ n_tokens_dev, long long T_max, int V, int H, float c, float* __restrict__ ref2) {
+    const long long t = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (t >= T_max) return;
+    const long long T = n_tokens_dev ? min((long long)*n_tokens_dev, T_max) : T_max;
+    const int y = t < T ? target[t] : -1;
+    if (y < 0 || y >= V) { if (lane == 0) ref2[t] = 0.0f; return; }
+    const uint4* hr = reinterpret_cast<const uint4*>(hidden + t * H);
+    const uint4* wr = reinterpret_cast<const uint4*>(W + (long long)y * H);
+    float acc = 0.0f;
+    for (int i = lane; i < H / 8; i += 32) {                         // H is a multiple of 64
+        const uint4 a = hr[i], b = wr[i];
+        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            acc = fmaf(__uint_as_float(aw[k] << 16), __uint_as_float(bw[k] << 16), acc);
+            acc = fmaf(__uint_as_float(aw[k] & 0xffff0000u), __uint_as_float(bw[k] & 0xffff0000u), acc);
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) ref2[t] = acc * c;
+}
 
 // One warp per token of the chunk: the row's tile partials -> base-2 log-sum-exp, then the loss's scalar
 // stage (lane 0) -> per-row loss terms, logp, lse and what the backward needs.
@@ -785,16 +842,13 @@ constexpr int kRowsWarps = 8;
 
 __global__ void __launch_bounds__(kRowsWarps * 32)
 lm_rows_kernel(const LossArgs a, const float2* __restrict__ part, const float* __restrict__ zy,
-               RowInfo* __restrict__ info, long long t0, long long tc, int n_ntiles) {
+               long long t0, long long tc, int n_ntiles) {
     const long long r = (long long)blockIdx.x * kRowsWarps + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (r >= tc) return;
     const long long t = t0 + r;
     const long long T = a.n_tokens_dev ? min((long long)*a.n_tokens_dev, a.T_max) : a.T_max;
-    if (t >= T) {                                                    // no token here: the backward sees g = 0
-        if (lane == 0) { RowInfo z; z.lse2_hi = 0.0f; z.lse2_lo = 0.0f; z.g_over_tau = 0.0f; z.y = -1; info[t] = z; }
-        return;
-    }
+    if (t >= T) return;                                              // no token here
     float M = -INFINITY, S = 0.0f;
     for (int i = lane; i < n_ntiles; i += 32) {
         const float2 q = part[r * n_ntiles + i];                     // every tile holds a vocabulary column: q.x is finite
@@ -813,86 +867,97 @@ lm_rows_kernel(const LossArgs a, const float2* __restrict__ part, const float* _
         RowInputs in;
         row_gather(a, t, in, false);
         if (in.state == 0) in.zy = (double)zy[r] / a.temperature;
-        const RowScalars rs = row_finish(a, t, in, M, S, true);
-        RowInfo ri;
-        ri.lse2_hi = rs.lse2_hi; ri.lse2_lo = rs.lse2_lo;
-        ri.g_over_tau = rs.valid ? rs.g_over_tau : 0.0f;
-        ri.y = rs.valid ? in.y : -1;
-        info[t] = ri;
+        row_finish(a, t, in, M, S, true);
     }
 }
 
-// Backward, step 1: dlogits of the chunk from the stored exponentials, D = g (onehot - softmax) / tau with
-// softmax = e * 2^(tile max - lse2), as bf16 [chunk tokens x ldd].  Both later contractions read this one copy:
-// dhidden = D W takes it K-major, dW = D^T hidden takes it MN-major.  Rows with g = 0 (no token, bad target) are
-// written as zeros without reading their exponentials.  One thread per 8 vocabulary entries of a row (8 divides
-// the tile width, so a thread's entries share one tile maximum).
-constexpr int kDlogitsThreads = 256;
-constexpr int kDlogitsVecs = 4;              // 16-byte vectors per thread, a block's width apart: their loads overlap
-
-__device__ __forceinline__ uint4 lm_dlogits_vec(uint4 q, float f, float g, int yrel) {
-    const float2 e0 = __half22float2(*reinterpret_cast<const __half2*>(&q.x));
-    const float2 e1 = __half22float2(*reinterpret_cast<const __half2*>(&q.y));
-    const float2 e2 = __half22float2(*reinterpret_cast<const __half2*>(&q.z));
-    const float2 e3 = __half22float2(*reinterpret_cast<const __half2*>(&q.w));
-    const float e[8] = {e0.x, e0.y, e1.x, e1.y, e2.x, e2.y, e3.x, e3.y};
-    float d[8];
+// Backward: one warp per token of the piece.  The tile sums of the row -> base-2 log-sum-exp (reference + log2 of
+// their sum, added in a fixed order), the loss's scalar stage (lane 0), then what turns E' into the gradient:
+// the row factor f, the replacement of the sampled token's entry, and the row of -f * hidden that dW contracts
+// with.  A row whose sum has left the range of the reference (the sampled token's log-prob below about -66) is
+// reported as DPPO_STATUS_RANGE, adds nothing to the loss and gets a zero gradient.
+__global__ void __launch_bounds__(kRowsWarps * 32)
+lm_rows_ref_kernel(const LossArgs a, const float* __restrict__ sums, const float* __restrict__ zy,
+                   const float* __restrict__ ref2, RowInfo* __restrict__ info, long long t0, long long tc, int n_ntiles,
+                   __nv_bfloat16* __restrict__ E, long long lde, const __nv_bfloat16* __restrict__ hidden, int H,
+                   __nv_bfloat16* __restrict__ hs) {
+    const long long r = (long long)blockIdx.x * kRowsWarps + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (r >= tc) return;
+    const long long t = t0 + r;
+    const long long T = a.n_tokens_dev ? min((long long)*a.n_tokens_dev, a.T_max) : a.T_max;
+    float f = 0.0f;
+    if (t < T) {
+        float S = 0.0f;
+        for (int i = lane; i < n_ntiles; i += 32) S += sums[r * n_ntiles + i];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) d[j] = fmaf(-f, e[j], (j == yrel) ? g : 0.0f);
-    const __nv_bfloat162 b0 = __floats2bfloat162_rn(d[0], d[1]), b1 = __floats2bfloat162_rn(d[2], d[3]);
-    const __nv_bfloat162 b2 = __floats2bfloat162_rn(d[4], d[5]), b3 = __floats2bfloat162_rn(d[6], d[7]);
-    uint4 pk;
-    pk.x = *reinterpret_cast<const uint32_t*>(&b0); pk.y = *reinterpret_cast<const uint32_t*>(&b1);
-    pk.z = *reinterpret_cast<const uint32_t*>(&b2); pk.w = *reinterpret_cast<const uint32_t*>(&b3);
-    return pk;
-}
-
-__global__ void __launch_bounds__(kDlogitsThreads)
-lm_dlogits_kernel(const __half* __restrict__ E, long long lde, const float2* __restrict__ part, int n_ntiles,
-                  const RowInfo* __restrict__ info, long long t0, int V, __nv_bfloat16* __restrict__ D, long long ldd) {
-    const long long r = blockIdx.y;
-    const int col0 = (blockIdx.x * kDlogitsVecs * kDlogitsThreads + threadIdx.x) * 8;
-    const RowInfo ri = info[t0 + r];
-    const float g = ri.g_over_tau;
-    const __half* erow = E + r * lde;
-    __nv_bfloat16* drow = D + r * ldd;
-    uint4 q[kDlogitsVecs];
-    float mx[kDlogitsVecs];
-#pragma unroll
-    for (int i = 0; i < kDlogitsVecs; ++i) {                         // lde, ldd and the columns are multiples of 8
-        const int col = col0 + i * kDlogitsThreads * 8;
-        q[i] = make_uint4(0u, 0u, 0u, 0u);
-        mx[i] = 0.0f;
-        if (g != 0.0f && col + 8 <= V) {
-            q[i] = __ldcs(reinterpret_cast<const uint4*>(erow + col));
-            mx[i] = part[r * n_ntiles + col / kBN].x;                // the same tile for the whole warp
-        }
-    }
-#pragma unroll
-    for (int i = 0; i < kDlogitsVecs; ++i) {
-        const int col = col0 + i * kDlogitsThreads * 8;
-        if (col >= V) break;
-        const float f = g != 0.0f ? g * lm_ex2((mx[i] - ri.lse2_hi) - ri.lse2_lo) : 0.0f;   // g * 2^(tile max - lse2)
-        if (col + 8 <= V) {
-            *reinterpret_cast<uint4*>(drow + col) = lm_dlogits_vec(q[i], f, g, ri.y - col);
-        } else {                                                     // the row's ragged end, element by element
-            const float ft = g != 0.0f ? g * lm_ex2((part[r * n_ntiles + col / kBN].x - ri.lse2_hi) - ri.lse2_lo) : 0.0f;
-            for (int j = 0; col + j < V; ++j) {
-                float dj = 0.0f;
-                if (g != 0.0f) dj = fmaf(-ft, __half2float(erow[col + j]), (col + j == ri.y) ? g : 0.0f);
-                drow[col + j] = __float2bfloat16_rn(dj);
+        for (int o = 16; o > 0; o >>= 1) S += __shfl_xor_sync(0xffffffffu, S, o);
+        if (lane == 0) {
+            const float ref = ref2[t];
+            RowInfo ri; ri.lse2_hi = 0.0f; ri.lse2_lo = 0.0f; ri.f = 0.0f; ri.y = -1;
+            RowInputs in;
+            row_gather(a, t, in, false);
+            // log2(S) is how far the log-sum-exp lies above the reference; S >= about 1 since the row holds the
+            // sampled token's own entry
+            const bool in_range = S > 0.0f && S < kMaxRowSum;         // no entry of the row reached the clamp
+            if (in.state == 0 && !in_range) {
+                set_status(a.status, DPPO_STATUS_RANGE);
+                const RowTerms zero = {0.0, 0.0, 0.0, 0.0};
+                a.terms[t] = zero;
+                if (a.logp_out) a.logp_out[t] = 0.0f;
+                if (a.lse_out) a.lse_out[t] = 0.0f;
+            } else {
+                if (in.state == 0) in.zy = (double)zy[r] / a.temperature;
+                const RowScalars rs = row_finish(a, t, in, ref, in_range ? S : 1.0f, true);
+                if (rs.valid && rs.g_over_tau != 0.0f) {
+                    ri.lse2_hi = rs.lse2_hi; ri.lse2_lo = rs.lse2_lo; ri.y = in.y;
+                    ri.f = rs.g_over_tau * lm_ex2((ref - rs.lse2_hi) - rs.lse2_lo);
+                    // the sampled token's entry carries the onehot term: -f (e_y - 2^(lse2 - ref)) = g - f e_y
+                    const float ey = lm_ex2(fminf(fmaf(zy[r], a.scale2, -ref), kMaxExp2));
+                    E[r * lde + in.y] = __float2bfloat16_rn(ey - lm_ex2((rs.lse2_hi - ref) + rs.lse2_lo));
+                }
             }
+            info[t] = ri;
+            f = ri.f;
         }
+        f = __shfl_sync(0xffffffffu, f, 0);
+    } else if (lane == 0) {                                            // no token here: the backward sees f = 0
+        RowInfo z; z.lse2_hi = 0.0f; z.lse2_lo = 0.0f; z.f = 0.0f; z.y = -1;
+        info[t] = z;
+    }
+    // the piece's operand of the dW contraction: hs[r, :] = -f * hidden[t, :] as bf16
+    const uint4* hr = reinterpret_cast<const uint4*>(hidden + t * H);
+    uint4* out = reinterpret_cast<uint4*>(hs + r * H);
+    const float nf = -f;
+    for (int i = lane; i < H / 8; i += 32) {
+        uint4 q = make_uint4(0u, 0u, 0u, 0u);
+        if (f != 0.0f) {
+            const uint4 x = hr[i];
+            const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+            uint32_t o[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const __nv_bfloat162 b2 = __floats2bfloat162_rn(nf * __uint_as_float(w[k] << 16), nf * __uint_as_float(w[k] & 0xffff0000u));
+                o[k] = *reinterpret_cast<const uint32_t*>(&b2);
+            }
+            q = make_uint4(o[0], o[1], o[2], o[3]);
+        }
+        out[i] = q;
     }
 }
 
-// C[rows x ldc] = acc as bf16 (dhidden).
-struct EpiStoreBf16 {
+// C[rows x ldc] = -f[row] * acc as bf16 (dhidden: the accumulator is E' W, the row factor turns E' into dlogits).
+struct EpiStoreScaledBf16 {
     static constexpr bool kTwoPass = false;
     __nv_bfloat16* C;
+    const RowInfo* info;         // per token; indexed by output row
     long long ldc, row0, rows;   // output row of tile row 0; rows that exist in C
     int cols;
-    __device__ __forceinline__ void row_begin(int, int, int) {}
+    float nf;
+    __device__ __forceinline__ void row_begin(int m, int, int row) {
+        const long long r = row0 + (long long)m * kBM + row;
+        nf = r < rows ? -info[r].f : 0.0f;
+    }
     __device__ __forceinline__ void chunk(int m, int n, int row, int ch, uint32_t (&v)[32], EpiCtx&) {
         const long long r = row0 + (long long)m * kBM + row;
         const int col0 = n * kBN + ch * 32;
@@ -902,7 +967,7 @@ struct EpiStoreBf16 {
             uint32_t pk[16];
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
-                const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+                const __nv_bfloat162 b2 = __floats2bfloat162_rn(nf * __uint_as_float(v[2 * j]), nf * __uint_as_float(v[2 * j + 1]));
                 pk[j] = *reinterpret_cast<const uint32_t*>(&b2);
             }
             uint4* d4 = reinterpret_cast<uint4*>(dst);
@@ -912,7 +977,7 @@ struct EpiStoreBf16 {
             d4[3] = make_uint4(pk[12], pk[13], pk[14], pk[15]);
         } else {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) if (col0 + j < cols) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
+            for (int j = 0; j < 32; ++j) if (col0 + j < cols) dst[j] = __float2bfloat16_rn(nf * __uint_as_float(v[j]));
         }
     }
     __device__ __forceinline__ void row_end(int, int, int) {}
@@ -1010,16 +1075,16 @@ static int make_map_out(CUtensorMap* map, const void* base, long long rows, long
     return DPPO_OK;
 }
 
-// fp16 [rows x cols] with row pitch ld elements as the target of the half-block stores: boxes of 64 columns x 32
+// bf16 [rows x cols] with row pitch ld elements as the target of the half-block stores: boxes of 64 columns x 32
 // rows (128-byte rows), 128B swizzle.
-static int make_map_out_f16(CUtensorMap* map, const void* base, long long rows, long long cols, long long ld) {
+static int make_map_out_bf16(CUtensorMap* map, const void* base, long long rows, long long cols, long long ld) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return fail(DPPO_ERR_CUDA, "lmhead: cuTensorMapEncodeTiled is not available from this driver");
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
     const cuuint32_t box[2] = {64, 32};
     const cuuint32_t estr[2] = {1, 1};
-    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(DPPO_ERR_CUDA, "lmhead: cuTensorMapEncodeTiled (exponentials) failed with %d", (int)r);
@@ -1085,28 +1150,39 @@ static int run_gemm(bool pair, const CUtensorMap& ma, const CUtensorMap& mb, con
 static long long round_up(long long x, long long m) { return (x + m - 1) / m * m; }
 
 struct LmWorkspace {
-    size_t terms, info, part, zy, z, d, dw32, total;   // byte offsets and the total
-    long long ld_v;                              // pitch of E and D (vocabulary)
+    size_t terms, info, ref, part, zy, e, hs, dw32, total;   // byte offsets and the total
+    long long ld_v;                              // pitch of E' (vocabulary)
     int n_ntiles;
 };
+
+// A chunk of tc tokens is taken in ceil(tc / sub) pieces of equal size, rounded up to whole row-tile pairs (the
+// last piece takes what is left): the size of a piece.
+static long long lm_piece_tokens(long long tc, int sub) {
+    if (sub < 256) sub = 256;
+    const long long n_pieces = (tc + sub - 1) / sub;
+    return n_pieces <= 1 ? tc : round_up((tc + n_pieces - 1) / n_pieces, 256);
+}
 
 static LmWorkspace lm_layout(const dppo_lmhead_params* p, bool backward) {
     LmWorkspace w;
     const long long T = p->loss.T_max > 0 ? p->loss.T_max : 1;
     auto al = [](size_t x) { return (x + 1023) & ~(size_t)1023; };
-    const int chunk = lm_tune(p->H).chunk_tokens;
-    const size_t rows = (size_t)(T < chunk ? round_up(T, kBM) : chunk);   // rows of the per-chunk buffers
+    const LmTune tune = lm_tune(p->H);
+    const size_t rows_d = (size_t)(T < tune.chunk_tokens ? round_up(T, kBM) : tune.chunk_tokens);   // rows of the dlogits scratch
+    // rows of the per-piece buffers: no piece of any chunk is longer than the piece size rounded up to a tile pair
+    const size_t rows = (size_t)std::min(round_up((long long)rows_d, 256), round_up(std::max(tune.sub_tokens, 256), 256));
     w.ld_v = round_up(p->loss.V, 8);
     w.n_ntiles = (p->loss.V + kBN - 1) / kBN;
     size_t off = 0;
     w.terms = off; off += al(loss_terms_bytes(T));
     w.info = off;  off += al((size_t)T * sizeof(RowInfo));
+    w.ref = off;   off += backward ? al((size_t)T * sizeof(float)) : 0;
     w.part = off;  off += al(rows * w.n_ntiles * sizeof(float2));
     w.zy = off;    off += al(rows * sizeof(float));
-    w.z = w.d = w.dw32 = off;
+    w.e = w.hs = w.dw32 = off;
     if (backward) {
-        w.z = off;  off += al(rows * w.ld_v * 2);
-        w.d = off;  off += al(rows * w.ld_v * 2);
+        w.e = off;   off += al(rows_d * w.ld_v * 2);                  // E' of a chunk
+        w.hs = off;  off += al(rows * (size_t)p->H * 2);              // -f * hidden of a piece
         if (p->dW_dtype == DPPO_BF16) { w.dw32 = off; off += al((size_t)p->loss.V * p->H * 4); }   // dW is accumulated in f32
     }
     w.total = off;
@@ -1190,8 +1266,9 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
         RowInfo* info = (RowInfo*)(ws + lay.info);
         float2* part = (float2*)(ws + lay.part);
         float* zy = (float*)(ws + lay.zy);
-        __half* E = backward ? (__half*)(ws + lay.z) : nullptr;
-        __nv_bfloat16* D = (__nv_bfloat16*)(ws + lay.d);
+        __nv_bfloat16* E = (__nv_bfloat16*)(ws + lay.e);                               // E' of the current chunk
+        __nv_bfloat16* hs = (__nv_bfloat16*)(ws + lay.hs);
+        float* ref2 = (float*)(ws + lay.ref);
         alignas(64) CUtensorMap map_w_mn;                                              // W as [K = V][N = H]
         alignas(64) CUtensorMap map_dw;
         if (backward) {
@@ -1199,6 +1276,10 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
             if (rc != DPPO_OK) return rc;
             rc = make_map_out(&map_dw, p->dW_dtype == DPPO_BF16 ? (void*)(ws + lay.dw32) : dW, V, H, H);
             if (rc != DPPO_OK) return rc;
+            // the rows' references: the sampled tokens' own logits
+            lm_ref_kernel<<<(unsigned)((T + 7) / 8), 256, 0, s>>>((const __nv_bfloat16*)hidden, (const __nv_bfloat16*)W, target,
+                                                               n_tokens_dev, T, V, H, a.scale2, ref2);
+            DPPO_CHECK_LAUNCH("lmhead reference launch");
             if (p->accumulate_dW && p->dW_dtype == DPPO_BF16) {        // the f32 sum starts from the caller's bf16 dW
                 const long long n = (long long)V * H;
                 lm_bf16_to_f32_kernel<<<(unsigned)((n / 8 + 255) / 256), 256, 0, s>>>((const __nv_bfloat16*)dW, (float*)(ws + lay.dw32), n);
@@ -1208,61 +1289,75 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
 
         const LmTune tune = lm_tune(H);
         const long long chunk = tune.chunk_tokens;
-        for (long long t0 = 0, c = 0; t0 < T; t0 += chunk, ++c) {
+        long long n_dw = 0;                                                            // dW launches so far
+        for (long long t0 = 0; t0 < T; t0 += chunk) {
             const long long tc = (T - t0) < chunk ? (T - t0) : chunk;                   // tokens in this chunk
-            // (1) logits of the chunk, tile by tile: per-tile (max, sum) of every row, z[y], and (backward) the
-            //     exponentials relative to the tile maxima, as fp16, into E [tc x V]
-            GemmShape g1 = gs0;
-            g1.n_mtiles = (int)((tc + kBM - 1) / kBM); g1.n_ntiles = lay.n_ntiles; g1.n_ksteps = H / kBK;
-            g1.a_row0 = (int)t0; g1.m_fast = 1;                                        // neighbours share the W tile
-            g1.group = tune.group_logits; g1.hint_a = tune.hints & 3; g1.hint_b = (tune.hints >> 2) & 3;
-            if (backward) {
-                EpiPartialExp e1 = {};
-                e1.part = part; e1.zy_out = zy; e1.target = target; e1.n_tokens_dev = n_tokens_dev;
-                e1.T_max = T; e1.t0 = t0; e1.tc = tc; e1.V = V; e1.n_ntiles = lay.n_ntiles; e1.c = a.scale2;
-                alignas(64) CUtensorMap map_e;
-                rc = make_map_out_f16(&map_e, E, tc, V, lay.ld_v);
+            const long long piece = lm_piece_tokens(tc, tune.sub_tokens);
+            for (long long s0 = t0; s0 < t0 + tc; s0 += piece) {
+                const long long ts = (t0 + tc - s0) < piece ? (t0 + tc - s0) : piece;   // tokens in this piece
+                // (1) logits of the piece, tile by tile.  Forward only: per-tile (max, sum) of every row and z[y].
+                //     Backward: the exponentials relative to the rows' references, as bf16, into the piece's rows of
+                //     E' [tc x V], their per-tile sums and z[y]
+                GemmShape g1 = gs0;
+                g1.n_mtiles = (int)((ts + kBM - 1) / kBM); g1.n_ntiles = lay.n_ntiles; g1.n_ksteps = H / kBK;
+                g1.a_row0 = (int)s0; g1.m_fast = 1;                                    // neighbours share the W tile
+                g1.group = tune.group_logits; g1.hint_a = tune.hints & 3; g1.hint_b = (tune.hints >> 2) & 3;
+                g1.hint_c = (tune.hints >> 12) & 3;
+                __nv_bfloat16* Ep = E + (s0 - t0) * lay.ld_v;
+                if (backward) {
+                    EpiExpRef e1 = {};
+                    e1.sums = (float*)part; e1.zy_out = zy; e1.ref2 = ref2; e1.target = target; e1.n_tokens_dev = n_tokens_dev;
+                    e1.T_max = T; e1.t0 = s0; e1.tc = ts; e1.V = V; e1.n_ntiles = lay.n_ntiles; e1.c = a.scale2;
+                    alignas(64) CUtensorMap map_e;
+                    rc = make_map_out_bf16(&map_e, Ep, ts, V, lay.ld_v);
+                    if (rc != DPPO_OK) return rc;
+                    rc = run_gemm<EpiExpRef, false, false>(pair, map_h, map_w, map_w_half, map_e, g1, e1, status, s, "lmhead logits launch");
+                } else {
+                    EpiPartial e1 = {};
+                    e1.part = part; e1.zy_out = zy; e1.target = target; e1.n_tokens_dev = n_tokens_dev;
+                    e1.T_max = T; e1.t0 = s0; e1.tc = ts; e1.V = V; e1.n_ntiles = lay.n_ntiles; e1.c = a.scale2;
+                    rc = run_gemm<EpiPartial, false, false>(pair, map_h, map_w, map_w_half, map_h, g1, e1, status, s, "lmhead logits launch");
+                }
                 if (rc != DPPO_OK) return rc;
-                rc = run_gemm<EpiPartialExp, false, false>(pair, map_h, map_w, map_w_half, map_e, g1, e1, status, s, "lmhead logits launch");
-            } else {
-                EpiPartial e1 = {};
-                e1.part = part; e1.zy_out = zy; e1.target = target; e1.n_tokens_dev = n_tokens_dev;
-                e1.T_max = T; e1.t0 = t0; e1.tc = tc; e1.V = V; e1.n_ntiles = lay.n_ntiles; e1.c = a.scale2;
-                rc = run_gemm<EpiPartial, false, false>(pair, map_h, map_w, map_w_half, map_h, g1, e1, status, s, "lmhead logits launch");
+                // (2) rows: log-sum-exp, logp, loss terms; backward: the row factors f, the sampled tokens' entries of
+                //     E' and the piece's -f * hidden
+                if (!backward) {
+                    lm_rows_kernel<<<(unsigned)((ts + kRowsWarps - 1) / kRowsWarps), kRowsWarps * 32, 0, s>>>(
+                        a, part, zy, s0, ts, lay.n_ntiles);
+                    DPPO_CHECK_LAUNCH("lmhead rows launch");
+                    continue;
+                }
+                lm_rows_ref_kernel<<<(unsigned)((ts + kRowsWarps - 1) / kRowsWarps), kRowsWarps * 32, 0, s>>>(
+                    a, (const float*)part, zy, ref2, info, s0, ts, lay.n_ntiles, Ep, lay.ld_v, (const __nv_bfloat16*)hidden, H, hs);
+                DPPO_CHECK_LAUNCH("lmhead rows launch");
+                // (3) dW (+)= E'^T (-f hidden)[s0 : s0+ts, :]   (M = V, N = H, K = tokens of the piece; both MN-major);
+                //     the K range stops at the piece: both maps have ts rows and fill with zeros beyond
+                alignas(64) CUtensorMap map_e_mn, map_hs_mn;
+                rc = make_map(&map_e_mn, Ep, ts, V, lay.ld_v, 64);
+                if (rc != DPPO_OK) return rc;
+                rc = make_map(&map_hs_mn, hs, ts, H, H, 64);
+                if (rc != DPPO_OK) return rc;
+                GemmShape g3 = gs0;
+                g3.n_mtiles = (V + kBM - 1) / kBM; g3.n_ntiles = (H + kBN - 1) / kBN; g3.n_ksteps = (int)((ts + kBK - 1) / kBK);
+                g3.group = tune.group_dw; g3.hint_a = (tune.hints >> 8) & 3; g3.hint_b = (tune.hints >> 10) & 3;
+                g3.hint_c = (tune.hints >> 14) & 3;
+                EpiAccumF32 e3 = {};
+                e3.rows = V; e3.cols = H; e3.accumulate = (n_dw > 0 || p->accumulate_dW) ? 1 : 0;
+                rc = run_gemm<EpiAccumF32, true, true>(pair, map_e_mn, map_hs_mn, map_hs_mn, map_dw, g3, e3, status, s, "lmhead dW launch");
+                if (rc != DPPO_OK) return rc;
+                ++n_dw;
             }
-            if (rc != DPPO_OK) return rc;
-            // (2) rows: log-sum-exp, logp, loss terms, dloss/dlogp
-            lm_rows_kernel<<<(unsigned)((tc + kRowsWarps - 1) / kRowsWarps), kRowsWarps * 32, 0, s>>>(
-                a, part, zy, info, t0, tc, lay.n_ntiles);
-            DPPO_CHECK_LAUNCH("lmhead rows launch");
             if (!backward) continue;
-            // (3) dlogits of the chunk: D [tc x V]
-            lm_dlogits_kernel<<<dim3((unsigned)((V + 8 * kDlogitsVecs * kDlogitsThreads - 1) / (8 * kDlogitsVecs * kDlogitsThreads)), (unsigned)tc),
-                                kDlogitsThreads, 0, s>>>(E, lay.ld_v, part, lay.n_ntiles, info, t0, V, D, lay.ld_v);
-            DPPO_CHECK_LAUNCH("lmhead dlogits launch");
-            // (4) dhidden[t0 : t0+tc, :] = D W            (M = tokens, N = H, K = V; D K-major, W MN-major)
-            alignas(64) CUtensorMap map_d, map_d_mn, map_h_mn;
-            rc = make_map(&map_d, D, tc, V, lay.ld_v, kBM);
+            // (4) dhidden[t0 : t0+tc, :] = -diag(f) (E' W)   (M = tokens of the chunk, N = H, K = V; E' K-major, W MN-major)
+            alignas(64) CUtensorMap map_e_k;
+            rc = make_map(&map_e_k, E, tc, V, lay.ld_v, kBM);
             if (rc != DPPO_OK) return rc;
             GemmShape g2 = gs0;
             g2.n_mtiles = (int)((tc + kBM - 1) / kBM); g2.n_ntiles = (H + kBN - 1) / kBN; g2.n_ksteps = (V + kBK - 1) / kBK;
             g2.hint_a = (tune.hints >> 4) & 3; g2.hint_b = (tune.hints >> 6) & 3;
-            EpiStoreBf16 e2 = {};
-            e2.C = (__nv_bfloat16*)dhidden; e2.ldc = H; e2.row0 = t0; e2.rows = T; e2.cols = H;
-            rc = run_gemm<EpiStoreBf16, false, true>(pair, map_d, map_w_mn, map_w_mn, map_d, g2, e2, status, s, "lmhead dhidden launch");
-            if (rc != DPPO_OK) return rc;
-            // (5) dW (+)= D^T hidden[t0 : t0+tc, :]       (M = V, N = H, K = tokens of the chunk; both MN-major);
-            //     the K range stops at the chunk: both maps have tc rows and fill with zeros beyond
-            rc = make_map(&map_d_mn, D, tc, V, lay.ld_v, 64);
-            if (rc != DPPO_OK) return rc;
-            rc = make_map(&map_h_mn, (const __nv_bfloat16*)hidden + t0 * H, tc, H, H, 64);
-            if (rc != DPPO_OK) return rc;
-            GemmShape g3 = gs0;
-            g3.n_mtiles = (V + kBM - 1) / kBM; g3.n_ntiles = (H + kBN - 1) / kBN; g3.n_ksteps = (int)((tc + kBK - 1) / kBK);
-            g3.group = tune.group_dw; g3.hint_a = (tune.hints >> 8) & 3; g3.hint_b = (tune.hints >> 10) & 3;
-            EpiAccumF32 e3 = {};
-            e3.rows = V; e3.cols = H; e3.accumulate = (c > 0 || p->accumulate_dW) ? 1 : 0;
-            rc = run_gemm<EpiAccumF32, true, true>(pair, map_d_mn, map_h_mn, map_h_mn, map_dw, g3, e3, status, s, "lmhead dW launch");
+            EpiStoreScaledBf16 e2 = {};
+            e2.C = (__nv_bfloat16*)dhidden; e2.info = info; e2.ldc = H; e2.row0 = t0; e2.rows = T; e2.cols = H;
+            rc = run_gemm<EpiStoreScaledBf16, false, true>(pair, map_e_k, map_w_mn, map_w_mn, map_e_k, g2, e2, status, s, "lmhead dhidden launch");
             if (rc != DPPO_OK) return rc;
         }
         if (backward && p->dW_dtype == DPPO_BF16) {

@@ -10,17 +10,20 @@
 
 namespace dppo {
 
-constexpr int kPackMaxUnits = 65536;           // bitmask of 2048 words in shared memory
+constexpr int kPackMaxUnits = 1 << 21;         // units per call (a dataset of two million prompts)
+constexpr int kPackSmemMask = 65536;           // up to this n_max the placed-bitmask (2048 words) sits in shared memory,
+                                               // above it in the caller's workspace
 constexpr int kPackSmemLens = 8192;            // stream lengths in a static shared array up to this n_max (stream in global)
 constexpr int kPackSmemAll = 16384;            // stream, lengths and loss tokens all in dynamic shared memory up to this
                                                // n_max (192 KB): covers a dataset of 7.5-8.5 k prompts packed at set-up
 
-struct PackWorkspace {                         // carved from the caller's workspace, all i32 [n_max]
-    int32_t* stream;                           // unit index of stream position j
-    int32_t* slen;                             // its length
+struct PackWorkspace {                         // carved from the caller's workspace
+    int32_t* stream;                           // i32 [n_max]: unit index of stream position j
+    int32_t* slen;                             // i32 [n_max]: its length
+    uint32_t* mask;                            // [n_max / 32] placed-bitmask, only for n_max > kPackSmemMask
 };
 
-template <bool kLensInSmem, bool kStreamInSmem>
+template <bool kLensInSmem, bool kStreamInSmem, bool kMaskInSmem = true>
 __global__ void __launch_bounds__(32)
 pack_prompts_kernel(dppo_pack_params prm, const int32_t* __restrict__ len,
                     const uint8_t* __restrict__ keep, const int32_t* __restrict__ loss_len,
@@ -28,7 +31,8 @@ pack_prompts_kernel(dppo_pack_params prm, const int32_t* __restrict__ len,
                     int32_t* __restrict__ off_in_row, int32_t* __restrict__ row_fill,
                     int32_t* __restrict__ cu_seqlens, int32_t* __restrict__ counts,
                     PackWorkspace ws, int32_t* status) {
-    __shared__ uint32_t placed[kPackMaxUnits / 32];
+    __shared__ uint32_t placed_smem[kMaskInSmem ? kPackSmemMask / 32 : 1];
+    uint32_t* placed = kMaskInSmem ? placed_smem : ws.mask;
     __shared__ int32_t lens_static[(kLensInSmem && !kStreamInSmem) ? kPackSmemLens : 1];
     extern __shared__ int32_t pack_dyn[];                      // kStreamInSmem: stream, loss tokens, lengths, [n_max] each
     int32_t* stream_s = pack_dyn;
@@ -60,7 +64,7 @@ pack_prompts_kernel(dppo_pack_params prm, const int32_t* __restrict__ len,
         total_tokens += t;
     }
     for (int w = lane; w < (n + 31) / 32; w += 32) placed[w] = 0u;
-    bad = __any_sync(0xffffffffu, bad);
+    bad = __any_sync(0xffffffffu, bad) || total_tokens > 0x7fffffffLL;   // the token counts are reported as i32
     __syncwarp();
     if (bad) {
         if (lane == 0) { set_status(status, DPPO_STATUS_BAD_LENGTH); counts[0] = counts[1] = counts[2] = counts[3] = 0; }
@@ -204,15 +208,18 @@ pack_prompts_kernel(dppo_pack_params prm, const int32_t* __restrict__ len,
 }
 
 static size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
+constexpr int kMaxDevices = 64;
 
 // ---- scratch for dppo_pack_prompts_static ------------------------------------------------------
-// Lives in the library's device image: every GPU that loads the library holds these 64 KB until the
-// process exits.  Layout: stream positions [0, kPackStaticMaxUnits), their lengths after that.
+// Lives in the library's device image: every GPU that loads the library holds these 32 KB until the
+// process exits.  It holds the stream (the unit index of every stream position); the lengths of the stream sit
+// in shared memory for streams of this size.
 constexpr int kPackStaticMaxUnits = 8192;
-static __device__ __align__(256) int32_t g_pack_static_scratch[2 * kPackStaticMaxUnits];
+static_assert(kPackStaticMaxUnits <= kPackSmemLens, "the static-scratch packer keeps the stream's lengths in shared memory");
+static __device__ __align__(256) int32_t g_pack_static_scratch[kPackStaticMaxUnits];
 
-constexpr int kMaxDevices = 64;
-static int32_t* g_pack_static_ptr[kMaxDevices];          // device address of the array, per device ordinal
+static int32_t* g_pack_static_ptr[kMaxDevices];          // device address of the array, per device ordinal; it
+                                                         // outlives neither cudaDeviceReset nor a new context
 
 // Device address of the scratch array on the current device.  In host code the array's name is only a
 // handle for the runtime; the address a kernel can use comes from cudaGetSymbolAddress, asked once per
@@ -238,7 +245,8 @@ static int pack_static_scratch(int32_t** out) {
 
 extern "C" size_t dppo_pack_workspace_bytes(const dppo_pack_params* p) {
     if (!p || p->n_max < 0 || p->n_max > dppo::kPackMaxUnits) return 0;
-    return 2 * dppo::align_up((size_t)(p->n_max > 0 ? p->n_max : 1) * sizeof(int32_t));
+    const size_t n = (size_t)(p->n_max > 0 ? p->n_max : 1);
+    return 2 * dppo::align_up(n * sizeof(int32_t)) + (p->n_max > dppo::kPackSmemMask ? dppo::align_up((n + 31) / 32 * 4) : 0);
 }
 
 extern "C" int dppo_pack_prompts(const dppo_pack_params* p, const int32_t* len, const uint8_t* keep,
@@ -261,21 +269,35 @@ extern "C" int dppo_pack_prompts(const dppo_pack_params* p, const int32_t* len, 
     if (!workspace || workspace_bytes < need)
         return fail(DPPO_ERR_WORKSPACE_TOO_SMALL, "pack_prompts: workspace %zu < %zu bytes", workspace_bytes, need);
     if (((uintptr_t)workspace & 15) != 0) return fail(DPPO_ERR_MISALIGNED, "pack_prompts: workspace not 16-byte aligned");
+    const size_t per_array = align_up((size_t)(p->n_max > 0 ? p->n_max : 1) * sizeof(int32_t));
     PackWorkspace ws;
     ws.stream = (int32_t*)workspace;
-    ws.slen = (int32_t*)((char*)workspace + need / 2);
+    ws.slen = (int32_t*)((char*)workspace + per_array);
+    ws.mask = (uint32_t*)((char*)workspace + 2 * per_array);          // used above kPackSmemMask units only
     cudaStream_t s = (cudaStream_t)stream;
     if (p->n_max <= kPackSmemAll) {
         // batch-sized streams: the stream and its loss-token counts sit in shared memory too, so a placement
         // costs shared-memory latency instead of two dependent global loads
         const size_t dyn = (size_t)(p->n_max > 0 ? p->n_max : 1) * 3 * sizeof(int32_t);
-        cudaError_t e = cudaFuncSetAttribute(pack_prompts_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
-        if (e != cudaSuccess) return cuda_fail(e, "pack_prompts: shared memory attribute");
+        // the limit is raised once per device to the largest size any call may ask for (a per-call value could be
+        // lowered by another host thread between this thread's set and its launch)
+        static bool raised[kMaxDevices];
+        int dev = -1;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); dev = -1; }
+        if (dev < 0 || !raised[dev]) {
+            cudaError_t e = cudaFuncSetAttribute(pack_prompts_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 (int)(kPackSmemAll * 3 * sizeof(int32_t)));
+            if (e != cudaSuccess) return cuda_fail(e, "pack_prompts: shared memory attribute");
+            if (dev >= 0) raised[dev] = true;
+        }
         pack_prompts_kernel<true, true><<<1, 32, dyn, s>>>(*p, len, keep, loss_len, order, row_of, off_in_row, row_fill,
                                                          cu_seqlens, counts, ws, status);
-    } else
+    } else if (p->n_max <= kPackSmemMask)
         pack_prompts_kernel<false, false><<<1, 32, 0, s>>>(*p, len, keep, loss_len, order, row_of, off_in_row, row_fill,
                                                     cu_seqlens, counts, ws, status);
+    else
+        pack_prompts_kernel<false, false, false><<<1, 32, 0, s>>>(*p, len, keep, loss_len, order, row_of, off_in_row,
+                                                                  row_fill, cu_seqlens, counts, ws, status);
     DPPO_CHECK_LAUNCH("pack_prompts launch");
     return DPPO_OK;
 }
@@ -303,7 +325,8 @@ extern "C" int dppo_pack_prompts_static(const dppo_pack_params* p, const int32_t
     if (rc != DPPO_OK) return rc;
     PackWorkspace ws;
     ws.stream = scratch;
-    ws.slen = scratch + kPackStaticMaxUnits;
+    ws.slen = nullptr;                                       // lengths: shared memory in this instantiation
+    ws.mask = nullptr;                                       // bitmask: shared memory at this size
     // Nothing in the scratch has to start at zero: the kernel writes every stream slot it later reads.
     pack_prompts_kernel<true, false><<<1, 32, 0, (cudaStream_t)stream>>>(*p, len, keep, loss_len, order, row_of, off_in_row,
                                                                   row_fill, cu_seqlens, counts, ws, status);

@@ -52,10 +52,10 @@ WORKLOADS = {
     # large fused loss pass
     "config3": Workload("config3", 32, 8, 151936, "bf16", ("const", 0), ("uniform", 64, 1024),
                         2.0, "softmax", "beta", 0.25, 0.25, 8192, 16),
-    # fused LM-head + loss
-    "config4_h2560": Workload("config4_h2560", 32, 8, 151936, "bf16", ("const", 0), ("uniform", 64, 1024),
+    # fused LM-head + loss: about 140 k retained tokens at pruning probabilities 0.5 / 0.5 (seed 4: 130,006)
+    "config4_h2560": Workload("config4_h2560", 64, 8, 151936, "bf16", ("const", 0), ("uniform", 64, 1024),
                               1.0, "uniform", "beta", 0.5, 0.5, 8192, 16, H=2560),
-    "config4_h4096": Workload("config4_h4096", 32, 8, 151936, "bf16", ("const", 0), ("uniform", 64, 1024),
+    "config4_h4096": Workload("config4_h4096", 64, 8, 151936, "bf16", ("const", 0), ("uniform", 64, 1024),
                               1.0, "uniform", "beta", 0.5, 0.5, 8192, 16, H=4096),
 }
 

@@ -76,6 +76,28 @@ def pick_rows(cu_seqlens, T, n_random, seed):
     return np.array(sorted(rows), dtype=np.int64)
 
 
+class Guarded:
+    """An output buffer with a guard band of sentinel elements before and after it (the library writes through
+    raw pointers, and no sanitizer runs in these tests): `t` is the tensor handed to the library, check() asserts
+    that nothing outside it was written.  The band is 256 elements, so `t` keeps the alignment of the allocation
+    up to 512 bytes."""
+    GUARD = 256
+
+    def __init__(self, shape, dtype, fill, device="cuda"):
+        n = 1
+        for d in shape:
+            n *= int(d)
+        self.sentinel = 77 if not dtype.is_floating_point else 1024.0          # exact in every dtype used here
+        self.buf = torch.full((n + 2 * self.GUARD,), self.sentinel, dtype=dtype, device=device)
+        self.t = self.buf[self.GUARD:self.GUARD + n].view(*shape)
+        self.t.fill_(fill)
+
+    def check(self):
+        g = self.GUARD
+        assert bool((self.buf[:g] == self.sentinel).all()), "write before the start of an output buffer"
+        assert bool((self.buf[-g:] == self.sentinel).all()), "write past the end of an output buffer"
+
+
 LOGP_TOL = {"f32": 2e-6, "bf16": 1e-5}      # |logp - oracle| with f32 accumulation of the row sum
 
 

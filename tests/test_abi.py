@@ -45,7 +45,10 @@ def test_struct_layouts_match_header(B):
 
 def test_workspace_queries(B):
     assert B.pack_workspace_bytes(B.PackParams(256, 8192, 16, 0)) >= 2 * 256 * 4
-    assert B.pack_workspace_bytes(B.PackParams(1 << 20, 8192, 16, 0)) == 0          # above the unit limit
+    assert B.pack_workspace_bytes(B.PackParams(65536, 8192, 16, 0)) == 2 * 65536 * 4
+    big = B.pack_workspace_bytes(B.PackParams(1 << 20, 8192, 16, 0))                 # dataset-sized: the placed-bitmask too
+    assert big >= 2 * (1 << 20) * 4 + (1 << 20) // 8
+    assert B.pack_workspace_bytes(B.PackParams((1 << 21) + 1, 8192, 16, 0)) == 0    # above the unit limit
     n = B.grpo_loss_workspace_bytes(B.LossParams(1000, 1024, 0, 1024, 4, 0, 0.2, 0.2, 0.04, 1.0))
     assert n >= 1000 * 32 and n % 256 == 0
 
@@ -67,7 +70,7 @@ def test_host_validation_needs_no_device(B):
         B.pack_prompts(B.PackParams(8, 0, 4, 0), *([None] * 9), None, 0)
     assert e.value.code == B.ERR_INVALID_ARG
     with pytest.raises(B.DppoError) as e:
-        B.pack_prompts(B.PackParams(1 << 20, 64, 4, 0), *([None] * 9), None, 0)
+        B.pack_prompts(B.PackParams((1 << 21) + 1, 64, 4, 0), *([None] * 9), None, 0)
     assert e.value.code == B.ERR_BAD_SHAPE
     with pytest.raises(B.DppoError) as e:
         B.grpo_loss_fwd_bwd(B.LossParams(8, 0, 0, 0, 1, 0, 0.2, 0.2, 0.04, 1.0), *([None] * 14), 0)
