@@ -109,6 +109,13 @@ __device__ __forceinline__ uint32_t exp_pair(uint32_t w, f32x2 c2, f32x2 nr2, f3
     return pack_half2(ea, eb);
 }
 
+// The same without keeping the exponentials (a forward-only call has no second pass).
+__device__ __forceinline__ void exp_pair_sum(uint32_t w, f32x2 c2, f32x2 nr2, f32x2& acc) {
+    float a, b;
+    unpair(fma2(pair_of(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u)), c2, nr2), a, b);
+    acc = add2(acc, pair_of(ex2(a), ex2(b)));
+}
+
 // f32 rows: one 16-byte vector = four logits -> their exponentials 2^(z c - r), in place; acc += the four.
 __device__ __forceinline__ uint4 exp_quad(uint4 q, f32x2 c2, f32x2 nr2, f32x2& acc0, f32x2& acc1) {
     float a, b, e0, e1;
@@ -147,7 +154,8 @@ __device__ __forceinline__ void remote_store_signal(uint32_t local_slot, uint32_
                  :: "r"(rslot), "l"(v), "r"(rbar) : "memory");
 }
 
-template <int THREADS, bool kF32>
+// kBackward = false: a forward-only call (no dlogits): the exponentials are summed and dropped.
+template <int THREADS, bool kF32, bool kBackward>
 __global__ void __launch_bounds__(THREADS)
 grpo_loss_cluster_kernel(const LossArgs a, const int C, const int vec_per_cta) {
     constexpr int kLog2PerVec = kF32 ? 2 : 3;               // elements per 16-byte vector: 4 f32 or 8 bf16
@@ -258,11 +266,15 @@ grpo_loss_cluster_kernel(const LossArgs a, const int C, const int vec_per_cta) {
             uint4 h;
             if constexpr (kF32) {
                 h = exp_quad(q, c2, nr2, acc0, acc1);
-            } else {
+                if constexpr (kBackward) slice[i] = h;
+            } else if constexpr (kBackward) {
                 h.x = exp_pair(q.x, c2, nr2, acc0); h.y = exp_pair(q.y, c2, nr2, acc1);
                 h.z = exp_pair(q.z, c2, nr2, acc0); h.w = exp_pair(q.w, c2, nr2, acc1);
+                slice[i] = h;
+            } else {
+                exp_pair_sum(q.x, c2, nr2, acc0); exp_pair_sum(q.y, c2, nr2, acc1);
+                exp_pair_sum(q.z, c2, nr2, acc0); exp_pair_sum(q.w, c2, nr2, acc1);
             }
-            slice[i] = h;
         }
         float s0, s1;
         unpair(add2(acc0, acc1), s0, s1);
@@ -319,7 +331,7 @@ grpo_loss_cluster_kernel(const LossArgs a, const int C, const int vec_per_cta) {
     const RowScalars rs = st.row;
 
     // ---- pass 2: dlogits = g/tau (onehot - 2^(z c - lse2)), shared memory -> streaming global stores
-    if (a.dlogits) {
+    if (kBackward && a.dlogits) {
         char* drow = a.dlogits + t * a.row_bytes;
         uint4* dst = reinterpret_cast<uint4*>(drow) + v0;
         const float ng = rs.valid ? -rs.g_over_tau : 0.0f;
@@ -378,9 +390,9 @@ constexpr size_t kClusterSmemMax = 220 * 1024;            // largest slice a CTA
 
 // The dynamic shared-memory limit of an instantiation is raised once per device to the largest slice any launch
 // may ask for (a per-call value could be lowered by another host thread between this thread's set and its launch).
-template <int THREADS, bool kF32>
+template <int THREADS, bool kF32, bool kBackward>
 static int cluster_prepare_t(int C, size_t dyn_bytes, cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, bool check_fit) {
-    auto kernel = grpo_loss_cluster_kernel<THREADS, kF32>;
+    auto kernel = grpo_loss_cluster_kernel<THREADS, kF32, kBackward>;
     static bool raised[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); dev = -1; }
@@ -407,17 +419,23 @@ static int cluster_prepare_t(int C, size_t dyn_bytes, cudaLaunchConfig_t* cfg, c
 }
 
 // launch = false: only the checks a launch would make (used by the kernel-choice query).
-template <int THREADS, bool kF32>
-static int launch_cluster_t(const LossArgs& a, int C, int vec_per_cta, size_t dyn_bytes, cudaStream_t s, bool launch) {
+template <int THREADS, bool kF32, bool kBackward>
+static int launch_cluster_tb(const LossArgs& a, int C, int vec_per_cta, size_t dyn_bytes, cudaStream_t s, bool launch) {
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[2];
     cfg.gridDim = dim3((unsigned)((a.T_max > 0 ? a.T_max : 1) * C), 1, 1);
     cfg.stream = s;
-    const int rc = cluster_prepare_t<THREADS, kF32>(C, dyn_bytes, &cfg, attr, true);
+    const int rc = cluster_prepare_t<THREADS, kF32, kBackward>(C, dyn_bytes, &cfg, attr, true);
     if (rc != DPPO_OK || !launch) return rc;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, grpo_loss_cluster_kernel<THREADS, kF32>, a, C, vec_per_cta);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, grpo_loss_cluster_kernel<THREADS, kF32, kBackward>, a, C, vec_per_cta);
     if (e != cudaSuccess) return cuda_fail(e, "grpo_loss cluster launch");
     return DPPO_OK;
+}
+
+template <int THREADS, bool kF32>
+static int launch_cluster_t(const LossArgs& a, int C, int vec_per_cta, size_t dyn_bytes, cudaStream_t s, bool launch) {
+    return a.dlogits ? launch_cluster_tb<THREADS, kF32, true>(a, C, vec_per_cta, dyn_bytes, s, launch)
+                     : launch_cluster_tb<THREADS, kF32, false>(a, C, vec_per_cta, dyn_bytes, s, launch);
 }
 
 int launch_rows_cluster(const LossArgs& a, int C, int threads, cudaStream_t s, bool launch) {

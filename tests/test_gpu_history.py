@@ -1,5 +1,6 @@
 """Several epochs of prompt / completion pruning with the dataset-wide history table (Eq. 16, Algorithm 1):
-the library's gather -> advantages -> prune -> scatter loop against the oracle's, bit for bit."""
+the library's epoch driver (gather -> advantages -> prune -> scatter -> pack per batch) against the oracle's loop,
+bit for bit."""
 import numpy as np
 import pytest
 import torch
@@ -23,31 +24,30 @@ def test_epochs_with_history_table_match_oracle(mode):
         batches.append([perm[i:i + P].tolist() for i in range(0, N, P)])
     table_ref, log = oracle.history_epochs(rewards, batches, N, G, r_q, r_o, seed=seed, mode=mode)
 
-    f32 = dict(dtype=torch.float32, device="cuda"); i32 = dict(dtype=torch.int32, device="cuda"); u8 = dict(dtype=torch.uint8, device="cuda")
-    table = torch.zeros(N, **f32)
-    H_prev = torch.zeros(P, **f32); adv = torch.zeros(P * G, **f32); mabs = torch.zeros(P, **f32)
-    cand_q = torch.zeros(P, **u8); cand_o = torch.zeros(P * G, **u8); keep_q = torch.zeros(P, **u8); keep_o = torch.zeros(P * G, **u8)
-    nq = torch.zeros(1, **i32); no = torch.zeros(P, **i32)
-    gq = torch.zeros(P, **f32); go = torch.zeros(P * G, **f32); ws = torch.zeros(P * G, **f32); H_next = torch.zeros(P, **f32)
-    status = torch.zeros(1, **i32)
-    i = 0
-    for t in range(epochs):
-        for b, ids in enumerate(batches[t]):
-            d_ids = torch.tensor(ids, **i32)
-            d_r = torch.from_numpy(rewards[t][ids].reshape(-1)).cuda()
-            B.history_gather(table, N, d_ids, P, H_prev, status)
-            B.group_advantages(d_r, P, G, adv, mabs)
-            prm = B.PruneParams(P, G, r_q, r_o, mode, 0, seed, t * 1000000 + b)
-            B.prune_and_rescale(prm, adv, mabs, None if t == 0 else H_prev, None, None, cand_q, cand_o, keep_q, keep_o,
-                                nq, no, gq, go, ws, H_next, status)
-            B.history_scatter(table, N, d_ids, P, H_next, status)
-            ref = log[i]; i += 1
-            assert np.array_equal(keep_q.cpu().numpy(), ref["keep_q"])
-            assert np.array_equal(keep_o.cpu().numpy(), ref["keep_o"].reshape(-1))
-            assert np.array_equal(cand_q.cpu().numpy(), ref["cand_q"])
-            assert np.array_equal(ws.cpu().numpy().view(np.uint32), ref["w_seq"].reshape(-1).view(np.uint32))
-    assert status.item() == 0
+    # the library's epoch driver owns the table and issues gather -> advantages -> prune -> scatter (-> pack) per batch
+    from paper_2603_04135_b200.step import DppoStep
+    st = DppoStep(P, G, 4096, 8, r_q, r_o, 1, "bf16", 1, mode=mode)
+    lens = rng.integers(16, 400, size=(N, G)).astype(np.int32)
+    seen = []
+
+    def on_batch(t, b, step):
+        ref = log[len(seen)]
+        seen.append((t, b))
+        assert np.array_equal(step.keep_q.cpu().numpy(), ref["keep_q"])
+        assert np.array_equal(step.keep_o.cpu().numpy(), ref["keep_o"].reshape(-1))
+        assert np.array_equal(step.cand_q.cpu().numpy(), ref["cand_q"])
+        assert np.array_equal(step.w_seq.cpu().numpy().view(np.uint32), ref["w_seq"].reshape(-1).view(np.uint32))
+        ids = batches[t][b]
+        pk = oracle.pack_prompts(lens[ids].reshape(-1), 4096, 8, keep=ref["keep_o"].reshape(-1))
+        assert tuple(int(x) for x in step.counts.cpu().numpy()) == tuple(pk["counts"])
+        assert list(step.order.cpu().numpy()[:pk["counts"][0]]) == list(pk["order"])
+
+    table = st.run_epochs(N, batches, lambda t, ids: rewards[t][ids], seed,
+                          lengths_fn=lambda t, ids: (lens[ids].reshape(-1), lens[ids].reshape(-1)), on_batch=on_batch)
+    assert len(seen) == epochs * (N // P) and st.status.item() == 0
     assert np.array_equal(table.cpu().numpy().view(np.uint32), table_ref.view(np.uint32))
+    f32 = dict(dtype=torch.float32, device="cuda"); i32 = dict(dtype=torch.int32, device="cuda")
+    status = st.status
     # an id outside the table is reported, not dereferenced
     bad = torch.tensor([0, N, 5, -1], **i32)
     out = torch.full((4,), 7.0, **f32)

@@ -617,3 +617,46 @@ def test_config3_full_size():
         pytest.skip("needs ~70 GB of free device memory")
     T = _run_config(synth.WORKLOADS["config3"], 3, 4096, all_rows="pool", in_place=True)
     assert T > 60000
+
+
+def test_rows_sharded_over_two_ranks_add_up():
+    # Rows dealt out to two ranks (dp.shard_rows), each rank's sweep run here one after the other on the one device:
+    # every rank uses the sequence weights of the WHOLE batch, so the five scalars add up to the whole batch's and each
+    # rank's dlogits are the whole batch's rows, bit for bit
+    w = synth.scaled(synth.WORKLOADS["config0"], P=8, G=4, V=2056, L_row=192, r_q=0.3, r_o=0.3)
+    seed = 9
+    batch = synth.make_batch(w, seed)
+    ref = oracle_prune_pack(batch, w, seed, step=1)
+    T = ref["pack"]["counts"][3]
+    st = _step(w, T)
+    st.set_batch(batch.rewards, batch.unit_len, batch.loss_len, ref["H_prev"])
+    st.prune_pack(seed=seed, step=1)
+    assert st.n_tokens() == T and ref["pack"]["counts"][1] >= 4
+    tok = synth.make_token_inputs(w, T, seed, device="cuda", sigma_old=0.3)
+    dl = torch.empty_like(tok.logits)
+    st.loss(tok.logits, tok.target, tok.logp_old, tok.logp_ref, dl)
+    whole = st.loss_out.double().cpu().numpy()
+    order = np.asarray(ref["pack"]["order"], dtype=np.int64)
+    full = oracle.grpo_loss(synth.to_f64_numpy(tok.logits), tok.target.cpu().numpy(), tok.logp_old.cpu().numpy(),
+                            tok.logp_ref.cpu().numpy(), ref["pack"]["cu_seqlens"], ref["adv"].reshape(-1)[order],
+                            ref["prune"]["w_seq"].reshape(-1)[order], w.eps, w.eps, w.beta, want_dlogits=False)
+    assert abs(whole[0] - full["loss"]) <= 1e-4 * abs(full["loss"]) + 1e-7 * full["abs_sum"]
+    parts = []
+    covered = 0
+    for rank in range(2):
+        sh = st.shard(2, rank)
+        a, b = sh["tok_lo"], sh["tok_hi"]
+        assert a == covered and b > a
+        covered = b
+        dl_r = torch.full((b - a, w.V), 7.0, device="cuda")
+        st.loss_shard(sh, tok.logits[a:b], tok.target[a:b], tok.logp_old[a:b], tok.logp_ref[a:b], dl_r)
+        torch.cuda.synchronize()
+        assert st.status.item() == 0
+        parts.append(st.loss_out.double().cpu().numpy())
+        assert torch.equal(dl_r.view(torch.int32), dl[a:b].view(torch.int32))
+    assert covered == T
+    total = parts[0][:3] + parts[1][:3]
+    for k in range(3):
+        assert abs(total[k] - whole[k]) <= 1e-6 * max(abs(whole[k]), 1e-6)
+    assert parts[0][4] + parts[1][4] == T == whole[4]
+    assert abs((parts[0][3] * parts[0][4] + parts[1][3] * parts[1][4]) / T - whole[3]) <= 1e-6
