@@ -1,5 +1,7 @@
 // Internal types shared by the loss-sweep kernels (not part of the ABI).
 #pragma once
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 
 namespace dppo {
@@ -98,6 +100,90 @@ template <> struct Elems<false> {
         reinterpret_cast<float*>(row)[v] = x;
     }
 };
+
+// ---- per-element arithmetic of the two row kernels that keep the exponentials (shared-memory and warp-per-row) ----
+namespace packed {
+
+__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
+    const __half2 h = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&h);
+}
+// Packed f32 pairs (one instruction works on both halves of a 64-bit register pair).
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pair_of(float lo, float hi) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpair(f32x2 p, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(p)); }
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+    f32x2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+    f32x2 d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+    f32x2 d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+// Two fp16 exponentials -> two bf16 gradient entries e * sc (sc2 = the scale in both halves).
+__device__ __forceinline__ uint32_t scale_pair(uint32_t h2, f32x2 sc2) {
+    const float2 e = __half22float2(*reinterpret_cast<const __half2*>(&h2));
+    float lo, hi;
+    unpair(mul2(pair_of(e.x, e.y), sc2), lo, hi);
+    const __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&b);
+}
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+// One 32-bit word = two bf16 logits -> their exponentials 2^(z c - r) as an fp16 pair; acc += the two (f32).
+__device__ __forceinline__ uint32_t exp_pair(uint32_t w, f32x2 c2, f32x2 nr2, f32x2& acc) {
+    float a, b;
+    unpair(fma2(pair_of(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u)), c2, nr2), a, b);
+    const float ea = ex2(a), eb = ex2(b);
+    acc = add2(acc, pair_of(ea, eb));
+    return pack_half2(ea, eb);
+}
+
+// The same without keeping the exponentials (a forward-only call has no second pass).
+__device__ __forceinline__ void exp_pair_sum(uint32_t w, f32x2 c2, f32x2 nr2, f32x2& acc) {
+    float a, b;
+    unpair(fma2(pair_of(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u)), c2, nr2), a, b);
+    acc = add2(acc, pair_of(ex2(a), ex2(b)));
+}
+
+// f32 rows: one 16-byte vector = four logits -> their exponentials 2^(z c - r), in place; acc += the four.
+__device__ __forceinline__ uint4 exp_quad(uint4 q, f32x2 c2, f32x2 nr2, f32x2& acc0, f32x2& acc1) {
+    float a, b, e0, e1;
+    unpair(fma2(pair_of(__uint_as_float(q.x), __uint_as_float(q.y)), c2, nr2), a, b);
+    e0 = ex2(a); e1 = ex2(b);
+    acc0 = add2(acc0, pair_of(e0, e1));
+    q.x = __float_as_uint(e0); q.y = __float_as_uint(e1);
+    unpair(fma2(pair_of(__uint_as_float(q.z), __uint_as_float(q.w)), c2, nr2), a, b);
+    e0 = ex2(a); e1 = ex2(b);
+    acc1 = add2(acc1, pair_of(e0, e1));
+    q.z = __float_as_uint(e0); q.w = __float_as_uint(e1);
+    return q;
+}
+__device__ __forceinline__ uint4 scale_quad(uint4 q, f32x2 sc2) {
+    float a, b;
+    unpair(mul2(pair_of(__uint_as_float(q.x), __uint_as_float(q.y)), sc2), a, b);
+    q.x = __float_as_uint(a); q.y = __float_as_uint(b);
+    unpair(mul2(pair_of(__uint_as_float(q.z), __uint_as_float(q.w)), sc2), a, b);
+    q.z = __float_as_uint(a); q.w = __float_as_uint(b);
+    return q;
+}
+
+}  // namespace packed
 
 // ---- scalar stage -------------------------------------------------------------------------------------
 // What one token row needs besides its logits; gathered once per row (one thread, or one warp ahead of

@@ -13,35 +13,11 @@
 #include "grpo_loss.cuh"
 
 namespace dppo {
+using namespace packed;
 namespace warprow {
 
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
-
-__device__ __forceinline__ float ex2(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-// Two bf16 logits in one word -> their exponentials 2^(z c + nr) as an fp16 pair; s += the two.
-__device__ __forceinline__ uint32_t exp_pair(uint32_t w, float c, float nr, float& s0, float& s1) {
-    const float e0 = ex2(fmaf(__uint_as_float(w << 16), c, nr));
-    const float e1 = ex2(fmaf(__uint_as_float(w & 0xffff0000u), c, nr));
-    s0 += e0; s1 += e1;
-    const __half2 h = __floats2half2_rn(e0, e1);
-    return *reinterpret_cast<const uint32_t*>(&h);
-}
-// Two fp16 exponentials -> two bf16 gradient entries e * sc.
-__device__ __forceinline__ uint32_t scale_pair(uint32_t h2, float sc) {
-    const float2 e = __half22float2(*reinterpret_cast<const __half2*>(&h2));
-    const __nv_bfloat162 b = __floats2bfloat162_rn(e.x * sc, e.y * sc);
-    return *reinterpret_cast<const uint32_t*>(&b);
-}
-__device__ __forceinline__ uint32_t exp_f32(uint32_t w, float c, float nr, float& s) {
-    const float e = ex2(fmaf(__uint_as_float(w), c, nr));
-    s += e;
-    return __float_as_uint(e);
-}
 
 // Word `wy` of vector `jy` of a lane's row registers.  Both indices are the same in every lane (they follow from the
 // sampled token's id), so a branch on them does not diverge and costs a few instructions, where selects over all
@@ -209,18 +185,20 @@ grpo_loss_warp_kernel(const LossArgs a) {
         const float r = m * c;                              // -inf only if the whole row is -inf
         const float nr = r > -INFINITY ? -r : 0.0f;
 
-        // ---- exponentials 2^(z c - r) in place, and their sum
-        float s0 = 0.0f, s1 = 0.0f;
+        // ---- exponentials 2^(z c - r) in place, and their sum (packed f32 pairs: one instruction for two elements)
+        const f32x2 c2 = pair_of(c, c), nr2 = pair_of(nr, nr);
+        f32x2 acc0 = pair_of(0.0f, 0.0f), acc1 = acc0;
 #pragma unroll
         for (int j = 0; j < kVPL; ++j) {
             if constexpr (kF32) {
-                d[j].x = exp_f32(d[j].x, c, nr, s0); d[j].y = exp_f32(d[j].y, c, nr, s1);
-                d[j].z = exp_f32(d[j].z, c, nr, s0); d[j].w = exp_f32(d[j].w, c, nr, s1);
+                d[j] = exp_quad(d[j], c2, nr2, acc0, acc1);
             } else {
-                d[j].x = exp_pair(d[j].x, c, nr, s0, s1); d[j].y = exp_pair(d[j].y, c, nr, s0, s1);
-                d[j].z = exp_pair(d[j].z, c, nr, s0, s1); d[j].w = exp_pair(d[j].w, c, nr, s0, s1);
+                d[j].x = exp_pair(d[j].x, c2, nr2, acc0); d[j].y = exp_pair(d[j].y, c2, nr2, acc1);
+                d[j].z = exp_pair(d[j].z, c2, nr2, acc0); d[j].w = exp_pair(d[j].w, c2, nr2, acc1);
             }
         }
+        float s0, s1;
+        unpair(add2(acc0, acc1), s0, s1);
         const float etail = ztail > -INFINITY ? ex2(fmaf(ztail, c, nr)) : 0.0f;
         const float s = warp_sum(s0 + s1 + etail);
 
@@ -241,17 +219,17 @@ grpo_loss_warp_kernel(const LossArgs a) {
             char* drow = a.dlogits + (long long)t * a.row_bytes;
             uint4* dst = reinterpret_cast<uint4*>(drow);
             const float sc = ng * ex2((r - lse2_hi) - lse2_lo);
+            const f32x2 sc2 = pair_of(sc, sc);
 #pragma unroll
             for (int j = 0; j < kVPL; ++j) {
                 const int i = lane + 32 * j;
                 if (i < nvec) {
                     uint4 o;
                     if constexpr (kF32) {
-                        o.x = __float_as_uint(__uint_as_float(d[j].x) * sc); o.y = __float_as_uint(__uint_as_float(d[j].y) * sc);
-                        o.z = __float_as_uint(__uint_as_float(d[j].z) * sc); o.w = __float_as_uint(__uint_as_float(d[j].w) * sc);
+                        o = scale_quad(d[j], sc2);
                     } else {
-                        o.x = scale_pair(d[j].x, sc); o.y = scale_pair(d[j].y, sc);
-                        o.z = scale_pair(d[j].z, sc); o.w = scale_pair(d[j].w, sc);
+                        o.x = scale_pair(d[j].x, sc2); o.y = scale_pair(d[j].y, sc2);
+                        o.z = scale_pair(d[j].z, sc2); o.w = scale_pair(d[j].w, sc2);
                     }
                     __stcs(dst + i, o);
                 }
