@@ -46,8 +46,8 @@ WORKLOAD_TEXT = WORKLOAD + ": P=32 G=8, response 64-1024 tokens, V=151936 bf16 l
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch over 8192 rows of this vocabulary.  Traffic
 # grows in proportion to the rows, so a launch over T rows moves T times the per-row figure.  The record
 # is tied to the kernel sources it was taken from: once they change, `traffic` is reported as null.
-TRAFFIC_CAPTURE = {"rows": 8192, "dram_bytes": 2489504000 + 2431640000,
-                   "source_sha256": "e9560dea6352e68770f24457c44a0df5462c8a9da2d58d5ba39d42e571b97d3b"}
+TRAFFIC_CAPTURE = {"rows": 8192, "dram_bytes": 2489485000 + 2432175000,
+                   "source_sha256": "2482415d6f07c889d19573b6fcd64e072262e8bf975348399d4f7e5601ea1a5b"}
 
 
 def captured_traffic_per_row():
