@@ -259,8 +259,8 @@ int dppo_grpo_loss_fwd_bwd(const dppo_loss_params* p, const void* logits, const 
                            int32_t* status, void* stream);
 
 /* Which kernel a dppo_grpo_loss_fwd_bwd call with these parameters runs on the current device (a host-side query:
- * it makes the same choice and the same device checks as the call and launches nothing).  Rows of up to 4 KB (bf16)
- * or 8 KB (f32) go to the warp-per-row kernel, rows that fit eight shared-memory slices to the shared-memory
+ * it makes the same choice and the same device checks as the call and launches nothing).  Rows of up to 8 KB
+ * go to the warp-per-row kernel, rows that fit eight shared-memory slices to the shared-memory
  * kernel, longer ones to the general two-pass kernel.  fell_back = 1 says that the device refused the kernel the
  * row length asked for (its shared memory or cluster size) and the slower general kernel runs instead.
  * Errors: INVALID_ARG; UNSUPPORTED when params.variant forces a kernel that cannot take the shape.

@@ -18,16 +18,17 @@ namespace dppo {
 // 55 KB slices (four per SM), else four or eight CTAs with slices up to 76 KB (three per SM).  Measured at rows of
 // 32 / 64 / 128 KB: 6.7 / 6.5 / 6.4 TB/s with 1 / 2 / 4 CTAs against 2.8 / 3.5 / 3.7 TB/s for the general kernel
 // and 2.6 / 4.4 / 6.4 with four CTAs throughout.  Below about 8 KB per row the grid's launch rate (one CTA per row,
-// about 250 rows per microsecond) is the limit: those rows go to the warp-per-row kernel (2 KB rows: 3.3-3.6 TB/s
-// against 1.0).
+// about 250 rows per microsecond) is the limit: rows of up to 8 KB go to the warp-per-row kernel (2 KB rows: 3.5-3.7
+// TB/s against 1.0).
 constexpr size_t kSliceMax1 = 44 * 1024;
 constexpr size_t kSliceMax2 = 55 * 1024;
 constexpr size_t kSliceMax48 = 76 * 1024;
-constexpr int kClusterThreads = 256;                // bf16 slices above 16 KB, f32 slices above 64 KB
+constexpr int kClusterThreads = 256;                // bf16 slices above 28 KB (24 KB rows: 6.3 TB/s with 128 threads, 5.5
+                                                    // with 256; 32 KB rows: 6.2 against 6.3), f32 slices above 64 KB
 constexpr int kClusterThreadsSmall = 128;           // shorter slices (f32 has half the arithmetic per byte)
 
-constexpr int kWarpRowMaxVecBf16 = 256;             // bf16 rows of up to 4 KB, f32 rows of up to 8 KB (an 8 KB bf16 row is
-constexpr int kWarpRowMaxVecF32 = 512;              // as fast in one CTA of the shared-memory kernel: 3.4 TB/s)
+constexpr int kWarpRowMaxVecBf16 = 512;             // rows of up to 8 KB in either dtype (8 KB bf16 rows: 4.35 TB/s against
+constexpr int kWarpRowMaxVecF32 = 512;              // 3.3 TB/s in one CTA of the shared-memory kernel)
 
 static int auto_cluster_size(int nvec) {
     const size_t limit[4] = {kSliceMax1, kSliceMax2, kSliceMax48, kSliceMax48};
@@ -270,8 +271,8 @@ int run_rows(LossArgs a, int variant, cudaStream_t s, bool launch, dppo_loss_ker
             refused = rc == DPPO_ERR_UNSUPPORTED;
         } else if (C > 0) {
             const size_t slice = (size_t)((nvec + C - 1) / C) * 16;
-            // 256 threads for bf16 slices above 16 KB and f32 slices above 64 KB, else 128
-            const int threads = slice > (a.bf16 ? 16u : 64u) * 1024 ? kClusterThreads : kClusterThreadsSmall;
+            // 256 threads for bf16 slices above 28 KB and f32 slices above 64 KB, else 128
+            const int threads = slice > (a.bf16 ? 28u : 64u) * 1024 ? kClusterThreads : kClusterThreadsSmall;
             ch.kernel = DPPO_KERNEL_SHARED; ch.ctas_per_row = C; ch.threads = threads;
             rc = launch_rows_cluster(a, C, threads, s, launch);
             refused = rc == DPPO_ERR_UNSUPPORTED;

@@ -386,7 +386,7 @@ def test_loss_warp_per_row_kernel(dtype):
     v = 2
     for V, seed in [(1, 300), (5, 301), (8, 302), (100, 303), (256, 304), (1000, 305), (1024, 306), (2047, 307)]:
         _loss_case(V, dtype, T=67, S=5, seed=seed, variant=v)
-    big = 4096 if dtype == "bf16" else 2048                                      # 16 vectors per lane
+    big = 4096 if dtype == "bf16" else 2048                                      # 16 vectors per lane (8 KB rows)
     _loss_case(big, dtype, T=40, S=3, seed=310, variant=v)
     _loss_case(1536, dtype, T=5000, S=40, seed=311, variant=v)                   # several rows per warp
     _loss_case(1024, dtype, T=50, S=4, seed=312, variant=v, in_place=True)
@@ -469,9 +469,9 @@ def test_loss_is_bit_reproducible(variant):
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
 def test_loss_kernel_choice_boundaries(dtype):
     # row lengths on both sides of every switch of the library's kernel choice: warp per row -> one CTA -> two ->
-    # four -> eight CTAs -> general kernel (limits in 16-byte vectors: 256 or 512, 2816, 7040, 19456, 38912)
+    # four -> eight CTAs -> general kernel (limits in 16-byte vectors: 512, 2816, 7040, 19456, 38912)
     per_vec = 8 if dtype == "bf16" else 4
-    warp_max = 256 if dtype == "bf16" else 512
+    warp_max = 512
     seed = 400
     for nvec in (warp_max, 2816, 7040, 19456, 38912):
         for V in (nvec * per_vec, nvec * per_vec + per_vec, nvec * per_vec + 3):
@@ -491,6 +491,7 @@ def test_loss_kernel_choice_query():
 
     assert choice(1024, B.BF16) == (B.KERNEL_WARP, 1, 32, 0)
     assert choice(2048, B.F32) == (B.KERNEL_WARP, 1, 32, 0)
+    assert choice(4096, B.BF16) == (B.KERNEL_WARP, 1, 32, 0)
     assert choice(8192, B.BF16) == (B.KERNEL_SHARED, 1, 128, 0)
     assert choice(16384, B.BF16) == (B.KERNEL_SHARED, 1, 256, 0)
     assert choice(32768, B.BF16) == (B.KERNEL_SHARED, 2, 256, 0)
