@@ -286,7 +286,7 @@ def run_profile_case(args):
         wseq = torch.full((S,), 1.0 / S, device="cuda")
         dl = tok.logits if args.in_place else torch.empty_like(tok.logits)
         prm = B.LossParams(T, w.V, B.BF16 if args.dtype == "bf16" else B.F32, w.V, S, args.variant, w.eps, w.eps, w.beta, 1.0)
-        ch = B.grpo_loss_kernel_choice(prm)
+        ch = B.grpo_loss_kernel_choice(prm, forward_only=args.forward_only)
         print("kernel: %s, %d CTA(s) per row, %d threads%s" % (B.KERNEL_NAMES[ch.kernel], ch.ctas_per_row, ch.threads,
                                                                   " (fell back)" if ch.fell_back else ""))
         nbytes = B.grpo_loss_workspace_bytes(prm)
@@ -509,6 +509,7 @@ def run_ours(args):
                            "frac": gbs / peak_m, "tokens_per_s": T / ms_mode * 1e3}
         modes["in_place"]["note"] = "dlogits written over the logits; after the first call the input is the previous gradient"
         modes["seq_ratio"]["note"] = "forward-only sweep + per-sequence mean log-ratio + gradient sweep: two reads, one write"
+        modes["forward_only"]["kernel"] = B.KERNEL_NAMES[B.grpo_loss_kernel_choice(st.loss_params, forward_only=True).kernel]
         ch = B.grpo_loss_kernel_choice(st.loss_params)
         modes["kernel_choice"] = {"kernel": B.KERNEL_NAMES[ch.kernel], "ctas_per_row": ch.ctas_per_row, "threads": ch.threads,
                                   "fell_back_to_general_kernel": bool(ch.fell_back)}

@@ -213,7 +213,8 @@ typedef struct {
     int64_t row_stride;     /* elements between consecutive rows (>= V; bytes a multiple of 16)      */
     int32_t S_max;          /* cu_seqlens has S_max+1 entries, non-decreasing, last >= true T        */
     int32_t variant;        /* 0: the library picks the kernel.  Tuning aid: 1 forces the general two-pass
-                               kernel, 2 the warp-per-row kernel (rows up to 8 KB), C*10000+threads the shared-memory kernel with C = 1, 2, 4 or 8
+                               kernel, 2 the warp-per-row kernel (rows up to 8 KB), 3 the streaming kernel (forward-only
+                               calls), C*10000+threads the shared-memory kernel with C = 1, 2, 4 or 8
                                CTAs per row and 128 / 256 / 512 / 1024 threads per CTA.
                                Self-test of the bounded waits: 1000000 + (0 or a C*10000+threads code) runs the
                                shared-memory kernel with every CTA expecting one exchange message more than is
@@ -261,18 +262,19 @@ int dppo_grpo_loss_fwd_bwd(const dppo_loss_params* p, const void* logits, const 
 /* Which kernel a dppo_grpo_loss_fwd_bwd call with these parameters runs on the current device (a host-side query:
  * it makes the same choice and the same device checks as the call and launches nothing).  Rows of up to 8 KB
  * go to the warp-per-row kernel, rows that fit eight shared-memory slices to the shared-memory
- * kernel, longer ones to the general two-pass kernel.  fell_back = 1 says that the device refused the kernel the
+ * kernel, longer ones to the general two-pass kernel; a forward-only call (forward_only != 0: the call will pass
+ * dlogits = NULL) on rows of 128 KB and more goes to the streaming kernel.  fell_back = 1 says that the device refused the kernel the
  * row length asked for (its shared memory or cluster size) and the slower general kernel runs instead.
  * Errors: INVALID_ARG; UNSUPPORTED when params.variant forces a kernel that cannot take the shape.
  */
-typedef enum { DPPO_KERNEL_GENERAL = 0, DPPO_KERNEL_WARP = 1, DPPO_KERNEL_SHARED = 2 } dppo_loss_kernel;
+typedef enum { DPPO_KERNEL_GENERAL = 0, DPPO_KERNEL_WARP = 1, DPPO_KERNEL_SHARED = 2, DPPO_KERNEL_STREAM = 3 } dppo_loss_kernel;
 typedef struct {
     int32_t kernel;         /* dppo_loss_kernel                                                      */
     int32_t ctas_per_row;   /* cluster size of the shared-memory kernel, else 1                      */
     int32_t threads;        /* threads that work on one row at a time in each CTA                    */
     int32_t fell_back;      /* 1: general kernel in place of the one the row length asked for        */
 } dppo_loss_kernel_choice;
-int dppo_grpo_loss_kernel_choice(const dppo_loss_params* p, dppo_loss_kernel_choice* out);
+int dppo_grpo_loss_kernel_choice(const dppo_loss_params* p, int forward_only, dppo_loss_kernel_choice* out);
 
 /* Mean token log-ratio of each sequence, out[s] = mean_t (logp[t] - logp_old[t]) over cu_seqlens[s] <= t <
  * cu_seqlens[s+1] (0 for an empty sequence): the log of the length-normalised sequence-level likelihood

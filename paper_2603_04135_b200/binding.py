@@ -52,8 +52,9 @@ class LossKernelChoice(ctypes.Structure):
                 ("fell_back", ctypes.c_int32)]
 
 
-KERNEL_GENERAL, KERNEL_WARP, KERNEL_SHARED = 0, 1, 2
-KERNEL_NAMES = {KERNEL_GENERAL: "general two-pass", KERNEL_WARP: "warp per row", KERNEL_SHARED: "shared memory"}
+KERNEL_GENERAL, KERNEL_WARP, KERNEL_SHARED, KERNEL_STREAM = 0, 1, 2, 3
+KERNEL_NAMES = {KERNEL_GENERAL: "general two-pass", KERNEL_WARP: "warp per row", KERNEL_SHARED: "shared memory",
+                KERNEL_STREAM: "streaming (forward only)"}
 LOSS_WAIT_SELF_TEST = 1000000      # added to dppo_loss_params.variant
 LMHEAD_WAIT_SELF_TEST = 100        # added to dppo_lmhead_params.variant
 
@@ -89,7 +90,7 @@ lib.dppo_grpo_loss_fwd_bwd.argtypes = [ctypes.POINTER(LossParams)] + [_vp] * 14 
 
 
 lib.dppo_grpo_loss_kernel_choice.restype = ctypes.c_int
-lib.dppo_grpo_loss_kernel_choice.argtypes = [ctypes.POINTER(LossParams), ctypes.POINTER(LossKernelChoice)]
+lib.dppo_grpo_loss_kernel_choice.argtypes = [ctypes.POINTER(LossParams), ctypes.c_int, ctypes.POINTER(LossKernelChoice)]
 lib.dppo_sequence_log_ratio.restype = ctypes.c_int
 lib.dppo_sequence_log_ratio.argtypes = [_vp, _vp, _vp, ctypes.c_int, _vp, _vp, _vp]
 lib.dppo_lmhead_workspace_bytes.restype = ctypes.c_size_t
@@ -186,10 +187,11 @@ def grpo_loss_fwd_bwd(params, logits, target, logp_old, logp_ref, cu_seqlens, n_
                                       _stream(stream)))
 
 
-def grpo_loss_kernel_choice(params):
-    """The kernel dppo_grpo_loss_fwd_bwd runs for these parameters on the current device, as a LossKernelChoice."""
+def grpo_loss_kernel_choice(params, forward_only=False):
+    """The kernel dppo_grpo_loss_fwd_bwd runs for these parameters on the current device (forward_only: the call
+    will pass no dlogits), as a LossKernelChoice."""
     out = LossKernelChoice()
-    _check(lib.dppo_grpo_loss_kernel_choice(ctypes.byref(params), ctypes.byref(out)))
+    _check(lib.dppo_grpo_loss_kernel_choice(ctypes.byref(params), int(bool(forward_only)), ctypes.byref(out)))
     return out
 
 

@@ -27,6 +27,7 @@ constexpr int kClusterThreads = 256;                // bf16 slices above 28 KB (
                                                     // with 256; 32 KB rows: 6.2 against 6.3), f32 slices above 64 KB
 constexpr int kClusterThreadsSmall = 128;           // shorter slices (f32 has half the arithmetic per byte)
 
+constexpr size_t kStreamMinRowBytes = 128 * 1024;   // forward-only calls: rows from this length on go to the streaming kernel
 constexpr int kWarpRowMaxVecBf16 = 512;             // rows of up to 8 KB in either dtype (8 KB bf16 rows: 4.35 TB/s against
 constexpr int kWarpRowMaxVecF32 = 512;              // 3.3 TB/s in one CTA of the shared-memory kernel)
 
@@ -236,8 +237,8 @@ LossArgs loss_args_from_params(const dppo_loss_params* p) {
 }
 
 // Picks the row kernel for `variant` and launches it (launch = true) or only runs the checks a launch would make.
-// variant: 0 picks the kernel from the shape; 1 forces the general kernel; 2 the warp-per-row kernel;
-// C*10000 + threads forces the shared-memory kernel with C CTAs per row (a tuning aid; unsupported shapes are an
+// variant: 0 picks the kernel from the shape; 1 forces the general kernel; 2 the warp-per-row kernel; 3 the
+// streaming kernel (forward-only calls); C*10000 + threads forces the shared-memory kernel with C CTAs per row (a tuning aid; unsupported shapes are an
 // error); kSelfTestVariant + one of those runs the self-test of the bounded waits on the shared-memory kernel.
 // choice (nullable) receives what was taken; fell_back = 1 when the device refused the kernel the shape asked for
 // and the general kernel took over.
@@ -257,6 +258,9 @@ int run_rows(LossArgs a, int variant, cudaStream_t s, bool launch, dppo_loss_ker
     } else if (variant == 2) {
         ch.kernel = DPPO_KERNEL_WARP; ch.threads = 32;
         rc = launch_rows_warp(a, s, launch);
+    } else if (variant == 3) {
+        ch.kernel = DPPO_KERNEL_STREAM; ch.threads = 512;
+        rc = launch_rows_stream(a, s, launch);
     } else if (variant >= 10000) {
         ch.kernel = DPPO_KERNEL_SHARED; ch.ctas_per_row = variant / 10000; ch.threads = variant % 10000;
         rc = launch_rows_cluster(a, ch.ctas_per_row, ch.threads, s, launch);
@@ -265,7 +269,13 @@ int run_rows(LossArgs a, int variant, cudaStream_t s, bool launch, dppo_loss_ker
         const int nvec = a.V >> (a.bf16 ? 3 : 2);
         const int C = auto_cluster_size(nvec);
         bool refused = false;
-        if (nvec <= (a.bf16 ? kWarpRowMaxVecBf16 : kWarpRowMaxVecF32)) {
+        if (a.dlogits == nullptr && (size_t)nvec * 16 >= kStreamMinRowBytes) {
+            // forward-only call on a long row: stream it (5.7 against 4.6 TB/s at 297 KB bf16 rows, 6.7 against 4.1 at
+            // 594 KB f32 rows; the shared-memory kernel stays ahead below about 128 KB: 4.6 against 3.7 at 64 KB)
+            ch.kernel = DPPO_KERNEL_STREAM; ch.threads = 512;
+            rc = launch_rows_stream(a, s, launch);
+            refused = rc == DPPO_ERR_UNSUPPORTED;
+        } else if (nvec <= (a.bf16 ? kWarpRowMaxVecBf16 : kWarpRowMaxVecF32)) {
             ch.kernel = DPPO_KERNEL_WARP; ch.threads = 32;
             rc = launch_rows_warp(a, s, launch);
             refused = rc == DPPO_ERR_UNSUPPORTED;
@@ -284,8 +294,8 @@ int run_rows(LossArgs a, int variant, cudaStream_t s, bool launch, dppo_loss_ker
     } else {
         rc = fail(DPPO_ERR_INVALID_ARG, "grpo_loss: variant %d", variant);
     }
-    if (rc == DPPO_OK && self_test && ch.kernel != DPPO_KERNEL_SHARED)
-        return fail(DPPO_ERR_UNSUPPORTED, "grpo_loss: the wait self-test runs on the shared-memory kernel only");
+    if (rc == DPPO_OK && self_test && ch.kernel != DPPO_KERNEL_SHARED && ch.kernel != DPPO_KERNEL_STREAM)
+        return fail(DPPO_ERR_UNSUPPORTED, "grpo_loss: the wait self-test runs on the shared-memory and streaming kernels only");
     if (choice) *choice = ch;
     return rc;
 }
@@ -344,13 +354,15 @@ extern "C" int dppo_grpo_loss_fwd_bwd(const dppo_loss_params* p, const void* log
     return launch_loss_reduce(a, loss_out, s);
 }
 
-extern "C" int dppo_grpo_loss_kernel_choice(const dppo_loss_params* p, dppo_loss_kernel_choice* out) {
+extern "C" int dppo_grpo_loss_kernel_choice(const dppo_loss_params* p, int forward_only, dppo_loss_kernel_choice* out) {
     using namespace dppo;
     if (!p || !out) return fail(DPPO_ERR_INVALID_ARG, "grpo_loss_kernel_choice: NULL argument");
     if (p->V < 1 || p->T_max < 0 || (p->dtype != DPPO_F32 && p->dtype != DPPO_BF16) || p->variant < 0 || !(p->temperature > 0.0))
         return fail(DPPO_ERR_INVALID_ARG, "grpo_loss_kernel_choice: V=%d T_max=%lld dtype=%d variant=%d", p->V,
                     (long long)p->T_max, p->dtype, p->variant);
-    return run_rows(loss_args_from_params(p), p->variant, nullptr, false, out);
+    LossArgs a = loss_args_from_params(p);
+    a.dlogits = forward_only ? nullptr : (char*)16;          // only tested against NULL on this path: nothing is launched
+    return run_rows(a, p->variant, nullptr, false, out);
 }
 
 extern "C" int dppo_sequence_log_ratio(const float* logp, const float* logp_old, const int32_t* cu_seqlens, int S_max,

@@ -302,6 +302,9 @@ int launch_rows_cluster(const LossArgs& a, int cluster, int threads, cudaStream_
 // Short rows (up to 512 16-byte vectors): one warp per row, the row in registers (grpo_loss_warp.cu).
 // Returns DPPO_ERR_UNSUPPORTED (nothing launched) for longer rows.
 int launch_rows_warp(const LossArgs& a, cudaStream_t s, bool launch = true);
+// Forward-only calls: persistent CTAs stream the rows through a shared-memory ring (grpo_loss_stream.cu).
+// Returns DPPO_ERR_UNSUPPORTED (nothing launched) when dlogits are asked for.
+int launch_rows_stream(const LossArgs& a, cudaStream_t s, bool launch = true);
 int launch_loss_reduce(const LossArgs& a, float* loss_out, cudaStream_t s);
 
 }  // namespace dppo

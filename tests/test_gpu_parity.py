@@ -397,6 +397,27 @@ def test_loss_warp_per_row_kernel(dtype):
     _loss_case(2040, dtype, T=80, S=6, seed=317, variant=v, seq_ratio=True, sigma_noise=0.3)
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_loss_streaming_forward_kernel(dtype):
+    # forward-only calls on the streaming kernel (forced): rows of less than a vector, of one piece, of several pieces
+    # with a ragged last one, ragged tails, more rows than CTAs, a device-side token count, a temperature, masked
+    # columns (a whole piece of -inf, and a masked start), a wide dynamic range, the sequence-level ratio's first sweep
+    v = 3
+    for V, T, seed in [(5, 20, 500), (8, 33, 501), (1000, 67, 502), (4099, 40, 503), (16384, 300, 504), (16384 + 24, 21, 505),
+                       (65536 + 8, 19, 506), (151936, 12, 507), (151936 - 5, 9, 508)]:
+        _loss_case(V, dtype, T=T, S=3, seed=seed, variant=v, forward_only=True)
+    _loss_case(40000, dtype, T=700, S=9, seed=510, variant=v, forward_only=True)             # several rows per CTA
+    _loss_case(40000, dtype, T=50, S=4, seed=511, variant=v, forward_only=True, n_tokens=37, tau=1.7, pad=8)
+    _loss_case(151936, dtype, T=6, S=2, seed=512, variant=v, forward_only=True, neg_inf_cols=(16384, 32768))
+    _loss_case(151936, dtype, T=6, S=2, seed=513, variant=v, forward_only=True, neg_inf_cols=(0, 37984))
+    _loss_case(151936, dtype, T=6, S=2, seed=514, variant=v, forward_only=True, neg_inf_cols=(151669, 151936))
+    _loss_case(70000, dtype, T=8, S=2, seed=515, variant=v, forward_only=True, logit_sigma=30.0, centre_on_oracle=True)
+    from paper_2603_04135_b200 import binding as B
+    with pytest.raises(B.DppoError) as e:                                        # it has no backward
+        _loss_case(1000, dtype, T=8, S=2, seed=516, variant=v)
+    assert e.value.code == B.ERR_UNSUPPORTED
+
+
 def test_loss_auto_dispatch_matches_forced_kernels():
     # variant 0 on a long bf16 row takes the cluster kernel; outputs agree with the general kernel's
     a = _loss_case(151936, "bf16", T=11, S=2, seed=60, variant=0)
@@ -498,6 +519,11 @@ def test_loss_kernel_choice_query():
     assert choice(151936, B.BF16) == (B.KERNEL_SHARED, 4, 256, 0)        # the benchmark's rows
     assert choice(151936, B.F32) == (B.KERNEL_SHARED, 8, 256, 0)
     assert choice(400000, B.BF16) == (B.KERNEL_GENERAL, 1, 512, 0)       # too long for eight slices: not a fall-back
+    prm = B.LossParams(64, 151936, B.BF16, 151936, 4, 0, 0.2, 0.2, 0.04, 1.0)
+    fwd = B.grpo_loss_kernel_choice(prm, forward_only=True)                # long rows, no dlogits: streamed
+    assert (fwd.kernel, fwd.fell_back) == (B.KERNEL_STREAM, 0)
+    prm = B.LossParams(64, 32768, B.BF16, 32768, 4, 0, 0.2, 0.2, 0.04, 1.0)
+    assert B.grpo_loss_kernel_choice(prm, forward_only=True).kernel == B.KERNEL_SHARED   # 64 KB rows stay
     assert choice(151936, B.BF16, variant=1)[0] == B.KERNEL_GENERAL
     assert choice(151936, B.BF16, variant=80128) == (B.KERNEL_SHARED, 8, 128, 0)
     with pytest.raises(B.DppoError) as e:

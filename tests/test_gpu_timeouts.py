@@ -76,6 +76,43 @@ def test_loss_sweep_waits_run_out(dtype, V, variant):
                            b.view(torch.int16) if b.dtype == torch.bfloat16 else b.view(torch.int32))
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_streaming_forward_kernel_waits_run_out(dtype):
+    """The forward-only streaming kernel: the first stage of every CTA's ring expects 8 bytes more than its copy
+    brings, so the consumers' first wait runs out after 1 ms; every CTA reports the time-out, lets its copies land
+    and leaves all of its rows as rows that add nothing."""
+    from paper_2603_04135_b200 import binding as B
+    T, S, V = 400, 3, 151936
+    w = synth.scaled(synth.WORKLOADS["config3"], V=V, dtype=dtype)
+    tok = synth.make_token_inputs(w, T, 12, device="cuda")
+    cu = torch.from_numpy(np.linspace(0, T, S + 1).astype(np.int32)).cuda()
+    adv = torch.ones(S, device="cuda"); wseq = torch.full((S,), 0.1, device="cuda")
+
+    def call(variant):
+        prm = B.LossParams(T, V, B.BF16 if dtype == "bf16" else B.F32, V, S, variant, 0.2, 0.2, 0.04, 1.0)
+        nbytes = B.grpo_loss_workspace_bytes(prm)
+        ws = torch.full((nbytes,), 0x7f, dtype=torch.uint8, device="cuda")     # garbage the kernel must overwrite
+        loss_out = torch.full((5,), 7.0, device="cuda")
+        logp_out = torch.full((T,), 7.0, device="cuda"); lse_out = torch.full((T,), 7.0, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        B.grpo_loss_fwd_bwd(prm, tok.logits, tok.target, tok.logp_old, tok.logp_ref, cu, None, adv, wseq, None, None,
+                            logp_out, lse_out, loss_out, ws, nbytes, status)
+        torch.cuda.synchronize()
+        return loss_out, logp_out, lse_out, int(status.item())
+
+    before = call(0)                                              # variant 0 takes the streaming kernel here
+    assert before[3] == 0 and float(before[0][4]) == T
+    loss_out, logp_out, lse_out, status = call(B.LOSS_WAIT_SELF_TEST)
+    assert status == B.STATUS_TIMEOUT
+    assert bool((logp_out == 0).all()) and bool((lse_out == 0).all())
+    lo = loss_out.cpu().numpy()
+    assert np.isfinite(lo).all() and (lo[:4] == 0).all() and lo[4] == T
+    after = call(0)
+    assert after[3] == 0
+    for a, b in zip(before[:3], after[:3]):
+        assert torch.equal(a.view(torch.int32), b.view(torch.int32))
+
+
 def test_wait_self_test_needs_the_shared_memory_kernel():
     from paper_2603_04135_b200 import binding as B
     prm = B.LossParams(8, 512, B.BF16, 512, 1, B.LOSS_WAIT_SELF_TEST, 0.2, 0.2, 0.04, 1.0)   # warp-per-row shape
