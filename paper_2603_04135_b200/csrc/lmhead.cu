@@ -745,7 +745,8 @@ struct EpiPartial {
 // gradient: with the one entry E'[t, y_t] replaced by e_y - 2^(lse2 - ref2) (lm_rows_ref_kernel),
 //     dlogits[t, :] = -f_t * E'[t, :],   f_t = (dloss/dlogp / temperature) * 2^(ref2 - lse2).
 // The two gradient contractions therefore read E' itself: dhidden = -diag(f) (E' W) scales the accumulator rows
-// in its epilogue, dW = E'^T (-diag(f) hidden) takes pre-scaled hidden rows.  No dlogits pass, no second copy.
+// in its epilogue, dW = E'^T (-diag(f) hidden) takes pre-scaled hidden rows (kept transposed: the token axis is
+// the contraction's K).  No dlogits pass, no second copy.
 // The row maximum is never below the sampled token's logit, so e >= 1 for the largest entry; bf16 has the exponent
 // range of f32, and the exponent is clamped at 100 so that sums of V such entries times weights stay far from the
 // f32 overflow in the two contractions.  A row counts as in range while its sum stays below 2^96, i.e. while its
@@ -873,20 +874,17 @@ lm_rows_kernel(const LossArgs a, const float2* __restrict__ part, const float* _
 
 // Backward: one warp per token of the piece.  The tile sums of the row -> base-2 log-sum-exp (reference + log2 of
 // their sum, added in a fixed order), the loss's scalar stage (lane 0), then what turns E' into the gradient:
-// the row factor f, the replacement of the sampled token's entry, and the row of -f * hidden that dW contracts
-// with.  A row whose sum has left the range of the reference (the sampled token's log-prob below about -66) is
+// the row factor f and the replacement of the sampled token's entry.  A row whose sum has left the range of the reference (the sampled token's log-prob below about -66) is
 // reported as DPPO_STATUS_RANGE, adds nothing to the loss and gets a zero gradient.
 __global__ void __launch_bounds__(kRowsWarps * 32)
 lm_rows_ref_kernel(const LossArgs a, const float* __restrict__ sums, const float* __restrict__ zy,
                    const float* __restrict__ ref2, RowInfo* __restrict__ info, long long t0, long long tc, int n_ntiles,
-                   __nv_bfloat16* __restrict__ E, long long lde, const __nv_bfloat16* __restrict__ hidden, int H,
-                   __nv_bfloat16* __restrict__ hs) {
+                   __nv_bfloat16* __restrict__ E, long long lde) {
     const long long r = (long long)blockIdx.x * kRowsWarps + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (r >= tc) return;
     const long long t = t0 + r;
     const long long T = a.n_tokens_dev ? min((long long)*a.n_tokens_dev, a.T_max) : a.T_max;
-    float f = 0.0f;
     if (t < T) {
         float S = 0.0f;
         for (int i = lane; i < n_ntiles; i += 32) S += sums[r * n_ntiles + i];
@@ -918,31 +916,45 @@ lm_rows_ref_kernel(const LossArgs a, const float* __restrict__ sums, const float
                 }
             }
             info[t] = ri;
-            f = ri.f;
         }
-        f = __shfl_sync(0xffffffffu, f, 0);
     } else if (lane == 0) {                                            // no token here: the backward sees f = 0
         RowInfo z; z.lse2_hi = 0.0f; z.lse2_lo = 0.0f; z.f = 0.0f; z.y = -1;
         info[t] = z;
     }
-    // the piece's operand of the dW contraction: hs[r, :] = -f * hidden[t, :] as bf16
-    const uint4* hr = reinterpret_cast<const uint4*>(hidden + t * H);
-    uint4* out = reinterpret_cast<uint4*>(hs + r * H);
-    const float nf = -f;
-    for (int i = lane; i < H / 8; i += 32) {
-        uint4 q = make_uint4(0u, 0u, 0u, 0u);
-        if (f != 0.0f) {
-            const uint4 x = hr[i];
-            const uint32_t w[4] = {x.x, x.y, x.z, x.w};
-            uint32_t o[4];
+}
+
+// The piece's operand of the dW contraction, K-major (the token axis contiguous, which is what the tensor core
+// reads fastest): hsT[k, r] = -f[t0 + r] * hidden[t0 + r, k] as bf16, row pitch ld (a multiple of 64; the columns
+// tc .. ld - 1 are written as zeros).  One CTA transposes a tile of 64 tokens x 64 hidden columns through
+// shared memory: 16-byte loads along the hidden rows, 16-byte stores along the token axis.
+constexpr int kTrTile = 64;
+__global__ void __launch_bounds__(256)
+lm_scaled_hidden_t_kernel(const __nv_bfloat16* __restrict__ hidden, const RowInfo* __restrict__ info, long long t0,
+                          long long tc, int H, __nv_bfloat16* __restrict__ hsT, long long ld) {
+    __shared__ __align__(16) unsigned short tile[kTrTile][kTrTile + 8];          // [hidden column][token], padded rows
+    const long long r0 = (long long)blockIdx.x * kTrTile;
+    const int k0 = blockIdx.y * kTrTile;
+    for (int v = threadIdx.x; v < kTrTile * (kTrTile / 8); v += 256) {
+        const int row = v >> 3, kv = (v & 7) * 8;
+        const long long r = r0 + row;
+        float nf = 0.0f;
+        if (r < tc) nf = -info[t0 + r].f;
+        uint4 x = make_uint4(0u, 0u, 0u, 0u);
+        if (nf != 0.0f && k0 + kv < H) x = *reinterpret_cast<const uint4*>(hidden + (t0 + r) * H + k0 + kv);
+        const uint32_t w[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const __nv_bfloat162 b2 = __floats2bfloat162_rn(nf * __uint_as_float(w[k] << 16), nf * __uint_as_float(w[k] & 0xffff0000u));
-                o[k] = *reinterpret_cast<const uint32_t*>(&b2);
-            }
-            q = make_uint4(o[0], o[1], o[2], o[3]);
+        for (int k = 0; k < 4; ++k) {
+            const __nv_bfloat162 b2 = __floats2bfloat162_rn(nf * __uint_as_float(w[k] << 16), nf * __uint_as_float(w[k] & 0xffff0000u));
+            const uint32_t o = nf != 0.0f ? *reinterpret_cast<const uint32_t*>(&b2) : 0u;
+            tile[kv + 2 * k][row] = (unsigned short)(o & 0xffffu);
+            tile[kv + 2 * k + 1][row] = (unsigned short)(o >> 16);
         }
-        out[i] = q;
+    }
+    __syncthreads();
+    for (int v = threadIdx.x; v < kTrTile * (kTrTile / 8); v += 256) {
+        const int k = v >> 3, rv = (v & 7) * 8;
+        if (k0 + k < H && r0 + rv < ld)
+            *reinterpret_cast<uint4*>(hsT + (long long)(k0 + k) * ld + r0 + rv) = *reinterpret_cast<const uint4*>(&tile[k][rv]);
     }
 }
 
@@ -1182,7 +1194,7 @@ static LmWorkspace lm_layout(const dppo_lmhead_params* p, bool backward) {
     w.e = w.hs = w.dw32 = off;
     if (backward) {
         w.e = off;   off += al(rows_d * w.ld_v * 2);                  // E' of a chunk
-        w.hs = off;  off += al(rows * (size_t)p->H * 2);              // -f * hidden of a piece
+        w.hs = off;  off += al((size_t)round_up((long long)rows, 64) * (size_t)p->H * 2);   // (-f * hidden)^T of a piece
         if (p->dW_dtype == DPPO_BF16) { w.dw32 = off; off += al((size_t)p->loss.V * p->H * 4); }   // dW is accumulated in f32
     }
     w.total = off;
@@ -1295,6 +1307,7 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
             const long long piece = lm_piece_tokens(tc, tune.sub_tokens);
             for (long long s0 = t0; s0 < t0 + tc; s0 += piece) {
                 const long long ts = (t0 + tc - s0) < piece ? (t0 + tc - s0) : piece;   // tokens in this piece
+                const long long hs_ld = round_up(ts, 64);                              // row pitch of (-f hidden)^T
                 // (1) logits of the piece, tile by tile.  Forward only: per-tile (max, sum) of every row and z[y].
                 //     Backward: the exponentials relative to the rows' references, as bf16, into the piece's rows of
                 //     E' [tc x V], their per-tile sums and z[y]
@@ -1328,14 +1341,20 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
                     continue;
                 }
                 lm_rows_ref_kernel<<<(unsigned)((ts + kRowsWarps - 1) / kRowsWarps), kRowsWarps * 32, 0, s>>>(
-                    a, (const float*)part, zy, ref2, info, s0, ts, lay.n_ntiles, Ep, lay.ld_v, (const __nv_bfloat16*)hidden, H, hs);
+                    a, (const float*)part, zy, ref2, info, s0, ts, lay.n_ntiles, Ep, lay.ld_v);
                 DPPO_CHECK_LAUNCH("lmhead rows launch");
-                // (3) dW (+)= E'^T (-f hidden)[s0 : s0+ts, :]   (M = V, N = H, K = tokens of the piece; both MN-major);
-                //     the K range stops at the piece: both maps have ts rows and fill with zeros beyond
-                alignas(64) CUtensorMap map_e_mn, map_hs_mn;
+                lm_scaled_hidden_t_kernel<<<dim3((unsigned)(hs_ld / kTrTile), (unsigned)((H + kTrTile - 1) / kTrTile)), 256, 0, s>>>(
+                    (const __nv_bfloat16*)hidden, info, s0, ts, H, hs, hs_ld);
+                DPPO_CHECK_LAUNCH("lmhead transposed operand launch");
+                // (3) dW (+)= E'^T (-f hidden)[s0 : s0+ts, :]   (M = V, N = H, K = tokens of the piece; E' MN-major,
+                //     (-f hidden)^T K-major); the K range stops at the piece: both maps have ts tokens and fill with
+                //     zeros beyond
+                alignas(64) CUtensorMap map_e_mn, map_hs_k, map_hs_k_half;
                 rc = make_map(&map_e_mn, Ep, ts, V, lay.ld_v, 64);
                 if (rc != DPPO_OK) return rc;
-                rc = make_map(&map_hs_mn, hs, ts, H, H, 64);
+                rc = make_map(&map_hs_k, hs, H, ts, hs_ld, kBN);
+                if (rc != DPPO_OK) return rc;
+                rc = make_map(&map_hs_k_half, hs, H, ts, hs_ld, kHalfBN);
                 if (rc != DPPO_OK) return rc;
                 GemmShape g3 = gs0;
                 g3.n_mtiles = (V + kBM - 1) / kBM; g3.n_ntiles = (H + kBN - 1) / kBN; g3.n_ksteps = (int)((ts + kBK - 1) / kBK);
@@ -1343,7 +1362,7 @@ extern "C" int dppo_lmhead_grpo_loss(const dppo_lmhead_params* p, const void* hi
                 g3.hint_c = (tune.hints >> 14) & 3;
                 EpiAccumF32 e3 = {};
                 e3.rows = V; e3.cols = H; e3.accumulate = (n_dw > 0 || p->accumulate_dW) ? 1 : 0;
-                rc = run_gemm<EpiAccumF32, true, true>(pair, map_e_mn, map_hs_mn, map_hs_mn, map_dw, g3, e3, status, s, "lmhead dW launch");
+                rc = run_gemm<EpiAccumF32, true, false>(pair, map_e_mn, map_hs_k, map_hs_k_half, map_dw, g3, e3, status, s, "lmhead dW launch");
                 if (rc != DPPO_OK) return rc;
                 ++n_dw;
             }
