@@ -267,7 +267,7 @@ int dppo_grpo_loss_fwd_bwd(const dppo_loss_params* p, const void* logits, const 
  * row length asked for (its shared memory or cluster size) and the slower general kernel runs instead.
  * Errors: INVALID_ARG; UNSUPPORTED when params.variant forces a kernel that cannot take the shape.
  */
-typedef enum { DPPO_KERNEL_GENERAL = 0, DPPO_KERNEL_WARP = 1, DPPO_KERNEL_SHARED = 2, DPPO_KERNEL_STREAM = 3 } dppo_loss_kernel;
+typedef enum { DPPO_KERNEL_GENERAL = 0, DPPO_KERNEL_WARP = 1, DPPO_KERNEL_SHARED = 2, DPPO_KERNEL_STREAM = 3, DPPO_KERNEL_TILE = 4 } dppo_loss_kernel;
 typedef struct {
     int32_t kernel;         /* dppo_loss_kernel                                                      */
     int32_t ctas_per_row;   /* cluster size of the shared-memory kernel, else 1                      */

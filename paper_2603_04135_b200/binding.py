@@ -52,9 +52,9 @@ class LossKernelChoice(ctypes.Structure):
                 ("fell_back", ctypes.c_int32)]
 
 
-KERNEL_GENERAL, KERNEL_WARP, KERNEL_SHARED, KERNEL_STREAM = 0, 1, 2, 3
+KERNEL_GENERAL, KERNEL_WARP, KERNEL_SHARED, KERNEL_STREAM, KERNEL_TILE = 0, 1, 2, 3, 4
 KERNEL_NAMES = {KERNEL_GENERAL: "general two-pass", KERNEL_WARP: "warp per row", KERNEL_SHARED: "shared memory",
-                KERNEL_STREAM: "streaming (forward only)"}
+                KERNEL_STREAM: "streaming (forward only)", KERNEL_TILE: "tiles of rows"}
 LOSS_WAIT_SELF_TEST = 1000000      # added to dppo_loss_params.variant
 LMHEAD_WAIT_SELF_TEST = 100        # added to dppo_lmhead_params.variant
 

@@ -261,6 +261,9 @@ int run_rows(LossArgs a, int variant, cudaStream_t s, bool launch, dppo_loss_ker
     } else if (variant == 3) {
         ch.kernel = DPPO_KERNEL_STREAM; ch.threads = 512;
         rc = launch_rows_stream(a, s, launch);
+    } else if (variant == 4) {
+        ch.kernel = DPPO_KERNEL_TILE; ch.threads = 512;
+        rc = launch_rows_tile(a, s, launch);
     } else if (variant >= 10000) {
         ch.kernel = DPPO_KERNEL_SHARED; ch.ctas_per_row = variant / 10000; ch.threads = variant % 10000;
         rc = launch_rows_cluster(a, ch.ctas_per_row, ch.threads, s, launch);
@@ -294,7 +297,7 @@ int run_rows(LossArgs a, int variant, cudaStream_t s, bool launch, dppo_loss_ker
     } else {
         rc = fail(DPPO_ERR_INVALID_ARG, "grpo_loss: variant %d", variant);
     }
-    if (rc == DPPO_OK && self_test && ch.kernel != DPPO_KERNEL_SHARED && ch.kernel != DPPO_KERNEL_STREAM)
+    if (rc == DPPO_OK && self_test && ch.kernel != DPPO_KERNEL_SHARED && ch.kernel != DPPO_KERNEL_STREAM && ch.kernel != DPPO_KERNEL_TILE)
         return fail(DPPO_ERR_UNSUPPORTED, "grpo_loss: the wait self-test runs on the shared-memory and streaming kernels only");
     if (choice) *choice = ch;
     return rc;

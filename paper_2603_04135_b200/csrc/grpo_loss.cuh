@@ -305,6 +305,9 @@ int launch_rows_warp(const LossArgs& a, cudaStream_t s, bool launch = true);
 // Forward-only calls: persistent CTAs stream the rows through a shared-memory ring (grpo_loss_stream.cu).
 // Returns DPPO_ERR_UNSUPPORTED (nothing launched) when dlogits are asked for.
 int launch_rows_stream(const LossArgs& a, cudaStream_t s, bool launch = true);
+// Calls with dlogits on dense rows of up to 32 KB: tiles of rows through a shared-memory ring, the scalar stage of
+// up to 32 rows in one pass (grpo_loss_tile.cu).  Returns DPPO_ERR_UNSUPPORTED (nothing launched) for other calls.
+int launch_rows_tile(const LossArgs& a, cudaStream_t s, bool launch = true);
 int launch_loss_reduce(const LossArgs& a, float* loss_out, cudaStream_t s);
 
 }  // namespace dppo

@@ -1,0 +1,446 @@
+// Loss sweep with dlogits for rows of up to 32 KB: tiles of consecutive rows go through a shared-memory ring, and
+// the three kinds of work a row needs are done by three kinds of warps that never wait for memory.
+//
+// A short row is dominated by what does not scale with its length: two warp reductions and, above all, the
+// binary64 scalar stage (a logarithm, two exponentials, the clip logic: several hundred instructions, and a warp
+// instruction costs the same with one lane active as with 32).  A warp that loads a row, reduces it, runs the
+// scalar stage and stores the row sees all of those latencies one after the other.  Here one persistent CTA per SM
+// splits the work:
+//   loader          one thread issues one bulk copy per TILE (up to 32 KB of consecutive rows, at most 32 units)
+//                   into a ring of stages, running ahead as far as the ring allows
+//   16 consumer     pass 1 on the tile's UNITS (a unit is a row, or a 2 KB part of a longer row; one warp per unit):
+//   warps           maximum, 2^(z c - r) once, kept in place as fp16 pairs (bf16 rows) or f32, the unit's (r, sum) to
+//                   shared memory.  Pass 2, two tiles later: the stored exponentials times the unit's factor go to
+//                   dlogits with streaming stores; the stage is then free
+//   scalar warps    lane q takes row q of a tile: joins the row's units, runs the scalar stage for up to 32 rows in
+//                   one pass, and leaves every unit's factor g/tau 2^(r - lse2) (and the one element per row that
+//                   also carries the onehot term) for pass 2.  The rows' per-token inputs and sequences are gathered
+//                   a tile ahead
+// HBM sees one read and one write per element.  Every wait is bounded; on a time-out the CTA raises an abort flag,
+// reports DPPO_STATUS_TIMEOUT, lets its copies in flight land (bounded) and leaves all of its rows as rows that add
+// nothing.
+#include <cuda_fp16.h>
+
+#include "common.cuh"
+#include "grpo_loss.cuh"
+
+namespace dppo {
+using namespace packed;
+
+namespace tile {
+
+constexpr int kConsumerWarps = 16;
+constexpr int kScalarWarps = 3;
+constexpr int kThreads = (kConsumerWarps + kScalarWarps + 1) * 32;       // + the loader's warp
+constexpr int kStages = 6;
+constexpr int kStageBytes = 32768;
+constexpr int kMaxUnits = 32;                             // units of a tile (and rows: one lane of a scalar warp each)
+constexpr int kSkew = 2;                                  // pass 2 of tile k runs after pass 1 of tile k + kSkew
+constexpr size_t kDynSmem = (size_t)kStages * kStageBytes;
+
+struct Meta {                                             // of one stage
+    float2 rs[kMaxUnits];                                 // per unit: reference r = max c, sum of 2^(z c - r)
+    float sc[kMaxUnits];                                  // per unit: the factor of its stored exponentials
+    int fix_y[kMaxUnits];                                 // per row: the element that also carries the onehot term, or -1
+    float fix_val[kMaxUnits];                             // its value
+};
+
+struct Shared {
+    unsigned long long full[kStages];                     // the tile's bytes have landed
+    unsigned long long p1_done[kStages];                  // all consumer warps have finished pass 1 of the tile
+    unsigned long long s_done[kStages];                   // the tile's scalar stage is done
+    unsigned long long free_[kStages];                    // all consumer warps have finished pass 2: the stage may be refilled
+    Meta meta[kStages];
+    int abort;
+};
+
+// How a row length maps to tiles: rows per tile R, parts per row P (units of a tile: R * P <= 32).
+struct Geometry {
+    int nvec;                                             // 16-byte vectors of a row that hold elements
+    int part_vecs;                                        // vectors per part (the last part of a row may have fewer)
+    int parts;                                            // parts per row
+    int rows;                                             // rows per tile
+};
+template <int kVPL>
+__host__ __device__ inline Geometry geometry(int V, int log2_per_vec, long long row_bytes) {
+    Geometry g;
+    g.nvec = V >> log2_per_vec;
+    g.part_vecs = 32 * kVPL;
+    g.parts = (g.nvec + g.part_vecs - 1) / g.part_vecs;
+    if (g.parts < 1) g.parts = 1;
+    const long long fit = kStageBytes / (row_bytes > 0 ? row_bytes : 1);
+    const int by_units = kMaxUnits / g.parts;
+    g.rows = (int)(fit < by_units ? fit : by_units);
+    return g;
+}
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ bool try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done != 0;
+}
+// Bounded wait on phase `parity`; also leaves (false) when another role has raised the abort flag.  A warp that waits
+// with all its lanes takes the vote of the lanes' results, so that it leaves as a whole.
+__device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned long long limit_ns) {
+    const unsigned long long t0 = global_ns();
+    for (;;) {
+        if (try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (global_ns() - t0 > limit_ns) { *abort_flag = 1; return false; }
+    }
+}
+__device__ __forceinline__ void arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(bar) : "memory");
+}
+
+}  // namespace tile
+
+using namespace tile;
+
+template <bool kF32, int kVPL>
+__global__ void __launch_bounds__(kThreads, 1)
+grpo_loss_tile_kernel(const LossArgs a) {
+    constexpr int kLog2PerVec = kF32 ? 2 : 3;               // elements per 16-byte vector: 4 f32 or 8 bf16
+    constexpr uint32_t kPad = kF32 ? 0xFF800000u : 0xFF80FF80u;   // -inf: adds nothing to the maximum or the sum
+    extern __shared__ __align__(128) unsigned char ring_raw[];
+    __shared__ Shared sh;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    volatile int* abort_flag = &sh.abort;
+    const long long T = a.n_tokens_dev ? min((long long)*a.n_tokens_dev, a.T_max) : a.T_max;
+    const Geometry geo = geometry<kVPL>(a.V, kLog2PerVec, a.row_bytes);
+    const int R = geo.rows, P = geo.parts;
+    const float c = a.scale2;
+    // this CTA's tiles: tile k covers rows (blockIdx.x + k gridDim.x) R ... of the batch
+    const long long total_tiles = (T + R - 1) / R;
+    const int n_tiles = (long long)blockIdx.x < total_tiles ? (int)((total_tiles - 1 - blockIdx.x) / gridDim.x) + 1 : 0;
+    auto tile_row0 = [&](int k) { return ((long long)blockIdx.x + (long long)k * gridDim.x) * R; };
+    auto tile_rows = [&](int k) { return (int)min((long long)R, T - tile_row0(k)); };
+
+    if (tid == 0) {
+        sh.abort = 0;
+        for (int s = 0; s < kStages; ++s) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(&sh.full[s])));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&sh.p1_done[s])), "r"(kConsumerWarps));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(&sh.s_done[s])));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&sh.free_[s])), "r"(kConsumerWarps));
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    if (warp == kConsumerWarps + kScalarWarps) {
+        // ------------------------------------------------------------------ loader
+        if (lane == 0) {
+            int k = 0;
+            for (; k < n_tiles && !*abort_flag; ++k) {
+                const uint32_t s = (uint32_t)k % kStages, use = (uint32_t)k / kStages;
+                if (use > 0 && !wait(smem_u32(&sh.free_[s]), (use - 1) & 1, abort_flag, a.wait_limit_ns)) break;
+                const uint32_t bytes = (uint32_t)tile_rows(k) * (uint32_t)a.row_bytes;
+                const uint32_t bar = smem_u32(&sh.full[s]);
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                             :: "r"(bar), "r"(bytes + (k == 0 ? (uint32_t)a.test_extra_tx : 0u)) : "memory");
+                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                             :: "r"(smem_u32(ring_raw + (size_t)s * kStageBytes)), "l"(a.logits + tile_row0(k) * a.row_bytes), "r"(bytes), "r"(bar)
+                             : "memory");
+            }
+            if (*abort_flag) {
+                // leaving early: the copies still in flight get a bounded chance to land before the CTA's shared
+                // memory goes away
+                const int pending = k < kStages ? k : kStages;
+                for (int i = 0; i < pending; ++i) {
+                    const uint32_t ki = (uint32_t)(k - 1 - i);
+                    const unsigned long long t0 = global_ns();
+                    while (!try_wait(smem_u32(&sh.full[ki % kStages]), (ki / kStages) & 1) && global_ns() - t0 <= a.wait_limit_ns) {}
+                }
+            }
+        }
+    } else if (warp < kConsumerWarps) {
+        // ------------------------------------------------------------------ consumers
+        for (int k = 0; k < n_tiles + kSkew && !*abort_flag; ++k) {
+            if (k < n_tiles) {
+                // ---- pass 1 of tile k: this warp's units
+                const uint32_t s = (uint32_t)k % kStages;
+                if (!__all_sync(0xffffffffu, wait(smem_u32(&sh.full[s]), ((uint32_t)k / kStages) & 1, abort_flag, a.wait_limit_ns))) break;
+                uint4* stage = reinterpret_cast<uint4*>(ring_raw + (size_t)s * kStageBytes);
+                const int units = tile_rows(k) * P;
+                for (int u = warp; u < units; u += kConsumerWarps) {
+                    const int row = u / P, part = u - row * P;
+                    uint4* src = stage + (size_t)row * (size_t)(a.row_bytes >> 4) + part * geo.part_vecs;
+                    const int nv = min(geo.part_vecs, geo.nvec - part * geo.part_vecs);
+                    uint4 d[kVPL];
+#pragma unroll
+                    for (int j = 0; j < kVPL; ++j) {
+                        const int i = lane + 32 * j;
+                        d[j] = i < nv ? src[i] : make_uint4(kPad, kPad, kPad, kPad);
+                    }
+                    float m;
+                    if constexpr (kF32) {
+                        m = -INFINITY;
+#pragma unroll
+                        for (int j = 0; j < kVPL; ++j)
+                            m = fmaxf(m, fmaxf(fmaxf(__uint_as_float(d[j].x), __uint_as_float(d[j].y)),
+                                               fmaxf(__uint_as_float(d[j].z), __uint_as_float(d[j].w))));
+                    } else {
+                        __nv_bfloat162 mx2 = __float2bfloat162_rn(-INFINITY);
+#pragma unroll
+                        for (int j = 0; j < kVPL; ++j) {
+                            mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&d[j].x));
+                            mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&d[j].y));
+                            mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&d[j].z));
+                            mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&d[j].w));
+                        }
+                        m = fmaxf(__low2float(mx2), __high2float(mx2));
+                    }
+                    m = warp_max(m);
+                    const float r = m * c;                          // -inf only if the whole unit is -inf
+                    const float nr = r > -INFINITY ? -r : 0.0f;
+                    const f32x2 c2 = pair_of(c, c), nr2 = pair_of(nr, nr);
+                    f32x2 acc0 = pair_of(0.0f, 0.0f), acc1 = acc0;
+#pragma unroll
+                    for (int j = 0; j < kVPL; ++j) {
+                        if constexpr (kF32) {
+                            d[j] = exp_quad(d[j], c2, nr2, acc0, acc1);
+                        } else {
+                            d[j].x = exp_pair(d[j].x, c2, nr2, acc0); d[j].y = exp_pair(d[j].y, c2, nr2, acc1);
+                            d[j].z = exp_pair(d[j].z, c2, nr2, acc0); d[j].w = exp_pair(d[j].w, c2, nr2, acc1);
+                        }
+                        const int i = lane + 32 * j;
+                        if (i < nv) src[i] = d[j];
+                    }
+                    float s0, s1;
+                    unpair(add2(acc0, acc1), s0, s1);
+                    const float sum = warp_sum(s0 + s1);
+                    if (lane == 0) sh.meta[s].rs[u] = make_float2(r, sum);
+                }
+                __syncwarp();
+                if (lane == 0) arrive(smem_u32(&sh.p1_done[s]));            // release: the scalar warp's wait acquires
+            }
+            if (k >= kSkew) {
+                // ---- pass 2 of tile k - kSkew
+                const int kk = k - kSkew;
+                const uint32_t s = (uint32_t)kk % kStages;
+                if (!__all_sync(0xffffffffu, wait(smem_u32(&sh.s_done[s]), ((uint32_t)kk / kStages) & 1, abort_flag, a.wait_limit_ns))) break;
+                const uint4* stage = reinterpret_cast<const uint4*>(ring_raw + (size_t)s * kStageBytes);
+                const int units = tile_rows(kk) * P;
+                const long long t0 = tile_row0(kk);
+                for (int u = warp; u < units; u += kConsumerWarps) {
+                    const int row = u / P, part = u - row * P;
+                    const uint4* src = stage + (size_t)row * (size_t)(a.row_bytes >> 4) + part * geo.part_vecs;
+                    char* drow = a.dlogits + (t0 + row) * a.row_bytes;
+                    uint4* dst = reinterpret_cast<uint4*>(drow) + part * geo.part_vecs;
+                    const int nv = min(geo.part_vecs, geo.nvec - part * geo.part_vecs);
+                    const float sc = sh.meta[s].sc[u];
+                    const f32x2 sc2 = pair_of(sc, sc);
+#pragma unroll
+                    for (int j = 0; j < kVPL; ++j) {
+                        const int i = lane + 32 * j;
+                        if (i < nv) {
+                            const uint4 e = src[i];
+                            uint4 o;
+                            if constexpr (kF32) {
+                                o = scale_quad(e, sc2);
+                            } else {
+                                o.x = scale_pair(e.x, sc2); o.y = scale_pair(e.y, sc2);
+                                o.z = scale_pair(e.z, sc2); o.w = scale_pair(e.w, sc2);
+                            }
+                            __stcs(dst + i, o);
+                        }
+                    }
+                    // the one element of the row that also carries the onehot term, if it lies in this unit
+                    const int y = sh.meta[s].fix_y[row];
+                    const int e0 = (part * geo.part_vecs) << kLog2PerVec;
+                    __syncwarp();                                           // after the lanes' stores of the unit
+                    if (lane == 0 && y >= e0 && y < e0 + (nv << kLog2PerVec)) Elems<!kF32>::store1(drow, y, sh.meta[s].fix_val[row]);
+                }
+                // the stage goes back to the loader: this warp's reads and writes of it come before the next copy into it
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) arrive(smem_u32(&sh.free_[s]));
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ scalar warps: lane q <-> row q of a tile
+        const int first = warp - kConsumerWarps;
+        // what the scalar stage needs besides (r, sum), gathered one tile ahead ("next"), used as "cur"
+        struct Gathered {
+            long long t;
+            int y;                                                          // -1 for a lane without a row
+            float lp_old, lp_ref, zy_raw;
+            double A, W, lr;
+            bool mine, seg_ok;
+        };
+        Gathered nxt, cur;
+        // first half: the per-token inputs (lane-indexed loads, consumed by the second half a scalar stage later)
+        auto gather_tokens = [&](int k) {
+            nxt.t = tile_row0(k) + lane;
+            nxt.mine = lane < tile_rows(k);
+            nxt.y = -1; nxt.lp_old = 0.0f; nxt.lp_ref = 0.0f;
+            if (nxt.mine) { nxt.y = a.target[nxt.t]; nxt.lp_old = a.logp_old[nxt.t]; nxt.lp_ref = a.logp_ref[nxt.t]; }
+        };
+        // second half: the rows' sequences (the whole warp searches cu_seqlens, 32 probes per round trip, once per
+        // sequence that the tile touches) and the sampled tokens' logits, from global memory: the stage's copy of
+        // the row is overwritten by pass 1
+        auto gather_rest = [&](int k) {
+            const long long t0 = tile_row0(k), t_end = t0 + tile_rows(k);
+            nxt.seg_ok = false;
+            int my_seg = 0, my_len = 1;
+            long long at = t0;                                              // first row not yet looked up
+            while (a.S_max >= 1 && at < t_end) {
+                int lo = 0, hi = a.S_max;
+                while (hi - lo > 1) {
+                    const int step = (hi - lo + 31) >> 5;
+                    const long long idx = (long long)lo + (long long)(lane + 1) * step;
+                    const bool le = idx < hi && (long long)a.cu_seqlens[idx] <= at;
+                    const int n = __popc(__ballot_sync(0xffffffffu, le));
+                    lo += n * step;
+                    hi = min(hi, lo + step);
+                }
+                const long long s_lo = a.cu_seqlens[lo], s_hi = a.cu_seqlens[lo + 1];
+                const bool ok = at >= s_lo && at < s_hi;
+                const long long upto = ok ? min(s_hi, t_end) : at + 1;      // rows [at, upto) are settled by this lookup
+                if (ok && nxt.t >= at && nxt.t < upto) { nxt.seg_ok = true; my_seg = lo; my_len = (int)(s_hi - s_lo); }
+                at = upto;
+            }
+            nxt.A = nxt.W = nxt.lr = 0.0;
+            if (nxt.mine && nxt.seg_ok) {
+                const int idx = a.seg_map ? a.seg_map[my_seg] : my_seg;
+                nxt.A = (double)a.adv[idx];
+                nxt.W = a.no_length_norm ? (double)a.w[idx] : (double)a.w[idx] / (double)my_len;
+                if (a.seq_log_ratio) nxt.lr = (double)a.seq_log_ratio[my_seg];
+            }
+            nxt.zy_raw = 0.0f;
+            if (nxt.mine && nxt.y >= 0 && nxt.y < a.V) nxt.zy_raw = Elems<!kF32>::load1(a.logits + nxt.t * a.row_bytes, nxt.y);
+        };
+        if (first < n_tiles) { gather_tokens(first); gather_rest(first); }
+        for (int k = first; k < n_tiles && !*abort_flag; k += kScalarWarps) {
+            const uint32_t s = (uint32_t)k % kStages;
+            if (!__all_sync(0xffffffffu, wait(smem_u32(&sh.p1_done[s]), ((uint32_t)k / kStages) & 1, abort_flag, a.wait_limit_ns))) break;
+            cur = nxt;
+            const bool more = k + kScalarWarps < n_tiles;
+            if (more) gather_tokens(k + kScalarWarps);                     // in flight during this tile's scalar stage
+            Meta& meta = sh.meta[s];
+            if (cur.mine) {
+                const int u0 = lane * P;
+                float r = -INFINITY, sum = 0.0f;                            // the row's units joined: sum of 2^(z c - r)
+                for (int p = 0; p < P; ++p) {
+                    const float2 q = meta.rs[u0 + p];
+                    const float hi = fmaxf(r, q.x);
+                    const float x = r > -INFINITY ? sum * ex2(r - hi) : 0.0f;
+                    const float y = q.x > -INFINITY ? q.y * ex2(q.x - hi) : 0.0f;
+                    r = hi; sum = x + y;
+                }
+                const bool y_ok = cur.y >= 0 && cur.y < a.V;
+                RowInputs in;
+                in.A = in.W = in.zy = in.logp_old = in.logp_ref = in.seq_lr = 0.0;
+                in.use_seq = 0; in.y = cur.y; in.state = 0;
+                if (!cur.seg_ok) in.state = DPPO_STATUS_BAD_SEGMENTS;
+                else if (!y_ok) in.state = DPPO_STATUS_BAD_TARGET;
+                else {
+                    in.A = cur.A; in.W = cur.W;
+                    if (a.seq_log_ratio) { in.use_seq = 1; in.seq_lr = cur.lr; }
+                    in.zy = (double)cur.zy_raw / a.temperature;
+                    in.logp_old = (double)cur.lp_old; in.logp_ref = (double)cur.lp_ref;
+                }
+                const RowScalars rs = row_finish(a, cur.t, in, r, sum, true);
+                const float ng = rs.valid ? -rs.g_over_tau : 0.0f;
+                // dlogits = g/tau (onehot - 2^(z c - lse2)): every unit's stored exponentials times its own factor
+                for (int p = 0; p < P; ++p) {
+                    const float rp = meta.rs[u0 + p].x;
+                    meta.sc[u0 + p] = rs.valid ? ng * ex2((rp - rs.lse2_hi) - rs.lse2_lo) : 0.0f;
+                }
+                int fix_y = -1;
+                float fix_val = 0.0f;
+                if (rs.valid) {
+                    // the element that also carries the onehot term: the same exponential as pass 1 formed (rounded
+                    // to fp16 where the stored ones are) times its unit's factor, minus g/tau
+                    const int py = (cur.y >> kLog2PerVec) / geo.part_vecs;
+                    const float rp = meta.rs[u0 + py].x;
+                    const float nr = rp > -INFINITY ? -rp : 0.0f;
+                    float e = cur.zy_raw > -INFINITY ? ex2(fmaf(cur.zy_raw, c, nr)) : 0.0f;
+                    if (!kF32) e = __half2float(__float2half_rn(e));
+                    fix_y = cur.y;
+                    fix_val = fmaf(e, meta.sc[u0 + py], -ng);
+                }
+                meta.fix_y[lane] = fix_y;
+                meta.fix_val[lane] = fix_val;
+            }
+            __syncwarp();
+            if (lane == 0) arrive(smem_u32(&sh.s_done[s]));                 // release: the consumers' waits acquire
+            if (more) gather_rest(k + kScalarWarps);
+        }
+    }
+
+    __syncthreads();
+    if (sh.abort) {
+        // a wait ran out somewhere in this CTA: report it, and leave every row of the CTA as a row that adds nothing
+        // (rows that were already finished included: which ones were is not worth tracking on this path)
+        if (tid == 0) set_status(a.status, DPPO_STATUS_TIMEOUT);
+        const RowTerms zero = {0.0, 0.0, 0.0, 0.0};
+        for (int k = 0; k < n_tiles; ++k) {
+            const long long t0 = tile_row0(k);
+            const int rows = tile_rows(k);
+            for (int q = tid; q < rows; q += kThreads) {
+                a.terms[t0 + q] = zero;
+                if (a.logp_out) a.logp_out[t0 + q] = 0.0f;
+                if (a.lse_out) a.lse_out[t0 + q] = 0.0f;
+            }
+            for (int i = tid; i < rows * geo.nvec; i += kThreads) {
+                const int q = i / geo.nvec, v = i - q * geo.nvec;
+                reinterpret_cast<uint4*>(a.dlogits + (t0 + q) * a.row_bytes)[v] = make_uint4(0u, 0u, 0u, 0u);
+            }
+        }
+    }
+}
+
+// ---- host side ---------------------------------------------------------------------------------------
+template <bool kF32, int kVPL>
+static int launch_tile_t(const LossArgs& a, cudaStream_t s, bool launch) {
+    auto kernel = grpo_loss_tile_kernel<kF32, kVPL>;
+    static bool raised[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); dev = -1; }
+    if (dev < 0 || !raised[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDynSmem);
+        if (e != cudaSuccess) { cudaGetLastError(); return fail(DPPO_ERR_UNSUPPORTED, "tile kernel: %zu bytes of shared memory refused", kDynSmem); }
+        if (dev >= 0) raised[dev] = true;
+    }
+    if (!launch) return DPPO_OK;
+    const Geometry geo = geometry<kVPL>(a.V, kF32 ? 2 : 3, a.row_bytes);
+    const long long tiles = (a.T_max + geo.rows - 1) / geo.rows;
+    const long long grid = tiles < sm_count() ? tiles : sm_count();
+    kernel<<<(unsigned)(grid > 0 ? grid : 1), kThreads, kDynSmem, s>>>(a);
+    DPPO_CHECK_LAUNCH("grpo_loss tile launch");
+    return DPPO_OK;
+}
+
+template <bool kF32>
+static int launch_tile_dtype(const LossArgs& a, int nvec, cudaStream_t s, bool launch) {
+    if (nvec <= 32) return launch_tile_t<kF32, 1>(a, s, launch);
+    if (nvec <= 64) return launch_tile_t<kF32, 2>(a, s, launch);
+    return launch_tile_t<kF32, 4>(a, s, launch);
+}
+
+// Calls with dlogits on dense rows: V a whole number of 16-byte vectors, the row pitch a multiple of 16 bytes and at
+// most 32 KB, both matrices 16-byte aligned.  DPPO_ERR_UNSUPPORTED (nothing launched) otherwise.
+int launch_rows_tile(const LossArgs& a, cudaStream_t s, bool launch) {
+    const int per_vec = a.bf16 ? 8 : 4;
+    if (!a.dlogits) return fail(DPPO_ERR_UNSUPPORTED, "tile kernel: calls with dlogits");
+    if (a.V < per_vec || a.V % per_vec != 0) return fail(DPPO_ERR_UNSUPPORTED, "tile kernel: V=%d is not a whole number of 16-byte vectors", a.V);
+    if (a.row_bytes % 16 != 0 || a.row_bytes > kStageBytes || a.row_bytes < (long long)a.V * (a.bf16 ? 2 : 4))
+        return fail(DPPO_ERR_UNSUPPORTED, "tile kernel: row pitch of %lld bytes", a.row_bytes);
+    if ((((uintptr_t)a.logits) | ((uintptr_t)a.dlogits)) & 15) return fail(DPPO_ERR_UNSUPPORTED, "tile kernel: matrices not 16-byte aligned");
+    const int nvec = a.V / per_vec;
+    return a.bf16 ? launch_tile_dtype<false>(a, nvec, s, launch) : launch_tile_dtype<true>(a, nvec, s, launch);
+}
+
+}  // namespace dppo

@@ -398,6 +398,33 @@ def test_loss_warp_per_row_kernel(dtype):
 
 
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_loss_tile_kernel(dtype):
+    # calls with dlogits on the tile kernel (forced): rows of one vector, of every vectors-per-lane form, rows that are
+    # split into several 2 KB units with a short last one, rows that fill a stage alone; fewer tiles than CTAs and
+    # several tiles per CTA (so that stages are reused many times), a last tile with fewer rows, sequences that end
+    # inside a tile, a padded row pitch, in place, a device-side token count, masked columns (a whole unit of -inf),
+    # a wide dynamic range
+    v = 4
+    per = 8 if dtype == "bf16" else 4
+    for nvec, T, seed in [(1, 67, 600), (3, 200, 601), (32, 67, 602), (33, 150, 603), (64, 67, 604), (65, 67, 605), (128, 67, 606),
+                          (129, 40, 607), (300, 67, 608), (512, 40, 609), (1000, 23, 610), (2048, 9, 611)]:
+        _loss_case(nvec * per, dtype, T=T, S=5, seed=seed, variant=v)
+    _loss_case(128 * per, dtype, T=40000, S=300, seed=620, variant=v, centre_on_oracle=True)                     # 17 tiles per CTA, short sequences
+    _loss_case(64 * per, dtype, T=30011, S=40, seed=621, variant=v, centre_on_oracle=True)
+    _loss_case(200 * per, dtype, T=5000, S=40, seed=622, variant=v, pad=3 * per, centre_on_oracle=True)          # padded pitch: the padding stays
+    _loss_case(128 * per, dtype, T=500, S=4, seed=623, variant=v, in_place=True)
+    _loss_case(96 * per, dtype, T=900, S=7, seed=624, variant=v, n_tokens=611, tau=1.7)
+    _loss_case(512 * per, dtype, T=50, S=2, seed=625, variant=v, neg_inf_cols=(128 * per, 256 * per))
+    _loss_case(512 * per, dtype, T=50, S=2, seed=626, variant=v, neg_inf_cols=(0, 300 * per))
+    _loss_case(128 * per, dtype, T=40, S=3, seed=627, variant=v, logit_sigma=40.0, centre_on_oracle=True)
+    from paper_2603_04135_b200 import binding as B
+    for bad in (dict(V=1004 if dtype == "bf16" else 1002, T=8), dict(V=4096 * per, T=8), dict(V=1024, T=8, forward_only=True)):
+        with pytest.raises(B.DppoError) as e:                                    # ragged tail, a row above 32 KB, no dlogits
+            _loss_case(bad.pop("V"), dtype, S=2, seed=630, variant=v, **bad)
+        assert e.value.code == B.ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
 def test_loss_streaming_forward_kernel(dtype):
     # forward-only calls on the streaming kernel (forced): rows of less than a vector, of one piece, of several pieces
     # with a ragged last one, ragged tails, more rows than CTAs, a device-side token count, a temperature, masked
