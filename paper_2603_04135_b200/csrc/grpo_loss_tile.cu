@@ -10,7 +10,7 @@
 //                   into a ring of stages, running ahead as far as the ring allows
 //   16 consumer     pass 1 on the tile's UNITS (a unit is a row, or a 2 KB part of a longer row; one warp per unit):
 //   warps           maximum, 2^(z c - r) once, kept in place as fp16 pairs (bf16 rows) or f32, the unit's (r, sum) to
-//                   shared memory.  Pass 2, two tiles later: the stored exponentials times the unit's factor go to
+//                   shared memory.  Pass 2, three tiles later: the stored exponentials times the unit's factor go to
 //                   dlogits with streaming stores; the stage is then free
 //   scalar warps    lane q takes row q of a tile: joins the row's units, runs the scalar stage for up to 32 rows in
 //                   one pass, and leaves every unit's factor g/tau 2^(r - lse2) (and the one element per row that
@@ -35,8 +35,9 @@ constexpr int kThreads = (kConsumerWarps + kScalarWarps + 1) * 32;       // + th
 constexpr int kStages = 6;
 constexpr int kStageBytes = 32768;
 constexpr int kMaxUnits = 32;                             // units of a tile (and rows: one lane of a scalar warp each)
-constexpr int kSkew = 2;                                  // pass 2 of tile k runs after pass 1 of tile k + kSkew
-constexpr size_t kDynSmem = (size_t)kStages * kStageBytes;
+constexpr int kSkew = 3;                                  // pass 2 of tile k runs after pass 1 of tile k + kSkew
+constexpr int kCuCache = 6144;                            // entries of cu_seqlens kept in shared memory (24 KB)
+constexpr size_t kDynSmem = (size_t)kStages * kStageBytes + (size_t)kCuCache * 4;
 
 struct Meta {                                             // of one stage
     float2 rs[kMaxUnits];                                 // per unit: reference r = max c, sum of 2^(z c - r)
@@ -57,7 +58,7 @@ struct Shared {
 // How a row length maps to tiles: rows per tile R, parts per row P (units of a tile: R * P <= 32).
 struct Geometry {
     int nvec;                                             // 16-byte vectors of a row that hold elements
-    int part_vecs;                                        // vectors per part (the last part of a row may have fewer)
+    int part_vecs;                                        // vectors per part, at most 32 kVPL (the last part of a row may have fewer)
     int parts;                                            // parts per row
     int rows;                                             // rows per tile
 };
@@ -65,9 +66,9 @@ template <int kVPL>
 __host__ __device__ inline Geometry geometry(int V, int log2_per_vec, long long row_bytes) {
     Geometry g;
     g.nvec = V >> log2_per_vec;
-    g.part_vecs = 32 * kVPL;
-    g.parts = (g.nvec + g.part_vecs - 1) / g.part_vecs;
+    g.parts = (g.nvec + 32 * kVPL - 1) / (32 * kVPL);
     if (g.parts < 1) g.parts = 1;
+    g.part_vecs = (g.nvec + g.parts - 1) / g.parts;       // equal parts (the last one may be a little shorter)
     const long long fit = kStageBytes / (row_bytes > 0 ? row_bytes : 1);
     const int by_units = kMaxUnits / g.parts;
     g.rows = (int)(fit < by_units ? fit : by_units);
@@ -80,20 +81,27 @@ __device__ __forceinline__ unsigned long long global_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
+// One try: the thread is suspended until the phase completes or about a microsecond has passed (a waiting warp
+// then issues a handful of instructions per microsecond instead of spinning against the working warps).
+constexpr uint32_t kSuspendNs = 1000;
 __device__ __forceinline__ bool try_wait(uint32_t bar, uint32_t parity) {
     uint32_t done;
     asm volatile("{\n\t.reg .pred p;\n\t"
-                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
                  "selp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+                 : "=r"(done) : "r"(bar), "r"(parity), "r"(kSuspendNs) : "memory");
     return done != 0;
 }
 // Bounded wait on phase `parity`; also leaves (false) when another role has raised the abort flag.  A warp that waits
-// with all its lanes takes the vote of the lanes' results, so that it leaves as a whole.
+// with all its lanes takes the vote of the lanes' results, so that it leaves as a whole.  The clock and the abort
+// flag are looked at once per eight tries (a try lasts up to a microsecond), not per try.
 __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned long long limit_ns) {
+    if (try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_ns();
     for (;;) {
-        if (try_wait(bar, parity)) return true;
+#pragma unroll 1
+        for (int i = 0; i < 8; ++i)
+            if (try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
         if (global_ns() - t0 > limit_ns) { *abort_flag = 1; return false; }
     }
@@ -108,7 +116,7 @@ using namespace tile;
 
 template <bool kF32, int kVPL>
 __global__ void __launch_bounds__(kThreads, 1)
-grpo_loss_tile_kernel(const LossArgs a) {
+grpo_loss_tile_kernel(const LossArgs a, const int rows_per_tile) {
     constexpr int kLog2PerVec = kF32 ? 2 : 3;               // elements per 16-byte vector: 4 f32 or 8 bf16
     constexpr uint32_t kPad = kF32 ? 0xFF800000u : 0xFF80FF80u;   // -inf: adds nothing to the maximum or the sum
     extern __shared__ __align__(128) unsigned char ring_raw[];
@@ -117,7 +125,7 @@ grpo_loss_tile_kernel(const LossArgs a) {
     volatile int* abort_flag = &sh.abort;
     const long long T = a.n_tokens_dev ? min((long long)*a.n_tokens_dev, a.T_max) : a.T_max;
     const Geometry geo = geometry<kVPL>(a.V, kLog2PerVec, a.row_bytes);
-    const int R = geo.rows, P = geo.parts;
+    const int R = rows_per_tile, P = geo.parts;               // R <= geo.rows: fewer for a batch of less than a full tile per SM
     const float c = a.scale2;
     // this CTA's tiles: tile k covers rows (blockIdx.x + k gridDim.x) R ... of the batch
     const long long total_tiles = (T + R - 1) / R;
@@ -125,6 +133,13 @@ grpo_loss_tile_kernel(const LossArgs a) {
     auto tile_row0 = [&](int k) { return ((long long)blockIdx.x + (long long)k * gridDim.x) * R; };
     auto tile_rows = [&](int k) { return (int)min((long long)R, T - tile_row0(k)); };
 
+    // cu_seqlens is searched once per tile by the scalar warps; a copy in shared memory (when its S_max + 1 entries
+    // fit) turns the three or four dependent round trips of a search into a fraction of a microsecond
+    int32_t* cu_copy = reinterpret_cast<int32_t*>(ring_raw + (size_t)kStages * kStageBytes);
+    const bool cu_cached = a.S_max >= 1 && a.S_max + 1 <= kCuCache;
+    if (cu_cached)
+        for (int i = tid; i <= a.S_max; i += kThreads) cu_copy[i] = a.cu_seqlens[i];
+    const int32_t* cu = cu_cached ? cu_copy : a.cu_seqlens;
     if (tid == 0) {
         sh.abort = 0;
         for (int s = 0; s < kStages; ++s) {
@@ -166,6 +181,21 @@ grpo_loss_tile_kernel(const LossArgs a) {
         }
     } else if (warp < kConsumerWarps) {
         // ------------------------------------------------------------------ consumers
+        // this warp's units of a tile, the same in every tile: unit u = warp + 16 i is part u % P of row u / P
+        constexpr int kUnitsPerWarp = kMaxUnits / kConsumerWarps;
+        int u_row[kUnitsPerWarp], u_nv[kUnitsPerWarp], u_e0[kUnitsPerWarp];
+        uint32_t u_vec[kUnitsPerWarp];                                     // 16-byte offset of the unit inside a stage
+        long long u_dst[kUnitsPerWarp];                                    // byte offset of the unit from its tile's first row
+#pragma unroll
+        for (int i = 0; i < kUnitsPerWarp; ++i) {
+            const int u = warp + i * kConsumerWarps;
+            const int row = u / P, part = u - row * P;
+            u_row[i] = row;
+            u_nv[i] = min(geo.part_vecs, geo.nvec - part * geo.part_vecs);
+            u_e0[i] = (part * geo.part_vecs) << kLog2PerVec;
+            u_vec[i] = (uint32_t)row * (uint32_t)(a.row_bytes >> 4) + (uint32_t)(part * geo.part_vecs);
+            u_dst[i] = (long long)row * a.row_bytes + (long long)part * geo.part_vecs * 16;
+        }
         for (int k = 0; k < n_tiles + kSkew && !*abort_flag; ++k) {
             if (k < n_tiles) {
                 // ---- pass 1 of tile k: this warp's units
@@ -173,10 +203,12 @@ grpo_loss_tile_kernel(const LossArgs a) {
                 if (!__all_sync(0xffffffffu, wait(smem_u32(&sh.full[s]), ((uint32_t)k / kStages) & 1, abort_flag, a.wait_limit_ns))) break;
                 uint4* stage = reinterpret_cast<uint4*>(ring_raw + (size_t)s * kStageBytes);
                 const int units = tile_rows(k) * P;
-                for (int u = warp; u < units; u += kConsumerWarps) {
-                    const int row = u / P, part = u - row * P;
-                    uint4* src = stage + (size_t)row * (size_t)(a.row_bytes >> 4) + part * geo.part_vecs;
-                    const int nv = min(geo.part_vecs, geo.nvec - part * geo.part_vecs);
+#pragma unroll
+                for (int ui = 0; ui < kUnitsPerWarp; ++ui) {
+                    const int u = warp + ui * kConsumerWarps;
+                    if (u >= units) break;
+                    uint4* src = stage + u_vec[ui];
+                    const int nv = u_nv[ui];
                     uint4 d[kVPL];
 #pragma unroll
                     for (int j = 0; j < kVPL; ++j) {
@@ -233,12 +265,15 @@ grpo_loss_tile_kernel(const LossArgs a) {
                 const uint4* stage = reinterpret_cast<const uint4*>(ring_raw + (size_t)s * kStageBytes);
                 const int units = tile_rows(kk) * P;
                 const long long t0 = tile_row0(kk);
-                for (int u = warp; u < units; u += kConsumerWarps) {
-                    const int row = u / P, part = u - row * P;
-                    const uint4* src = stage + (size_t)row * (size_t)(a.row_bytes >> 4) + part * geo.part_vecs;
+#pragma unroll
+                for (int ui = 0; ui < kUnitsPerWarp; ++ui) {
+                    const int u = warp + ui * kConsumerWarps;
+                    if (u >= units) break;
+                    const int row = u_row[ui];
+                    const uint4* src = stage + u_vec[ui];
                     char* drow = a.dlogits + (t0 + row) * a.row_bytes;
-                    uint4* dst = reinterpret_cast<uint4*>(drow) + part * geo.part_vecs;
-                    const int nv = min(geo.part_vecs, geo.nvec - part * geo.part_vecs);
+                    uint4* dst = reinterpret_cast<uint4*>(a.dlogits + t0 * a.row_bytes + u_dst[ui]);
+                    const int nv = u_nv[ui];
                     const float sc = sh.meta[s].sc[u];
                     const f32x2 sc2 = pair_of(sc, sc);
 #pragma unroll
@@ -258,7 +293,7 @@ grpo_loss_tile_kernel(const LossArgs a) {
                     }
                     // the one element of the row that also carries the onehot term, if it lies in this unit
                     const int y = sh.meta[s].fix_y[row];
-                    const int e0 = (part * geo.part_vecs) << kLog2PerVec;
+                    const int e0 = u_e0[ui];
                     __syncwarp();                                           // after the lanes' stores of the unit
                     if (lane == 0 && y >= e0 && y < e0 + (nv << kLog2PerVec)) Elems<!kF32>::store1(drow, y, sh.meta[s].fix_val[row]);
                 }
@@ -287,7 +322,7 @@ grpo_loss_tile_kernel(const LossArgs a) {
             nxt.y = -1; nxt.lp_old = 0.0f; nxt.lp_ref = 0.0f;
             if (nxt.mine) { nxt.y = a.target[nxt.t]; nxt.lp_old = a.logp_old[nxt.t]; nxt.lp_ref = a.logp_ref[nxt.t]; }
         };
-        // second half: the rows' sequences (the whole warp searches cu_seqlens, 32 probes per round trip, once per
+        // second half: the rows' sequences (the whole warp searches cu_seqlens, 32 probes per step, once per
         // sequence that the tile touches) and the sampled tokens' logits, from global memory: the stage's copy of
         // the row is overwritten by pass 1
         auto gather_rest = [&](int k) {
@@ -300,12 +335,12 @@ grpo_loss_tile_kernel(const LossArgs a) {
                 while (hi - lo > 1) {
                     const int step = (hi - lo + 31) >> 5;
                     const long long idx = (long long)lo + (long long)(lane + 1) * step;
-                    const bool le = idx < hi && (long long)a.cu_seqlens[idx] <= at;
+                    const bool le = idx < hi && (long long)cu[idx] <= at;
                     const int n = __popc(__ballot_sync(0xffffffffu, le));
                     lo += n * step;
                     hi = min(hi, lo + step);
                 }
-                const long long s_lo = a.cu_seqlens[lo], s_hi = a.cu_seqlens[lo + 1];
+                const long long s_lo = cu[lo], s_hi = cu[lo + 1];
                 const bool ok = at >= s_lo && at < s_hi;
                 const long long upto = ok ? min(s_hi, t_end) : at + 1;      // rows [at, upto) are settled by this lookup
                 if (ok && nxt.t >= at && nxt.t < upto) { nxt.seg_ok = true; my_seg = lo; my_len = (int)(s_hi - s_lo); }
@@ -415,10 +450,14 @@ static int launch_tile_t(const LossArgs& a, cudaStream_t s, bool launch) {
         if (dev >= 0) raised[dev] = true;
     }
     if (!launch) return DPPO_OK;
+    // rows per tile: as many as a stage and the 32 units allow; a batch that would leave SMs without a tile takes
+    // smaller tiles instead
     const Geometry geo = geometry<kVPL>(a.V, kF32 ? 2 : 3, a.row_bytes);
-    const long long tiles = (a.T_max + geo.rows - 1) / geo.rows;
+    const long long per_sm = (a.T_max + sm_count() - 1) / sm_count();
+    const int rows = (int)(per_sm < geo.rows ? (per_sm > 1 ? per_sm : 1) : geo.rows);
+    const long long tiles = (a.T_max + rows - 1) / rows;
     const long long grid = tiles < sm_count() ? tiles : sm_count();
-    kernel<<<(unsigned)(grid > 0 ? grid : 1), kThreads, kDynSmem, s>>>(a);
+    kernel<<<(unsigned)(grid > 0 ? grid : 1), kThreads, kDynSmem, s>>>(a, rows);
     DPPO_CHECK_LAUNCH("grpo_loss tile launch");
     return DPPO_OK;
 }

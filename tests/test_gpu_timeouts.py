@@ -34,7 +34,7 @@ def _loss_call(B, prm, tok, cu, adv, wseq, T, stride, tdt):
     ("bf16", 151936, 80128),      # eight CTAs
     ("bf16", 151936 - 5, 20512),  # two CTAs, ragged tail
     ("f32", 151936, 0),           # eight CTAs, f32 rows
-    ("bf16", 16384, 0),           # one CTA per row: the exchange with itself
+    ("bf16", 16384, 10256),       # one CTA per row: the exchange with itself
     ("f32", 12, 40128),           # most slices empty
 ])
 def test_loss_sweep_waits_run_out(dtype, V, variant):
@@ -113,9 +113,43 @@ def test_streaming_forward_kernel_waits_run_out(dtype):
         assert torch.equal(a.view(torch.int32), b.view(torch.int32))
 
 
-def test_wait_self_test_needs_the_shared_memory_kernel():
+@pytest.mark.parametrize("dtype,V,T", [("bf16", 1024, 5000), ("f32", 2048, 2000), ("bf16", 64, 40000)])
+def test_tile_kernel_waits_run_out(dtype, V, T):
+    """The tile kernel: the first tile of every CTA is announced with 8 bytes more than its copy brings, so the
+    consumers' first wait runs out after 1 ms; every CTA reports the time-out, lets its copies land and leaves all
+    of its rows as rows that add nothing (dlogits of zeros)."""
     from paper_2603_04135_b200 import binding as B
-    prm = B.LossParams(8, 512, B.BF16, 512, 1, B.LOSS_WAIT_SELF_TEST, 0.2, 0.2, 0.04, 1.0)   # warp-per-row shape
+    S = 5
+    w = synth.scaled(synth.WORKLOADS["config3"], V=V, dtype=dtype)
+    tok = synth.make_token_inputs(w, T, 13, device="cuda")
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    cu = torch.from_numpy(np.linspace(0, T, S + 1).astype(np.int32)).cuda()
+    rng = np.random.default_rng(13)
+    adv = torch.from_numpy(rng.normal(size=S).astype(np.float32)).cuda()
+    wseq = torch.from_numpy((rng.random(S) * 0.1).astype(np.float32)).cuda()
+
+    def params(v):
+        return B.LossParams(T, V, B.BF16 if dtype == "bf16" else B.F32, V, S, v, 0.2, 0.2, 0.04, 1.0)
+
+    assert B.grpo_loss_kernel_choice(params(0)).kernel == B.KERNEL_TILE
+    before = _loss_call(B, params(0), tok, cu, adv, wseq, T, V, tdt)
+    assert before[4] == 0 and float(before[1][4]) == T
+    dl, loss_out, logp_out, lse_out, status = _loss_call(B, params(B.LOSS_WAIT_SELF_TEST), tok, cu, adv, wseq, T, V, tdt)
+    assert status == B.STATUS_TIMEOUT
+    assert bool((dl == 0).all())
+    assert bool((logp_out == 0).all()) and bool((lse_out == 0).all())
+    lo = loss_out.cpu().numpy()
+    assert np.isfinite(lo).all() and (lo[:4] == 0).all() and lo[4] == T
+    after = _loss_call(B, params(0), tok, cu, adv, wseq, T, V, tdt)
+    assert after[4] == 0
+    for a, b in zip(before[:4], after[:4]):
+        assert torch.equal(a.view(torch.int16) if a.dtype == torch.bfloat16 else a.view(torch.int32),
+                           b.view(torch.int16) if b.dtype == torch.bfloat16 else b.view(torch.int32))
+
+
+def test_wait_self_test_needs_a_kernel_that_waits():
+    from paper_2603_04135_b200 import binding as B
+    prm = B.LossParams(8, 508, B.BF16, 512, 1, B.LOSS_WAIT_SELF_TEST, 0.2, 0.2, 0.04, 1.0)   # warp-per-row shape
     with pytest.raises(B.DppoError) as e:
         B.grpo_loss_kernel_choice(prm)
     assert e.value.code == B.ERR_UNSUPPORTED
