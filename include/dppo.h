@@ -214,7 +214,7 @@ typedef struct {
     int32_t S_max;          /* cu_seqlens has S_max+1 entries, non-decreasing, last >= true T        */
     int32_t variant;        /* 0: the library picks the kernel.  Tuning aid: 1 forces the general two-pass
                                kernel, 2 the warp-per-row kernel (rows up to 8 KB), 3 the streaming kernel (forward-only
-                               calls), 4 the tile kernel (calls with dlogits; dense rows of up to 32 KB),
+                               calls), 4 the tile kernel (dense rows of up to 32 KB),
                                C*10000+threads the shared-memory kernel with C = 1, 2, 4 or 8
                                CTAs per row and 128 / 256 / 512 / 1024 threads per CTA.
                                Self-test of the bounded waits: 1000000 + (0, 3, 4 or a C*10000+threads code) runs
@@ -261,8 +261,8 @@ int dppo_grpo_loss_fwd_bwd(const dppo_loss_params* p, const void* logits, const 
                            int32_t* status, void* stream);
 
 /* Which kernel a dppo_grpo_loss_fwd_bwd call with these parameters runs on the current device (a host-side query:
- * it makes the same choice and the same device checks as the call and launches nothing).  With dlogits, dense rows
- * (V a whole number of 16-byte vectors) of up to 16 KB, and of exactly 32 KB, go to the tile kernel.  Other rows of
+ * it makes the same choice and the same device checks as the call and launches nothing).  Dense rows (V a whole
+ * number of 16-byte vectors) of up to 16 KB, and with dlogits of exactly 32 KB, go to the tile kernel.  Other rows of
  * up to 8 KB go to the warp-per-row kernel, rows that fit eight shared-memory slices to the shared-memory
  * kernel, longer ones to the general two-pass kernel; a forward-only call (forward_only != 0: the call will pass
  * dlogits = NULL) on rows of 128 KB and more goes to the streaming kernel.  fell_back = 1 says that the device refused the kernel the

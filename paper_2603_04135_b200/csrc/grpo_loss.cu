@@ -238,23 +238,25 @@ LossArgs loss_args_from_params(const dppo_loss_params* p) {
 
 // Picks the row kernel for `variant` and launches it (launch = true) or only runs the checks a launch would make.
 // variant: 0 picks the kernel from the shape; 1 forces the general kernel; 2 the warp-per-row kernel; 3 the
-// streaming kernel (forward-only calls); 4 the tile kernel (calls with dlogits); C*10000 + threads forces the shared-memory kernel with C CTAs per row (a tuning aid; unsupported shapes are an
+// streaming kernel (forward-only calls); 4 the tile kernel; C*10000 + threads forces the shared-memory kernel with C CTAs per row (a tuning aid; unsupported shapes are an
 // error); kSelfTestVariant + one of those runs the self-test of the bounded waits (shared-memory, streaming and tile kernels).
 // choice (nullable) receives what was taken; fell_back = 1 when the device refused the kernel the shape asked for
 // and the general kernel took over.
 constexpr int kSelfTestVariant = 1000000;
 
-// Rows the tile kernel is chosen for when dlogits are asked for: dense rows (no ragged tail of less than a vector,
-// 16-byte aligned) of up to 16 KB, and rows that fill one of its 32 KB stages exactly.  Measured against the
+// Rows the tile kernel is chosen for: dense rows (no ragged tail of less than a vector, 16-byte aligned) of up to
+// 16 KB and, with dlogits, rows that fill one of its 32 KB stages exactly.  With dlogits, measured against the
 // warp-per-row kernel (rows up to 8 KB) it is 1.2 to 2.8 times as fast (bf16 V = 1024: 5.6 against 3.5 TB/s; rows
 // of 128 B: 0.75 against 0.27), against one CTA per row of the shared-memory kernel 1.1 to 1.5 times (bf16 rows
 // of 9 to 16 KB: 4.7-5.7 against 3.4-4.9 TB/s).  Rows of 16 to 32 KB leave a stage partly empty (one row per tile)
-// and stay with the shared-memory kernel (20 KB: 4.0 against 5.4), except at 32 KB (5.7 against 5.4).
+// and stay with the shared-memory kernel (20 KB: 4.0 against 5.4), except at 32 KB (5.7 against 5.4).  Forward
+// only: 4.0-4.1 TB/s on bf16 rows of 2 to 16 KB against 2.1-3.3, 4.4-4.8 on f32 rows against 2.2-4.6; at 32 KB
+// the shared-memory kernel is ahead (4.3 against 3.6).
 static bool tile_kernel_takes(const LossArgs& a) {
     const int per_vec = a.bf16 ? 8 : 4;
     if (a.V < per_vec || a.V % per_vec != 0 || a.row_bytes % 16 != 0) return false;
     if ((((uintptr_t)a.logits) | ((uintptr_t)a.dlogits)) & 15) return false;
-    return a.row_bytes <= 16384 || a.row_bytes == 32768;
+    return a.row_bytes <= 16384 || (a.dlogits != nullptr && a.row_bytes == 32768);
 }
 
 int run_rows(LossArgs a, int variant, cudaStream_t s, bool launch, dppo_loss_kernel_choice* choice) {
@@ -291,7 +293,7 @@ int run_rows(LossArgs a, int variant, cudaStream_t s, bool launch, dppo_loss_ker
             ch.kernel = DPPO_KERNEL_STREAM; ch.threads = 512;
             rc = launch_rows_stream(a, s, launch);
             refused = rc == DPPO_ERR_UNSUPPORTED;
-        } else if (a.dlogits != nullptr && tile_kernel_takes(a)) {
+        } else if (tile_kernel_takes(a)) {
             ch.kernel = DPPO_KERNEL_TILE; ch.threads = 512;
             rc = launch_rows_tile(a, s, launch);
             refused = rc == DPPO_ERR_UNSUPPORTED;

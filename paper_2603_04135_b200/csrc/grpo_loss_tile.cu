@@ -1,4 +1,4 @@
-// Loss sweep with dlogits for rows of up to 32 KB: tiles of consecutive rows go through a shared-memory ring, and
+// Loss sweep for rows of up to 32 KB: tiles of consecutive rows go through a shared-memory ring, and
 // the three kinds of work a row needs are done by three kinds of warps that never wait for memory.
 //
 // A short row is dominated by what does not scale with its length: two warp reductions and, above all, the
@@ -16,10 +16,14 @@
 //                   one pass, and leaves every unit's factor g/tau 2^(r - lse2) (and the one element per row that
 //                   also carries the onehot term) for pass 2.  The rows' per-token inputs and sequences are gathered
 //                   a tile ahead
+// A forward-only call (no dlogits) runs pass 1 without the write-back and the scalar stage; a stage is free as soon
+// as pass 1 has read it.
 // HBM sees one read and one write per element.  Every wait is bounded; on a time-out the CTA raises an abort flag,
 // reports DPPO_STATUS_TIMEOUT, lets its copies in flight land (bounded) and leaves all of its rows as rows that add
 // nothing.
 #include <cuda_fp16.h>
+
+#include <type_traits>
 
 #include "common.cuh"
 #include "grpo_loss.cuh"
@@ -127,6 +131,7 @@ grpo_loss_tile_kernel(const LossArgs a, const int rows_per_tile) {
     const Geometry geo = geometry<kVPL>(a.V, kLog2PerVec, a.row_bytes);
     const int R = rows_per_tile, P = geo.parts;               // R <= geo.rows: fewer for a batch of less than a full tile per SM
     const float c = a.scale2;
+    const bool backward = a.dlogits != nullptr;           // else forward only: pass 1 and the scalar stage
     // this CTA's tiles: tile k covers rows (blockIdx.x + k gridDim.x) R ... of the batch
     const long long total_tiles = (T + R - 1) / R;
     const int n_tiles = (long long)blockIdx.x < total_tiles ? (int)((total_tiles - 1 - blockIdx.x) / gridDim.x) + 1 : 0;
@@ -196,11 +201,15 @@ grpo_loss_tile_kernel(const LossArgs a, const int rows_per_tile) {
             u_vec[i] = (uint32_t)row * (uint32_t)(a.row_bytes >> 4) + (uint32_t)(part * geo.part_vecs);
             u_dst[i] = (long long)row * a.row_bytes + (long long)part * geo.part_vecs * 16;
         }
-        for (int k = 0; k < n_tiles + kSkew && !*abort_flag; ++k) {
+        for (int k = 0; k < n_tiles + (backward ? kSkew : 0) && !*abort_flag; ++k) {
             if (k < n_tiles) {
                 // ---- pass 1 of tile k: this warp's units
-                const uint32_t s = (uint32_t)k % kStages;
-                if (!__all_sync(0xffffffffu, wait(smem_u32(&sh.full[s]), ((uint32_t)k / kStages) & 1, abort_flag, a.wait_limit_ns))) break;
+                const uint32_t s = (uint32_t)k % kStages, use = (uint32_t)k / kStages;
+                if (!__all_sync(0xffffffffu, wait(smem_u32(&sh.full[s]), use & 1, abort_flag, a.wait_limit_ns))) break;
+                // forward only: there is no pass 2 whose wait would tell that the scalar warp has read this stage's
+                // (r, sum) of the previous round
+                if (!backward && use > 0 &&
+                    !__all_sync(0xffffffffu, wait(smem_u32(&sh.s_done[s]), (use - 1) & 1, abort_flag, a.wait_limit_ns))) break;
                 uint4* stage = reinterpret_cast<uint4*>(ring_raw + (size_t)s * kStageBytes);
                 const int units = tile_rows(k) * P;
 #pragma unroll
@@ -247,7 +256,7 @@ grpo_loss_tile_kernel(const LossArgs a, const int rows_per_tile) {
                             d[j].z = exp_pair(d[j].z, c2, nr2, acc0); d[j].w = exp_pair(d[j].w, c2, nr2, acc1);
                         }
                         const int i = lane + 32 * j;
-                        if (i < nv) src[i] = d[j];
+                        if (backward && i < nv) src[i] = d[j];
                     }
                     float s0, s1;
                     unpair(add2(acc0, acc1), s0, s1);
@@ -255,9 +264,12 @@ grpo_loss_tile_kernel(const LossArgs a, const int rows_per_tile) {
                     if (lane == 0) sh.meta[s].rs[u] = make_float2(r, sum);
                 }
                 __syncwarp();
-                if (lane == 0) arrive(smem_u32(&sh.p1_done[s]));            // release: the scalar warp's wait acquires
+                if (lane == 0) {
+                    arrive(smem_u32(&sh.p1_done[s]));                       // release: the scalar warp's wait acquires
+                    if (!backward) arrive(smem_u32(&sh.free_[s]));          // forward only: the stage has been read, that is all
+                }
             }
-            if (k >= kSkew) {
+            if (backward && k >= kSkew) {
                 // ---- pass 2 of tile k - kSkew
                 const int kk = k - kSkew;
                 const uint32_t s = (uint32_t)kk % kStages;
@@ -306,29 +318,28 @@ grpo_loss_tile_kernel(const LossArgs a, const int rows_per_tile) {
     } else {
         // ------------------------------------------------------------------ scalar warps: lane q <-> row q of a tile
         const int first = warp - kConsumerWarps;
-        // what the scalar stage needs besides (r, sum), gathered one tile ahead ("next"), used as "cur"
+        // What the scalar stage needs besides (r, sum), gathered one tile ahead ("next", used as "cur") in two halves, so
+        // that no load is waited for where it is issued: values stay as loaded (conversions wait for the load) and
+        // the loads that depend on loaded values (the sampled logit on the token id, advantage and weight on the mapped
+        // sequence index) go out a scalar stage after those.
         struct Gathered {
             long long t;
             int y;                                                          // -1 for a lane without a row
-            float lp_old, lp_ref, zy_raw;
-            double A, W, lr;
+            int seg, idx, len;                                              // sequence position, mapped index, length
+            float lp_old, lp_ref, adv, w, lr;
+            typename std::conditional<kF32, float, __nv_bfloat16>::type zy;
             bool mine, seg_ok;
         };
         Gathered nxt, cur;
-        // first half: the per-token inputs (lane-indexed loads, consumed by the second half a scalar stage later)
-        auto gather_tokens = [&](int k) {
-            nxt.t = tile_row0(k) + lane;
-            nxt.mine = lane < tile_rows(k);
+        // first half: the per-token inputs (lane-indexed loads) and the rows' sequences: the whole warp searches the
+        // copy of cu_seqlens, 32 probes per step, once per sequence that the tile touches
+        auto gather_first = [&](int k) {
+            const long long t0 = tile_row0(k), t_end = t0 + tile_rows(k);
+            nxt.t = t0 + lane;
+            nxt.mine = nxt.t < t_end;
             nxt.y = -1; nxt.lp_old = 0.0f; nxt.lp_ref = 0.0f;
             if (nxt.mine) { nxt.y = a.target[nxt.t]; nxt.lp_old = a.logp_old[nxt.t]; nxt.lp_ref = a.logp_ref[nxt.t]; }
-        };
-        // second half: the rows' sequences (the whole warp searches cu_seqlens, 32 probes per step, once per
-        // sequence that the tile touches) and the sampled tokens' logits, from global memory: the stage's copy of
-        // the row is overwritten by pass 1
-        auto gather_rest = [&](int k) {
-            const long long t0 = tile_row0(k), t_end = t0 + tile_rows(k);
-            nxt.seg_ok = false;
-            int my_seg = 0, my_len = 1;
+            nxt.seg_ok = false; nxt.seg = 0; nxt.len = 1;
             long long at = t0;                                              // first row not yet looked up
             while (a.S_max >= 1 && at < t_end) {
                 int lo = 0, hi = a.S_max;
@@ -343,26 +354,32 @@ grpo_loss_tile_kernel(const LossArgs a, const int rows_per_tile) {
                 const long long s_lo = cu[lo], s_hi = cu[lo + 1];
                 const bool ok = at >= s_lo && at < s_hi;
                 const long long upto = ok ? min(s_hi, t_end) : at + 1;      // rows [at, upto) are settled by this lookup
-                if (ok && nxt.t >= at && nxt.t < upto) { nxt.seg_ok = true; my_seg = lo; my_len = (int)(s_hi - s_lo); }
+                if (ok && nxt.t >= at && nxt.t < upto) { nxt.seg_ok = true; nxt.seg = lo; nxt.len = (int)(s_hi - s_lo); }
                 at = upto;
             }
-            nxt.A = nxt.W = nxt.lr = 0.0;
-            if (nxt.mine && nxt.seg_ok) {
-                const int idx = a.seg_map ? a.seg_map[my_seg] : my_seg;
-                nxt.A = (double)a.adv[idx];
-                nxt.W = a.no_length_norm ? (double)a.w[idx] : (double)a.w[idx] / (double)my_len;
-                if (a.seq_log_ratio) nxt.lr = (double)a.seq_log_ratio[my_seg];
-            }
-            nxt.zy_raw = 0.0f;
-            if (nxt.mine && nxt.y >= 0 && nxt.y < a.V) nxt.zy_raw = Elems<!kF32>::load1(a.logits + nxt.t * a.row_bytes, nxt.y);
+            nxt.idx = nxt.seg;
+            if (nxt.mine && nxt.seg_ok && a.seg_map) nxt.idx = a.seg_map[nxt.seg];
         };
-        if (first < n_tiles) { gather_tokens(first); gather_rest(first); }
+        // second half: what needs the first half's loads.  The sampled token's logit comes from global memory: the
+        // stage's copy of the row is overwritten by pass 1
+        auto gather_second = [&]() {
+            nxt.adv = nxt.w = nxt.lr = 0.0f;
+            if (nxt.mine && nxt.seg_ok) {
+                nxt.adv = a.adv[nxt.idx];
+                nxt.w = a.w[nxt.idx];
+                if (a.seq_log_ratio) nxt.lr = a.seq_log_ratio[nxt.seg];
+            }
+            nxt.zy = 0.0f;
+            if (nxt.mine && nxt.y >= 0 && nxt.y < a.V)
+                nxt.zy = reinterpret_cast<const decltype(nxt.zy)*>(a.logits + nxt.t * a.row_bytes)[nxt.y];
+        };
+        if (first < n_tiles) { gather_first(first); gather_second(); }
         for (int k = first; k < n_tiles && !*abort_flag; k += kScalarWarps) {
             const uint32_t s = (uint32_t)k % kStages;
             if (!__all_sync(0xffffffffu, wait(smem_u32(&sh.p1_done[s]), ((uint32_t)k / kStages) & 1, abort_flag, a.wait_limit_ns))) break;
             cur = nxt;
             const bool more = k + kScalarWarps < n_tiles;
-            if (more) gather_tokens(k + kScalarWarps);                     // in flight during this tile's scalar stage
+            if (more) gather_first(k + kScalarWarps);                      // in flight during this tile's scalar stage
             Meta& meta = sh.meta[s];
             if (cur.mine) {
                 const int u0 = lane * P;
@@ -375,15 +392,17 @@ grpo_loss_tile_kernel(const LossArgs a, const int rows_per_tile) {
                     r = hi; sum = x + y;
                 }
                 const bool y_ok = cur.y >= 0 && cur.y < a.V;
+                const float zy_raw = (float)cur.zy;
                 RowInputs in;
                 in.A = in.W = in.zy = in.logp_old = in.logp_ref = in.seq_lr = 0.0;
                 in.use_seq = 0; in.y = cur.y; in.state = 0;
                 if (!cur.seg_ok) in.state = DPPO_STATUS_BAD_SEGMENTS;
                 else if (!y_ok) in.state = DPPO_STATUS_BAD_TARGET;
                 else {
-                    in.A = cur.A; in.W = cur.W;
-                    if (a.seq_log_ratio) { in.use_seq = 1; in.seq_lr = cur.lr; }
-                    in.zy = (double)cur.zy_raw / a.temperature;
+                    in.A = (double)cur.adv;
+                    in.W = a.no_length_norm ? (double)cur.w : (double)cur.w / (double)cur.len;
+                    if (a.seq_log_ratio) { in.use_seq = 1; in.seq_lr = (double)cur.lr; }
+                    in.zy = (double)zy_raw / a.temperature;
                     in.logp_old = (double)cur.lp_old; in.logp_ref = (double)cur.lp_ref;
                 }
                 const RowScalars rs = row_finish(a, cur.t, in, r, sum, true);
@@ -401,7 +420,7 @@ grpo_loss_tile_kernel(const LossArgs a, const int rows_per_tile) {
                     const int py = (cur.y >> kLog2PerVec) / geo.part_vecs;
                     const float rp = meta.rs[u0 + py].x;
                     const float nr = rp > -INFINITY ? -rp : 0.0f;
-                    float e = cur.zy_raw > -INFINITY ? ex2(fmaf(cur.zy_raw, c, nr)) : 0.0f;
+                    float e = zy_raw > -INFINITY ? ex2(fmaf(zy_raw, c, nr)) : 0.0f;
                     if (!kF32) e = __half2float(__float2half_rn(e));
                     fix_y = cur.y;
                     fix_val = fmaf(e, meta.sc[u0 + py], -ng);
@@ -411,7 +430,7 @@ grpo_loss_tile_kernel(const LossArgs a, const int rows_per_tile) {
             }
             __syncwarp();
             if (lane == 0) arrive(smem_u32(&sh.s_done[s]));                 // release: the consumers' waits acquire
-            if (more) gather_rest(k + kScalarWarps);
+            if (more) gather_second();
         }
     }
 
@@ -429,7 +448,7 @@ grpo_loss_tile_kernel(const LossArgs a, const int rows_per_tile) {
                 if (a.logp_out) a.logp_out[t0 + q] = 0.0f;
                 if (a.lse_out) a.lse_out[t0 + q] = 0.0f;
             }
-            for (int i = tid; i < rows * geo.nvec; i += kThreads) {
+            for (int i = tid; backward && i < rows * geo.nvec; i += kThreads) {
                 const int q = i / geo.nvec, v = i - q * geo.nvec;
                 reinterpret_cast<uint4*>(a.dlogits + (t0 + q) * a.row_bytes)[v] = make_uint4(0u, 0u, 0u, 0u);
             }
@@ -469,15 +488,14 @@ static int launch_tile_dtype(const LossArgs& a, int nvec, cudaStream_t s, bool l
     return launch_tile_t<kF32, 4>(a, s, launch);
 }
 
-// Calls with dlogits on dense rows: V a whole number of 16-byte vectors, the row pitch a multiple of 16 bytes and at
+// Dense rows, with dlogits or forward only: V a whole number of 16-byte vectors, the row pitch a multiple of 16 bytes and at
 // most 32 KB, both matrices 16-byte aligned.  DPPO_ERR_UNSUPPORTED (nothing launched) otherwise.
 int launch_rows_tile(const LossArgs& a, cudaStream_t s, bool launch) {
     const int per_vec = a.bf16 ? 8 : 4;
-    if (!a.dlogits) return fail(DPPO_ERR_UNSUPPORTED, "tile kernel: calls with dlogits");
     if (a.V < per_vec || a.V % per_vec != 0) return fail(DPPO_ERR_UNSUPPORTED, "tile kernel: V=%d is not a whole number of 16-byte vectors", a.V);
     if (a.row_bytes % 16 != 0 || a.row_bytes > kStageBytes || a.row_bytes < (long long)a.V * (a.bf16 ? 2 : 4))
         return fail(DPPO_ERR_UNSUPPORTED, "tile kernel: row pitch of %lld bytes", a.row_bytes);
-    if ((((uintptr_t)a.logits) | ((uintptr_t)a.dlogits)) & 15) return fail(DPPO_ERR_UNSUPPORTED, "tile kernel: matrices not 16-byte aligned");
+    if ((((uintptr_t)a.logits) | ((uintptr_t)a.dlogits)) & 15) return fail(DPPO_ERR_UNSUPPORTED, "tile kernel: matrices not 16-byte aligned");   // dlogits may be null
     const int nvec = a.V / per_vec;
     return a.bf16 ? launch_tile_dtype<false>(a, nvec, s, launch) : launch_tile_dtype<true>(a, nvec, s, launch);
 }

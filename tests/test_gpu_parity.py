@@ -418,8 +418,13 @@ def test_loss_tile_kernel(dtype):
     _loss_case(512 * per, dtype, T=50, S=2, seed=626, variant=v, neg_inf_cols=(0, 300 * per))
     _loss_case(128 * per, dtype, T=40, S=3, seed=627, variant=v, logit_sigma=40.0, centre_on_oracle=True)
     from paper_2603_04135_b200 import binding as B
-    for bad in (dict(V=1004 if dtype == "bf16" else 1002, T=8), dict(V=4096 * per, T=8), dict(V=1024, T=8, forward_only=True)):
-        with pytest.raises(B.DppoError) as e:                                    # ragged tail, a row above 32 KB, no dlogits
+    # forward only: pass 1 and the scalar stage; stages reused many times, the sequence-level ratio's two sweeps
+    _loss_case(128 * per, dtype, T=40000, S=300, seed=640, variant=v, forward_only=True, centre_on_oracle=True)
+    _loss_case(300 * per, dtype, T=67, S=5, seed=641, variant=v, forward_only=True)
+    _loss_case(16 * per, dtype, T=9000, S=50, seed=642, variant=v, forward_only=True, n_tokens=8000, tau=0.8)
+    _loss_case(255 * per, dtype, T=80, S=6, seed=643, variant=v, seq_ratio=True, sigma_noise=0.3)
+    for bad in (dict(V=1004 if dtype == "bf16" else 1002, T=8), dict(V=4096 * per, T=8)):
+        with pytest.raises(B.DppoError) as e:                                    # ragged tail, a row above 32 KB
             _loss_case(bad.pop("V"), dtype, S=2, seed=630, variant=v, **bad)
         assert e.value.code == B.ERR_UNSUPPORTED
 
@@ -539,10 +544,10 @@ def test_loss_kernel_choice_query():
         c = B.grpo_loss_kernel_choice(B.LossParams(64, V, dtype, stride, 4, variant, 0.2, 0.2, 0.04, 1.0))
         return (c.kernel, c.ctas_per_row, c.threads, c.fell_back)
 
-    assert choice(1024, B.BF16) == (B.KERNEL_TILE, 1, 512, 0)            # dense rows of up to 16 KB, with dlogits
+    assert choice(1024, B.BF16) == (B.KERNEL_TILE, 1, 512, 0)            # dense rows of up to 16 KB
     assert choice(2048, B.F32) == (B.KERNEL_TILE, 1, 512, 0)
     assert choice(8192, B.BF16) == (B.KERNEL_TILE, 1, 512, 0)
-    assert choice(16384, B.BF16) == (B.KERNEL_TILE, 1, 512, 0)           # 32 KB: fills a stage exactly
+    assert choice(16384, B.BF16) == (B.KERNEL_TILE, 1, 512, 0)           # 32 KB with dlogits: fills a stage exactly
     assert choice(1020, B.BF16) == (B.KERNEL_WARP, 1, 32, 0)             # a ragged tail of 4 elements
     assert choice(4092, B.BF16) == (B.KERNEL_WARP, 1, 32, 0)
     assert choice(8200, B.BF16) == (B.KERNEL_SHARED, 1, 128, 0)          # 16,400 B: one row would leave half a stage empty
@@ -550,7 +555,9 @@ def test_loss_kernel_choice_query():
     assert choice(16392, B.BF16) == (B.KERNEL_SHARED, 1, 256, 0)
     assert choice(32768, B.BF16) == (B.KERNEL_SHARED, 2, 256, 0)
     fwd_short = B.grpo_loss_kernel_choice(B.LossParams(64, 1024, B.BF16, 1024, 4, 0, 0.2, 0.2, 0.04, 1.0), forward_only=True)
-    assert (fwd_short.kernel, fwd_short.threads) == (B.KERNEL_WARP, 32)  # no dlogits: the warp-per-row kernel
+    assert fwd_short.kernel == B.KERNEL_TILE                             # forward only as well
+    fwd_32k = B.grpo_loss_kernel_choice(B.LossParams(64, 16384, B.BF16, 16384, 4, 0, 0.2, 0.2, 0.04, 1.0), forward_only=True)
+    assert fwd_32k.kernel == B.KERNEL_SHARED                             # but not at 32 KB
     assert choice(151936, B.BF16) == (B.KERNEL_SHARED, 4, 256, 0)        # the benchmark's rows
     assert choice(151936, B.F32) == (B.KERNEL_SHARED, 8, 256, 0)
     assert choice(400000, B.BF16) == (B.KERNEL_GENERAL, 1, 512, 0)       # too long for eight slices: not a fall-back
