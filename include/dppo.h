@@ -262,7 +262,7 @@ int dppo_grpo_loss_fwd_bwd(const dppo_loss_params* p, const void* logits, const 
 
 /* Which kernel a dppo_grpo_loss_fwd_bwd call with these parameters runs on the current device (a host-side query:
  * it makes the same choice and the same device checks as the call and launches nothing).  Dense rows (V a whole
- * number of 16-byte vectors) of up to 16 KB, and with dlogits of exactly 32 KB, go to the tile kernel.  Other rows of
+ * number of 16-byte vectors) of up to 16 KB go to the tile kernel.  Other rows of
  * up to 8 KB go to the warp-per-row kernel, rows that fit eight shared-memory slices to the shared-memory
  * kernel, longer ones to the general two-pass kernel; a forward-only call (forward_only != 0: the call will pass
  * dlogits = NULL) on rows of 128 KB and more goes to the streaming kernel.  fell_back = 1 says that the device refused the kernel the

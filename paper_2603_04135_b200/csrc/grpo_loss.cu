@@ -245,18 +245,16 @@ LossArgs loss_args_from_params(const dppo_loss_params* p) {
 constexpr int kSelfTestVariant = 1000000;
 
 // Rows the tile kernel is chosen for: dense rows (no ragged tail of less than a vector, 16-byte aligned) of up to
-// 16 KB and, with dlogits, rows that fill one of its 32 KB stages exactly.  With dlogits, measured against the
-// warp-per-row kernel (rows up to 8 KB) it is 1.2 to 2.8 times as fast (bf16 V = 1024: 5.6 against 3.5 TB/s; rows
-// of 128 B: 0.75 against 0.27), against one CTA per row of the shared-memory kernel 1.1 to 1.5 times (bf16 rows
-// of 9 to 16 KB: 4.7-5.7 against 3.4-4.9 TB/s).  Rows of 16 to 32 KB leave a stage partly empty (one row per tile)
-// and stay with the shared-memory kernel (20 KB: 4.0 against 5.4), except at 32 KB (5.7 against 5.4).  Forward
-// only: 4.0-4.1 TB/s on bf16 rows of 2 to 16 KB against 2.1-3.3, 4.4-4.8 on f32 rows against 2.2-4.6; at 32 KB
-// the shared-memory kernel is ahead (4.3 against 3.6).
+// 16 KB.  With dlogits, measured on the call a training step makes: bf16 rows of 2 to 16 KB 5.6-5.7 TB/s (the
+// warp-per-row kernel 3.5-4.5, one CTA per row of the shared-memory kernel 4.2-5.0), 1 KB rows 4.7 (2.2), f32 rows
+// of 2 to 16 KB 6.2-6.5 (3.8-5.2).  Rows of 16 to 32 KB leave a stage partly empty (one row per tile) and stay with
+// the shared-memory kernel (bf16 rows of 20 KB: 4.0 against 5.4; of 32 KB, which fill a stage: 5.7 against 6.2-6.4).
+// Forward only: 4.0-4.1 TB/s on bf16 rows of 2 to 16 KB against 2.1-3.3, 4.4-4.8 on f32 rows against 2.2-4.6.
 static bool tile_kernel_takes(const LossArgs& a) {
     const int per_vec = a.bf16 ? 8 : 4;
     if (a.V < per_vec || a.V % per_vec != 0 || a.row_bytes % 16 != 0) return false;
     if ((((uintptr_t)a.logits) | ((uintptr_t)a.dlogits)) & 15) return false;
-    return a.row_bytes <= 16384 || (a.dlogits != nullptr && a.row_bytes == 32768);
+    return a.row_bytes <= 16384;
 }
 
 int run_rows(LossArgs a, int variant, cudaStream_t s, bool launch, dppo_loss_kernel_choice* choice) {

@@ -70,10 +70,12 @@ template <int kVPL>
 __host__ __device__ inline Geometry geometry(int V, int log2_per_vec, long long row_bytes) {
     Geometry g;
     g.nvec = V >> log2_per_vec;
-    g.parts = (g.nvec + 32 * kVPL - 1) / (32 * kVPL);
-    if (g.parts < 1) g.parts = 1;
-    g.part_vecs = (g.nvec + g.parts - 1) / g.parts;       // equal parts (the last one may be a little shorter)
     const long long fit = kStageBytes / (row_bytes > 0 ? row_bytes : 1);
+    // parts per row: as few as keep a part within 32 kVPL vectors (more, smaller parts that would fill the 16 consumer
+    // warps more evenly measured slower: a unit's fixed cost, its two warp reductions, is what counts)
+    g.parts = g.nvec > 32 * kVPL ? (g.nvec + 32 * kVPL - 1) / (32 * kVPL) : 1;
+    g.part_vecs = (g.nvec + g.parts - 1) / g.parts;       // equal parts (the last one may be a little shorter)
+    if (g.part_vecs < 1) g.part_vecs = 1;
     const int by_units = kMaxUnits / g.parts;
     g.rows = (int)(fit < by_units ? fit : by_units);
     return g;

@@ -526,9 +526,9 @@ def test_loss_kernel_choice_boundaries(dtype):
     per_vec = 8 if dtype == "bf16" else 4
     warp_max = 512
     seed = 400
-    # (dense rows of up to 1024 vectors, and of 2048, take the tile kernel when dlogits are asked for: both sides of
-    # those limits too, and a ragged row next to each, which stays with the other kernels)
-    for nvec in (warp_max, 1024, 2048, 2816, 7040, 19456, 38912):
+    # (dense rows of up to 1024 vectors take the tile kernel: both sides of that limit too, and a ragged row next to
+    # each, which stays with the other kernels)
+    for nvec in (warp_max, 1024, 2816, 7040, 19456, 38912):
         for V in (nvec * per_vec, nvec * per_vec + per_vec, nvec * per_vec + 3):
             seed += 1
             _loss_case(V, dtype, T=5, S=2, seed=seed, variant=0)
@@ -547,7 +547,7 @@ def test_loss_kernel_choice_query():
     assert choice(1024, B.BF16) == (B.KERNEL_TILE, 1, 512, 0)            # dense rows of up to 16 KB
     assert choice(2048, B.F32) == (B.KERNEL_TILE, 1, 512, 0)
     assert choice(8192, B.BF16) == (B.KERNEL_TILE, 1, 512, 0)
-    assert choice(16384, B.BF16) == (B.KERNEL_TILE, 1, 512, 0)           # 32 KB with dlogits: fills a stage exactly
+    assert choice(16384, B.BF16) == (B.KERNEL_SHARED, 1, 256, 0)
     assert choice(1020, B.BF16) == (B.KERNEL_WARP, 1, 32, 0)             # a ragged tail of 4 elements
     assert choice(4092, B.BF16) == (B.KERNEL_WARP, 1, 32, 0)
     assert choice(8200, B.BF16) == (B.KERNEL_SHARED, 1, 128, 0)          # 16,400 B: one row would leave half a stage empty
@@ -556,8 +556,6 @@ def test_loss_kernel_choice_query():
     assert choice(32768, B.BF16) == (B.KERNEL_SHARED, 2, 256, 0)
     fwd_short = B.grpo_loss_kernel_choice(B.LossParams(64, 1024, B.BF16, 1024, 4, 0, 0.2, 0.2, 0.04, 1.0), forward_only=True)
     assert fwd_short.kernel == B.KERNEL_TILE                             # forward only as well
-    fwd_32k = B.grpo_loss_kernel_choice(B.LossParams(64, 16384, B.BF16, 16384, 4, 0, 0.2, 0.2, 0.04, 1.0), forward_only=True)
-    assert fwd_32k.kernel == B.KERNEL_SHARED                             # but not at 32 KB
     assert choice(151936, B.BF16) == (B.KERNEL_SHARED, 4, 256, 0)        # the benchmark's rows
     assert choice(151936, B.F32) == (B.KERNEL_SHARED, 8, 256, 0)
     assert choice(400000, B.BF16) == (B.KERNEL_GENERAL, 1, 512, 0)       # too long for eight slices: not a fall-back
