@@ -39,7 +39,9 @@ constexpr int kThreads = (kConsumerWarps + kScalarWarps + 1) * 32;       // + th
 constexpr int kStages = 6;
 constexpr int kStageBytes = 32768;
 constexpr int kMaxUnits = 32;                             // units of a tile (and rows: one lane of a scalar warp each)
-constexpr int kSkew = 3;                                  // pass 2 of tile k runs after pass 1 of tile k + kSkew
+constexpr int kGroups = 2;                                // the consumer warps work in groups on alternate tiles
+constexpr int kGroupWarps = kConsumerWarps / kGroups;
+constexpr int kGroupSkew = 1;                             // a group runs pass 2 of a tile after pass 1 of its kGroupSkew-th next tile
 constexpr int kCuCache = 6144;                            // entries of cu_seqlens kept in shared memory (24 KB)
 constexpr size_t kDynSmem = (size_t)kStages * kStageBytes + (size_t)kCuCache * 4;
 
@@ -52,9 +54,9 @@ struct Meta {                                             // of one stage
 
 struct Shared {
     unsigned long long full[kStages];                     // the tile's bytes have landed
-    unsigned long long p1_done[kStages];                  // all consumer warps have finished pass 1 of the tile
+    unsigned long long p1_done[kStages];                  // the tile's group of consumer warps has finished pass 1
     unsigned long long s_done[kStages];                   // the tile's scalar stage is done
-    unsigned long long free_[kStages];                    // all consumer warps have finished pass 2: the stage may be refilled
+    unsigned long long free_[kStages];                    // ... and pass 2: the stage may be refilled
     Meta meta[kStages];
     int abort;
 };
@@ -120,11 +122,125 @@ __device__ __forceinline__ void arrive(uint32_t bar) {
 
 using namespace tile;
 
+// Pass 1 on N units of one warp at once, so that their instruction streams interleave (the shuffle chains of one unit
+// run under the exponentials of the other): per unit the maximum, 2^(z c - r) for every element (kept in place as fp16
+// pairs or f32 when write_back), and (r, sum) of the unit.
+template <bool kF32, int kVPL, int N>
+__device__ __forceinline__ void pass1_units(uint4* const (&src)[N], const int (&nv)[N], int lane, float c, bool write_back,
+                                            float2 (&out)[N]) {
+    constexpr uint32_t kPad = kF32 ? 0xFF800000u : 0xFF80FF80u;   // -inf: adds nothing to the maximum or the sum
+    uint4 d[N][kVPL];
+#pragma unroll
+    for (int n = 0; n < N; ++n)
+#pragma unroll
+        for (int j = 0; j < kVPL; ++j) {
+            const int i = lane + 32 * j;
+            d[n][j] = i < nv[n] ? src[n][i] : make_uint4(kPad, kPad, kPad, kPad);
+        }
+    float m[N];
+#pragma unroll
+    for (int n = 0; n < N; ++n) {
+        if constexpr (kF32) {
+            m[n] = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < kVPL; ++j)
+                m[n] = fmaxf(m[n], fmaxf(fmaxf(__uint_as_float(d[n][j].x), __uint_as_float(d[n][j].y)),
+                                         fmaxf(__uint_as_float(d[n][j].z), __uint_as_float(d[n][j].w))));
+        } else {
+            __nv_bfloat162 mx2 = __float2bfloat162_rn(-INFINITY);
+#pragma unroll
+            for (int j = 0; j < kVPL; ++j) {
+                mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&d[n][j].x));
+                mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&d[n][j].y));
+                mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&d[n][j].z));
+                mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&d[n][j].w));
+            }
+            m[n] = fmaxf(__low2float(mx2), __high2float(mx2));
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+        for (int n = 0; n < N; ++n) m[n] = fmaxf(m[n], __shfl_xor_sync(0xffffffffu, m[n], o));
+    float sum[N];
+#pragma unroll
+    for (int n = 0; n < N; ++n) {
+        const float r = m[n] * c;                                  // -inf only if the whole unit is -inf
+        const float nr = r > -INFINITY ? -r : 0.0f;
+        const f32x2 c2 = pair_of(c, c), nr2 = pair_of(nr, nr);
+        f32x2 acc0 = pair_of(0.0f, 0.0f), acc1 = acc0;
+        if (write_back) {
+#pragma unroll
+            for (int j = 0; j < kVPL; ++j) {
+                if constexpr (kF32) {
+                    d[n][j] = exp_quad(d[n][j], c2, nr2, acc0, acc1);
+                } else {
+                    d[n][j].x = exp_pair(d[n][j].x, c2, nr2, acc0); d[n][j].y = exp_pair(d[n][j].y, c2, nr2, acc1);
+                    d[n][j].z = exp_pair(d[n][j].z, c2, nr2, acc0); d[n][j].w = exp_pair(d[n][j].w, c2, nr2, acc1);
+                }
+                const int i = lane + 32 * j;
+                if (i < nv[n]) src[n][i] = d[n][j];
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < kVPL; ++j) {
+                if constexpr (kF32) {
+                    exp_quad(d[n][j], c2, nr2, acc0, acc1);
+                } else {
+                    exp_pair_sum(d[n][j].x, c2, nr2, acc0); exp_pair_sum(d[n][j].y, c2, nr2, acc1);
+                    exp_pair_sum(d[n][j].z, c2, nr2, acc0); exp_pair_sum(d[n][j].w, c2, nr2, acc1);
+                }
+            }
+        }
+        float s0, s1;
+        unpair(add2(acc0, acc1), s0, s1);
+        sum[n] = s0 + s1;
+        out[n].x = r;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+        for (int n = 0; n < N; ++n) sum[n] += __shfl_xor_sync(0xffffffffu, sum[n], o);
+#pragma unroll
+    for (int n = 0; n < N; ++n) out[n].y = sum[n];
+}
+
+// Pass 2 on N units of one warp at once: the stored exponentials times the unit's factor, to dlogits.
+template <bool kF32, int kVPL, int N>
+__device__ __forceinline__ void pass2_units(const uint4* const (&src)[N], uint4* const (&dst)[N], const int (&nv)[N],
+                                            const float (&sc)[N], int lane) {
+    uint4 e[N][kVPL];
+#pragma unroll
+    for (int n = 0; n < N; ++n)
+#pragma unroll
+        for (int j = 0; j < kVPL; ++j) {
+            const int i = lane + 32 * j;
+            e[n][j] = i < nv[n] ? src[n][i] : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+    for (int n = 0; n < N; ++n) {
+        const f32x2 sc2 = pair_of(sc[n], sc[n]);
+#pragma unroll
+        for (int j = 0; j < kVPL; ++j) {
+            const int i = lane + 32 * j;
+            if (i < nv[n]) {
+                uint4 o;
+                if constexpr (kF32) {
+                    o = scale_quad(e[n][j], sc2);
+                } else {
+                    o.x = scale_pair(e[n][j].x, sc2); o.y = scale_pair(e[n][j].y, sc2);
+                    o.z = scale_pair(e[n][j].z, sc2); o.w = scale_pair(e[n][j].w, sc2);
+                }
+                __stcs(dst[n] + i, o);
+            }
+        }
+    }
+}
+
 template <bool kF32, int kVPL>
 __global__ void __launch_bounds__(kThreads, 1)
 grpo_loss_tile_kernel(const LossArgs a, const int rows_per_tile) {
     constexpr int kLog2PerVec = kF32 ? 2 : 3;               // elements per 16-byte vector: 4 f32 or 8 bf16
-    constexpr uint32_t kPad = kF32 ? 0xFF800000u : 0xFF80FF80u;   // -inf: adds nothing to the maximum or the sum
     extern __shared__ __align__(128) unsigned char ring_raw[];
     __shared__ Shared sh;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -151,9 +267,9 @@ grpo_loss_tile_kernel(const LossArgs a, const int rows_per_tile) {
         sh.abort = 0;
         for (int s = 0; s < kStages; ++s) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(&sh.full[s])));
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&sh.p1_done[s])), "r"(kConsumerWarps));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&sh.p1_done[s])), "r"(kGroupWarps));
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(&sh.s_done[s])));
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&sh.free_[s])), "r"(kConsumerWarps));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(&sh.free_[s])), "r"(kGroupWarps));
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -188,14 +304,18 @@ grpo_loss_tile_kernel(const LossArgs a, const int rows_per_tile) {
         }
     } else if (warp < kConsumerWarps) {
         // ------------------------------------------------------------------ consumers
-        // this warp's units of a tile, the same in every tile: unit u = warp + 16 i is part u % P of row u / P
-        constexpr int kUnitsPerWarp = kMaxUnits / kConsumerWarps;
+        // Two groups of eight warps take the tiles alternately (group g: tiles g, g + 2, ...), so that the groups are
+        // in different phases of their tiles (one in its exponentials while the other reduces, waits or stores) instead
+        // of all sixteen warps wanting the same pipe at the same time.  A warp works on its units two at a time.
+        // This warp's units of a tile, the same in every tile: unit u = wid + 8 i is part u % P of row u / P.
+        const int group = warp / kGroupWarps, wid = warp - group * kGroupWarps;
+        constexpr int kUnitsPerWarp = kMaxUnits / kGroupWarps;
         int u_row[kUnitsPerWarp], u_nv[kUnitsPerWarp], u_e0[kUnitsPerWarp];
         uint32_t u_vec[kUnitsPerWarp];                                     // 16-byte offset of the unit inside a stage
         long long u_dst[kUnitsPerWarp];                                    // byte offset of the unit from its tile's first row
 #pragma unroll
         for (int i = 0; i < kUnitsPerWarp; ++i) {
-            const int u = warp + i * kConsumerWarps;
+            const int u = wid + i * kGroupWarps;
             const int row = u / P, part = u - row * P;
             u_row[i] = row;
             u_nv[i] = min(geo.part_vecs, geo.nvec - part * geo.part_vecs);
@@ -203,9 +323,11 @@ grpo_loss_tile_kernel(const LossArgs a, const int rows_per_tile) {
             u_vec[i] = (uint32_t)row * (uint32_t)(a.row_bytes >> 4) + (uint32_t)(part * geo.part_vecs);
             u_dst[i] = (long long)row * a.row_bytes + (long long)part * geo.part_vecs * 16;
         }
-        for (int k = 0; k < n_tiles + (backward ? kSkew : 0) && !*abort_flag; ++k) {
+        for (int j = 0; !*abort_flag; ++j) {
+            const int k = group + kGroups * j;                              // pass 1 of tile k
+            const int kk = k - kGroups * kGroupSkew;                        // pass 2 of tile kk
+            if (k >= n_tiles && (!backward || kk >= n_tiles)) break;
             if (k < n_tiles) {
-                // ---- pass 1 of tile k: this warp's units
                 const uint32_t s = (uint32_t)k % kStages, use = (uint32_t)k / kStages;
                 if (!__all_sync(0xffffffffu, wait(smem_u32(&sh.full[s]), use & 1, abort_flag, a.wait_limit_ns))) break;
                 // forward only: there is no pass 2 whose wait would tell that the scalar warp has read this stage's
@@ -215,55 +337,21 @@ grpo_loss_tile_kernel(const LossArgs a, const int rows_per_tile) {
                 uint4* stage = reinterpret_cast<uint4*>(ring_raw + (size_t)s * kStageBytes);
                 const int units = tile_rows(k) * P;
 #pragma unroll
-                for (int ui = 0; ui < kUnitsPerWarp; ++ui) {
-                    const int u = warp + ui * kConsumerWarps;
-                    if (u >= units) break;
-                    uint4* src = stage + u_vec[ui];
-                    const int nv = u_nv[ui];
-                    uint4 d[kVPL];
-#pragma unroll
-                    for (int j = 0; j < kVPL; ++j) {
-                        const int i = lane + 32 * j;
-                        d[j] = i < nv ? src[i] : make_uint4(kPad, kPad, kPad, kPad);
+                for (int i = 0; i < kUnitsPerWarp; i += 2) {
+                    const int ua = wid + i * kGroupWarps, ub = ua + kGroupWarps;
+                    if (ub < units) {
+                        uint4* const src[2] = {stage + u_vec[i], stage + u_vec[i + 1]};
+                        const int nv[2] = {u_nv[i], u_nv[i + 1]};
+                        float2 rs[2];
+                        pass1_units<kF32, kVPL, 2>(src, nv, lane, c, backward, rs);
+                        if (lane == 0) { sh.meta[s].rs[ua] = rs[0]; sh.meta[s].rs[ub] = rs[1]; }
+                    } else if (ua < units) {
+                        uint4* const src[1] = {stage + u_vec[i]};
+                        const int nv[1] = {u_nv[i]};
+                        float2 rs[1];
+                        pass1_units<kF32, kVPL, 1>(src, nv, lane, c, backward, rs);
+                        if (lane == 0) sh.meta[s].rs[ua] = rs[0];
                     }
-                    float m;
-                    if constexpr (kF32) {
-                        m = -INFINITY;
-#pragma unroll
-                        for (int j = 0; j < kVPL; ++j)
-                            m = fmaxf(m, fmaxf(fmaxf(__uint_as_float(d[j].x), __uint_as_float(d[j].y)),
-                                               fmaxf(__uint_as_float(d[j].z), __uint_as_float(d[j].w))));
-                    } else {
-                        __nv_bfloat162 mx2 = __float2bfloat162_rn(-INFINITY);
-#pragma unroll
-                        for (int j = 0; j < kVPL; ++j) {
-                            mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&d[j].x));
-                            mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&d[j].y));
-                            mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&d[j].z));
-                            mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162*>(&d[j].w));
-                        }
-                        m = fmaxf(__low2float(mx2), __high2float(mx2));
-                    }
-                    m = warp_max(m);
-                    const float r = m * c;                          // -inf only if the whole unit is -inf
-                    const float nr = r > -INFINITY ? -r : 0.0f;
-                    const f32x2 c2 = pair_of(c, c), nr2 = pair_of(nr, nr);
-                    f32x2 acc0 = pair_of(0.0f, 0.0f), acc1 = acc0;
-#pragma unroll
-                    for (int j = 0; j < kVPL; ++j) {
-                        if constexpr (kF32) {
-                            d[j] = exp_quad(d[j], c2, nr2, acc0, acc1);
-                        } else {
-                            d[j].x = exp_pair(d[j].x, c2, nr2, acc0); d[j].y = exp_pair(d[j].y, c2, nr2, acc1);
-                            d[j].z = exp_pair(d[j].z, c2, nr2, acc0); d[j].w = exp_pair(d[j].w, c2, nr2, acc1);
-                        }
-                        const int i = lane + 32 * j;
-                        if (backward && i < nv) src[i] = d[j];
-                    }
-                    float s0, s1;
-                    unpair(add2(acc0, acc1), s0, s1);
-                    const float sum = warp_sum(s0 + s1);
-                    if (lane == 0) sh.meta[s].rs[u] = make_float2(r, sum);
                 }
                 __syncwarp();
                 if (lane == 0) {
@@ -271,45 +359,42 @@ grpo_loss_tile_kernel(const LossArgs a, const int rows_per_tile) {
                     if (!backward) arrive(smem_u32(&sh.free_[s]));          // forward only: the stage has been read, that is all
                 }
             }
-            if (backward && k >= kSkew) {
-                // ---- pass 2 of tile k - kSkew
-                const int kk = k - kSkew;
+            if (backward && kk >= 0 && kk < n_tiles) {
                 const uint32_t s = (uint32_t)kk % kStages;
                 if (!__all_sync(0xffffffffu, wait(smem_u32(&sh.s_done[s]), ((uint32_t)kk / kStages) & 1, abort_flag, a.wait_limit_ns))) break;
                 const uint4* stage = reinterpret_cast<const uint4*>(ring_raw + (size_t)s * kStageBytes);
                 const int units = tile_rows(kk) * P;
                 const long long t0 = tile_row0(kk);
+                char* tile_dst = a.dlogits + t0 * a.row_bytes;
 #pragma unroll
-                for (int ui = 0; ui < kUnitsPerWarp; ++ui) {
-                    const int u = warp + ui * kConsumerWarps;
-                    if (u >= units) break;
-                    const int row = u_row[ui];
-                    const uint4* src = stage + u_vec[ui];
-                    char* drow = a.dlogits + (t0 + row) * a.row_bytes;
-                    uint4* dst = reinterpret_cast<uint4*>(a.dlogits + t0 * a.row_bytes + u_dst[ui]);
-                    const int nv = u_nv[ui];
-                    const float sc = sh.meta[s].sc[u];
-                    const f32x2 sc2 = pair_of(sc, sc);
-#pragma unroll
-                    for (int j = 0; j < kVPL; ++j) {
-                        const int i = lane + 32 * j;
-                        if (i < nv) {
-                            const uint4 e = src[i];
-                            uint4 o;
-                            if constexpr (kF32) {
-                                o = scale_quad(e, sc2);
-                            } else {
-                                o.x = scale_pair(e.x, sc2); o.y = scale_pair(e.y, sc2);
-                                o.z = scale_pair(e.z, sc2); o.w = scale_pair(e.w, sc2);
-                            }
-                            __stcs(dst + i, o);
-                        }
+                for (int i = 0; i < kUnitsPerWarp; i += 2) {
+                    const int ua = wid + i * kGroupWarps, ub = ua + kGroupWarps;
+                    if (ub < units) {
+                        const uint4* const src[2] = {stage + u_vec[i], stage + u_vec[i + 1]};
+                        uint4* const dst[2] = {reinterpret_cast<uint4*>(tile_dst + u_dst[i]), reinterpret_cast<uint4*>(tile_dst + u_dst[i + 1])};
+                        const int nv[2] = {u_nv[i], u_nv[i + 1]};
+                        const float sc[2] = {sh.meta[s].sc[ua], sh.meta[s].sc[ub]};
+                        pass2_units<kF32, kVPL, 2>(src, dst, nv, sc, lane);
+                    } else if (ua < units) {
+                        const uint4* const src[1] = {stage + u_vec[i]};
+                        uint4* const dst[1] = {reinterpret_cast<uint4*>(tile_dst + u_dst[i])};
+                        const int nv[1] = {u_nv[i]};
+                        const float sc[1] = {sh.meta[s].sc[ua]};
+                        pass2_units<kF32, kVPL, 1>(src, dst, nv, sc, lane);
                     }
-                    // the one element of the row that also carries the onehot term, if it lies in this unit
-                    const int y = sh.meta[s].fix_y[row];
-                    const int e0 = u_e0[ui];
-                    __syncwarp();                                           // after the lanes' stores of the unit
-                    if (lane == 0 && y >= e0 && y < e0 + (nv << kLog2PerVec)) Elems<!kF32>::store1(drow, y, sh.meta[s].fix_val[row]);
+                }
+                // the one element of a row that also carries the onehot term, where it lies in one of this warp's units
+                __syncwarp();                                               // after the lanes' stores of the units
+                if (lane < kUnitsPerWarp) {
+                    int row = 0, e0 = 0, nv = 0;
+#pragma unroll
+                    for (int i = 0; i < kUnitsPerWarp; ++i)
+                        if (lane == i) { row = u_row[i]; e0 = u_e0[i]; nv = u_nv[i]; }
+                    if (wid + lane * kGroupWarps < units) {
+                        const int y = sh.meta[s].fix_y[row];
+                        if (y >= e0 && y < e0 + (nv << kLog2PerVec))
+                            Elems<!kF32>::store1(tile_dst + (long long)row * a.row_bytes, y, sh.meta[s].fix_val[row]);
+                    }
                 }
                 // the stage goes back to the loader: this warp's reads and writes of it come before the next copy into it
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
