@@ -46,8 +46,8 @@ WORKLOAD_TEXT = WORKLOAD + ": P=32 G=8, response 64-1024 tokens, V=151936 bf16 l
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch over 8192 rows of this vocabulary.  Traffic
 # grows in proportion to the rows, so a launch over T rows moves T times the per-row figure.  The record
 # is tied to the kernel sources it was taken from: once they change, `traffic` is reported as null.
-TRAFFIC_CAPTURE = {"rows": 8192, "dram_bytes": 2489531000 + 2431551000,
-                   "source_sha256": "579e608420e874657a7134b5630237f74d88f61552209af201eeb0f088e1ab64"}
+TRAFFIC_CAPTURE = {"rows": 8192, "dram_bytes": 2489449000 + 2432122000,
+                   "source_sha256": "d86ff3052c1d82b57f08f193f805e11838b448ac96fe6cbbd238bb0b51579171"}
 
 
 def captured_traffic_per_row():
