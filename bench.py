@@ -284,8 +284,14 @@ def run_profile_case(args):
         cu = torch.from_numpy(np.linspace(0, T, S + 1).astype(np.int32)).cuda()
         adv = torch.from_numpy(rng.normal(size=S).astype(np.float32)).cuda()
         wseq = torch.full((S,), 1.0 / S, device="cuda")
+        per16 = 8 if args.dtype == "bf16" else 4                  # rows start on 16-byte boundaries: pad the pitch
+        stride = -(-w.V // per16) * per16
+        if stride != w.V:
+            padded = torch.zeros((T, stride), dtype=tok.logits.dtype, device="cuda")
+            padded[:, :w.V] = tok.logits
+            tok.logits = padded
         dl = tok.logits if args.in_place else torch.empty_like(tok.logits)
-        prm = B.LossParams(T, w.V, B.BF16 if args.dtype == "bf16" else B.F32, w.V, S, args.variant, w.eps, w.eps, w.beta, 1.0)
+        prm = B.LossParams(T, w.V, B.BF16 if args.dtype == "bf16" else B.F32, stride, S, args.variant, w.eps, w.eps, w.beta, 1.0)
         ch = B.grpo_loss_kernel_choice(prm, forward_only=args.forward_only)
         print("kernel: %s, %d CTA(s) per row, %d threads%s" % (B.KERNEL_NAMES[ch.kernel], ch.ctas_per_row, ch.threads,
                                                                   " (fell back)" if ch.fell_back else ""))
