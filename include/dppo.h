@@ -250,8 +250,9 @@ size_t dppo_grpo_loss_workspace_bytes(const dppo_loss_params* p);
  *   logp_out, lse_out   f32 [T_max] or NULL
  *   loss_out     f32 [5]: loss, policy-gradient part -sum W surr, sum W kl, clipped fraction, T
  * Errors: INVALID_ARG, BAD_SHAPE, MISALIGNED (logits/dlogits base or row stride), UNSUPPORTED
- * (dtype), WORKSPACE_TOO_SMALL.  Device status: BAD_TARGET (that row's dlogits are zeroed and it
- * adds nothing to the loss), BAD_SEGMENTS.
+ * (dtype), WORKSPACE_TOO_SMALL.  Device status: BAD_TARGET, BAD_SEGMENTS (a row below T that cu_seqlens does not
+ * cover): such a row's dlogits are zero, its logp_out is 0 (its lse_out is still the row's log-sum-exp) and it adds
+ * nothing to the loss; the other rows are not affected.
  */
 int dppo_grpo_loss_fwd_bwd(const dppo_loss_params* p, const void* logits, const int32_t* target,
                            const float* logp_old, const float* logp_ref, const int32_t* cu_seqlens,

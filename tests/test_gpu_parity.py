@@ -418,6 +418,9 @@ def test_loss_tile_kernel(dtype):
     _loss_case(512 * per, dtype, T=50, S=2, seed=626, variant=v, neg_inf_cols=(0, 300 * per))
     _loss_case(128 * per, dtype, T=40, S=3, seed=627, variant=v, logit_sigma=40.0, centre_on_oracle=True)
     from paper_2603_04135_b200 import binding as B
+    _loss_case(64 * per, dtype, T=30000, S=7000, seed=650, variant=v, centre_on_oracle=True)   # more sequences than the shared-memory copy of cu_seqlens holds
+    _loss_case(128 * per, dtype, T=3, S=2, seed=651, variant=v)                                # fewer rows than a tile
+    _loss_case(128 * per, dtype, T=1, S=1, seed=652, variant=v)
     # forward only: pass 1 and the scalar stage; stages reused many times, the sequence-level ratio's two sweeps
     _loss_case(128 * per, dtype, T=40000, S=300, seed=640, variant=v, forward_only=True, centre_on_oracle=True)
     _loss_case(300 * per, dtype, T=67, S=5, seed=641, variant=v, forward_only=True)
@@ -569,6 +572,51 @@ def test_loss_kernel_choice_query():
     with pytest.raises(B.DppoError) as e:
         choice(151936, B.F32, variant=10256)                              # one CTA cannot hold 594 KB
     assert e.value.code == B.ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("dtype,V,variant,forward_only", [
+    ("bf16", 1024, 1, False), ("bf16", 1016, 2, False), ("bf16", 1024, 4, False), ("f32", 4096, 4, False), ("bf16", 1024, 4, True),
+    ("bf16", 16384, 10256, False), ("bf16", 65536, 0, False), ("bf16", 151936, 3, True)])
+def test_loss_rows_that_no_sequence_covers(dtype, V, variant, forward_only):
+    """cu_seqlens that ends before the token count (a caller's mistake): the rows past its last entry belong to no
+    sequence.  Every kernel reports DPPO_STATUS_BAD_SEGMENTS, leaves those rows as rows that add nothing (dlogits and
+    logp_out of zero) and gives the covered rows exactly what a call on the covered rows alone gives."""
+    from paper_2603_04135_b200 import binding as B
+    T, covered, S = 45, 29, 3
+    per16 = 8 if dtype == "bf16" else 4
+    stride = -(-V // per16) * per16
+    w = synth.scaled(synth.WORKLOADS["config0"], V=stride, dtype=dtype)
+    tok = synth.make_token_inputs(w, T, 700, device="cuda")
+    tok.target.clamp_(max=V - 1)
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    rng = np.random.default_rng(700)
+    adv = torch.from_numpy(rng.normal(size=S).astype(np.float32)).cuda()
+    wseq = torch.from_numpy((rng.random(S) * 0.1).astype(np.float32)).cuda()
+    cu = torch.tensor([0, 10, 17, covered], dtype=torch.int32, device="cuda")
+
+    def call(T_call):
+        prm = B.LossParams(T_call, V, B.BF16 if dtype == "bf16" else B.F32, stride, S, variant, 0.2, 0.2, 0.04, 1.0)
+        nbytes = B.grpo_loss_workspace_bytes(prm)
+        ws = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+        dl = None if forward_only else torch.full((T, stride), 7.0, dtype=tdt, device="cuda")
+        loss_out = torch.full((5,), 7.0, device="cuda")
+        logp_out = torch.full((T,), 7.0, device="cuda"); lse_out = torch.full((T,), 7.0, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        B.grpo_loss_fwd_bwd(prm, tok.logits, tok.target, tok.logp_old, tok.logp_ref, cu, None, adv, wseq, None, dl,
+                            logp_out, lse_out, loss_out, ws, nbytes, status)
+        torch.cuda.synchronize()
+        return dl, logp_out, lse_out, loss_out, int(status.item())
+
+    dl, logp_out, lse_out, loss_out, status = call(T)
+    ref_dl, ref_logp, ref_lse, ref_loss, ref_status = call(covered)
+    assert ref_status == 0 and status == B.STATUS_BAD_SEGMENTS
+    assert bool((logp_out[covered:] == 0).all()) and bool(torch.isfinite(lse_out).all())
+    assert torch.equal(logp_out[:covered], ref_logp[:covered]) and torch.equal(lse_out[:covered], ref_lse[:covered])
+    assert torch.equal(loss_out[:4], ref_loss[:4]) and float(loss_out[4]) == T and float(ref_loss[4]) == covered
+    if not forward_only:
+        assert bool((dl[covered:, :V] == 0).all())
+        assert torch.equal(dl[:covered].view(torch.int16 if dtype == "bf16" else torch.int32),
+                           ref_dl[:covered].view(torch.int16 if dtype == "bf16" else torch.int32))
 
 
 def test_loss_bad_target_and_empty():
