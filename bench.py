@@ -268,6 +268,46 @@ def time_lmhead(H, dev, gpu_index, iters=10, warmup=3, sample_clocks=True):
                          "note": "executed flops = 6 T V H: logits, dhidden, dW (a chunk's exponentials are kept as bf16, nothing is recomputed)"}}
 
 
+def time_row_length(dtype, V, rows, dev, iters=8, warmup=3):
+    """The loss sweep (forward + dlogits, the call a training step makes: device-side token count, sequence map,
+    log-prob and lse outputs) on `rows` rows of another vocabulary size, with the library's own kernel choice:
+    `iters` back-to-back calls after `warmup`, CUDA events around each."""
+    from paper_2603_04135_b200 import binding as B
+    w = synth.scaled(synth.WORKLOADS["config3"], V=V, dtype=dtype)
+    S = 2000
+    tok = synth.make_token_inputs(w, rows, 0, device=dev)
+    rng = np.random.default_rng(0)
+    cu = torch.from_numpy(np.linspace(0, rows, S + 1).astype(np.int32)).to(dev)
+    adv = torch.from_numpy(rng.normal(size=S).astype(np.float32)).to(dev)
+    wseq = torch.full((S,), 1.0 / S, device=dev)
+    dl = torch.empty_like(tok.logits)
+    prm = B.LossParams(rows, V, B.BF16 if dtype == "bf16" else B.F32, V, S, 0, w.eps, w.eps, w.beta, 1.0)
+    ch = B.grpo_loss_kernel_choice(prm)
+    nbytes = B.grpo_loss_workspace_bytes(prm)
+    ws = torch.zeros(nbytes, dtype=torch.uint8, device=dev)
+    loss_out = torch.zeros(5, device=dev); status = torch.zeros(1, dtype=torch.int32, device=dev)
+    ntd = torch.tensor([rows], dtype=torch.int32, device=dev)
+    seg_map = torch.arange(S, dtype=torch.int32, device=dev)
+    logp_out = torch.zeros(rows, device=dev); lse_out = torch.zeros(rows, device=dev)
+    evs = []
+    for it in range(warmup + iters):
+        a_, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a_.record()
+        B.grpo_loss_fwd_bwd(prm, tok.logits, tok.target, tok.logp_old, tok.logp_ref, cu, ntd, adv, wseq, seg_map, dl,
+                            logp_out, lse_out, loss_out, ws, nbytes, status)
+        b_.record()
+        evs.append((a_, b_))
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    ms = sum(x.elapsed_time(y) for x, y in evs[warmup:]) / iters
+    esize = 2 if dtype == "bf16" else 4
+    gbs = 2.0 * rows * V * esize / (ms / 1e3) / 1e9
+    peak, _ = measured_peaks()
+    return {"dtype": dtype, "V": V, "row_bytes": V * esize, "rows": rows, "kernel": B.KERNEL_NAMES[ch.kernel],
+            "ctas_per_row": ch.ctas_per_row, "ms": ms, "achieved_gbs": gbs, "frac": gbs / peak,
+            "tokens_per_s": rows / ms * 1e3}
+
+
 # --------------------------------------------------------------------------------------- profile cases
 def run_profile_case(args):
     """A small, self-contained run of one entry point for timing and profiler captures: prints the event-timed
@@ -474,7 +514,7 @@ def run_ours(args):
     loss_value = float(st.loss_out[0].item())
 
     # ---- the same kernel in its other modes (rank 0 of a single-GPU run; a few calls each, CUDA events)
-    modes = None
+    modes = other_rows = None
     if rank == 0 and world == 1 and not args.no_modes:
         from paper_2603_04135_b200 import binding as B
 
@@ -519,6 +559,11 @@ def run_ours(args):
         ch = B.grpo_loss_kernel_choice(st.loss_params)
         modes["kernel_choice"] = {"kernel": B.KERNEL_NAMES[ch.kernel], "ctas_per_row": ch.ctas_per_row, "threads": ch.threads,
                                   "fell_back_to_general_kernel": bool(ch.fell_back)}
+
+        # ---- the same entry point on other row lengths (about 2 GB of logits each): the short-row and mid-row kernels
+        other_rows = [time_row_length(dt, V_, n_, dev) for dt, V_, n_ in
+                      (("bf16", 1024, 1000000), ("bf16", 4096, 250000), ("f32", 2048, 250000), ("bf16", 32768, 40000))]
+        torch.cuda.empty_cache()
 
     # ---- end to end: host buffers in, loss scalars out, through DppoStep.step_from_host
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
@@ -603,6 +648,7 @@ def run_ours(args):
         if modes is not None:
             line["roofline"]["kernel_choice"] = modes.pop("kernel_choice")
             line["loss_sweep_modes"] = modes
+            line["loss_sweep_other_row_lengths"] = other_rows
         if lm is not None:
             line["lmhead"] = lm
             line["lmhead_h4096"] = lm_wide
