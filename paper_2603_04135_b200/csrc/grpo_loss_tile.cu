@@ -8,10 +8,11 @@
 // splits the work:
 //   loader          one thread issues one bulk copy per TILE (up to 32 KB of consecutive rows, at most 32 units)
 //                   into a ring of stages, running ahead as far as the ring allows
-//   16 consumer     pass 1 on the tile's UNITS (a unit is a row, or a 2 KB part of a longer row; one warp per unit):
-//   warps           maximum, 2^(z c - r) once, kept in place as fp16 pairs (bf16 rows) or f32, the unit's (r, sum) to
-//                   shared memory.  Pass 2, three tiles later: the stored exponentials times the unit's factor go to
-//                   dlogits with streaming stores; the stage is then free
+//   16 consumer     two groups of eight take the tiles alternately.  Pass 1 on the tile's UNITS (a unit is a row, or
+//   warps           one of the equal parts of at most 2 KB of a longer row; a warp works on two units at a time):
+//                   maximum, 2^(z c - r) once, kept in place as fp16 pairs (bf16 rows) or f32, the unit's (r, sum) to
+//                   shared memory.  Pass 2, after pass 1 of the group's next tile: the stored exponentials times the
+//                   unit's factor go to dlogits with streaming stores; the stage is then free
 //   scalar warps    lane q takes row q of a tile: joins the row's units, runs the scalar stage for up to 32 rows in
 //                   one pass, and leaves every unit's factor g/tau 2^(r - lse2) (and the one element per row that
 //                   also carries the onehot term) for pass 2.  The rows' per-token inputs and sequences are gathered
