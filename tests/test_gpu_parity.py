@@ -734,6 +734,62 @@ def test_config3_full_size():
     assert T > 60000
 
 
+@pytest.mark.parametrize("dtype,V,T", [("bf16", 1024, 1000000), ("f32", 2048, 250000)])
+def test_short_rows_at_the_timed_size(dtype, V, T):
+    """The short-row cases the benchmark line times (`loss_sweep_other_row_lengths`), in the call form it uses: the
+    library's own kernel choice (the tile kernel), device-side token count, sequence map, log-prob and lse outputs,
+    2,000 sequences.  dlogits element-wise on the first and last row of every sequence plus random rows; log-probs,
+    lse and the loss sums against the oracle over ALL rows."""
+    from paper_2603_04135_b200 import binding as B
+    S, seed = 2000, 800
+    w = synth.scaled(synth.WORKLOADS["config3"], V=V, dtype=dtype)
+    tok = synth.make_token_inputs(w, T, seed, device="cuda")
+    rng = np.random.default_rng(seed)
+    cu = np.linspace(0, T, S + 1).astype(np.int32)
+    adv = rng.normal(size=S).astype(np.float32)
+    wseq = np.full(S, 1.0 / S, dtype=np.float32)
+    seg_map = rng.permutation(S).astype(np.int32)
+    prm = B.LossParams(T, V, B.BF16 if dtype == "bf16" else B.F32, V, S, 0, w.eps, w.eps, w.beta, 1.0)
+    assert B.grpo_loss_kernel_choice(prm).kernel == B.KERNEL_TILE
+    nbytes = B.grpo_loss_workspace_bytes(prm)
+    ws = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+    dl = torch.empty_like(tok.logits)
+    loss_out = torch.zeros(5, device="cuda"); status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    logp_out = torch.zeros(T, device="cuda"); lse_out = torch.zeros(T, device="cuda")
+    ntd = torch.tensor([T], dtype=torch.int32, device="cuda")
+    B.grpo_loss_fwd_bwd(prm, tok.logits, tok.target, tok.logp_old, tok.logp_ref, torch.from_numpy(cu).cuda(), ntd,
+                        torch.from_numpy(adv).cuda(), torch.from_numpy(wseq).cuda(), torch.from_numpy(seg_map).cuda(), dl,
+                        logp_out, lse_out, loss_out, ws, nbytes, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    adv_seg, w_seg = adv[seg_map], wseq[seg_map]
+    target = tok.target.cpu().numpy(); lo = tok.logp_old.cpu().numpy(); lr = tok.logp_ref.cpu().numpy()
+    tol = LOGP_TOL[dtype]
+    logp_got = logp_out.cpu().numpy(); lse_got = lse_out.cpu().numpy()
+    rows_all = pick_rows(cu, T, 1024, seed)
+    n_stable = 0
+    for a in range(0, len(rows_all), 1024):
+        rows = rows_all[a:a + 1024]
+        sub = oracle.grpo_loss(rows_to_f64(tok.logits, rows), target, lo, lr, cu, adv_seg, w_seg, w.eps, w.eps, w.beta,
+                               rows=rows, chunk=256)
+        stable = clip_decision_is_stable(sub["rho"], w.eps, w.eps)
+        n_stable += int(stable.sum())
+        assert_dlogits_close(rows_to_f64(dl, rows), sub, dtype, w.beta, rows_ok=stable)
+        assert np.abs(logp_got[rows] - sub["logp"]).max() <= tol
+        assert np.abs(lse_got[rows] - sub["lse"]).max() <= tol
+    assert len(rows_all) > 4096 and n_stable > 0.99 * len(rows_all)
+    full = oracle_forward_all_rows(tok.logits, target, lo, lr, cu, adv_seg, w_seg, w.eps, w.eps, w.beta, rows_per_task=16384)
+    out = loss_out.cpu().numpy().astype(np.float64)
+    assert out[4] == T
+    assert np.abs(logp_got - full["logp"]).max() <= tol and np.abs(lse_got - full["lse"]).max() <= tol
+    assert abs(out[0] - full["loss"]) <= 1e-4 * abs(full["loss"]) + 1e-7 * full["abs_sum"]
+    assert abs(out[1] - full["pg"]) <= 1e-4 * full["abs_sum"]
+    assert abs(out[2] - full["kl"]) <= 1e-4 * full["kl"] + 1e-9
+    # a row whose ratio sits within the margin of a clip bound may take the other branch in f32 (same loss there)
+    unstable = int((~clip_decision_is_stable(full["rho"], w.eps, w.eps)).sum())
+    assert abs(out[3] - full["clip_frac"]) <= (unstable + 2.0) / T
+
+
 def test_rows_sharded_over_two_ranks_add_up():
     # Rows dealt out to two ranks (dp.shard_rows), each rank's sweep run here one after the other on the one device:
     # every rank uses the sequence weights of the WHOLE batch, so the five scalars add up to the whole batch's and each
