@@ -49,16 +49,26 @@ __device__ __forceinline__ unsigned long long global_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait on phase `parity`; also leaves (false) when another role has raised the abort flag.
+// One try: the thread is suspended until the phase completes or about a microsecond has passed (a waiting warp
+// then issues a handful of instructions per microsecond instead of spinning against the working warps).
+constexpr uint32_t kSuspendNs = 1000;
+__device__ __forceinline__ bool try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(bar), "r"(parity), "r"(kSuspendNs) : "memory");
+    return done != 0;
+}
+// Bounded wait on phase `parity`; also leaves (false) when another role has raised the abort flag.  The clock and
+// the abort flag are looked at once per eight tries.
 __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned long long limit_ns) {
+    if (try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_ns();
     for (;;) {
-        uint32_t done;
-        asm volatile("{\n\t.reg .pred p;\n\t"
-                     "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-                     "selp.u32 %0, 1, 0, p;\n\t}"
-                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-        if (done) return true;
+#pragma unroll 1
+        for (int i = 0; i < 8; ++i)
+            if (try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
         if (global_ns() - t0 > limit_ns) { *abort_flag = 1; return false; }
     }
