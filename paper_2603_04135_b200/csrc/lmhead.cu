@@ -92,11 +92,15 @@ __device__ __forceinline__ bool lm_try(uint32_t bar, uint32_t parity) {
     return done != 0;
 }
 
-// Bounded wait; also leaves when another role has raised the abort flag.
+// Bounded wait; also leaves when another role has raised the abort flag.  The clock and the flag are looked at once
+// per sixteen tries (a try already suspends the thread for a short, hardware-chosen time), not per try.
 __device__ __forceinline__ bool lm_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned long long limit_ns) {
+    if (lm_try(bar, parity)) return true;
     const unsigned long long t0 = lm_global_ns();
     for (;;) {
-        if (lm_try(bar, parity)) return true;
+#pragma unroll 1
+        for (int i = 0; i < 16; ++i)
+            if (lm_try(bar, parity)) return true;
         if (*abort_flag) return false;
         if (lm_global_ns() - t0 > limit_ns) { *abort_flag = 1; return false; }
     }
@@ -104,9 +108,12 @@ __device__ __forceinline__ bool lm_wait(uint32_t bar, uint32_t parity, volatile 
 
 // Bounded wait that ignores the abort flag (used on the way out).
 __device__ __forceinline__ bool lm_wait_plain(uint32_t bar, uint32_t parity, unsigned long long limit_ns) {
+    if (lm_try(bar, parity)) return true;
     const unsigned long long t0 = lm_global_ns();
     for (;;) {
-        if (lm_try(bar, parity)) return true;
+#pragma unroll 1
+        for (int i = 0; i < 16; ++i)
+            if (lm_try(bar, parity)) return true;
         if (lm_global_ns() - t0 > limit_ns) return false;
     }
 }
